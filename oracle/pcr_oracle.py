@@ -1,0 +1,199 @@
+"""ctypes front end of the CPU oracle (`pcr_oracle.c`).
+
+TEST INFRASTRUCTURE ONLY: tests, the smoke check and the benchmark's CPU-baseline leg may
+import this; the CUDA library and its Python binding never do.  The C file is compiled on
+first use with the host compiler; it links nothing but libm.
+
+Follows the paper's Section 3 (record = metadata + scan groups, prefix read = fidelity k)
+and Section 5 "Decoding" (reassemble scans 1..k, terminate with EOI, JPEG-decode).
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "pcr_oracle.c")
+_LIB = os.path.join(_HERE, "libpcr_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(["gcc", "-O2", "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    with _lock:
+        if _lib is None:
+            lib = C.CDLL(build())
+            vp, sz = C.c_void_p, C.c_size_t
+            lib.oracle_record_info.argtypes = [vp, sz, C.POINTER(C.c_int), C.POINTER(C.c_int)]
+            lib.oracle_image_info.argtypes = [vp, sz, C.c_int, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32), C.POINTER(C.c_int32)]
+            lib.oracle_prefix_bytes.restype = C.c_longlong
+            lib.oracle_prefix_bytes.argtypes = [vp, sz, C.c_int]
+            lib.oracle_reassemble.restype = C.c_longlong
+            lib.oracle_reassemble.argtypes = [vp, sz, C.c_int, C.c_int, vp, sz]
+            lib.oracle_decode_image.argtypes = [vp, sz, C.c_int, C.c_int, vp, sz, vp]
+            lib.oracle_jpeg_decode.argtypes = [vp, sz, vp, sz, vp, vp, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]
+            lib.oracle_jpeg_dims.argtypes = [vp, sz, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]
+            lib.oracle_pixels_from_coeffs.argtypes = [vp, C.c_uint32, C.c_uint32, vp, vp, vp, vp, vp]
+            lib.oracle_num_blocks.restype = sz
+            lib.oracle_num_blocks.argtypes = [C.c_uint32, C.c_uint32]
+            lib.oracle_block_idct.argtypes = [vp, vp, vp]
+            lib.oracle_ycc_to_rgb.argtypes = [C.c_int, C.c_int, C.c_int, vp]
+            lib.oracle_ycc_to_rgb_array.argtypes = [vp, sz, vp]
+            _lib = lib
+    return _lib
+
+
+class OracleError(RuntimeError):
+    def __init__(self, code):
+        super().__init__(f"oracle error {code}")
+        self.code = code
+
+
+def _chk(rc):
+    if rc < 0:
+        raise OracleError(rc)
+    return rc
+
+
+def _u8(buf) -> np.ndarray:
+    a = np.frombuffer(buf, dtype=np.uint8) if not isinstance(buf, np.ndarray) else buf
+    return np.ascontiguousarray(a, dtype=np.uint8)
+
+
+def record_info(rec):
+    """(number of images, number of scan groups)."""
+    rec = _u8(rec)
+    n, g = C.c_int(), C.c_int()
+    _chk(_load().oracle_record_info(rec.ctypes.data, rec.size, C.byref(n), C.byref(g)))
+    return n.value, g.value
+
+
+def image_info(rec, i):
+    """(width, height, label) of image i, from the record's sample metadata."""
+    rec = _u8(rec)
+    W, H, lab = C.c_uint32(), C.c_uint32(), C.c_int32()
+    _chk(_load().oracle_image_info(rec.ctypes.data, rec.size, i, C.byref(W), C.byref(H), C.byref(lab)))
+    return W.value, H.value, lab.value
+
+
+def prefix_bytes(rec, k) -> int:
+    rec = _u8(rec)
+    return _chk(_load().oracle_prefix_bytes(rec.ctypes.data, rec.size, k))
+
+
+def reassemble(rec, i, k) -> bytes:
+    """Scans 1..k of image i followed by EOI: a JPEG file any stock decoder renders."""
+    rec = _u8(rec)
+    lib = _load()
+    n = _chk(lib.oracle_reassemble(rec.ctypes.data, rec.size, i, k, None, 0))
+    out = np.empty(n, dtype=np.uint8)
+    _chk(lib.oracle_reassemble(rec.ctypes.data, rec.size, i, k, out.ctypes.data, out.size))
+    return out.tobytes()
+
+
+def num_blocks(W, H) -> int:
+    return int(_load().oracle_num_blocks(W, H))
+
+
+def decode_image(rec, i, k, want_rgb=True):
+    """Image i at fidelity k -> (coefficients (blocks, 64) int16 zigzag, RGB (H, W, 3) uint8 or None)."""
+    rec = _u8(rec)
+    W, H, _ = image_info(rec, i)
+    coef = np.empty((num_blocks(W, H), 64), dtype=np.int16)
+    rgb = np.empty((H, W, 3), dtype=np.uint8) if want_rgb else None
+    _chk(_load().oracle_decode_image(rec.ctypes.data, rec.size, i, k, coef.ctypes.data, coef.size,
+                                     rgb.ctypes.data if want_rgb else None))
+    return coef, rgb
+
+
+def jpeg_decode(jpg: bytes, want_planes=False):
+    """A progressive JPEG byte string -> (coefficients, RGB[, (Y, Cb, Cr) padded planes])."""
+    lib = _load()
+    a = _u8(jpg)
+    W, H = C.c_uint32(), C.c_uint32()
+    _chk(lib.oracle_jpeg_dims(a.ctypes.data, a.size, C.byref(W), C.byref(H)))
+    W, H = W.value, H.value
+    coef = np.empty((num_blocks(W, H), 64), dtype=np.int16)
+    rgb = np.empty((H, W, 3), dtype=np.uint8)
+    mx, my = (W + 15) // 16, (H + 15) // 16
+    planes = np.empty(384 * mx * my, dtype=np.uint8) if want_planes else None
+    _chk(lib.oracle_jpeg_decode(a.ctypes.data, a.size, coef.ctypes.data, coef.size, rgb.ctypes.data,
+                                planes.ctypes.data if want_planes else None, None, None))
+    if not want_planes:
+        return coef, rgb
+    ny = 256 * mx * my
+    Y = planes[:ny].reshape(16 * my, 16 * mx)
+    Cb = planes[ny:ny + 64 * mx * my].reshape(8 * my, 8 * mx)
+    Cr = planes[ny + 64 * mx * my:].reshape(8 * my, 8 * mx)
+    return coef, rgb, (Y, Cb, Cr)
+
+
+def pixels_from_coeffs(coef, W, H, qy_zz, qc_zz, want_planes=False):
+    """Sequential-style decode of given coefficients: canonical (blocks, 64) int16 + zigzag-order
+    quantisers -> RGB (H, W, 3)."""
+    coef = np.ascontiguousarray(coef, dtype=np.int16)
+    qy = np.ascontiguousarray(qy_zz, dtype=np.uint16)
+    qc = np.ascontiguousarray(qc_zz, dtype=np.uint16)
+    rgb = np.empty((H, W, 3), dtype=np.uint8)
+    mx, my = (W + 15) // 16, (H + 15) // 16
+    planes = np.empty(384 * mx * my, dtype=np.uint8) if want_planes else None
+    _chk(_load().oracle_pixels_from_coeffs(coef.ctypes.data, W, H, qy.ctypes.data, qc.ctypes.data, qc.ctypes.data,
+                                           rgb.ctypes.data, planes.ctypes.data if want_planes else None))
+    if not want_planes:
+        return rgb
+    ny = 256 * mx * my
+    return rgb, (planes[:ny].reshape(16 * my, 16 * mx), planes[ny:ny + 64 * mx * my].reshape(8 * my, 8 * mx),
+                 planes[ny + 64 * mx * my:].reshape(8 * my, 8 * mx))
+
+
+def block_idct(coef_zz, q_zz) -> np.ndarray:
+    c = np.ascontiguousarray(coef_zz, dtype=np.int16)
+    q = np.ascontiguousarray(q_zz, dtype=np.uint16)
+    out = np.empty(64, dtype=np.uint8)
+    _load().oracle_block_idct(c.ctypes.data, q.ctypes.data, out.ctypes.data)
+    return out.reshape(8, 8)
+
+
+def ycc_to_rgb(Y, cb, cr):
+    out = np.empty(3, dtype=np.uint8)
+    _load().oracle_ycc_to_rgb(int(Y), int(cb), int(cr), out.ctypes.data)
+    return tuple(int(v) for v in out)
+
+
+def ycc_to_rgb_array(ycc: np.ndarray) -> np.ndarray:
+    """(n, 3) uint8 Y,Cb,Cr triples -> (n, 3) uint8 R,G,B."""
+    a = np.ascontiguousarray(ycc, dtype=np.uint8).reshape(-1, 3)
+    out = np.empty_like(a)
+    _load().oracle_ycc_to_rgb_array(a.ctypes.data, a.shape[0], out.ctypes.data)
+    return out
+
+
+def decode_record(rec, k, images=None, want_rgb=True):
+    """Decode every image (or the listed ones) of a record at fidelity k, one after the other."""
+    n, _ = record_info(rec)
+    idx = range(n) if images is None else images
+    return [decode_image(rec, i, k, want_rgb) for i in idx]
+
+
+def _pool_worker(args):
+    path_or_bytes, k, lo, hi = args
+    rec = np.load(path_or_bytes, mmap_mode="r") if isinstance(path_or_bytes, str) else _u8(path_or_bytes)
+    rec = np.ascontiguousarray(rec)
+    npx = 0
+    for i in range(lo, hi):
+        _, rgb = decode_image(rec, i, k, True)
+        npx += rgb.shape[0] * rgb.shape[1]
+    return hi - lo, npx
