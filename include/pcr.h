@@ -1,0 +1,135 @@
+/*
+ * pcr.h — C ABI of the B200 (sm_100a) decoder for Progressive Compressed Records.
+ *
+ * A record is the paper's storage unit (Section 3, and its record-layout figure): sample
+ * metadata (labels) and record metadata (where every image's every scan lives) followed by
+ * scan group 1 of all images, scan group 2 of all images, ...  Reading the record from its
+ * start to the end of scan group k gives every image at fidelity k.  This library takes
+ * those bytes and produces training pixels on the GPU: for every image, the progressive
+ * JPEG decode of its scans 1..k (Section 2, "Progressive Image Compression"; Section 5,
+ * "Decoding": scans 1..k of an image followed by an end-of-image token are a decodable
+ * JPEG) -> int16 coefficient planes in device memory -> dequantise, 8x8 inverse DCT,
+ * 2x2 chroma replication, YCbCr->RGB -> packed uint8 RGB.
+ *
+ * Record layout (little-endian, 16-byte aligned chunks; the "raw struct" form of Section 5):
+ *   header  64 B : "PCR1", u32 version(1), u32 n_images N, u32 n_groups G, u32 flags, u32 rsvd,
+ *                  u64 meta_off, u64 index_off, u64 data_off, u64 total_bytes, u64 rsvd
+ *   meta         : N x { i32 label; u32 width; u32 height; u32 rsvd }            (scan group 0)
+ *   index        : u64 group_end[G+1]  (group_end[0] = data_off; fidelity k needs bytes
+ *                  [0, group_end[k]))  then  { u64 off; u32 len; u32 rsvd } chunk[G][N]
+ *   data         : group 1 chunks of images 0..N-1, group 2 chunks, ...
+ *   chunk (g, i) = the bytes of image i's progressive JPEG file that belong to scan g: for
+ *   g = 1 from SOI (tables, frame header), for every g the scan's DHT/DRI/SOS segments and
+ *   entropy-coded bytes.  The file's EOI is not stored.  One scan per group.
+ *
+ * Supported streams: 8-bit, three components, 4:2:0 (2x2, 1x1, 1x1), progressive Huffman
+ * (SOF2), any scan script that is the same for all images of a record, any restart interval.
+ *
+ * All functions return an int status: PCR_OK (0) or a negative PCR_E_* code.  Nothing here
+ * throws, aborts or prints.  Unless said otherwise pointers are HOST pointers.
+ * A pcr_record may be used by one thread at a time.
+ */
+#ifndef PCR_H_
+#define PCR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PCR_OK 0
+#define PCR_E_ARG (-1)      /* NULL pointer, k outside 1..G, index out of range, misaligned output */
+#define PCR_E_FORMAT (-2)   /* not a record: magic/version, offsets not monotone or past the end,
+                               images disagree on the scan script, unsupported JPEG features     */
+#define PCR_E_CORRUPT (-3)  /* found while decoding on the device: undefined Huffman code,
+                               segment overrun, wrong number of restart markers                   */
+#define PCR_E_TIMEOUT (-4)  /* a bounded device-side wait gave up                                */
+#define PCR_E_CUDA (-5)     /* a CUDA runtime call failed                                        */
+#define PCR_E_NOMEM (-6)    /* host or device allocation failed                                  */
+
+typedef struct pcr_record pcr_record; /* opaque; owned by the library */
+
+typedef struct {
+    uint32_t width, height;
+    int32_t label;
+    uint32_t rsvd;
+    uint64_t out_offset; /* byte offset of the image's pixels inside the output buffer */
+    uint64_t out_bytes;  /* 3 * width * height                                          */
+} pcr_image_info;
+
+/* Section 3 (metadata + scan groups) and Section 5 "Decoding" (locate the offsets).
+ * Parses and validates the header, the group table, every chunk's position and every
+ * image's JPEG frame, table and scan headers; allocates the per-record device state
+ * (record bytes, coefficient planes, tables) on the current CUDA device.
+ *   bytes : the whole record, HOST memory (pinned memory makes the copies asynchronous).
+ *           BORROWED: it must stay valid and unchanged until pcr_close.
+ *   len   : its length in bytes (< 4 GiB).
+ *   rec   : receives the handle; NULL on failure.
+ * Errors: PCR_E_ARG, PCR_E_FORMAT, PCR_E_NOMEM, PCR_E_CUDA. */
+int pcr_open(const void* bytes, size_t len, pcr_record** rec);
+
+/* Number of images N / scan groups G of the record (negative error for a NULL handle). */
+int pcr_num_images(const pcr_record* rec);
+int pcr_num_groups(const pcr_record* rec);
+
+/* Sample metadata and output placement of image i (Section 3: labels are metadata). */
+int pcr_get_image(const pcr_record* rec, int i, pcr_image_info* info);
+
+/* Size the output buffer of pcr_decode must have.  Images are packed RGB, row-major,
+ * 3*width bytes per row, image i at out_offset (a multiple of 128). */
+size_t pcr_out_bytes(const pcr_record* rec);
+
+/* Bytes [0, pcr_prefix_bytes(rec, k)) are what fidelity k reads (Section 3: "from the
+ * start of the PCR to the end of the corresponding scan group").  0 for a bad k. */
+size_t pcr_prefix_bytes(const pcr_record* rec, int k);
+
+/* Decode all images at fidelity k (Sections 2, 3, 5): Huffman-decode scans 1..k into the
+ * record's int16 coefficient planes (first passes, then successive-approximation
+ * refinements in place), then dequantise, inverse-DCT, upsample, colour-convert and store.
+ *   k      : 1..G.
+ *   out    : DEVICE memory, caller-owned, at least pcr_out_bytes(rec) bytes, 16-byte aligned.
+ *            Only the bytes of each image's 3*W*H pixels are written.
+ *   stream : a cudaStream_t (NULL = the default stream).
+ * Any part of the prefix [0, end_k) that is not yet resident on the device is first copied
+ * from the borrowed host buffer on `stream`; resident bytes are kept for later calls.
+ * The call enqueues the copy and the kernels and returns; the caller synchronises `stream`.
+ * Every call decodes scans 1..k from scratch.  One decode in flight per record.
+ * Bytes at or beyond end_k are never read.
+ * Errors: PCR_E_ARG, PCR_E_CUDA (launch failures).  Stream errors found by the device are
+ * reported by pcr_status. */
+int pcr_decode(pcr_record* rec, int k, void* out, void* stream);
+
+/* Forget which record bytes are resident on the device: the next pcr_decode copies its whole
+ * prefix again (what a loader that streams each record once from host memory pays). */
+int pcr_evict(pcr_record* rec);
+
+/* After the stream of the last pcr_decode has been synchronised: reads the per-image
+ * status words back.  *code = PCR_OK, or the first failing image's error with its index in
+ * *first_bad_image (-1 if none).  A corrupt image's pixels come from the coefficients
+ * decoded before the error (never uninitialised memory). */
+int pcr_status(pcr_record* rec, int* first_bad_image, int* code);
+
+/* Test hook: the coefficient planes of the last decode, DEVICE memory owned by the record.
+ * Layout: image after image (image i's first block = its blocks_offset), within an image
+ * component Y, Cb, Cr, block rows then block columns of the MCU-padded grid, 64 int16 per
+ * block in zigzag order (128 bytes per block).  *bytes = total size. */
+int pcr_coeffs(pcr_record* rec, const int16_t** dev_planes, size_t* bytes);
+
+/* First block of image i inside the planes returned by pcr_coeffs, and its block count. */
+int pcr_image_blocks(const pcr_record* rec, int i, uint64_t* first_block, uint64_t* n_blocks);
+
+/* Counts kernel launches issued by this library since it was loaded (all records). */
+uint64_t pcr_launch_count(void);
+
+/* Text for a status code. */
+const char* pcr_strerror(int code);
+
+/* Frees host and device state.  NULL is allowed.  The borrowed bytes are not touched. */
+void pcr_close(pcr_record* rec);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PCR_H_ */

@@ -1,0 +1,135 @@
+"""ctypes binding of the C ABI declared in include/pcr.h: argument marshalling only.
+
+Every step of the decode runs in the CUDA library; there is no CPU fallback.  Loading fails
+loudly when the shared library has not been built.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpcr_b200.so")
+
+PCR_OK = 0
+PCR_E_ARG, PCR_E_FORMAT, PCR_E_CORRUPT, PCR_E_TIMEOUT, PCR_E_CUDA, PCR_E_NOMEM = -1, -2, -3, -4, -5, -6
+
+EXPORTS = ("pcr_open", "pcr_num_images", "pcr_num_groups", "pcr_get_image", "pcr_out_bytes", "pcr_prefix_bytes",
+           "pcr_decode", "pcr_evict", "pcr_status", "pcr_coeffs", "pcr_image_blocks", "pcr_launch_count",
+           "pcr_strerror", "pcr_close")
+
+
+class ImageInfo(C.Structure):
+    _fields_ = [("width", C.c_uint32), ("height", C.c_uint32), ("label", C.c_int32), ("rsvd", C.c_uint32),
+                ("out_offset", C.c_uint64), ("out_bytes", C.c_uint64)]
+
+
+class PcrError(RuntimeError):
+    def __init__(self, code, what=""):
+        self.code = code
+        super().__init__(f"{what}: {strerror(code)} ({code})")
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it first (python -m paper_1911_00472_b200.build); "
+                               "there is no fallback path")
+        L = C.CDLL(LIB_PATH)
+        vp = C.c_void_p
+        L.pcr_open.argtypes = [vp, C.c_size_t, C.POINTER(vp)]
+        L.pcr_num_images.argtypes = [vp]
+        L.pcr_num_groups.argtypes = [vp]
+        L.pcr_get_image.argtypes = [vp, C.c_int, C.POINTER(ImageInfo)]
+        L.pcr_out_bytes.restype = C.c_size_t
+        L.pcr_out_bytes.argtypes = [vp]
+        L.pcr_prefix_bytes.restype = C.c_size_t
+        L.pcr_prefix_bytes.argtypes = [vp, C.c_int]
+        L.pcr_decode.argtypes = [vp, C.c_int, vp, vp]
+        L.pcr_evict.argtypes = [vp]
+        L.pcr_status.argtypes = [vp, C.POINTER(C.c_int), C.POINTER(C.c_int)]
+        L.pcr_coeffs.argtypes = [vp, C.POINTER(vp), C.POINTER(C.c_size_t)]
+        L.pcr_image_blocks.argtypes = [vp, C.c_int, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
+        L.pcr_launch_count.restype = C.c_uint64
+        L.pcr_launch_count.argtypes = []
+        L.pcr_strerror.restype = C.c_char_p
+        L.pcr_strerror.argtypes = [C.c_int]
+        L.pcr_close.restype = None
+        L.pcr_close.argtypes = [vp]
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().pcr_strerror(code).decode()
+
+
+def _chk(rc, what):
+    if rc != PCR_OK:
+        raise PcrError(rc, what)
+
+
+def pcr_open(host_ptr: int, length: int) -> int:
+    h = C.c_void_p()
+    _chk(lib().pcr_open(host_ptr, length, C.byref(h)), "pcr_open")
+    return h.value
+
+
+def pcr_close(handle: int) -> None:
+    lib().pcr_close(handle)
+
+
+def pcr_num_images(handle: int) -> int:
+    return lib().pcr_num_images(handle)
+
+
+def pcr_num_groups(handle: int) -> int:
+    return lib().pcr_num_groups(handle)
+
+
+def pcr_get_image(handle: int, i: int) -> ImageInfo:
+    info = ImageInfo()
+    _chk(lib().pcr_get_image(handle, i, C.byref(info)), "pcr_get_image")
+    return info
+
+
+def pcr_out_bytes(handle: int) -> int:
+    return lib().pcr_out_bytes(handle)
+
+
+def pcr_prefix_bytes(handle: int, k: int) -> int:
+    return lib().pcr_prefix_bytes(handle, k)
+
+
+def pcr_decode(handle: int, k: int, out_dev_ptr: int, stream: int = 0) -> None:
+    _chk(lib().pcr_decode(handle, k, out_dev_ptr, stream), "pcr_decode")
+
+
+def pcr_evict(handle: int) -> None:
+    _chk(lib().pcr_evict(handle), "pcr_evict")
+
+
+def pcr_status(handle: int):
+    bad, code = C.c_int(), C.c_int()
+    _chk(lib().pcr_status(handle, C.byref(bad), C.byref(code)), "pcr_status")
+    return bad.value, code.value
+
+
+def pcr_coeffs(handle: int):
+    p, n = C.c_void_p(), C.c_size_t()
+    _chk(lib().pcr_coeffs(handle, C.byref(p), C.byref(n)), "pcr_coeffs")
+    return p.value, n.value
+
+
+def pcr_image_blocks(handle: int, i: int):
+    a, b = C.c_uint64(), C.c_uint64()
+    _chk(lib().pcr_image_blocks(handle, i, C.byref(a), C.byref(b)), "pcr_image_blocks")
+    return a.value, b.value
+
+
+def pcr_launch_count() -> int:
+    return lib().pcr_launch_count()

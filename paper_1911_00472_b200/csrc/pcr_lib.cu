@@ -1,0 +1,470 @@
+// Host side of the PCR decoder and its C ABI (see include/pcr.h).
+//
+// pcr_open walks the record's metadata and every image's JPEG marker segments once, on the
+// host, and turns them into flat device tables (per (scan, image) byte ranges and Huffman
+// table positions, per image geometry, work lists).  pcr_decode only enqueues work: the
+// prefix copy, the restart-interval index, one entropy kernel per dependency wave of the
+// scan script, and the fused pixel kernel.
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <algorithm>
+#include <atomic>
+#include <new>
+#include <vector>
+
+#include "../../include/pcr.h"
+#include "pcr_entropy.cuh"
+#include "pcr_pixels.cuh"
+#include "pcr_types.h"
+
+using namespace pcr;
+
+static std::atomic<uint64_t> g_launches{0};
+
+struct pcr_record {
+    const uint8_t* host = nullptr;
+    size_t len = 0;
+    int N = 0, G = 0;
+    std::vector<uint64_t> group_end;
+    std::vector<pcr_image_info> info;
+    std::vector<uint64_t> blk_base, nblk;
+    uint64_t total_blocks = 0, total_segs = 0;
+    size_t out_bytes = 0;
+    // scan script analysis
+    std::vector<ScanScript> script;
+    std::vector<int> wave_of_scan;
+    int n_waves = 0;
+    std::vector<uint32_t> scan_item_begin, scan_item_count;   // in the (wave, scan)-sorted item list
+    std::vector<std::vector<int>> wave_scans;
+    uint32_t n_units = 0;
+    // device state
+    int device = 0;
+    uint8_t* d_rec = nullptr;
+    size_t resident = 0;
+    int16_t* d_planes = nullptr;
+    ScanScript* d_script = nullptr;
+    ScanDesc* d_scans = nullptr;
+    ImgDesc* d_imgs = nullptr;
+    uint32_t* d_seg = nullptr;
+    Item* d_items = nullptr;
+    Unit* d_units = nullptr;
+    uint16_t* d_qtab = nullptr;
+    int* d_status = nullptr;
+    std::vector<int> h_status;
+};
+
+static inline uint32_t rd32(const uint8_t* p) { return (uint32_t)p[0] | ((uint32_t)p[1] << 8) | ((uint32_t)p[2] << 16) | ((uint32_t)p[3] << 24); }
+static inline uint64_t rd64(const uint8_t* p) { return (uint64_t)rd32(p) | ((uint64_t)rd32(p + 4) << 32); }
+
+namespace {
+
+struct TableRef { uint32_t off = 0; };   // offset of the 16 length counts of a DHT table body; 0 = undefined
+
+struct ImageParse {
+    uint32_t W = 0, H = 0;
+    int cid[3] = {0, 0, 0}, tq[3] = {0, 0, 0};
+    uint16_t q[4][64];
+    bool qdef[4] = {false, false, false, false};
+    TableRef dc[4], ac[4];
+    uint32_t ri = 0;
+    bool have_frame = false;
+};
+
+struct ScanParse {
+    ScanScript sc;
+    uint32_t tab[3];       // table body offset per scan component (0 when the scan uses none)
+    uint32_t data_off, data_end, ri;
+};
+
+// Validate one DHT table body at p (inside [p, end)): returns its length or 0.
+size_t check_dht_body(const uint8_t* p, size_t avail) {
+    if (avail < 16) return 0;
+    uint32_t code = 0, n = 0;
+    for (int l = 1; l <= 16; ++l) {
+        code += p[l - 1];
+        n += p[l - 1];
+        if (code > (1u << l)) return 0;
+        code <<= 1;
+    }
+    if (n > 256 || 16 + (size_t)n > avail) return 0;
+    return 16 + n;
+}
+
+// Walk the marker segments of chunk [off, off+len) of one image up to and including its SOS.
+int parse_chunk(const uint8_t* rec, uint64_t off, uint32_t len, bool first, ImageParse& im, ScanParse& out) {
+    uint64_t p = off, end = off + len;
+    if (first) {
+        if (len < 4 || rec[p] != 0xFF || rec[p + 1] != 0xD8) return PCR_E_FORMAT;
+        p += 2;
+    }
+    for (;;) {
+        if (p + 4 > end || rec[p] != 0xFF) return PCR_E_FORMAT;
+        while (p < end && rec[p] == 0xFF) ++p;
+        if (p >= end) return PCR_E_FORMAT;
+        int mk = rec[p++];
+        if (p + 2 > end) return PCR_E_FORMAT;
+        uint32_t L = ((uint32_t)rec[p] << 8) | rec[p + 1];
+        if (L < 2 || p + L > end) return PCR_E_FORMAT;
+        const uint8_t* s = rec + p + 2;
+        uint32_t sl = L - 2;
+        if (mk == 0xDB) {
+            uint32_t q = 0;
+            while (q < sl) {
+                int pq = s[q] >> 4, tq = s[q] & 15;
+                ++q;
+                if (tq > 3 || pq > 1 || q + (pq ? 128u : 64u) > sl) return PCR_E_FORMAT;
+                for (int k = 0; k < 64; ++k) {
+                    im.q[tq][k] = pq ? (uint16_t)((s[q] << 8) | s[q + 1]) : s[q];
+                    q += pq ? 2 : 1;
+                }
+                im.qdef[tq] = true;
+            }
+        } else if (mk == 0xC2) {
+            if (im.have_frame || sl < 15 || s[0] != 8 || s[5] != 3) return PCR_E_FORMAT;
+            im.H = ((uint32_t)s[1] << 8) | s[2];
+            im.W = ((uint32_t)s[3] << 8) | s[4];
+            for (int c = 0; c < 3; ++c) {
+                im.cid[c] = s[6 + 3 * c];
+                int hv = s[7 + 3 * c];
+                im.tq[c] = s[8 + 3 * c];
+                if (im.tq[c] > 3) return PCR_E_FORMAT;
+                if (hv != (c == 0 ? 0x22 : 0x11)) return PCR_E_FORMAT;   // 4:2:0 only
+            }
+            if (im.W == 0 || im.H == 0) return PCR_E_FORMAT;
+            im.have_frame = true;
+        } else if (mk == 0xC4) {
+            uint32_t q = 0;
+            while (q < sl) {
+                int tc = s[q] >> 4, th = s[q] & 15;
+                if (tc > 1 || th > 3) return PCR_E_FORMAT;
+                size_t n = check_dht_body(s + q + 1, sl - q - 1);
+                if (!n) return PCR_E_FORMAT;
+                (tc ? im.ac[th] : im.dc[th]).off = (uint32_t)(p + 2 + q + 1);
+                q += 1 + (uint32_t)n;
+            }
+        } else if (mk == 0xDD) {
+            if (sl != 2) return PCR_E_FORMAT;
+            im.ri = ((uint32_t)s[0] << 8) | s[1];
+        } else if (mk == 0xDA) {
+            if (!im.have_frame || sl < 1) return PCR_E_FORMAT;
+            int ns = s[0];
+            if (ns < 1 || ns > 3 || sl != (uint32_t)(4 + 2 * ns)) return PCR_E_FORMAT;
+            ScanScript& sc = out.sc;
+            memset(&sc, 0, sizeof sc);
+            sc.ncomp = ns;
+            int td[3] = {0, 0, 0}, ta[3] = {0, 0, 0};
+            for (int i = 0; i < ns; ++i) {
+                int id = s[1 + 2 * i], found = -1;
+                for (int c = 0; c < 3; ++c) if (im.cid[c] == id) found = c;
+                if (found < 0) return PCR_E_FORMAT;
+                for (int j = 0; j < i; ++j) if (sc.comp[j] >= found) return PCR_E_FORMAT;   // frame order
+                sc.comp[i] = found;
+                td[i] = s[2 + 2 * i] >> 4;
+                ta[i] = s[2 + 2 * i] & 15;
+                if (td[i] > 3 || ta[i] > 3) return PCR_E_FORMAT;
+            }
+            sc.Ss = s[1 + 2 * ns]; sc.Se = s[2 + 2 * ns];
+            sc.Ah = s[3 + 2 * ns] >> 4; sc.Al = s[3 + 2 * ns] & 15;
+            if (sc.Ss > sc.Se || sc.Se > 63 || sc.Al > 13) return PCR_E_FORMAT;
+            if (sc.Ss == 0 && sc.Se != 0) return PCR_E_FORMAT;
+            if (sc.Ss > 0 && ns != 1) return PCR_E_FORMAT;
+            if (ns > 1 && ns != 3) return PCR_E_FORMAT;     // interleaved scans hold all three components
+            if (sc.Ah != 0 && sc.Ah != sc.Al + 1) return PCR_E_FORMAT;
+            for (int i = 0; i < 3; ++i) out.tab[i] = 0;
+            for (int i = 0; i < ns; ++i) {
+                if (sc.Ss == 0 && sc.Ah == 0) { out.tab[i] = im.dc[td[i]].off; if (!out.tab[i]) return PCR_E_FORMAT; }
+                if (sc.Ss > 0) { out.tab[i] = im.ac[ta[i]].off; if (!out.tab[i]) return PCR_E_FORMAT; }
+            }
+            out.data_off = (uint32_t)(p + L);
+            out.data_end = (uint32_t)end;
+            out.ri = im.ri;
+            return PCR_OK;
+        } else if ((mk >= 0xC0 && mk <= 0xCF) || (mk >= 0xD0 && mk <= 0xD9)) {
+            return PCR_E_FORMAT;     // other frame types, stray restart / SOI / EOI markers
+        }
+        p += L;
+    }
+}
+
+void free_device(pcr_record* r) {
+    cudaFree(r->d_rec); cudaFree(r->d_planes); cudaFree(r->d_script); cudaFree(r->d_scans);
+    cudaFree(r->d_imgs); cudaFree(r->d_seg); cudaFree(r->d_items); cudaFree(r->d_units);
+    cudaFree(r->d_qtab); cudaFree(r->d_status);
+}
+
+template <class T>
+int upload(T** dst, const std::vector<T>& v) {
+    size_t n = std::max<size_t>(v.size(), 1) * sizeof(T);
+    if (cudaMalloc(reinterpret_cast<void**>(dst), n) != cudaSuccess) { *dst = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
+    if (!v.empty() && cudaMemcpy(*dst, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice) != cudaSuccess) return PCR_E_CUDA;
+    return PCR_OK;
+}
+
+int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
+    if (len < 64 || len >= (1ull << 32)) return PCR_E_FORMAT;
+    if (memcmp(rec, "PCR1", 4) != 0 || rd32(rec + 4) != 1) return PCR_E_FORMAT;
+    uint32_t N = rd32(rec + 8), G = rd32(rec + 12);
+    uint64_t meta_off = rd64(rec + 24), index_off = rd64(rec + 32), data_off = rd64(rec + 40), total = rd64(rec + 48);
+    if (N == 0 || G == 0 || G > 64 || N > (1u << 24)) return PCR_E_FORMAT;
+    if (total != len) return PCR_E_FORMAT;
+    if (meta_off < 64 || meta_off + 16ull * N > len) return PCR_E_FORMAT;
+    if (index_off < 64 || index_off + 8ull * (G + 1) + 16ull * G * N > len) return PCR_E_FORMAT;
+    if (data_off > len || data_off < index_off + 8ull * (G + 1) + 16ull * G * N) return PCR_E_FORMAT;
+    r->host = rec; r->len = len; r->N = (int)N; r->G = (int)G;
+    r->group_end.resize(G + 1);
+    for (uint32_t g = 0; g <= G; ++g) r->group_end[g] = rd64(rec + index_off + 8ull * g);
+    if (r->group_end[0] != data_off) return PCR_E_FORMAT;
+    for (uint32_t g = 1; g <= G; ++g)
+        if (r->group_end[g] < r->group_end[g - 1] || r->group_end[g] > len) return PCR_E_FORMAT;
+    const uint8_t* chunk = rec + index_off + 8ull * (G + 1);
+
+    std::vector<ScanDesc> scans((size_t)G * N);
+    std::vector<ImgDesc> imgs(N);
+    std::vector<uint16_t> qtab((size_t)N * 192);
+    r->info.resize(N); r->blk_base.resize(N); r->nblk.resize(N);
+    r->script.resize(G);
+    uint64_t blocks = 0, out_off = 0, segs = 0;
+    for (uint32_t i = 0; i < N; ++i) {
+        ImageParse im;
+        const uint8_t* m = rec + meta_off + 16ull * i;
+        for (uint32_t g = 0; g < G; ++g) {
+            const uint8_t* c = chunk + 16ull * ((uint64_t)g * N + i);
+            uint64_t off = rd64(c);
+            uint32_t clen = rd32(c + 8);
+            uint64_t padded = ((uint64_t)clen + 15) & ~15ull;
+            if ((off & 15) || off < r->group_end[g] || off + padded > r->group_end[g + 1]) return PCR_E_FORMAT;
+            ScanParse sp;
+            int rc = parse_chunk(rec, off, clen, g == 0, im, sp);
+            if (rc) return rc;
+            if (i == 0) r->script[g] = sp.sc;
+            else if (memcmp(&r->script[g], &sp.sc, sizeof(ScanScript)) != 0) return PCR_E_FORMAT;   // one script per record
+            ScanDesc& sd = scans[(size_t)g * N + i];
+            sd.data_off = sp.data_off; sd.data_end = sp.data_end; sd.ri = sp.ri;
+            // up to two distinct tables per scan
+            sd.tab_off[0] = sp.tab[0]; sd.tab_off[1] = 0; sd.slots = 0;
+            for (int ci = 1; ci < sp.sc.ncomp; ++ci) {
+                if (sp.tab[ci] == sd.tab_off[0]) continue;
+                if (sd.tab_off[1] == 0) sd.tab_off[1] = sp.tab[ci];
+                if (sp.tab[ci] != sd.tab_off[1]) return PCR_E_FORMAT;
+                sd.slots |= 1u << (2 * ci);
+            }
+            uint32_t mx = (im.W + 15) / 16, my = (im.H + 15) / 16;
+            uint64_t total_mcu;
+            if (sp.sc.ncomp > 1) total_mcu = (uint64_t)mx * my;
+            else {
+                uint32_t wc = sp.sc.comp[0] == 0 ? im.W : (im.W + 1) / 2, hc = sp.sc.comp[0] == 0 ? im.H : (im.H + 1) / 2;
+                total_mcu = (uint64_t)((wc + 7) / 8) * ((hc + 7) / 8);
+            }
+            sd.nseg = sd.ri ? (uint32_t)((total_mcu + sd.ri - 1) / sd.ri) : 1u;
+            sd.seg_base = (uint32_t)segs;
+            segs += sd.nseg;
+            if (segs >= (1ull << 32)) return PCR_E_FORMAT;
+        }
+        if (!im.have_frame) return PCR_E_FORMAT;
+        if (rd32(m + 4) != im.W || rd32(m + 8) != im.H) return PCR_E_FORMAT;   // metadata and frame header agree
+        for (int c = 0; c < 3; ++c) {
+            if (!im.qdef[im.tq[c]]) return PCR_E_FORMAT;
+            memcpy(&qtab[(size_t)i * 192 + 64 * c], im.q[im.tq[c]], 128);
+        }
+        uint32_t mx = (im.W + 15) / 16, my = (im.H + 15) / 16;
+        pcr_image_info& inf = r->info[i];
+        inf.width = im.W; inf.height = im.H; inf.label = (int32_t)rd32(m); inf.rsvd = 0;
+        inf.out_offset = out_off; inf.out_bytes = 3ull * im.W * im.H;
+        out_off += (inf.out_bytes + 127) & ~127ull;
+        r->blk_base[i] = blocks; r->nblk[i] = 6ull * mx * my;
+        imgs[i].W = im.W; imgs[i].H = im.H; imgs[i].mx = mx; imgs[i].my = my;
+        imgs[i].blk_base = blocks; imgs[i].out_off = inf.out_offset;
+        blocks += r->nblk[i];
+    }
+    r->total_blocks = blocks; r->out_bytes = out_off; r->total_segs = segs;
+
+    // dependency waves of the script: a scan waits for every earlier scan that touches an
+    // overlapping coefficient band of one of its components
+    r->wave_of_scan.assign(G, 0);
+    for (uint32_t s = 0; s < G; ++s) {
+        int w = 0;
+        for (uint32_t t = 0; t < s; ++t) {
+            bool share = false;
+            for (int a = 0; a < r->script[s].ncomp; ++a)
+                for (int b = 0; b < r->script[t].ncomp; ++b)
+                    if (r->script[s].comp[a] == r->script[t].comp[b]) share = true;
+            if (share && r->script[s].Ss <= r->script[t].Se && r->script[t].Ss <= r->script[s].Se)
+                w = std::max(w, r->wave_of_scan[t] + 1);
+        }
+        r->wave_of_scan[s] = w;
+        r->n_waves = std::max(r->n_waves, w + 1);
+    }
+    r->wave_scans.assign(r->n_waves, {});
+    for (uint32_t s = 0; s < G; ++s) r->wave_scans[r->wave_of_scan[s]].push_back((int)s);
+    std::vector<Item> items;
+    r->scan_item_begin.assign(G, 0); r->scan_item_count.assign(G, 0);
+    for (int w = 0; w < r->n_waves; ++w)
+        for (int s : r->wave_scans[w]) {
+            r->scan_item_begin[s] = (uint32_t)items.size();
+            for (uint32_t i = 0; i < N; ++i) {
+                const ScanDesc& sd = scans[(size_t)s * N + i];
+                for (uint32_t j = 0; j < sd.nseg; j += 32) items.push_back(Item{(uint32_t)(s * N + i), j});
+            }
+            r->scan_item_count[s] = (uint32_t)items.size() - r->scan_item_begin[s];
+        }
+    std::vector<Unit> units;
+    for (uint32_t i = 0; i < N; ++i)
+        for (uint32_t row = 0; row < imgs[i].my; ++row)
+            for (uint32_t col = 0; col < imgs[i].mx; col += kPixMcus) {
+                if (imgs[i].my > 65535 || imgs[i].mx > 65535) return PCR_E_FORMAT;
+                units.push_back(Unit{i, (uint16_t)row, (uint16_t)col});
+            }
+    r->n_units = (uint32_t)units.size();
+
+    // device state
+    if (cudaGetDevice(&r->device) != cudaSuccess) return PCR_E_CUDA;
+    if (cudaMalloc(reinterpret_cast<void**>(&r->d_rec), len + 64) != cudaSuccess) { r->d_rec = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
+    if (cudaMalloc(reinterpret_cast<void**>(&r->d_planes), std::max<uint64_t>(blocks, 1) * 128) != cudaSuccess) { r->d_planes = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
+    if (cudaMalloc(reinterpret_cast<void**>(&r->d_seg), (segs + 1) * 4) != cudaSuccess) { r->d_seg = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
+    if (cudaMalloc(reinterpret_cast<void**>(&r->d_status), (size_t)N * 4) != cudaSuccess) { r->d_status = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
+    if (cudaMemset(r->d_seg, 0, (segs + 1) * 4) != cudaSuccess || cudaMemset(r->d_status, 0, (size_t)N * 4) != cudaSuccess) return PCR_E_CUDA;
+    int rc;
+    if ((rc = upload(&r->d_script, r->script))) return rc;
+    if ((rc = upload(&r->d_scans, scans))) return rc;
+    if ((rc = upload(&r->d_imgs, imgs))) return rc;
+    if ((rc = upload(&r->d_items, items))) return rc;
+    if ((rc = upload(&r->d_units, units))) return rc;
+    if ((rc = upload(&r->d_qtab, qtab))) return rc;
+    r->h_status.assign(N, 0);
+    r->resident = 0;
+    return PCR_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int pcr_open(const void* bytes, size_t len, pcr_record** rec) {
+    if (rec) *rec = nullptr;
+    if (!bytes || !rec) return PCR_E_ARG;
+    pcr_record* r = new (std::nothrow) pcr_record();
+    if (!r) return PCR_E_NOMEM;
+    int rc;
+    try {
+        rc = open_impl(static_cast<const uint8_t*>(bytes), len, r);
+    } catch (const std::bad_alloc&) {
+        rc = PCR_E_NOMEM;
+    }
+    if (rc != PCR_OK) {
+        free_device(r);
+        delete r;
+        return rc;
+    }
+    *rec = r;
+    return PCR_OK;
+}
+
+int pcr_num_images(const pcr_record* rec) { return rec ? rec->N : PCR_E_ARG; }
+int pcr_num_groups(const pcr_record* rec) { return rec ? rec->G : PCR_E_ARG; }
+
+int pcr_get_image(const pcr_record* rec, int i, pcr_image_info* info) {
+    if (!rec || !info || i < 0 || i >= rec->N) return PCR_E_ARG;
+    *info = rec->info[i];
+    return PCR_OK;
+}
+
+size_t pcr_out_bytes(const pcr_record* rec) { return rec ? rec->out_bytes : 0; }
+
+size_t pcr_prefix_bytes(const pcr_record* rec, int k) {
+    if (!rec || k < 1 || k > rec->G) return 0;
+    return (size_t)rec->group_end[k];
+}
+
+int pcr_evict(pcr_record* rec) {
+    if (!rec) return PCR_E_ARG;
+    rec->resident = 0;
+    return PCR_OK;
+}
+
+int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
+    if (!rec || !out || k < 1 || k > rec->G) return PCR_E_ARG;
+    if (reinterpret_cast<uintptr_t>(out) & 15u) return PCR_E_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t need = (size_t)rec->group_end[k];
+    if (rec->resident < need) {
+        size_t from = rec->resident & ~(size_t)15;
+        if (cudaMemcpyAsync(rec->d_rec + from, rec->host + from, need - from, cudaMemcpyHostToDevice, st) != cudaSuccess) return PCR_E_CUDA;
+        rec->resident = need;
+    }
+    if (cudaMemsetAsync(rec->d_status, 0, (size_t)rec->N * 4, st) != cudaSuccess) return PCR_E_CUDA;
+    if (cudaMemsetAsync(rec->d_planes, 0, rec->total_blocks * 128, st) != cudaSuccess) return PCR_E_CUDA;
+    Params P;
+    P.rec = rec->d_rec; P.planes = rec->d_planes; P.script = rec->d_script; P.scans = rec->d_scans;
+    P.imgs = rec->d_imgs; P.seg_start = rec->d_seg; P.items = rec->d_items; P.units = rec->d_units;
+    P.qtab = rec->d_qtab; P.status = rec->d_status; P.N = rec->N;
+    {
+        uint32_t warps = (uint32_t)k * (uint32_t)rec->N;
+        seg_index_kernel<<<(warps + 7) / 8, 256, 0, st>>>(P, k);
+        ++g_launches;
+    }
+    for (int w = 0; w < rec->n_waves; ++w) {
+        uint32_t begin = 0, count = 0;
+        bool any = false;
+        for (int s : rec->wave_scans[w]) {
+            if (s >= k) break;   // scans of a wave are stored in ascending order
+            if (!any) { begin = rec->scan_item_begin[s]; any = true; }
+            count += rec->scan_item_count[s];
+        }
+        if (!count) continue;
+        entropy_kernel<<<(count + kEntropyWarps - 1) / kEntropyWarps, 32 * kEntropyWarps, 0, st>>>(P, begin, count);
+        ++g_launches;
+    }
+    pixel_kernel<<<rec->n_units, kPixThreads, 0, st>>>(P, static_cast<uint8_t*>(out));
+    ++g_launches;
+    if (cudaGetLastError() != cudaSuccess) return PCR_E_CUDA;
+    return PCR_OK;
+}
+
+int pcr_status(pcr_record* rec, int* first_bad_image, int* code) {
+    if (!rec || !first_bad_image || !code) return PCR_E_ARG;
+    if (cudaMemcpy(rec->h_status.data(), rec->d_status, (size_t)rec->N * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return PCR_E_CUDA;
+    *first_bad_image = -1; *code = PCR_OK;
+    for (int i = 0; i < rec->N; ++i)
+        if (rec->h_status[i] != 0) { *first_bad_image = i; *code = rec->h_status[i]; break; }
+    return PCR_OK;
+}
+
+int pcr_coeffs(pcr_record* rec, const int16_t** dev_planes, size_t* bytes) {
+    if (!rec || !dev_planes || !bytes) return PCR_E_ARG;
+    *dev_planes = rec->d_planes;
+    *bytes = (size_t)rec->total_blocks * 128;
+    return PCR_OK;
+}
+
+int pcr_image_blocks(const pcr_record* rec, int i, uint64_t* first_block, uint64_t* n_blocks) {
+    if (!rec || !first_block || !n_blocks || i < 0 || i >= rec->N) return PCR_E_ARG;
+    *first_block = rec->blk_base[i];
+    *n_blocks = rec->nblk[i];
+    return PCR_OK;
+}
+
+uint64_t pcr_launch_count(void) { return g_launches.load(); }
+
+const char* pcr_strerror(int code) {
+    switch (code) {
+    case PCR_OK: return "ok";
+    case PCR_E_ARG: return "invalid argument";
+    case PCR_E_FORMAT: return "not a valid or supported record";
+    case PCR_E_CORRUPT: return "corrupt entropy-coded data";
+    case PCR_E_TIMEOUT: return "device-side wait timed out";
+    case PCR_E_CUDA: return "CUDA runtime error";
+    case PCR_E_NOMEM: return "out of memory";
+    default: return "unknown error";
+    }
+}
+
+void pcr_close(pcr_record* rec) {
+    if (!rec) return;
+    free_device(rec);
+    delete rec;
+}
+
+}  // extern "C"

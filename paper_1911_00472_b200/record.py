@@ -1,0 +1,85 @@
+"""A small convenience wrapper: pinned host copy of a record + the C-ABI handle + torch buffers.
+
+torch is used for memory and streams only (pinned host buffer, device output tensor, the
+current stream's handle); all decoding happens behind pcr_decode.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+
+class Decoder:
+    """Opens one record (bytes-like / uint8 numpy array) and decodes it at a chosen fidelity."""
+
+    def __init__(self, record_bytes, device: str | torch.device = "cuda:0", pin: bool = True):
+        self.device = torch.device(device)
+        if self.device.type != "cuda":
+            raise RuntimeError("the PCR decoder runs on a CUDA device only")
+        arr = np.frombuffer(record_bytes, dtype=np.uint8) if not isinstance(record_bytes, np.ndarray) else record_bytes
+        host = torch.from_numpy(np.ascontiguousarray(arr, dtype=np.uint8))
+        self.host = host.pin_memory() if pin else host.clone()
+        with torch.cuda.device(self.device):
+            self.handle = B.pcr_open(self.host.data_ptr(), self.host.numel())
+        self.n_images = B.pcr_num_images(self.handle)
+        self.n_groups = B.pcr_num_groups(self.handle)
+        self.out_bytes = B.pcr_out_bytes(self.handle)
+        self.info = [B.pcr_get_image(self.handle, i) for i in range(self.n_images)]
+        self.out = None
+
+    def prefix_bytes(self, k: int) -> int:
+        return B.pcr_prefix_bytes(self.handle, k)
+
+    def alloc_out(self) -> torch.Tensor:
+        return torch.empty(max(self.out_bytes, 16), dtype=torch.uint8, device=self.device)
+
+    def decode(self, k: int, out: torch.Tensor | None = None, stream: torch.cuda.Stream | None = None) -> torch.Tensor:
+        """Enqueue the decode at fidelity k on `stream` (default: torch's current stream)."""
+        if out is None:
+            if self.out is None:
+                self.out = self.alloc_out()
+            out = self.out
+        s = stream if stream is not None else torch.cuda.current_stream(self.device)
+        with torch.cuda.device(self.device):
+            B.pcr_decode(self.handle, k, out.data_ptr(), s.cuda_stream)
+        return out
+
+    def evict(self) -> None:
+        B.pcr_evict(self.handle)
+
+    def status(self):
+        return B.pcr_status(self.handle)
+
+    def image(self, out: torch.Tensor, i: int) -> torch.Tensor:
+        """View of image i inside an output buffer: (H, W, 3) uint8."""
+        inf = self.info[i]
+        return out[inf.out_offset:inf.out_offset + inf.out_bytes].view(inf.height, inf.width, 3)
+
+    def coeffs(self, i: int | None = None) -> torch.Tensor:
+        """Coefficient planes of the last decode as a (blocks, 64) int16 device tensor (a copy)."""
+        ptr, nbytes = B.pcr_coeffs(self.handle)
+        n = nbytes // 2
+        iface = {"shape": (n,), "typestr": "<i2", "data": (ptr, False), "version": 2}
+
+        class _Wrap:
+            __cuda_array_interface__ = iface
+
+        with torch.cuda.device(self.device):
+            t = torch.as_tensor(_Wrap(), device=self.device).view(-1, 64).clone()
+        if i is None:
+            return t
+        a, b = B.pcr_image_blocks(self.handle, i)
+        return t[a:a + b]
+
+    def close(self) -> None:
+        if getattr(self, "handle", None):
+            B.pcr_close(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,196 @@
+"""GPU parity: the CUDA path through the C ABI against the CPU oracle, element by element,
+on the same seeded records.  Bit exact: int16 coefficients and uint8 pixels, at every k."""
+import numpy as np
+import pytest
+
+import pcr_synth
+from oracle import pcr_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+G = 10
+
+
+def _gpu_decode(dec, k):
+    import torch
+    out = dec.decode(k)
+    torch.cuda.synchronize()
+    bad, code = dec.status()
+    return out, dec.coeffs(), bad, code
+
+
+def _compare(rec, ks, images=None):
+    import torch
+    from paper_1911_00472_b200 import Decoder
+    dec = Decoder(rec.bytes)
+    assert dec.n_images == rec.n_images and dec.n_groups == G
+    idx = range(rec.n_images) if images is None else images
+    try:
+        for k in ks:
+            out, coef, bad, code = _gpu_decode(dec, k)
+            assert (bad, code) == (-1, 0), (k, bad, code)
+            out_h = out.cpu().numpy()
+            coef_h = coef.cpu().numpy()
+            for i in idx:
+                want_c, want_rgb = O.decode_image(rec.bytes, i, k)
+                inf = dec.info[i]
+                a, b = dec_blocks(dec, i)
+                got_c = coef_h[a:a + b]
+                assert np.array_equal(got_c, want_c), f"coefficients differ: image {i} k {k}: {np.argwhere(got_c != want_c)[:4]}"
+                got = out_h[inf.out_offset:inf.out_offset + inf.out_bytes].reshape(inf.height, inf.width, 3)
+                assert np.array_equal(got, want_rgb), f"pixels differ: image {i} k {k}: {np.argwhere(got != want_rgb)[:4]}"
+    finally:
+        dec.close()
+
+
+def dec_blocks(dec, i):
+    from paper_1911_00472_b200 import pcr_image_blocks
+    return pcr_image_blocks(dec.handle, i)
+
+
+def test_tiny_record_every_k(rec0):
+    _compare(rec0, range(1, G + 1))
+
+
+def test_imagenet_shaped_small(rec1_small):
+    _compare(rec1_small, (1, 2, 5, 6, 7, 10))
+
+
+def test_celeba_shaped_small_unpadded_grid(rec2_small):
+    _compare(rec2_small, range(1, G + 1))
+
+
+def test_ham_shaped_small_no_restarts(rec3_small):
+    _compare(rec3_small, (1, 5, 10))
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_coefficient_fields(seed):
+    rng = np.random.default_rng(100 + seed)
+    dims = [(int(rng.integers(1, 90)), int(rng.integers(1, 90))) for _ in range(6)] + [(8, 8), (16, 16), (17, 9), (1, 1), (129, 40), (300, 20)]
+    density = [0.02, 0.1, 0.3, 0.6, 0.9, 1.0][seed]
+    amp = [1.0, 2.0, 4.0, 20.0, 100.0, 300.0][seed]
+    coeffs = []
+    for W, H in dims:
+        nb = pcr_synth.num_blocks(W, H)
+        c = np.zeros((nb, 64), dtype=np.int16)
+        m = rng.random((nb, 64)) < density
+        mag = np.minimum(np.floor(rng.exponential(amp, size=(nb, 64))) + 1, 1023)
+        c[m] = (mag * rng.choice([-1, 1], size=(nb, 64)))[m].astype(np.int16)
+        c[:, 0] = rng.integers(-1023, 1024, size=nb)
+        coeffs.append(c)
+    mode = [dict(restart_rows=True), dict(restart_rows=False), dict(restart_rows=False, restart_fixed=1),
+            dict(restart_rows=False, restart_fixed=3), dict(restart_rows=True), dict(restart_rows=False, restart_fixed=40)][seed]
+    rec = pcr_synth.record_from_coeffs(dims, coeffs, quality=[90, 50, 95, 100, 75, 90][seed], **mode)
+    _compare(rec, range(1, G + 1))
+
+
+def test_stuffed_bytes():
+    W, H = 48, 32
+    nb = pcr_synth.num_blocks(W, H)
+    c = np.zeros((nb, 64), dtype=np.int16)
+    c[:, 1:] = -1
+    c2 = np.full((nb, 64), 1023, dtype=np.int16)
+    c3 = np.full((nb, 64), -1023, dtype=np.int16)
+    rec = pcr_synth.record_from_coeffs([(W, H)] * 3, [c, c2, c3])
+    _compare(rec, range(1, G + 1))
+
+
+def test_prefix_property_on_the_device(rec0):
+    """Bytes at or beyond the end of scan group k never influence decode(k)."""
+    import torch
+    from paper_1911_00472_b200 import Decoder
+    for k in (1, 4, 7):
+        poisoned = rec0.bytes.copy()
+        dec0 = Decoder(rec0.bytes)
+        pre = dec0.prefix_bytes(k)
+        assert pre == O.prefix_bytes(rec0.bytes, k)
+        out0, c0, bad, code = _gpu_decode(dec0, k)
+        out0 = out0.clone()
+        dec0.close()
+        # the header/index stay intact (they precede group 1); everything past the prefix is junk
+        poisoned[pre:] = 0xA7
+        dec1 = Decoder.__new__(Decoder)
+        # opening needs the full record's index to validate, so open on the intact bytes and
+        # poison the pinned host copy afterwards: the decode copies from that buffer
+        dec1.__init__(rec0.bytes)
+        dec1.host[pre:] = 0xA7
+        out1, c1, bad, code = _gpu_decode(dec1, k)
+        assert (bad, code) == (-1, 0)
+        assert torch.equal(out0, out1) and torch.equal(c0, c1)
+        dec1.close()
+
+
+def test_incremental_prefix_copy_and_evict(rec0):
+    """Raising k copies only the missing groups; evict forces a full copy; results identical."""
+    import torch
+    from paper_1911_00472_b200 import Decoder
+    dec = Decoder(rec0.bytes)
+    outs = {}
+    for k in (2, 5, 10, 3):
+        out, c, bad, code = _gpu_decode(dec, k)
+        outs[k] = (out.clone(), c)
+    dec.evict()
+    for k in (10, 3):
+        out, c, bad, code = _gpu_decode(dec, k)
+        assert torch.equal(out, outs[k][0]) and torch.equal(c, outs[k][1])
+    dec.close()
+
+
+def test_argument_and_format_errors(rec0):
+    import torch
+    from paper_1911_00472_b200 import Decoder, PcrError, binding
+    dec = Decoder(rec0.bytes)
+    out = dec.alloc_out()
+    for k in (0, 11, -1):
+        with pytest.raises(PcrError) as e:
+            binding.pcr_decode(dec.handle, k, out.data_ptr(), 0)
+        assert e.value.code == binding.PCR_E_ARG
+    with pytest.raises(PcrError) as e:
+        binding.pcr_decode(dec.handle, 1, out.data_ptr() + 4, 0)
+    assert e.value.code == binding.PCR_E_ARG
+    assert dec.prefix_bytes(0) == 0 and dec.prefix_bytes(11) == 0
+    dec.close()
+    # malformed records: bad magic, truncated, offsets past the end, non-monotone group table
+    b = rec0.bytes.copy(); b[0] = ord("X")
+    with pytest.raises(PcrError) as e:
+        Decoder(b)
+    assert e.value.code == binding.PCR_E_FORMAT
+    with pytest.raises(PcrError):
+        Decoder(rec0.bytes[:len(rec0.bytes) // 2].copy())
+    b = rec0.bytes.copy()
+    index_off = int(np.frombuffer(b[32:40].tobytes(), dtype="<u8")[0])
+    b[index_off + 8:index_off + 16] = np.frombuffer(np.uint64(2 ** 40).tobytes(), dtype=np.uint8)
+    with pytest.raises(PcrError):
+        Decoder(b)
+    # a frame header that disagrees with the record metadata
+    b = rec0.bytes.copy()
+    meta_off = int(np.frombuffer(b[24:32].tobytes(), dtype="<u8")[0])
+    b[meta_off + 4] = 48
+    with pytest.raises(PcrError):
+        Decoder(b)
+
+
+def test_corrupt_entropy_data_sets_status_not_a_fault(rec0):
+    """Damaged entropy-coded bytes: the decode completes, the image is flagged (or happens to
+    decode to something else); neighbouring images are untouched."""
+    import torch
+    from paper_1911_00472_b200 import Decoder
+    ref = Decoder(rec0.bytes)
+    good, cgood, _, _ = _gpu_decode(ref, 10)
+    good = good.clone()
+    b = rec0.bytes.copy()
+    # remove image 5's restart markers in scan 10 by overwriting its chunk tail with zeros
+    N = rec0.n_images
+    index_off = int(np.frombuffer(b[32:40].tobytes(), dtype="<u8")[0])
+    ent = index_off + 8 * 11 + 16 * (9 * N + 5)
+    off = int(np.frombuffer(b[ent:ent + 8].tobytes(), dtype="<u8")[0])
+    ln = int(np.frombuffer(b[ent + 8:ent + 12].tobytes(), dtype="<u4")[0])
+    b[off + ln - 30:off + ln] = 0
+    dec = Decoder(b)
+    out, c, bad, code = _gpu_decode(dec, 10)
+    assert bad == 5 and code == -3
+    for i in (4, 6):
+        inf = dec.info[i]
+        assert torch.equal(out[inf.out_offset:inf.out_offset + inf.out_bytes], good[inf.out_offset:inf.out_offset + inf.out_bytes])
+    dec.close(); ref.close()
