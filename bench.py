@@ -1,0 +1,419 @@
+#!/usr/bin/env python
+"""Benchmark of the PCR decode path: decoded images/s at scan group k on B200.
+
+One step = one pcr_decode of one synthetic ImageNet-shaped record (1024 images, sizes
+256..496, quality 90, 4:2:0, ten scans, restart every MCU row) at fidelity k: restart-interval
+index, Huffman decode of scans 1..k into int16 coefficient planes, refinement in place,
+dequantise / inverse DCT / upsample / colour convert to packed RGB.  `value` is measured with the
+record already resident in device memory; `e2e` copies the record prefix from pinned host
+memory inside every step and reads the status words back.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--k 10] [--impl ours|reference]
+
+With N > 1 (launched by torchrun, one rank per GPU) every rank decodes its own record of the
+same distribution: independent units, no collective on the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decoded images/sec at scan group k"
+UNIT = "images/s"
+WORKLOAD = 1                 # ImageNet-shaped record
+WORKLOAD_DESC = ("imagenet_shaped: 1 record x 1024 images per GPU, W,H in {256..496 step 16}, q90, 4:2:0, "
+                 "10-scan script, restart per MCU row")
+FALLBACK_HBM_GBS = 6650.0
+
+
+# ----------------------------------------------------------------------------------------
+# pieces shared by every rank (kept importable: the CPU tests exercise them over gloo)
+# ----------------------------------------------------------------------------------------
+def rank_record_index(rank: int) -> int:
+    """Rank r decodes record r of the workload's distribution (weak scaling, no exchange)."""
+    return rank
+
+
+def _reduce(value: float, world_size: int, op_name: str) -> float:
+    if world_size <= 1:
+        return value
+    import torch
+    import torch.distributed as dist
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([value], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=getattr(dist.ReduceOp, op_name))
+    return float(t.item())
+
+
+def reduce_max(value: float, world_size: int) -> float:
+    """Max over ranks of a host-side scalar (the timed region)."""
+    return _reduce(value, world_size, "MAX")
+
+
+def reduce_sum(value: float, world_size: int) -> float:
+    return _reduce(value, world_size, "SUM")
+
+
+def whole_job_rate(images_this_rank: int, steps: int, ms_this_rank: float, world_size: int) -> float:
+    """Images of all ranks / slowest rank's time."""
+    total = reduce_sum(float(images_this_rank), world_size)
+    ms = reduce_max(ms_this_rank, world_size)
+    return total * steps / (ms / 1000.0)
+
+
+def algorithmic_bytes(scans, infos, k: int):
+    """Bytes the method has to move for one decode at fidelity k, per stage.
+
+    scans: [(ncomp, comp0, Ss, Se, Ah, wave, group_bytes)], infos: [(W, H)].
+      index    : bytes of scan groups <= k, read once
+      entropyW : compressed bytes of the wave's scans + 2 bytes per coefficient of every
+                 block the scan visits (written once by a first pass, read and written by a
+                 refinement)
+      clear    : 128 bytes per block
+      pixels   : 128 bytes per block read + 3 bytes per pixel written
+    """
+    out = {"index": 0.0, "clear": 0.0, "pixels": 0.0}
+    blocks_pad = 0
+    blocks_unp = [0, 0, 0]
+    px = 0
+    for W, H in infos:
+        mx, my = (W + 15) // 16, (H + 15) // 16
+        blocks_pad += 6 * mx * my
+        cw, ch = (W + 1) // 2, (H + 1) // 2
+        blocks_unp[0] += ((W + 7) // 8) * ((H + 7) // 8)
+        blocks_unp[1] += ((cw + 7) // 8) * ((ch + 7) // 8)
+        blocks_unp[2] += ((cw + 7) // 8) * ((ch + 7) // 8)
+        px += W * H
+    out["clear"] = 128.0 * blocks_pad
+    out["pixels"] = 128.0 * blocks_pad + 3.0 * px
+    for s, (ncomp, comp0, Ss, Se, Ah, wave, gbytes) in enumerate(scans):
+        if s >= k:
+            break
+        out["index"] += gbytes
+        band = Se - Ss + 1
+        nb = blocks_pad if ncomp > 1 else blocks_unp[comp0]
+        coef = 2.0 * band * nb * (2 if Ah else 1)
+        key = f"entropy{wave}"
+        out[key] = out.get(key, 0.0) + gbytes + coef
+    out["total"] = sum(out.values())
+    return out
+
+
+class ClockSampler:
+    """SM clock and throttle-reason samples (NVML, read-only queries) taken by a thread while
+    the timed region runs."""
+
+    def __init__(self, gpu_index: int, period_s: float = 0.005):
+        self.rows = []
+        self.ok = False
+        self._stop = threading.Event()
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            phys = gpu_index
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            if vis:
+                ids = [v.strip() for v in vis.split(",") if v.strip()]
+                if gpu_index < len(ids) and ids[gpu_index].isdigit():
+                    phys = int(ids[gpu_index])
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.sm_max = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.period = period_s
+            self.ok = True
+            self.t = threading.Thread(target=self._run, daemon=True)
+            self.t.start()
+        except Exception as e:   # no NVML: report that, never guess
+            self.err = repr(e)
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                sm = float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    rs = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    rs = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                try:
+                    pw = nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0
+                except Exception:
+                    pw = 0.0
+                self.rows.append((time.perf_counter(), sm, rs, pw))
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def stop(self, t0: float, t1: float):
+        if not self.ok:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["NVML unavailable: " + getattr(self, "err", "")]}
+        self._stop.set()
+        self.t.join(timeout=2)
+        rows = [r for r in self.rows if t0 <= r[0] <= t1]
+        where = "timed region"
+        if not rows:
+            rows, where = self.rows, "whole run (timed region shorter than one sample)"
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": ["no samples"]}
+        bits = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
+        reasons = [n for n, b in bits.items() if any(r[2] & b for r in rows)]
+        return {"sm_mhz": statistics.median(r[1] for r in rows), "sm_max_mhz": self.sm_max,
+                "power_w_max": max(r[3] for r in rows), "samples": len(rows), "window": where, "reasons": reasons}
+
+
+# ----------------------------------------------------------------------------------------
+# CPU oracle timing (the reported baseline, and the --impl reference arm)
+# ----------------------------------------------------------------------------------------
+def _oracle_worker(args):
+    path, k, lo, hi = args
+    import numpy as np
+    from oracle import pcr_oracle as O
+    rec = np.load(path)
+    for i in range(lo, hi):
+        O.decode_image(rec, i, k, True)
+    return hi - lo
+
+
+def time_oracle(pool, cores: int, rec_path: str, k: int, n_images: int, passes: int = 1) -> float:
+    """Images/s of the oracle decoding images [0, n_images) on `cores` processes."""
+    per = max(1, (n_images + cores * 4 - 1) // (cores * 4))
+    shards = [(rec_path, k, lo, min(lo + per, n_images)) for lo in range(0, n_images, per)]
+    t0 = time.perf_counter()
+    done = 0
+    for _ in range(passes):
+        done += sum(pool.map(_oracle_worker, shards))
+    return done / (time.perf_counter() - t0)
+
+
+def run_reference(args, rank: int):
+    """The CPU oracle, as it stands, on this machine's host cores: same metric, config and unit."""
+    if rank != 0:
+        return
+    import multiprocessing as mp
+    import tempfile
+    import numpy as np
+    import pcr_synth
+    from oracle import pcr_oracle as O
+    O.build()
+    cores = len(os.sched_getaffinity(0))
+    rec = pcr_synth.make_record(WORKLOAD, 0)
+    sample = min(rec.n_images, 256)
+    with tempfile.TemporaryDirectory() as td:
+        path = os.path.join(td, "rec.npy")
+        np.save(path, rec.bytes)
+        with mp.get_context("spawn").Pool(cores) as pool:
+            for _ in range(max(args.warmup, 1)):
+                time_oracle(pool, cores, path, args.k, min(sample, 64))
+            t0 = time.perf_counter()
+            for _ in range(args.steps):
+                time_oracle(pool, cores, path, args.k, sample)
+            dt = time.perf_counter() - t0
+    value = sample * args.steps / dt
+    desc = f"first {sample} images of the record per step, decoded by the single-threaded oracle in {cores} processes"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1000.0 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int16/u8", "data": "synthetic",
+        "config": {"workload": WORKLOAD_DESC, "k": args.k},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ----------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--k", type=int, default=10, help="scan group (fidelity) of the headline number")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--images", type=int, default=0, help="images per record (default: the workload's 1024)")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    args.warmup = max(args.warmup, 3)
+
+    import multiprocessing as mp
+    import tempfile
+    import numpy as np
+    import pcr_synth
+
+    # input record of this rank; the oracle's process pool starts before the first GPU call
+    rec = pcr_synth.make_record(WORKLOAD, rank_record_index(rank), n_images=args.images or None)
+    pool = None
+    tmpdir = None
+    cores = len(os.sched_getaffinity(0))
+    do_cpu = (rank == 0 and world == 1 and not args.no_cpu_baseline)
+    if do_cpu:
+        from oracle import pcr_oracle as O
+        O.build()
+        tmpdir = tempfile.TemporaryDirectory()
+        rec_path = os.path.join(tmpdir.name, "rec.npy")
+        np.save(rec_path, rec.bytes)
+        pool = mp.get_context("spawn").Pool(cores)
+        time_oracle(pool, cores, rec_path, 1, min(64, rec.n_images))   # start the workers
+
+    import torch
+    import torch.distributed as dist
+    from paper_1911_00472_b200 import Decoder, binding
+    from paper_1911_00472_b200 import build as libbuild
+    libbuild.build()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    dec = Decoder(rec.bytes, device=dev)
+    out = dec.alloc_out()
+    stream = torch.cuda.current_stream(dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)     # > 126 MB L2
+    k = args.k
+    n_img = dec.n_images
+    scans = []
+    for s in range(dec.n_groups):
+        si = binding.pcr_get_scan(dec.handle, s)
+        scans.append((si.ncomp, si.comp[0], si.Ss, si.Se, si.Ah, si.wave, si.bytes))
+    infos = [(i.width, i.height) for i in dec.info]
+
+    def sync_all():
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize(dev)
+
+    def timed_steps(kk, steps):
+        """Sum of per-step device times (ms): L2 flushed before every step, events on the launch stream."""
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for a, b in evs:
+            flush.fill_(1)
+            a.record(stream)
+            dec.decode(kk, out)
+            b.record(stream)
+        torch.cuda.synchronize(dev)
+        return sum(a.elapsed_time(b) for a, b in evs)
+
+    dec.decode(k, out)
+    torch.cuda.synchronize(dev)
+    bad, code = dec.status()
+    if code != 0:
+        raise RuntimeError(f"decode reported error {code} on image {bad}")
+
+    sampler = ClockSampler(local_rank)
+    for _ in range(args.warmup):
+        dec.decode(k, out)
+    sync_all()
+    launches0 = binding.pcr_launch_count()
+    t0 = time.perf_counter()
+    ms = timed_steps(k, args.steps)
+    t1 = time.perf_counter()
+    launches = binding.pcr_launch_count() - launches0
+    sync_all()
+    clocks = sampler.stop(t0, t1)
+    ms_max = reduce_max(ms, world)
+    total_images = reduce_sum(float(n_img), world)
+    value = total_images * args.steps / (ms_max / 1000.0)
+
+    # end to end: prefix copied from pinned host memory inside every step, status words read back
+    prefix = dec.prefix_bytes(k)
+    for _ in range(2):
+        dec.evict(); dec.decode(k, out); torch.cuda.synchronize(dev); dec.status()
+    sync_all()
+    te = time.perf_counter()
+    for _ in range(args.steps):
+        dec.evict()
+        dec.decode(k, out)
+        torch.cuda.synchronize(dev)
+        dec.status()
+    e2e_s = reduce_max(time.perf_counter() - te, world)
+    e2e = {"value": total_images * args.steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(prefix),
+           "d2h_bytes_per_step": 4 * n_img, "ms_per_step": 1000.0 * e2e_s / args.steps,
+           "note": "pcr_evict + pcr_decode from pinned host bytes + synchronise + pcr_status, wall clock; "
+                   "pixels stay on the device for the training step"}
+
+    # per-k numbers and the stage profile (this rank's GPU)
+    per_k = {}
+    for kk in pcr_synth.WORKLOADS[WORKLOAD].ks:
+        for _ in range(2):
+            dec.decode(kk, out)
+        torch.cuda.synchronize(dev)
+        st = 5
+        per_k[str(kk)] = n_img * st / (timed_steps(kk, st) / 1000.0)
+    binding.pcr_set_profiling(dec.handle, True)
+    stage_ms, stage_n = {}, {}
+    reps = 5
+    for _ in range(reps):
+        flush.fill_(1)
+        dec.decode(k, out)
+        torch.cuda.synchronize(dev)
+        for name, t, nl in binding.pcr_get_profile(dec.handle):
+            stage_ms[name] = stage_ms.get(name, 0.0) + t / reps
+            stage_n[name] = nl
+    binding.pcr_set_profiling(dec.handle, False)
+    model = algorithmic_bytes(scans, infos, k)
+    kernels = {n: t for n, t in stage_ms.items() if stage_n.get(n, 0) > 0}
+    dom = max(kernels, key=kernels.get)
+    peak, peak_src = FALLBACK_HBM_GBS, "fallback"
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            peak = float(json.load(f)["hbm_gbs"])
+            peak_src = "measured"
+    except Exception:
+        pass
+    achieved = model[dom] / (kernels[dom] * 1e-3) / 1e9
+    whole = model["total"] / (ms_max / args.steps * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None, "peak_source": peak_src, "kernel_ms": kernels[dom],
+                "algorithmic_bytes_per_launch": model[dom],
+                "whole_path": {"algorithmic_bytes_per_step": model["total"], "achieved": whole, "frac": whole / peak},
+                "stages_ms": stage_ms,
+                "stage_frac_of_peak": {n: (model.get(n, 0.0) / (t * 1e-3) / 1e9 / peak if t > 0 else None)
+                                       for n, t in stage_ms.items()}}
+
+    cpu_baseline = None
+    if do_cpu:
+        n_s = min(n_img, 512)
+        v = time_oracle(pool, cores, rec_path, k, n_s, passes=2)
+        t1c = time.perf_counter()
+        n1 = sum(pool.map(_oracle_worker, [(rec_path, k, 0, min(n_img, 48))]))      # one shard = one process
+        v1 = n1 / (time.perf_counter() - t1c)
+        pool.close(); pool.join()
+        cpu_baseline = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                        "sample": f"images 0..{n_s - 1} of the same record at k={k}, 2 passes, {cores} processes of the single-threaded oracle",
+                        "one_core": v1}
+        tmpdir.cleanup()
+
+    if rank == 0:
+        comp = [s[6] for s in scans]
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_max / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int16/u8", "data": "synthetic",
+            "config": {"workload": WORKLOAD_DESC, "k": k, "images_per_step_per_gpu": n_img,
+                       "l2": "flushed by a 256 MiB write before every timed step",
+                       "record_bytes": int(rec.bytes.size), "prefix_bytes_at_k": int(prefix),
+                       "mean_compressed_bytes_per_image_by_scan": [c / n_img for c in comp]},
+            "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
+            "cpu_baseline": cpu_baseline, "images_per_s_by_k": per_k,
+        }))
+    dec.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

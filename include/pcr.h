@@ -120,6 +120,33 @@ int pcr_coeffs(pcr_record* rec, const int16_t** dev_planes, size_t* bytes);
 /* First block of image i inside the planes returned by pcr_coeffs, and its block count. */
 int pcr_image_blocks(const pcr_record* rec, int i, uint64_t* first_block, uint64_t* n_blocks);
 
+/* One scan of the record's scan script (Section 2: scans are ordered groups of deltas; the
+ * spectral band Ss..Se and the bit positions Ah/Al are the two progressive dimensions) and
+ * the dependency wave the decoder runs it in (scans of one wave touch disjoint data). */
+typedef struct {
+    int32_t ncomp;      /* components in the scan (1, or 3 interleaved)             */
+    int32_t comp[3];    /* 0 = Y, 1 = Cb, 2 = Cr                                     */
+    int32_t Ss, Se;     /* zigzag band                                               */
+    int32_t Ah, Al;     /* successive approximation: previous / current bit position */
+    int32_t wave;       /* 0-based dependency wave                                   */
+    int32_t rsvd;
+    uint64_t bytes;     /* bytes of this scan group in the record                    */
+} pcr_scan_info;
+int pcr_get_scan(const pcr_record* rec, int s, pcr_scan_info* info);   /* s in 0..G-1 */
+
+/* Stage timing for benchmarks.  With profiling enabled every pcr_decode records CUDA events
+ * on its stream around each stage; after the stream has been synchronised pcr_get_profile
+ * returns, for the last decode, up to `cap` entries {name, milliseconds, kernel launches}.
+ * Stages: "h2d" (prefix copy), "clear" (status and plane clearing), "index" (restart-interval
+ * index), "entropy0".."entropyW" (one per wave that ran), "pixels".  *n = entries written. */
+typedef struct {
+    char name[24];
+    float ms;
+    int32_t launches;
+} pcr_stage_time;
+int pcr_set_profiling(pcr_record* rec, int enable);
+int pcr_get_profile(pcr_record* rec, pcr_stage_time* out, int cap, int* n);
+
 /* Counts kernel launches issued by this library since it was loaded (all records). */
 uint64_t pcr_launch_count(void);
 

@@ -16,12 +16,21 @@ PCR_E_ARG, PCR_E_FORMAT, PCR_E_CORRUPT, PCR_E_TIMEOUT, PCR_E_CUDA, PCR_E_NOMEM =
 
 EXPORTS = ("pcr_open", "pcr_num_images", "pcr_num_groups", "pcr_get_image", "pcr_out_bytes", "pcr_prefix_bytes",
            "pcr_decode", "pcr_evict", "pcr_status", "pcr_coeffs", "pcr_image_blocks", "pcr_launch_count",
-           "pcr_strerror", "pcr_close")
+           "pcr_strerror", "pcr_close", "pcr_get_scan", "pcr_set_profiling", "pcr_get_profile")
 
 
 class ImageInfo(C.Structure):
     _fields_ = [("width", C.c_uint32), ("height", C.c_uint32), ("label", C.c_int32), ("rsvd", C.c_uint32),
                 ("out_offset", C.c_uint64), ("out_bytes", C.c_uint64)]
+
+
+class ScanInfo(C.Structure):
+    _fields_ = [("ncomp", C.c_int32), ("comp", C.c_int32 * 3), ("Ss", C.c_int32), ("Se", C.c_int32),
+                ("Ah", C.c_int32), ("Al", C.c_int32), ("wave", C.c_int32), ("rsvd", C.c_int32), ("bytes", C.c_uint64)]
+
+
+class StageTime(C.Structure):
+    _fields_ = [("name", C.c_char * 24), ("ms", C.c_float), ("launches", C.c_int32)]
 
 
 class PcrError(RuntimeError):
@@ -54,6 +63,9 @@ def lib():
         L.pcr_status.argtypes = [vp, C.POINTER(C.c_int), C.POINTER(C.c_int)]
         L.pcr_coeffs.argtypes = [vp, C.POINTER(vp), C.POINTER(C.c_size_t)]
         L.pcr_image_blocks.argtypes = [vp, C.c_int, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
+        L.pcr_get_scan.argtypes = [vp, C.c_int, C.POINTER(ScanInfo)]
+        L.pcr_set_profiling.argtypes = [vp, C.c_int]
+        L.pcr_get_profile.argtypes = [vp, C.POINTER(StageTime), C.c_int, C.POINTER(C.c_int)]
         L.pcr_launch_count.restype = C.c_uint64
         L.pcr_launch_count.argtypes = []
         L.pcr_strerror.restype = C.c_char_p
@@ -133,3 +145,21 @@ def pcr_image_blocks(handle: int, i: int):
 
 def pcr_launch_count() -> int:
     return lib().pcr_launch_count()
+
+
+def pcr_get_scan(handle: int, s: int) -> ScanInfo:
+    info = ScanInfo()
+    _chk(lib().pcr_get_scan(handle, s, C.byref(info)), "pcr_get_scan")
+    return info
+
+
+def pcr_set_profiling(handle: int, enable: bool) -> None:
+    _chk(lib().pcr_set_profiling(handle, 1 if enable else 0), "pcr_set_profiling")
+
+
+def pcr_get_profile(handle: int):
+    """[(stage name, milliseconds, kernel launches)] of the last decode (after a synchronise)."""
+    arr = (StageTime * 16)()
+    n = C.c_int()
+    _chk(lib().pcr_get_profile(handle, arr, 16, C.byref(n)), "pcr_get_profile")
+    return [(arr[i].name.decode(), float(arr[i].ms), int(arr[i].launches)) for i in range(n.value)]

@@ -7,6 +7,7 @@
 // scan script, and the fused pixel kernel.
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
 
@@ -54,7 +55,13 @@ struct pcr_record {
     uint16_t* d_qtab = nullptr;
     int* d_status = nullptr;
     std::vector<int> h_status;
+    // optional stage timing
+    bool profiling = false;
+    std::vector<cudaEvent_t> events;
+    std::vector<pcr_stage_time> stages;   // names and launch counts of the last decode
 };
+
+static const int kMaxStages = 16;
 
 static inline uint32_t rd32(const uint8_t* p) { return (uint32_t)p[0] | ((uint32_t)p[1] << 8) | ((uint32_t)p[2] << 16) | ((uint32_t)p[3] << 24); }
 static inline uint64_t rd64(const uint8_t* p) { return (uint64_t)rd32(p) | ((uint64_t)rd32(p + 4) << 32); }
@@ -190,6 +197,8 @@ int parse_chunk(const uint8_t* rec, uint64_t off, uint32_t len, bool first, Imag
 }
 
 void free_device(pcr_record* r) {
+    for (cudaEvent_t e : r->events) cudaEventDestroy(e);
+    r->events.clear();
     cudaFree(r->d_rec); cudaFree(r->d_planes); cudaFree(r->d_script); cudaFree(r->d_scans);
     cudaFree(r->d_imgs); cudaFree(r->d_seg); cudaFree(r->d_items); cudaFree(r->d_units);
     cudaFree(r->d_qtab); cudaFree(r->d_status);
@@ -389,13 +398,27 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
     if (reinterpret_cast<uintptr_t>(out) & 15u) return PCR_E_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t need = (size_t)rec->group_end[k];
+    const bool prof = rec->profiling;
+    rec->stages.clear();
+    auto mark = [&](const char* name, int launches) {
+        if (!prof || rec->stages.size() + 1 >= rec->events.size()) return;
+        pcr_stage_time t;
+        memset(&t, 0, sizeof t);
+        strncpy(t.name, name, sizeof t.name - 1);
+        t.launches = launches;
+        rec->stages.push_back(t);
+        cudaEventRecord(rec->events[rec->stages.size()], st);
+    };
+    if (prof) cudaEventRecord(rec->events[0], st);
     if (rec->resident < need) {
         size_t from = rec->resident & ~(size_t)15;
         if (cudaMemcpyAsync(rec->d_rec + from, rec->host + from, need - from, cudaMemcpyHostToDevice, st) != cudaSuccess) return PCR_E_CUDA;
         rec->resident = need;
     }
+    mark("h2d", 0);
     if (cudaMemsetAsync(rec->d_status, 0, (size_t)rec->N * 4, st) != cudaSuccess) return PCR_E_CUDA;
     if (cudaMemsetAsync(rec->d_planes, 0, rec->total_blocks * 128, st) != cudaSuccess) return PCR_E_CUDA;
+    mark("clear", 0);
     Params P;
     P.rec = rec->d_rec; P.planes = rec->d_planes; P.script = rec->d_script; P.scans = rec->d_scans;
     P.imgs = rec->d_imgs; P.seg_start = rec->d_seg; P.items = rec->d_items; P.units = rec->d_units;
@@ -404,6 +427,7 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
         uint32_t warps = (uint32_t)k * (uint32_t)rec->N;
         seg_index_kernel<<<(warps + 7) / 8, 256, 0, st>>>(P, k);
         ++g_launches;
+        mark("index", 1);
     }
     for (int w = 0; w < rec->n_waves; ++w) {
         uint32_t begin = 0, count = 0;
@@ -416,9 +440,13 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
         if (!count) continue;
         entropy_kernel<<<(count + kEntropyWarps - 1) / kEntropyWarps, 32 * kEntropyWarps, 0, st>>>(P, begin, count);
         ++g_launches;
+        char name[24];
+        snprintf(name, sizeof name, "entropy%d", w);
+        mark(name, 1);
     }
     pixel_kernel<<<rec->n_units, kPixThreads, 0, st>>>(P, static_cast<uint8_t*>(out));
     ++g_launches;
+    mark("pixels", 1);
     if (cudaGetLastError() != cudaSuccess) return PCR_E_CUDA;
     return PCR_OK;
 }
@@ -443,6 +471,42 @@ int pcr_image_blocks(const pcr_record* rec, int i, uint64_t* first_block, uint64
     if (!rec || !first_block || !n_blocks || i < 0 || i >= rec->N) return PCR_E_ARG;
     *first_block = rec->blk_base[i];
     *n_blocks = rec->nblk[i];
+    return PCR_OK;
+}
+
+int pcr_get_scan(const pcr_record* rec, int s, pcr_scan_info* info) {
+    if (!rec || !info || s < 0 || s >= rec->G) return PCR_E_ARG;
+    const ScanScript& sc = rec->script[s];
+    info->ncomp = sc.ncomp;
+    for (int i = 0; i < 3; ++i) info->comp[i] = sc.comp[i];
+    info->Ss = sc.Ss; info->Se = sc.Se; info->Ah = sc.Ah; info->Al = sc.Al;
+    info->wave = rec->wave_of_scan[s];
+    info->rsvd = 0;
+    info->bytes = rec->group_end[s + 1] - rec->group_end[s];
+    return PCR_OK;
+}
+
+int pcr_set_profiling(pcr_record* rec, int enable) {
+    if (!rec) return PCR_E_ARG;
+    if (enable && rec->events.empty()) {
+        for (int i = 0; i <= kMaxStages; ++i) {
+            cudaEvent_t e;
+            if (cudaEventCreate(&e) != cudaSuccess) return PCR_E_CUDA;
+            rec->events.push_back(e);
+        }
+    }
+    rec->profiling = enable != 0;
+    return PCR_OK;
+}
+
+int pcr_get_profile(pcr_record* rec, pcr_stage_time* out, int cap, int* n) {
+    if (!rec || !out || !n || cap < 0) return PCR_E_ARG;
+    *n = 0;
+    for (size_t i = 0; i < rec->stages.size() && (int)i < cap; ++i) {
+        out[i] = rec->stages[i];
+        if (cudaEventElapsedTime(&out[i].ms, rec->events[i], rec->events[i + 1]) != cudaSuccess) return PCR_E_CUDA;
+        ++*n;
+    }
     return PCR_OK;
 }
 
