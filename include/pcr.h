@@ -147,6 +147,37 @@ typedef struct {
 int pcr_set_profiling(pcr_record* rec, int enable);
 int pcr_get_profile(pcr_record* rec, pcr_stage_time* out, int cap, int* n);
 
+/* The pixel stage alone, for one image, without any allocation.  (The paper has no
+ * counterpart; this is a convenience of this library.)
+ *
+ * Who needs it: code that is handed a fixed set of device buffers and must not grow the
+ * device heap or call into an allocator while it runs: a data-loader plug-in running inside
+ * another framework's memory pool, a worker that runs after the training job has claimed all
+ * device memory, or code on a path where cudaMalloc's implicit device synchronisation is not
+ * acceptable.  pcr_open/pcr_decode allocate their tables with cudaMalloc; this call does not
+ * call cudaMalloc, cudaFree or any allocating library routine.
+ *
+ * It turns the int16 coefficient planes of ONE image into packed RGB exactly as pcr_decode's
+ * last stage does (dequantise, inverse DCT, 2x2 chroma replication, colour conversion, crop).
+ *   dev_coeffs : DEVICE, caller-owned: 6*ceil(W/16)*ceil(H/16) blocks of 64 int16 in the
+ *                layout of pcr_coeffs (Y, Cb, Cr; block rows, block columns; zigzag), 4-byte
+ *                aligned.  Not modified.
+ *   width, height : at most 4096 each; larger images are refused with PCR_E_ARG.
+ *   host_qtab  : HOST, 3 x 64 uint16 quantisers (Y, Cb, Cr) in zigzag order; copied by value.
+ *   dev_rgb    : DEVICE, caller-owned, 3*W*H bytes, 4-byte aligned start recommended.
+ *   stream     : a cudaStream_t (NULL = default stream).  The call only enqueues work.
+ * The kernel's small tables (image descriptor, work-unit list, quantisers: about 65 KB) live
+ * in one fixed array inside the library's device image, which every GPU that loads the
+ * library holds until the process exits.  All calls on a device share that array and each
+ * call rewrites the part it uses, so two calls whose work overlaps on the GPU (different
+ * streams, no ordering between them) race; order them on one stream or with events.
+ * The first call on each device looks the array's device address up (cudaGetSymbolAddress,
+ * with that device current); make that first call before starting any stream capture.
+ * Errors: PCR_E_ARG (NULL, zero or too-large size, misaligned coefficients, device index
+ * beyond 63), PCR_E_CUDA. */
+int pcr_pixels_noalloc(const int16_t* dev_coeffs, uint32_t width, uint32_t height, const uint16_t* host_qtab,
+                       uint8_t* dev_rgb, void* stream);
+
 /* Counts kernel launches issued by this library since it was loaded (all records). */
 uint64_t pcr_launch_count(void);
 

@@ -16,7 +16,8 @@ PCR_E_ARG, PCR_E_FORMAT, PCR_E_CORRUPT, PCR_E_TIMEOUT, PCR_E_CUDA, PCR_E_NOMEM =
 
 EXPORTS = ("pcr_open", "pcr_num_images", "pcr_num_groups", "pcr_get_image", "pcr_out_bytes", "pcr_prefix_bytes",
            "pcr_decode", "pcr_evict", "pcr_status", "pcr_coeffs", "pcr_image_blocks", "pcr_launch_count",
-           "pcr_strerror", "pcr_close", "pcr_get_scan", "pcr_set_profiling", "pcr_get_profile")
+           "pcr_strerror", "pcr_close", "pcr_get_scan", "pcr_set_profiling", "pcr_get_profile",
+           "pcr_pixels_noalloc")
 
 
 class ImageInfo(C.Structure):
@@ -66,6 +67,7 @@ def lib():
         L.pcr_get_scan.argtypes = [vp, C.c_int, C.POINTER(ScanInfo)]
         L.pcr_set_profiling.argtypes = [vp, C.c_int]
         L.pcr_get_profile.argtypes = [vp, C.POINTER(StageTime), C.c_int, C.POINTER(C.c_int)]
+        L.pcr_pixels_noalloc.argtypes = [vp, C.c_uint32, C.c_uint32, vp, vp, vp]
         L.pcr_launch_count.restype = C.c_uint64
         L.pcr_launch_count.argtypes = []
         L.pcr_strerror.restype = C.c_char_p
@@ -163,3 +165,11 @@ def pcr_get_profile(handle: int):
     n = C.c_int()
     _chk(lib().pcr_get_profile(handle, arr, 16, C.byref(n)), "pcr_get_profile")
     return [(arr[i].name.decode(), float(arr[i].ms), int(arr[i].launches)) for i in range(n.value)]
+
+
+def pcr_pixels_noalloc(dev_coeffs_ptr: int, width: int, height: int, host_qtab_ptr: int, dev_rgb_ptr: int,
+                       stream: int = 0) -> None:
+    """Pixel stage of one image with no allocation inside the library (see include/pcr.h):
+    device coefficients + host quantisers -> device RGB, enqueued on `stream`."""
+    _chk(lib().pcr_pixels_noalloc(dev_coeffs_ptr, width, height, host_qtab_ptr, dev_rgb_ptr, stream),
+         "pcr_pixels_noalloc")

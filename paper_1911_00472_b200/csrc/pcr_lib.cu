@@ -525,6 +525,82 @@ const char* pcr_strerror(int code) {
     }
 }
 
+// ---------------------------------------------------------------------------------------
+// pcr_pixels_noalloc: the pixel stage for one image, for callers that may not allocate.
+// The pixel kernel reads an image descriptor, a work-unit list and the quantisers from
+// global memory; pcr_open puts those in cudaMalloc'd tables.  Here they live in one
+// file-scope device array that a small kernel fills on every call.
+// ---------------------------------------------------------------------------------------
+namespace {
+
+constexpr uint32_t kNoAllocMaxDim = 4096;                                         // pixels per side
+constexpr uint32_t kNoAllocMaxUnits = (kNoAllocMaxDim / 16) * (kNoAllocMaxDim / 16 / kPixMcus);
+struct NoAllocScratch {
+    ImgDesc img;
+    uint16_t qtab[192];
+    Unit units[kNoAllocMaxUnits];
+};
+static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocScratch)];
+
+struct QuantArg { uint16_t q[192]; };
+
+__global__ void noalloc_fill_kernel(uint32_t W, uint32_t H, QuantArg qa) {
+    NoAllocScratch* s = reinterpret_cast<NoAllocScratch*>(g_noalloc_scratch);   // device code may name the array
+    const uint32_t mx = (W + 15) / 16, my = (H + 15) / 16;
+    const uint32_t per_row = (mx + kPixMcus - 1) / kPixMcus;
+    const uint32_t tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+    if (tid == 0) {
+        s->img.W = W; s->img.H = H; s->img.mx = mx; s->img.my = my;
+        s->img.blk_base = 0; s->img.out_off = 0;
+    }
+    if (tid < 192) s->qtab[tid] = qa.q[tid];
+    for (uint32_t u = tid; u < per_row * my; u += nth) {
+        Unit un;
+        un.img = 0; un.mrow = (uint16_t)(u / per_row); un.mcol0 = (uint16_t)((u % per_row) * kPixMcus);
+        s->units[u] = un;
+    }
+}
+
+constexpr int kMaxDevices = 64;
+void* g_noalloc_ptr[kMaxDevices];          // device address of the array, per device
+std::atomic<int> g_noalloc_ready[kMaxDevices];
+
+}  // namespace
+
+int pcr_pixels_noalloc(const int16_t* dev_coeffs, uint32_t width, uint32_t height, const uint16_t* host_qtab,
+                       uint8_t* dev_rgb, void* stream) {
+    if (!dev_coeffs || !host_qtab || !dev_rgb || width == 0 || height == 0) return PCR_E_ARG;
+    if (width > kNoAllocMaxDim || height > kNoAllocMaxDim) return PCR_E_ARG;   // beyond the fixed scratch
+    if (reinterpret_cast<uintptr_t>(dev_coeffs) & 3u) return PCR_E_ARG;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return PCR_E_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return PCR_E_ARG;
+    if (!g_noalloc_ready[dev].load(std::memory_order_acquire)) {
+        // In host code the array's name is only a handle; its device address has to be asked for,
+        // once per device, with that device current.
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) { cudaGetLastError(); return PCR_E_CUDA; }
+        g_noalloc_ptr[dev] = p;
+        g_noalloc_ready[dev].store(1, std::memory_order_release);
+    }
+    NoAllocScratch* s = static_cast<NoAllocScratch*>(g_noalloc_ptr[dev]);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const uint32_t mx = (width + 15) / 16, my = (height + 15) / 16;
+    const uint32_t n_units = ((mx + kPixMcus - 1) / kPixMcus) * my;
+    QuantArg qa;
+    memcpy(qa.q, host_qtab, sizeof qa.q);
+    noalloc_fill_kernel<<<(n_units + 255) / 256, 256, 0, st>>>(width, height, qa);
+    ++g_launches;
+    Params P;
+    memset(&P, 0, sizeof P);
+    P.planes = const_cast<int16_t*>(dev_coeffs);     // read only by the pixel kernel
+    P.imgs = &s->img; P.units = s->units; P.qtab = s->qtab; P.N = 1;
+    pixel_kernel<<<n_units, kPixThreads, 0, st>>>(P, dev_rgb);
+    ++g_launches;
+    if (cudaGetLastError() != cudaSuccess) return PCR_E_CUDA;
+    return PCR_OK;
+}
+
 void pcr_close(pcr_record* rec) {
     if (!rec) return;
     free_device(rec);
