@@ -76,8 +76,9 @@ def algorithmic_bytes(scans, infos, k: int):
     scans: [(ncomp, comp0, Ss, Se, Ah, wave, group_bytes)], infos: [(W, H)].
       index    : bytes of scan groups <= k, read once
       entropyW : compressed bytes of the wave's scans + 2 bytes per coefficient of every
-                 block the scan visits (written once by a first pass, read and written by a
-                 refinement)
+                 block a first pass visits (written once)
+      finalize : 2 bytes read + 2 bytes written per coefficient of every block a refinement
+                 scan visits (the in-place update of the planes)
       clear    : 128 bytes per block
       pixels   : 128 bytes per block read + 3 bytes per pixel written
     """
@@ -101,9 +102,14 @@ def algorithmic_bytes(scans, infos, k: int):
         out["index"] += gbytes
         band = Se - Ss + 1
         nb = blocks_pad if ncomp > 1 else blocks_unp[comp0]
-        coef = 2.0 * band * nb * (2 if Ah else 1)
         key = f"entropy{wave}"
-        out[key] = out.get(key, 0.0) + gbytes + coef
+        out[key] = out.get(key, 0.0) + gbytes
+        if Ah and Ss > 0:
+            out["finalize"] = out.get("finalize", 0.0) + 4.0 * band * nb
+        elif Ah:
+            out[key] += 4.0 * band * nb
+        else:
+            out[key] += 2.0 * band * nb
     out["total"] = sum(out.values())
     return out
 

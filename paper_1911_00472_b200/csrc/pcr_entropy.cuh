@@ -1,9 +1,19 @@
-// Entropy stage of the PCR decoder: restart-interval index and progressive Huffman decode
-// of one wave of scans into the int16 coefficient planes.
+// Entropy stage of the PCR decoder: restart-interval index, progressive Huffman decode of one
+// wave of scans, and the pass that folds the refinement scans into the coefficient planes.
 //
 // Parallel decomposition: one LANE per restart interval.  A warp takes up to 32 consecutive
 // restart intervals of one (scan, image) pair, so its lanes share the scan's Huffman tables
-// (held as lookup tables in shared memory) and run the same scan kind in lock step.
+// (lookup tables in shared memory).  Every lane runs ONE flat loop whose iteration decodes one
+// Huffman symbol (or one block of an end-of-band run); block changes are a few predicated
+// instructions inside that loop, so lanes that sit in different blocks stay converged.
+//
+// First passes write coefficients straight into the (pre-zeroed) planes.  An AC refinement
+// needs, per block, only WHICH band positions are already non-zero: a 64-bit mask.  First-pass
+// AC scans leave that mask as side data; a refinement lane reads it, decodes with bit
+// operations (skipping r zero positions = dropping r set bits of the inverted mask; one
+// correction bit per set bit of the mask passed over) and leaves {new mask, correction bits,
+// new positions, their signs} as side data.  finalize_kernel then updates the planes in place,
+// one lane per coefficient pair, fully coalesced.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -14,8 +24,8 @@ namespace pcr {
 
 constexpr int kErrCorrupt = -3;
 
-constexpr int kLutBits = 9;
-constexpr int kEntropyWarps = 8;
+constexpr int kLutBits = 11;
+constexpr int kEntropyWarps = 4;
 
 // Decoder tables of one Huffman table: a direct lookup on the next kLutBits bits for short
 // codes, and the canonical first-code / count / index triple per length for the rest.
@@ -36,16 +46,21 @@ __device__ __forceinline__ void build_hufftab(HuffTab& t, const uint8_t* __restr
         code = (code + c) << 1;
         p += c;
     }
-    if (p > 256) p = 256;
-    for (uint32_t j = lane; j < p; j += 32) t.vals[j] = dht[16 + j];
+    const uint32_t nvals = min(p, 256u);
+    for (uint32_t j = lane; j < nvals; j += 32) t.vals[j] = dht[16 + j];
+    uint32_t* lw = reinterpret_cast<uint32_t*>(t.lut);
+    for (int e = lane; e < (1 << kLutBits) / 2; e += 32) lw[e] = 0;
     __syncwarp();
-    for (int e = lane; e < (1 << kLutBits); e += 32) {
-        uint32_t entry = 0;
-        for (int l = 1; l <= kLutBits; ++l) {
-            uint32_t d = ((uint32_t)e >> (kLutBits - l)) - t.first[l];
-            if (d < t.cnt[l]) { entry = ((uint32_t)l << 8) | t.vals[t.idx[l] + d]; break; }
+    // every symbol with a short code fills its 2^(kLutBits - length) entries, all lanes together
+    uint32_t j = 0;
+    for (int l = 1; l <= kLutBits; ++l) {
+        const uint32_t c = t.cnt[l], f = t.first[l], span = 1u << (kLutBits - l);
+        for (uint32_t i = 0; i < c && j < nvals; ++i, ++j) {
+            const uint32_t base = (f + i) << (kLutBits - l);
+            const uint16_t entry = (uint16_t)(((uint32_t)l << 8) | t.vals[j]);
+            if (base + span <= (1u << kLutBits))
+                for (uint32_t e = lane; e < span; e += 32) t.lut[base + e] = entry;
         }
-        t.lut[e] = (uint16_t)entry;
     }
     __syncwarp();
 }
@@ -171,6 +186,7 @@ struct Geometry {
     uint32_t mx, my;          // MCU grid
     uint32_t bw[3], ubw[3], ubh[3];
     uint64_t coff[3];         // first block of each component (global block index)
+    uint64_t loff[3];         // first block of each component counted inside its component
 };
 
 __device__ __forceinline__ Geometry make_geometry(const ImgDesc& im) {
@@ -183,17 +199,21 @@ __device__ __forceinline__ Geometry make_geometry(const ImgDesc& im) {
     g.coff[0] = im.blk_base;
     g.coff[1] = im.blk_base + 4ull * im.mx * im.my;
     g.coff[2] = im.blk_base + 5ull * im.mx * im.my;
+    const uint64_t mcus_before = im.blk_base / 6;      // every image holds 6 blocks per MCU
+    g.loff[0] = 4 * mcus_before; g.loff[1] = g.loff[2] = mcus_before;
     return g;
 }
 
+__device__ __forceinline__ uint64_t low_mask(int p) { return p >= 64 ? ~0ull : ((1ull << p) - 1ull); }
+
 __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, uint32_t item_begin, uint32_t item_count) {
     __shared__ HuffTab tabs[kEntropyWarps][2];
-    int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    uint32_t it = blockIdx.x * kEntropyWarps + wid;
+    const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t it = blockIdx.x * kEntropyWarps + wid;
     if (it >= item_count) return;
     const Item item = P.items[item_begin + it];
     const ScanDesc sd = P.scans[item.si];
-    int s = item.si / P.N, img = item.si % P.N;
+    const int s = item.si / P.N, img = item.si % P.N;
     const ScanScript sc = P.script[s];
     const ImgDesc im = P.imgs[img];
     const Geometry g = make_geometry(im);
@@ -203,19 +223,19 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
         build_hufftab(tabs[wid][0], P.rec + sd.tab_off[0], lane);
         if (sd.tab_off[1]) build_hufftab(tabs[wid][1], P.rec + sd.tab_off[1], lane);
     }
-    uint32_t seg = item.seg0 + lane;
-    if (seg >= sd.nseg) return;
+    const uint32_t seg = item.seg0 + lane;
+    if ((uint32_t)lane >= item.count || seg >= sd.nseg) return;
 
     const bool inter = sc.ncomp > 1;
     const int c0 = sc.comp[0];
-    uint32_t mcu_w = inter ? g.mx : g.ubw[c0];
-    uint32_t mcu_h = inter ? g.my : g.ubh[c0];
-    uint32_t total = mcu_w * mcu_h;
-    uint32_t m0 = sd.ri ? seg * sd.ri : 0;
-    uint32_t m1 = sd.ri ? min(m0 + sd.ri, total) : total;
+    const uint32_t mcu_w = inter ? g.mx : g.ubw[c0];
+    const uint32_t mcu_h = inter ? g.my : g.ubh[c0];
+    const uint32_t total = mcu_w * mcu_h;
+    const uint32_t m0 = sd.ri ? seg * sd.ri : 0;
+    const uint32_t m1 = sd.ri ? min(m0 + sd.ri, total) : total;
     const uint32_t* segtab = P.seg_start + sd.seg_base;
-    uint32_t bstart = segtab[seg];
-    uint32_t bend = (seg + 1 < sd.nseg) ? segtab[seg + 1] - 2 : sd.data_end;
+    const uint32_t bstart = segtab[seg];
+    const uint32_t bend = (seg + 1 < sd.nseg) ? segtab[seg + 1] - 2 : sd.data_end;
     if (bstart < sd.data_off || bend > sd.data_end || bend < bstart) {   // a missing marker left a hole
         atomicMin(&P.status[img], kErrCorrupt);
         return;
@@ -224,26 +244,28 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
     br.init(P.rec, bstart, bend);
     bool bad = false;
     const int Al = sc.Al, p1 = 1 << sc.Al;
-    uint32_t mrow = m0 / mcu_w, mcol = m0 % mcu_w;
 
     if (dc) {
-        int pred[3] = {0, 0, 0};
+        // DC scans: every lane walks the same MCU structure, so the loop nest stays converged.
+        uint32_t mrow = m0 / mcu_w, mcol = m0 % mcu_w;
+        int pred0 = 0, pred1 = 0, pred2 = 0;
         for (uint32_t m = m0; m < m1 && !bad; ++m) {
             for (int ci = 0; ci < sc.ncomp; ++ci) {
-                int c = sc.comp[ci];
-                int hv = (inter && c == 0) ? 2 : 1;
-                const HuffTab& tab = tabs[wid][(sd.slots >> (2 * ci)) & 3u];
+                const int c = sc.comp[ci];
+                const int hv = (inter && c == 0) ? 2 : 1;
+                const HuffTab& tab = tabs[wid][(sd.slots >> (2 * ci)) & 1u];
                 for (int sub = 0; sub < hv * hv; ++sub) {
-                    uint64_t blk = g.coff[c] + (uint64_t)(mrow * hv + (sub >> (hv - 1))) * g.bw[c] + mcol * hv + (sub & (hv - 1));
+                    const uint64_t blk = g.coff[c] + (uint64_t)(mrow * hv + (sub >> (hv - 1))) * g.bw[c] + mcol * hv + (sub & (hv - 1));
                     int16_t* cf = P.planes + blk * 64;
                     br.refill();
                     if (sc.Ah == 0) {
-                        int sz = huff_decode(tab, br, bad);
+                        const int sz = huff_decode(tab, br, bad);
                         if (sz > 15) bad = true;
                         if (bad) break;
-                        int d = extend_bits(br.take(sz), sz);
-                        pred[c] += d;
-                        cf[0] = (int16_t)(pred[c] << Al);
+                        const int d = extend_bits(br.take(sz), sz);
+                        int pv = (c == 0 ? pred0 : (c == 1 ? pred1 : pred2)) + d;
+                        if (c == 0) pred0 = pv; else if (c == 1) pred1 = pv; else pred2 = pv;
+                        cf[0] = (int16_t)(pv << Al);
                     } else {
                         if (br.take(1)) cf[0] = (int16_t)(cf[0] | p1);
                     }
@@ -253,86 +275,193 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
             if (++mcol == mcu_w) { mcol = 0; ++mrow; }
         }
     } else {
-        const HuffTab& tab = tabs[wid][sd.slots & 3u];
+        const HuffTab& tab = tabs[wid][0];
         const int c = c0, Ss = sc.Ss, Se = sc.Se;
+        const ScanAux ax = P.saux[s];
+        const uint32_t bw = g.bw[c];
+        uint32_t m = m0, brow = m0 / mcu_w, bcol = m0 % mcu_w;
         uint32_t eobrun = 0;
+        int k = Ss;
         if (sc.Ah == 0) {
-            uint32_t m = m0;
+            // ---- AC first pass: one Huffman symbol per iteration
+            uint64_t* maskp = P.aux + ax.base + g.loff[c];
+            uint64_t M = 0;
             while (m < m1 && !bad) {
-                if (eobrun > 0) {                       // whole blocks inside an end-of-band run
-                    uint32_t sk = min(eobrun, m1 - m);
-                    eobrun -= sk; m += sk;
-                    continue;
+                br.refill();
+                const int rs = huff_decode(tab, br, bad);
+                if (bad) break;
+                const int r = rs >> 4, sz = rs & 15;
+                bool done;
+                if (sz) {
+                    k += r;
+                    if (k > Se) { bad = true; break; }
+                    const int v = extend_bits(br.take(sz), sz) * p1;
+                    P.planes[(g.coff[c] + (uint64_t)brow * bw + bcol) * 64 + k] = (int16_t)v;
+                    M |= 1ull << k;
+                    ++k;
+                    done = k > Se;
+                } else if (r == 15) {
+                    k += 16;
+                    done = k > Se;
+                } else {
+                    eobrun = (1u << r) + (r ? br.take(r) : 0u) - 1u;
+                    done = true;
                 }
-                uint32_t brow = m / mcu_w, bcol = m % mcu_w;
-                int16_t* cf = P.planes + (g.coff[c] + (uint64_t)brow * g.bw[c] + bcol) * 64;
-                int k = Ss;
-                while (k <= Se) {
-                    br.refill();
-                    int rs = huff_decode(tab, br, bad);
-                    if (bad) break;
-                    int r = rs >> 4, sz = rs & 15;
-                    if (sz) {
-                        k += r;
-                        if (k > Se) { bad = true; break; }
-                        cf[k] = (int16_t)(extend_bits(br.take(sz), sz) * p1);
-                        ++k;
-                    } else if (r == 15) {
-                        k += 16;
-                    } else {
-                        eobrun = (1u << r) + (r ? br.take(r) : 0u) - 1u;
-                        break;
+                if (done) {
+                    if (M) maskp[(uint64_t)brow * bw + bcol] = M;
+                    uint32_t adv = 1;
+                    if (eobrun) {                      // the following blocks of the run are empty
+                        const uint32_t extra = min(eobrun, m1 - (m + 1));
+                        eobrun -= extra;
+                        adv += extra;
                     }
+                    m += adv;
+                    if (adv == 1) { if (++bcol == mcu_w) { bcol = 0; ++brow; } }
+                    else { brow = m / mcu_w; bcol = m % mcu_w; }
+                    k = Ss; M = 0;
                 }
-                ++m;
             }
         } else {
-            for (uint32_t m = m0; m < m1 && !bad; ++m) {
-                uint32_t brow = m / mcu_w, bcol = m % mcu_w;
-                int16_t* cf = P.planes + (g.coff[c] + (uint64_t)brow * g.bw[c] + bcol) * 64;
-                int k = Ss;
-                if (eobrun == 0) {
-                    while (k <= Se) {
-                        br.refill();
-                        int rs = huff_decode(tab, br, bad);
-                        if (bad) break;
-                        int r = rs >> 4, sz = rs & 15, newval = 0;
-                        if (sz) {
-                            if (sz != 1) { bad = true; break; }
-                            newval = br.take(1) ? p1 : -p1;
-                        } else if (r < 15) {
-                            eobrun = (1u << r) + (r ? br.take(r) : 0u);
-                            break;
-                        }
-                        while (k <= Se) {
-                            int v = cf[k];
-                            if (v != 0) {
-                                br.refill();
-                                if (br.take(1) && (v & p1) == 0) cf[k] = (int16_t)(v >= 0 ? v + p1 : v - p1);
-                            } else {
-                                if (r == 0) break;
-                                --r;
-                            }
-                            ++k;
-                        }
-                        if (sz && k <= Se) cf[k] = (int16_t)newval;
-                        ++k;
+            // ---- AC refinement: one Huffman symbol, or one block of an end-of-band run, per iteration
+            const uint64_t band = low_mask(Se + 1) & ~low_mask(Ss);
+            const uint64_t* srcp[4];
+            uint32_t srcs[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const ScanAux sx = P.saux[ax.src[i < ax.nsrc ? i : 0]];
+                srcp[i] = P.aux + sx.base + (uint64_t)g.loff[c] * sx.stride;
+                srcs[i] = sx.stride;
+            }
+            uint64_t* outp = P.aux + ax.base + g.loff[c] * 4ull;
+            auto load_hist = [&](uint32_t row, uint32_t col) -> uint64_t {
+                const uint64_t bi = (uint64_t)row * bw + col;
+                uint64_t h = srcp[0][bi * srcs[0]];
+                if (ax.nsrc > 1) h |= srcp[1][bi * srcs[1]];
+                if (ax.nsrc > 2) h |= srcp[2][bi * srcs[2]];
+                if (ax.nsrc > 3) h |= srcp[3][bi * srcs[3]];
+                return h & band;
+            };
+            uint64_t H = load_hist(brow, bcol);
+            uint32_t nrow = brow, ncol = bcol + 1;
+            if (ncol == mcu_w) { ncol = 0; ++nrow; }
+            uint64_t Hn = (m + 1 < m1) ? load_hist(nrow, ncol) : 0ull;      // the next block's mask is already in flight
+            uint64_t cstr = 0, Nw = 0, NS = 0;
+            int cn = 0;
+            while (m < m1 && !bad) {
+                bool eob = eobrun > 0;
+                int r = 0, sz = 0;
+                uint32_t sign = 0;
+                if (!eob) {
+                    br.refill();
+                    const int rs = huff_decode(tab, br, bad);
+                    if (bad) break;
+                    r = rs >> 4; sz = rs & 15;
+                    if (sz) {
+                        if (sz != 1) { bad = true; break; }
+                        sign = br.take(1);
+                    } else if (r < 15) {
+                        eobrun = (1u << r) + (r ? br.take(r) : 0u);
+                        eob = true;
                     }
                 }
-                if (eobrun > 0 && !bad) {
-                    for (; k <= Se; ++k) {
-                        int v = cf[k];
-                        if (v != 0) {
-                            br.refill();
-                            if (br.take(1) && (v & p1) == 0) cf[k] = (int16_t)(v >= 0 ? v + p1 : v - p1);
-                        }
-                    }
-                    --eobrun;
+                const uint64_t from = ~0ull << k;                      // k <= Se <= 63 here
+                int pos = Se + 1;
+                if (!eob) {
+                    uint64_t Z = ~H & band & from;                     // zero-valued positions still ahead
+                    for (; r > 0 && Z; --r) Z &= Z - 1;                // pass over r of them
+                    if (Z) pos = __ffsll((long long)Z) - 1;
+                }
+                const uint64_t hist = H & from & low_mask(pos);        // non-zero positions passed: one correction bit each
+                const int n = __popcll(hist);
+                if (n) {
+                    if (cn + n > 64) { bad = true; break; }
+                    br.refill();
+                    uint64_t bits = br.take(min(n, 32));
+                    if (n > 32) { br.refill(); bits = (bits << (n - 32)) | br.take(n - 32); }
+                    cstr |= bits << (64 - cn - n);
+                    cn += n;
+                }
+                if (sz && pos <= Se) { Nw |= 1ull << pos; NS |= (uint64_t)sign << pos; }
+                k = pos + 1;
+                if (eob) --eobrun;
+                if (k > Se) {                                          // block finished
+                    uint64_t* o = outp + ((uint64_t)brow * bw + bcol) * 4;
+                    *reinterpret_cast<ulonglong2*>(o) = make_ulonglong2(H | Nw, cstr);
+                    *reinterpret_cast<ulonglong2*>(o + 2) = make_ulonglong2(Nw, NS);
+                    ++m;
+                    brow = nrow; bcol = ncol;
+                    H = Hn;
+                    if (++ncol == mcu_w) { ncol = 0; ++nrow; }
+                    if (m + 1 < m1) Hn = load_hist(nrow, ncol);
+                    k = Ss; cstr = 0; Nw = 0; NS = 0; cn = 0;
                 }
             }
         }
     }
     if (bad || br.overran()) atomicMin(&P.status[img], kErrCorrupt);
+}
+
+// ---------------------------------------------------------------------------------------
+// Fold the side data of the AC refinement scans into the coefficient planes, in scan order.
+// One thread per block; the work is proportional to the coefficients that actually change:
+// the thread walks the set bits of the "already non-zero" mask while correction bits equal to 1
+// remain (a correction moves the coefficient away from zero by 2^Al if its bit Al is still
+// clear), then the set bits of the "newly non-zero" mask (value +-2^Al).
+// ---------------------------------------------------------------------------------------
+constexpr int kFinalizeThreads = 192;      // four units of 48 blocks
+
+__global__ void __launch_bounds__(kFinalizeThreads) finalize_kernel(Params P, FinalizeList fl, uint32_t n_units) {
+    const uint32_t t = blockIdx.x * kFinalizeThreads + threadIdx.x;
+    const uint32_t unit = t / 48;
+    const int j = (int)(t % 48);
+    if (unit >= n_units) return;
+    const Unit un = P.units[unit];
+    const ImgDesc im = P.imgs[un.img];
+    const int nm = min(8, (int)im.mx - (int)un.mcol0);
+    const uint64_t mcus_before = im.blk_base / 6;
+    // same block order as the pixel kernel: Y row 0 (16), Y row 1 (16), Cb (8), Cr (8)
+    int c;
+    uint64_t local, blk;
+    if (j < 32) {
+        const int r = j >> 4, col = j & 15;
+        if (col >= 2 * nm) return;
+        c = 0;
+        local = (uint64_t)(2 * un.mrow + r) * (2 * im.mx) + 2 * un.mcol0 + col;
+        blk = im.blk_base + local;
+        local += 4 * mcus_before;
+    } else {
+        const int col = (j - 32) & 7;
+        if (col >= nm) return;
+        c = 1 + ((j - 32) >> 3);
+        local = (uint64_t)un.mrow * im.mx + un.mcol0 + col;
+        blk = im.blk_base + (c == 1 ? 4ull : 5ull) * im.mx * im.my + local;
+        local += mcus_before;
+    }
+    int16_t* cf = P.planes + blk * 64;
+    for (int i = 0; i < fl.n[c]; ++i) {
+        const int s = fl.scan[c][i];
+        const int p1 = fl.p1[c][i];
+        const ulonglong2* o = reinterpret_cast<const ulonglong2*>(P.aux + fl.base[c][i] + local * 4);
+        const ulonglong2 a = __ldg(o), b = __ldg(o + 1);       // {mask, corrections}, {new, signs}
+        (void)s;
+        uint64_t h = a.x & ~b.x, cc = a.y;
+        while (cc) {
+            const int pos = __ffsll((long long)h) - 1;
+            if (pos < 0) break;
+            h &= h - 1;
+            if (cc >> 63) {
+                const int v = cf[pos];
+                if ((v & p1) == 0) cf[pos] = (int16_t)(v >= 0 ? v + p1 : v - p1);
+            }
+            cc <<= 1;
+        }
+        uint64_t nw = b.x;
+        while (nw) {
+            const int pos = __ffsll((long long)nw) - 1;
+            nw &= nw - 1;
+            cf[pos] = (int16_t)(((b.y >> pos) & 1ull) ? p1 : -p1);
+        }
+    }
 }
 
 }  // namespace pcr

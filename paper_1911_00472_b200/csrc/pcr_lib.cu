@@ -47,6 +47,9 @@ struct pcr_record {
     size_t resident = 0;
     int16_t* d_planes = nullptr;
     ScanScript* d_script = nullptr;
+    ScanAux* d_saux = nullptr;
+    uint64_t* d_aux = nullptr;
+    std::vector<ScanAux> saux;
     ScanDesc* d_scans = nullptr;
     ImgDesc* d_imgs = nullptr;
     uint32_t* d_seg = nullptr;
@@ -199,7 +202,7 @@ int parse_chunk(const uint8_t* rec, uint64_t off, uint32_t len, bool first, Imag
 void free_device(pcr_record* r) {
     for (cudaEvent_t e : r->events) cudaEventDestroy(e);
     r->events.clear();
-    cudaFree(r->d_rec); cudaFree(r->d_planes); cudaFree(r->d_script); cudaFree(r->d_scans);
+    cudaFree(r->d_rec); cudaFree(r->d_planes); cudaFree(r->d_script); cudaFree(r->d_saux); cudaFree(r->d_aux); cudaFree(r->d_scans);
     cudaFree(r->d_imgs); cudaFree(r->d_seg); cudaFree(r->d_items); cudaFree(r->d_units);
     cudaFree(r->d_qtab); cudaFree(r->d_status);
 }
@@ -315,7 +318,11 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
             r->scan_item_begin[s] = (uint32_t)items.size();
             for (uint32_t i = 0; i < N; ++i) {
                 const ScanDesc& sd = scans[(size_t)s * N + i];
-                for (uint32_t j = 0; j < sd.nseg; j += 32) items.push_back(Item{(uint32_t)(s * N + i), j});
+                // split the restart intervals evenly over as few warps as needed
+                const uint32_t parts = (sd.nseg + kSegsPerItem - 1) / kSegsPerItem;
+                const uint32_t per = (sd.nseg + parts - 1) / parts;
+                for (uint32_t j = 0; j < sd.nseg; j += per)
+                    items.push_back(Item{(uint32_t)(s * N + i), j, std::min(per, sd.nseg - j), 0u});
             }
             r->scan_item_count[s] = (uint32_t)items.size() - r->scan_item_begin[s];
         }
@@ -328,8 +335,47 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
             }
     r->n_units = (uint32_t)units.size();
 
+    // side data of the AC scans: one word per block for a first pass, four for a refinement
+    const uint64_t total_mcus = blocks / 6;
+    uint64_t aux_words = 0;
+    r->saux.assign(G, ScanAux{});
+    int n_refine[3] = {0, 0, 0};
+    for (uint32_t s = 0; s < G; ++s)
+        if (r->script[s].Ss > 0 && r->script[s].Ah > 0 && ++n_refine[r->script[s].comp[0]] > 4) return PCR_E_FORMAT;
+    for (uint32_t s = 0; s < G; ++s) {
+        const ScanScript& sc = r->script[s];
+        ScanAux& ax = r->saux[s];
+        if (sc.Ss == 0) continue;
+        ax.stride = sc.Ah ? 4u : 1u;
+        ax.base = aux_words;
+        aux_words += (sc.comp[0] == 0 ? 4ull : 1ull) * total_mcus * ax.stride;
+        aux_words = (aux_words + 1) & ~1ull;      // 16-byte alignment of every scan's area
+        if (sc.Ah) {
+            // positions already non-zero = union of the masks of earlier scans on this band; an
+            // earlier scan is covered by a later refinement whose band contains its own
+            std::vector<int> src;
+            for (uint32_t t = 0; t < s; ++t) {
+                const ScanScript& st = r->script[t];
+                if (st.Ss == 0 || st.comp[0] != sc.comp[0] || st.Ss > sc.Se || sc.Ss > st.Se) continue;
+                src.push_back((int)t);
+            }
+            std::vector<int> keep;
+            for (int t : src) {
+                bool covered = false;
+                for (int u : src)
+                    if (u > t && r->script[u].Ah && r->script[u].Ss <= r->script[t].Ss && r->script[u].Se >= r->script[t].Se) covered = true;
+                if (!covered) keep.push_back(t);
+            }
+            if (keep.empty() || keep.size() > 4) return PCR_E_FORMAT;
+            ax.nsrc = (int)keep.size();
+            for (size_t i = 0; i < keep.size(); ++i) ax.src[i] = keep[i];
+        }
+    }
+
     // device state
     if (cudaGetDevice(&r->device) != cudaSuccess) return PCR_E_CUDA;
+    if (cudaMalloc(reinterpret_cast<void**>(&r->d_aux), std::max<uint64_t>(aux_words, 2) * 8) != cudaSuccess) { r->d_aux = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
+    if (cudaMemset(r->d_aux, 0, std::max<uint64_t>(aux_words, 2) * 8) != cudaSuccess) return PCR_E_CUDA;
     if (cudaMalloc(reinterpret_cast<void**>(&r->d_rec), len + 64) != cudaSuccess) { r->d_rec = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
     if (cudaMalloc(reinterpret_cast<void**>(&r->d_planes), std::max<uint64_t>(blocks, 1) * 128) != cudaSuccess) { r->d_planes = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
     if (cudaMalloc(reinterpret_cast<void**>(&r->d_seg), (segs + 1) * 4) != cudaSuccess) { r->d_seg = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
@@ -337,6 +383,7 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     if (cudaMemset(r->d_seg, 0, (segs + 1) * 4) != cudaSuccess || cudaMemset(r->d_status, 0, (size_t)N * 4) != cudaSuccess) return PCR_E_CUDA;
     int rc;
     if ((rc = upload(&r->d_script, r->script))) return rc;
+    if ((rc = upload(&r->d_saux, r->saux))) return rc;
     if ((rc = upload(&r->d_scans, scans))) return rc;
     if ((rc = upload(&r->d_imgs, imgs))) return rc;
     if ((rc = upload(&r->d_items, items))) return rc;
@@ -421,6 +468,7 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
     mark("clear", 0);
     Params P;
     P.rec = rec->d_rec; P.planes = rec->d_planes; P.script = rec->d_script; P.scans = rec->d_scans;
+    P.saux = rec->d_saux; P.aux = rec->d_aux;
     P.imgs = rec->d_imgs; P.seg_start = rec->d_seg; P.items = rec->d_items; P.units = rec->d_units;
     P.qtab = rec->d_qtab; P.status = rec->d_status; P.N = rec->N;
     {
@@ -443,6 +491,29 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
         char name[24];
         snprintf(name, sizeof name, "entropy%d", w);
         mark(name, 1);
+    }
+    {
+        FinalizeList fl;
+        memset(&fl, 0, sizeof fl);
+        bool any = false;
+        for (int s = 0; s < k; ++s) {
+            const ScanScript& sc = rec->script[s];
+            if (sc.Ss == 0 || sc.Ah == 0) continue;
+            int c = sc.comp[0];
+            if (fl.n[c] < 4) {
+                fl.scan[c][fl.n[c]] = s;
+                fl.p1[c][fl.n[c]] = 1 << sc.Al;
+                fl.base[c][fl.n[c]] = rec->saux[s].base;
+                ++fl.n[c];
+                any = true;
+            }
+        }
+        if (any) {
+            const uint64_t threads = (uint64_t)rec->n_units * 48;
+            finalize_kernel<<<(unsigned)((threads + kFinalizeThreads - 1) / kFinalizeThreads), kFinalizeThreads, 0, st>>>(P, fl, rec->n_units);
+            ++g_launches;
+            mark("finalize", 1);
+        }
     }
     pixel_kernel<<<rec->n_units, kPixThreads, 0, st>>>(P, static_cast<uint8_t*>(out));
     ++g_launches;

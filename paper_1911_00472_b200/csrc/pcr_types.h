@@ -11,6 +11,30 @@ struct ScanScript {
     int32_t Ss, Se, Ah, Al;
 };
 
+// Where an AC scan keeps its per-block side data in the auxiliary array (units of uint64,
+// indexed by the block's number inside its component across the whole record):
+//  - a first-pass AC scan writes one word per block: the mask of zigzag positions it made non-zero;
+//  - an AC refinement scan writes four words per block: {mask of non-zero positions of its band
+//    after the scan, correction bits in reading order (first bit at bit 63), mask of newly
+//    non-zero positions, mask of those that are positive}.  The coefficient planes are updated
+//    from these by the finalize kernel.
+// A refinement scan finds the positions that were non-zero before it by OR-ing the masks of up
+// to four earlier scans (src), each read with its own stride.
+struct ScanAux {
+    uint64_t base;        // first word of this scan's side data
+    uint32_t stride;      // words per block: 1 or 4
+    int32_t nsrc;
+    int32_t src[4];       // scan indices
+};
+
+// Refinement scans to apply per component, in scan order (built per decode for the chosen k).
+struct FinalizeList {
+    int32_t n[3];
+    int32_t scan[3][4];
+    int32_t p1[3][4];      // 1 << Al of the scan
+    uint64_t base[3][4];   // first word of the scan's side data
+};
+
 // One (scan, image) pair: where its entropy-coded bytes and Huffman tables live.
 struct ScanDesc {
     uint32_t data_off;    // first entropy-coded byte (offset in the record)
@@ -28,10 +52,19 @@ struct ImgDesc {
     uint64_t out_off;     // first byte of the image in the output buffer
 };
 
-// Entropy work item: up to 32 consecutive restart intervals of one (scan, image).
+// Restart intervals one warp takes (one lane each).  Fewer than 32 leaves lanes idle but
+// gives more warps to hide the latency of the serial decode chains.
+#ifndef PCR_SEGS_PER_ITEM
+#define PCR_SEGS_PER_ITEM 32
+#endif
+constexpr int kSegsPerItem = PCR_SEGS_PER_ITEM;
+
+// Entropy work item: up to kSegsPerItem consecutive restart intervals of one (scan, image).
 struct Item {
     uint32_t si;          // scan * N + image
     uint32_t seg0;        // first restart interval of the item
+    uint32_t count;       // restart intervals in the item (<= kSegsPerItem)
+    uint32_t rsvd;
 };
 
 // Pixel work unit: a run of MCUs in one MCU row of one image.
@@ -44,6 +77,8 @@ struct Params {
     const uint8_t* rec;         // record bytes on the device
     int16_t* planes;            // coefficient planes, 64 int16 per block, zigzag order
     const ScanScript* script;   // [G]
+    const ScanAux* saux;        // [G]
+    uint64_t* aux;              // side data of the AC scans
     const ScanDesc* scans;      // [G][N]
     const ImgDesc* imgs;        // [N]
     uint32_t* seg_start;        // segment table: first byte of every restart interval
