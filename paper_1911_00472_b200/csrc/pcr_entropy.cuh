@@ -65,63 +65,30 @@ __device__ __forceinline__ void build_hufftab(HuffTab& t, const uint8_t* __restr
     __syncwarp();
 }
 
-// MSB-first bit reader over one restart interval, removing the stuffed zero byte after 0xFF.
-// Past the end of the interval it feeds zero bits and counts them, so that over-reading is
-// detected at the end instead of touching bytes of another interval.
+// MSB-first bit reader over the unstuffed copy of the entropy-coded bytes (see
+// unstuff_index_kernel): the copy holds big-endian 32-bit words, so the next 32 bits at any
+// bit position are two aligned word loads and one funnel shift, and consuming bits is an add.
 struct BitReader {
-    const uint8_t* base;
-    uint32_t pos, end;
-    uint64_t buf;     // left aligned
-    int nbits;        // bits held in buf
-    int fake;         // zero bits appended past the end
+    const uint32_t* w;   // word 0 of the (scan, image) chunk in the unstuffed copy
+    uint32_t pos;        // next bit, relative to w
+    uint32_t end;        // first bit past the restart interval
 
-    __device__ __forceinline__ void init(const uint8_t* b, uint32_t p, uint32_t e) {
-        base = b; pos = p; end = e; buf = 0; nbits = 0; fake = 0;
+    __device__ __forceinline__ uint32_t peek() const {
+        const uint32_t i = pos >> 5;
+        return __funnelshift_l(__ldg(w + i + 1), __ldg(w + i), pos);
     }
-    // afterwards at least 33 bits are held
-    __device__ __forceinline__ void refill() {
-        while (nbits <= 32) {
-            if ((pos & 3u) == 0 && pos + 4 <= end) {
-                uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(base + pos));
-                uint32_t ff = ((w & 0x7F7F7F7Fu) + 0x01010101u) & w & 0x80808080u;
-                if (ff == 0) {
-                    buf |= (uint64_t)__byte_perm(w, 0, 0x0123) << (32 - nbits);
-                    nbits += 32;
-                    pos += 4;
-                    continue;
-                }
-            }
-            uint32_t b = 0;
-            if (pos < end) {
-                b = __ldg(base + pos);
-                pos += (b == 0xFF) ? 2 : 1;
-            } else {
-                fake += 8;
-            }
-            buf |= (uint64_t)b << (56 - nbits);
-            nbits += 8;
-        }
-    }
-    __device__ __forceinline__ uint32_t peek16() const { return (uint32_t)(buf >> 48); }
-    __device__ __forceinline__ void skip(int n) { buf <<= n; nbits -= n; }
-    // n in 0..32, bits must be held
-    __device__ __forceinline__ uint32_t take(int n) {
-        uint32_t v = n ? (uint32_t)(buf >> (64 - n)) : 0u;
-        skip(n);
-        return v;
-    }
-    __device__ __forceinline__ bool overran() const { return nbits < fake; }
+    __device__ __forceinline__ bool overran() const { return pos > end; }
 };
 
-__device__ __forceinline__ int huff_decode(const HuffTab& t, BitReader& br, bool& bad) {
-    uint32_t w = br.peek16();
-    uint32_t e = t.lut[w >> (16 - kLutBits)];
-    if (e) { br.skip((int)(e >> 8)); return (int)(e & 255u); }
+// Huffman symbol at the top of the 32-bit window; returns (length << 8) | symbol, 0 if undefined
+__device__ __forceinline__ uint32_t huff_lookup(const HuffTab& t, uint32_t win) {
+    uint32_t e = t.lut[win >> (32 - kLutBits)];
+    if (e) return e;
+    const uint32_t w16 = win >> 16;
     for (int l = kLutBits + 1; l <= 16; ++l) {
-        uint32_t d = (w >> (16 - l)) - t.first[l];
-        if (d < t.cnt[l]) { br.skip(l); return t.vals[t.idx[l] + d]; }
+        uint32_t d = (w16 >> (16 - l)) - t.first[l];
+        if (d < t.cnt[l]) return ((uint32_t)l << 8) | t.vals[t.idx[l] + d];
     }
-    bad = true;
     return 0;
 }
 
@@ -129,54 +96,75 @@ __device__ __forceinline__ int extend_bits(uint32_t v, int s) {
     // value of an s-bit magnitude field: the top bit clear means negative
     return s == 0 ? 0 : ((v >> (s - 1)) ? (int)v : (int)v - (1 << s) + 1);
 }
+// the top n bits of x (n in 0..32)
+__device__ __forceinline__ uint32_t top_bits(uint32_t x, int n) { return n ? x >> (32 - n) : 0u; }
 
 // ---------------------------------------------------------------------------------------
-// Restart-interval index: for every (scan < nscans, image), the first byte of each restart
-// interval.  One warp per pair; markers found per 16-byte lane slice, ordinals by a warp
-// prefix sum.
+// Restart-interval index and unstuffing, one warp per (scan < nscans, image).
+// Copies the pair's entropy-coded bytes into P.ubuf with the zero byte after every 0xFF
+// removed, bytes of each aligned group of four stored in reverse (big-endian words), at the
+// same start offset as in the record.  Records, in offsets of that copy, the first byte of every
+// restart interval (the byte after each RSTn marker) plus one final entry = end of data + 2, so
+// interval j spans [seg[j], seg[j+1] - 2).  Lanes take 16-byte slices; positions come from a
+// warp prefix sum of the bytes each slice keeps.
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) seg_index_kernel(Params P, int nscans) {
-    int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    int lane = threadIdx.x & 31;
+__global__ void __launch_bounds__(256) unstuff_index_kernel(Params P, int nscans) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
     if (warp >= nscans * P.N) return;
     const ScanDesc sd = P.scans[warp];
-    int img = warp % P.N;
+    const int img = warp % P.N;
     uint32_t* seg = P.seg_start + sd.seg_base;
-    if (lane == 0) seg[0] = sd.data_off;
-    if (sd.nseg <= 1) return;
-    uint32_t a = sd.data_off, b = sd.data_end;
-    uint32_t found = 0;  // markers seen so far (warp uniform)
+    const uint32_t a = sd.data_off, b = sd.data_end;
+    if (lane == 0) seg[0] = a;
+    uint32_t found = 0;      // markers seen so far (warp uniform)
+    uint32_t kept = 0;       // bytes written so far (warp uniform)
     for (uint32_t p0 = a & ~15u; p0 < b; p0 += 512) {
-        uint32_t p = p0 + 16u * lane;
+        const uint32_t p = p0 + 16u * lane;
         uint4 v = make_uint4(0, 0, 0, 0);
-        uint32_t nxt = 0;
+        uint32_t nxt = 0, prev = 0;
         if (p < b) v = __ldg(reinterpret_cast<const uint4*>(P.rec + p));   // chunks are padded to 16 bytes
         if (p + 16 < b) nxt = __ldg(P.rec + p + 16);
-        uint32_t w[5] = {v.x, v.y, v.z, v.w, nxt};
-        uint32_t mask = 0;
+        if (p > a && p < b) prev = __ldg(P.rec + p - 1);
+        const uint32_t w[5] = {v.x, v.y, v.z, v.w, nxt};
+        uint32_t keep = 0, mark = 0;
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-            uint32_t c0 = (w[j >> 2] >> (8 * (j & 3))) & 255u;
-            uint32_t c1 = (w[(j + 1) >> 2] >> (8 * ((j + 1) & 3))) & 255u;
-            uint32_t q = p + j;
-            if (c0 == 0xFFu && (c1 & 0xF8u) == 0xD0u && q >= a && q + 1 < b) mask |= 1u << j;
+            const uint32_t c0 = (w[j >> 2] >> (8 * (j & 3))) & 255u;
+            const uint32_t c1 = (w[(j + 1) >> 2] >> (8 * ((j + 1) & 3))) & 255u;
+            const uint32_t cp = j ? (w[(j - 1) >> 2] >> (8 * ((j - 1) & 3))) & 255u : prev;
+            const uint32_t q = p + j;
+            const bool in = q >= a && q < b;
+            if (in && !(c0 == 0u && cp == 0xFFu && q > a)) keep |= 1u << j;
+            if (in && q + 1 < b && c0 == 0xFFu && (c1 & 0xF8u) == 0xD0u) mark |= 1u << j;
         }
-        uint32_t cnt = __popc(mask), incl = cnt;
+        // exclusive prefix sums over lanes of kept bytes and of markers
+        uint32_t kc = __popc(keep), mc = __popc(mark), kin = kc, min_ = mc;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
-            uint32_t o = __shfl_up_sync(0xffffffffu, incl, d);
-            if (lane >= d) incl += o;
+            const uint32_t ok = __shfl_up_sync(0xffffffffu, kin, d), om = __shfl_up_sync(0xffffffffu, min_, d);
+            if (lane >= d) { kin += ok; min_ += om; }
         }
-        uint32_t ord = found + incl - cnt;
-        while (mask) {
-            int j = __ffs(mask) - 1;
-            mask &= mask - 1;
-            ++ord;
-            if (ord < sd.nseg) seg[ord] = p + j + 2;
+        const uint32_t obase = a + kept + kin - kc;
+        uint32_t ord = found + min_ - mc;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            if ((keep >> j) & 1u) {
+                const uint32_t o = obase + __popc(keep & ((1u << j) - 1u));
+                P.ubuf[o ^ 3u] = (uint8_t)((w[j >> 2] >> (8 * (j & 3))) & 255u);
+                if ((mark >> j) & 1u) {
+                    ++ord;
+                    if (ord < sd.nseg) seg[ord] = o + 2;
+                }
+            }
         }
-        found += __shfl_sync(0xffffffffu, incl, 31);
+        kept += __shfl_sync(0xffffffffu, kin, 31);
+        found += __shfl_sync(0xffffffffu, min_, 31);
     }
-    if (lane == 0 && found != sd.nseg - 1) atomicMin(&P.status[img], kErrCorrupt);
+    if (lane == 0) {
+        seg[sd.nseg] = a + kept + 2;
+        if (found != sd.nseg - 1) atomicMin(&P.status[img], kErrCorrupt);
+    }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -212,19 +200,27 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
     const uint32_t it = blockIdx.x * kEntropyWarps + wid;
     if (it >= item_count) return;
     const Item item = P.items[item_begin + it];
-    const ScanDesc sd = P.scans[item.si];
-    const int s = item.si / P.N, img = item.si % P.N;
+    const ScanDesc sd0 = P.scans[item.si];
+    const int s = item.si / P.N;
     const ScanScript sc = P.script[s];
-    const ImgDesc im = P.imgs[img];
-    const Geometry g = make_geometry(im);
     const bool dc = sc.Ss == 0;
     const bool huff = !(dc && sc.Ah != 0);
+    // tables: a DC scan may use two tables of one image; an AC item may span two images
+    const bool two_images = item.rsvd != 0;
     if (huff) {
-        build_hufftab(tabs[wid][0], P.rec + sd.tab_off[0], lane);
-        if (sd.tab_off[1]) build_hufftab(tabs[wid][1], P.rec + sd.tab_off[1], lane);
+        build_hufftab(tabs[wid][0], P.rec + sd0.tab_off[0], lane);
+        if (two_images) build_hufftab(tabs[wid][1], P.rec + P.scans[item.si + 1].tab_off[0], lane);
+        else if (sd0.tab_off[1]) build_hufftab(tabs[wid][1], P.rec + sd0.tab_off[1], lane);
     }
-    const uint32_t seg = item.seg0 + lane;
-    if ((uint32_t)lane >= item.count || seg >= sd.nseg) return;
+    if ((uint32_t)lane >= item.count) return;
+    const uint32_t rem0 = sd0.nseg - item.seg0;           // restart intervals left in the first image
+    const int which = (two_images && (uint32_t)lane >= rem0) ? 1 : 0;
+    const uint32_t seg = which ? (uint32_t)lane - rem0 : item.seg0 + lane;
+    const ScanDesc sd = which ? P.scans[item.si + 1] : sd0;
+    const int img = (int)(item.si % P.N) + which;
+    if (seg >= sd.nseg) return;
+    const ImgDesc im = P.imgs[img];
+    const Geometry g = make_geometry(im);
 
     const bool inter = sc.ncomp > 1;
     const int c0 = sc.comp[0];
@@ -235,13 +231,16 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
     const uint32_t m1 = sd.ri ? min(m0 + sd.ri, total) : total;
     const uint32_t* segtab = P.seg_start + sd.seg_base;
     const uint32_t bstart = segtab[seg];
-    const uint32_t bend = (seg + 1 < sd.nseg) ? segtab[seg + 1] - 2 : sd.data_end;
+    const uint32_t bend = segtab[seg + 1] - 2;
     if (bstart < sd.data_off || bend > sd.data_end || bend < bstart) {   // a missing marker left a hole
         atomicMin(&P.status[img], kErrCorrupt);
         return;
     }
     BitReader br;
-    br.init(P.rec, bstart, bend);
+    const uint32_t wbase = sd.data_off & ~3u;
+    br.w = reinterpret_cast<const uint32_t*>(P.ubuf + wbase);
+    br.pos = (bstart - wbase) * 8;
+    br.end = (bend - wbase) * 8;
     bool bad = false;
     const int Al = sc.Al, p1 = 1 << sc.Al;
 
@@ -257,17 +256,20 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
                 for (int sub = 0; sub < hv * hv; ++sub) {
                     const uint64_t blk = g.coff[c] + (uint64_t)(mrow * hv + (sub >> (hv - 1))) * g.bw[c] + mcol * hv + (sub & (hv - 1));
                     int16_t* cf = P.planes + blk * 64;
-                    br.refill();
+                    if (br.overran()) { bad = true; break; }
+                    const uint32_t win = br.peek();
                     if (sc.Ah == 0) {
-                        const int sz = huff_decode(tab, br, bad);
-                        if (sz > 15) bad = true;
-                        if (bad) break;
-                        const int d = extend_bits(br.take(sz), sz);
+                        const uint32_t e = huff_lookup(tab, win);
+                        const int len = (int)(e >> 8), sz = (int)(e & 255u);
+                        if (e == 0 || sz > 15) { bad = true; break; }
+                        const int d = extend_bits(top_bits(win << len, sz), sz);
+                        br.pos += len + sz;
                         int pv = (c == 0 ? pred0 : (c == 1 ? pred1 : pred2)) + d;
                         if (c == 0) pred0 = pv; else if (c == 1) pred1 = pv; else pred2 = pv;
                         cf[0] = (int16_t)(pv << Al);
                     } else {
-                        if (br.take(1)) cf[0] = (int16_t)(cf[0] | p1);
+                        if (win >> 31) cf[0] = (int16_t)(cf[0] | p1);
+                        br.pos += 1;
                     }
                 }
                 if (bad) break;
@@ -275,40 +277,47 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
             if (++mcol == mcu_w) { mcol = 0; ++mrow; }
         }
     } else {
-        const HuffTab& tab = tabs[wid][0];
+        const HuffTab& tab = tabs[wid][which];
         const int c = c0, Ss = sc.Ss, Se = sc.Se;
         const ScanAux ax = P.saux[s];
         const uint32_t bw = g.bw[c];
-        uint32_t m = m0, brow = m0 / mcu_w, bcol = m0 % mcu_w;
+        const uint32_t wrap = bw - mcu_w + 1;              // step of the block index at the end of a block row
+        uint32_t m = m0, bcol = m0 % mcu_w;
+        uint32_t bi = (m0 / mcu_w) * bw + bcol;            // block index inside the image's component
         uint32_t eobrun = 0;
         int k = Ss;
         if (sc.Ah == 0) {
             // ---- AC first pass: one Huffman symbol per iteration
             uint64_t* maskp = P.aux + ax.base + g.loff[c];
+            int16_t* plane = P.planes + g.coff[c] * 64;
             uint64_t M = 0;
-            while (m < m1 && !bad) {
-                br.refill();
-                const int rs = huff_decode(tab, br, bad);
-                if (bad) break;
-                const int r = rs >> 4, sz = rs & 15;
+            while (m < m1) {
+                if (br.overran()) { bad = true; break; }
+                const uint32_t win = br.peek();
+                const uint32_t e = huff_lookup(tab, win);
+                if (e == 0) { bad = true; break; }
+                const int len = (int)(e >> 8), r = (int)(e >> 4) & 15, sz = (int)(e & 15u);
+                const uint32_t rest = win << len;
                 bool done;
                 if (sz) {
                     k += r;
                     if (k > Se) { bad = true; break; }
-                    const int v = extend_bits(br.take(sz), sz) * p1;
-                    P.planes[(g.coff[c] + (uint64_t)brow * bw + bcol) * 64 + k] = (int16_t)v;
+                    plane[(uint64_t)bi * 64 + k] = (int16_t)(extend_bits(top_bits(rest, sz), sz) * p1);
+                    br.pos += len + sz;
                     M |= 1ull << k;
                     ++k;
                     done = k > Se;
                 } else if (r == 15) {
+                    br.pos += len;
                     k += 16;
                     done = k > Se;
                 } else {
-                    eobrun = (1u << r) + (r ? br.take(r) : 0u) - 1u;
+                    eobrun = (1u << r) + top_bits(rest, r) - 1u;
+                    br.pos += len + r;
                     done = true;
                 }
                 if (done) {
-                    if (M) maskp[(uint64_t)brow * bw + bcol] = M;
+                    if (M) maskp[bi] = M;
                     uint32_t adv = 1;
                     if (eobrun) {                      // the following blocks of the run are empty
                         const uint32_t extra = min(eobrun, m1 - (m + 1));
@@ -316,52 +325,59 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
                         adv += extra;
                     }
                     m += adv;
-                    if (adv == 1) { if (++bcol == mcu_w) { bcol = 0; ++brow; } }
-                    else { brow = m / mcu_w; bcol = m % mcu_w; }
+                    if (adv == 1) { if (++bcol == mcu_w) { bcol = 0; bi += wrap; } else ++bi; }
+                    else { bcol = m % mcu_w; bi = (m / mcu_w) * bw + bcol; }
                     k = Ss; M = 0;
                 }
             }
         } else {
             // ---- AC refinement: one Huffman symbol, or one block of an end-of-band run, per iteration
             const uint64_t band = low_mask(Se + 1) & ~low_mask(Ss);
-            const uint64_t* srcp[4];
-            uint32_t srcs[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const ScanAux sx = P.saux[ax.src[i < ax.nsrc ? i : 0]];
-                srcp[i] = P.aux + sx.base + (uint64_t)g.loff[c] * sx.stride;
-                srcs[i] = sx.stride;
+            const uint64_t* src0 = nullptr; const uint64_t* src1 = nullptr; const uint64_t* src2 = nullptr; const uint64_t* src3 = nullptr;
+            uint32_t st0 = 0, st1 = 0, st2 = 0, st3 = 0;
+            {
+                const ScanAux x0 = P.saux[ax.src[0]];
+                src0 = P.aux + x0.base + g.loff[c] * x0.stride; st0 = x0.stride;
+                if (ax.nsrc > 1) { const ScanAux x = P.saux[ax.src[1]]; src1 = P.aux + x.base + g.loff[c] * x.stride; st1 = x.stride; }
+                if (ax.nsrc > 2) { const ScanAux x = P.saux[ax.src[2]]; src2 = P.aux + x.base + g.loff[c] * x.stride; st2 = x.stride; }
+                if (ax.nsrc > 3) { const ScanAux x = P.saux[ax.src[3]]; src3 = P.aux + x.base + g.loff[c] * x.stride; st3 = x.stride; }
             }
             uint64_t* outp = P.aux + ax.base + g.loff[c] * 4ull;
-            auto load_hist = [&](uint32_t row, uint32_t col) -> uint64_t {
-                const uint64_t bi = (uint64_t)row * bw + col;
-                uint64_t h = srcp[0][bi * srcs[0]];
-                if (ax.nsrc > 1) h |= srcp[1][bi * srcs[1]];
-                if (ax.nsrc > 2) h |= srcp[2][bi * srcs[2]];
-                if (ax.nsrc > 3) h |= srcp[3][bi * srcs[3]];
+            auto load_hist = [&](uint32_t b) -> uint64_t {
+                uint64_t h = src0[(uint64_t)b * st0];
+                if (src1) h |= src1[(uint64_t)b * st1];
+                if (src2) h |= src2[(uint64_t)b * st2];
+                if (src3) h |= src3[(uint64_t)b * st3];
                 return h & band;
             };
-            uint64_t H = load_hist(brow, bcol);
-            uint32_t nrow = brow, ncol = bcol + 1;
-            if (ncol == mcu_w) { ncol = 0; ++nrow; }
-            uint64_t Hn = (m + 1 < m1) ? load_hist(nrow, ncol) : 0ull;      // the next block's mask is already in flight
+            uint64_t H = load_hist(bi);
+            uint32_t ncol = bcol + 1, nbi = bi + 1;
+            if (ncol == mcu_w) { ncol = 0; nbi = bi + wrap; }
+            uint64_t Hn = (m + 1 < m1) ? load_hist(nbi) : 0ull;      // the next block's mask is already in flight
             uint64_t cstr = 0, Nw = 0, NS = 0;
             int cn = 0;
-            while (m < m1 && !bad) {
+            while (m < m1) {
+                if (br.overran()) { bad = true; break; }
                 bool eob = eobrun > 0;
                 int r = 0, sz = 0;
                 uint32_t sign = 0;
                 if (!eob) {
-                    br.refill();
-                    const int rs = huff_decode(tab, br, bad);
-                    if (bad) break;
-                    r = rs >> 4; sz = rs & 15;
+                    const uint32_t win = br.peek();
+                    const uint32_t e = huff_lookup(tab, win);
+                    if (e == 0) { bad = true; break; }
+                    const int len = (int)(e >> 8);
+                    r = (int)(e >> 4) & 15; sz = (int)(e & 15u);
+                    const uint32_t rest = win << len;
                     if (sz) {
                         if (sz != 1) { bad = true; break; }
-                        sign = br.take(1);
+                        sign = rest >> 31;
+                        br.pos += len + 1;
                     } else if (r < 15) {
-                        eobrun = (1u << r) + (r ? br.take(r) : 0u);
+                        eobrun = (1u << r) + top_bits(rest, r);
+                        br.pos += len + r;
                         eob = true;
+                    } else {
+                        br.pos += len;
                     }
                 }
                 const uint64_t from = ~0ull << k;                      // k <= Se <= 63 here
@@ -375,9 +391,9 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
                 const int n = __popcll(hist);
                 if (n) {
                     if (cn + n > 64) { bad = true; break; }
-                    br.refill();
-                    uint64_t bits = br.take(min(n, 32));
-                    if (n > 32) { br.refill(); bits = (bits << (n - 32)) | br.take(n - 32); }
+                    uint64_t bits = top_bits(br.peek(), min(n, 32));
+                    br.pos += min(n, 32);
+                    if (n > 32) { bits = (bits << (n - 32)) | top_bits(br.peek(), n - 32); br.pos += n - 32; }
                     cstr |= bits << (64 - cn - n);
                     cn += n;
                 }
@@ -385,14 +401,14 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
                 k = pos + 1;
                 if (eob) --eobrun;
                 if (k > Se) {                                          // block finished
-                    uint64_t* o = outp + ((uint64_t)brow * bw + bcol) * 4;
+                    uint64_t* o = outp + (uint64_t)bi * 4;
                     *reinterpret_cast<ulonglong2*>(o) = make_ulonglong2(H | Nw, cstr);
                     *reinterpret_cast<ulonglong2*>(o + 2) = make_ulonglong2(Nw, NS);
                     ++m;
-                    brow = nrow; bcol = ncol;
+                    bi = nbi;
                     H = Hn;
-                    if (++ncol == mcu_w) { ncol = 0; ++nrow; }
-                    if (m + 1 < m1) Hn = load_hist(nrow, ncol);
+                    if (++ncol == mcu_w) { ncol = 0; nbi += wrap; } else ++nbi;
+                    if (m + 1 < m1) Hn = load_hist(nbi);
                     k = Ss; cstr = 0; Nw = 0; NS = 0; cn = 0;
                 }
             }

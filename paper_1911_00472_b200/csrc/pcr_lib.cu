@@ -44,6 +44,7 @@ struct pcr_record {
     // device state
     int device = 0;
     uint8_t* d_rec = nullptr;
+    uint8_t* d_ubuf = nullptr;
     size_t resident = 0;
     int16_t* d_planes = nullptr;
     ScanScript* d_script = nullptr;
@@ -202,7 +203,7 @@ int parse_chunk(const uint8_t* rec, uint64_t off, uint32_t len, bool first, Imag
 void free_device(pcr_record* r) {
     for (cudaEvent_t e : r->events) cudaEventDestroy(e);
     r->events.clear();
-    cudaFree(r->d_rec); cudaFree(r->d_planes); cudaFree(r->d_script); cudaFree(r->d_saux); cudaFree(r->d_aux); cudaFree(r->d_scans);
+    cudaFree(r->d_rec); cudaFree(r->d_ubuf); cudaFree(r->d_planes); cudaFree(r->d_script); cudaFree(r->d_saux); cudaFree(r->d_aux); cudaFree(r->d_scans);
     cudaFree(r->d_imgs); cudaFree(r->d_seg); cudaFree(r->d_items); cudaFree(r->d_units);
     cudaFree(r->d_qtab); cudaFree(r->d_status);
 }
@@ -272,7 +273,7 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
             }
             sd.nseg = sd.ri ? (uint32_t)((total_mcu + sd.ri - 1) / sd.ri) : 1u;
             sd.seg_base = (uint32_t)segs;
-            segs += sd.nseg;
+            segs += sd.nseg + 1;                      // one closing entry per (scan, image)
             if (segs >= (1ull << 32)) return PCR_E_FORMAT;
         }
         if (!im.have_frame) return PCR_E_FORMAT;
@@ -318,12 +319,23 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
             r->scan_item_begin[s] = (uint32_t)items.size();
             for (uint32_t i = 0; i < N; ++i) {
                 const ScanDesc& sd = scans[(size_t)s * N + i];
-                // split the restart intervals evenly over as few warps as needed
-                const uint32_t parts = (sd.nseg + kSegsPerItem - 1) / kSegsPerItem;
-                const uint32_t per = (sd.nseg + parts - 1) / parts;
-                for (uint32_t j = 0; j < sd.nseg; j += per)
-                    items.push_back(Item{(uint32_t)(s * N + i), j, std::min(per, sd.nseg - j), 0u});
+                // full warps of 32 restart intervals; in AC scans the last warp of an image
+                // runs on into the first intervals of the next image (two tables per warp)
+                const bool ac = r->script[s].Ss > 0;
+                uint32_t j = 0;
+                if (ac && !items.empty() && items.back().rsvd == 2) {     // continued from the previous image
+                    Item& prev = items.back();
+                    const uint32_t take = std::min<uint32_t>(kSegsPerItem - prev.count, sd.nseg);
+                    prev.count += take; prev.rsvd = 1;
+                    j = take;
+                }
+                for (; j < sd.nseg; j += kSegsPerItem) {
+                    const uint32_t cnt = std::min<uint32_t>(kSegsPerItem, sd.nseg - j);
+                    // rsvd == 2 marks an unfilled last item that the next image may extend
+                    items.push_back(Item{(uint32_t)(s * N + i), j, cnt, (ac && cnt < (uint32_t)kSegsPerItem && i + 1 < N) ? 2u : 0u});
+                }
             }
+            if (!items.empty() && items.back().rsvd == 2) items.back().rsvd = 0;
             r->scan_item_count[s] = (uint32_t)items.size() - r->scan_item_begin[s];
         }
     std::vector<Unit> units;
@@ -377,6 +389,8 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     if (cudaMalloc(reinterpret_cast<void**>(&r->d_aux), std::max<uint64_t>(aux_words, 2) * 8) != cudaSuccess) { r->d_aux = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
     if (cudaMemset(r->d_aux, 0, std::max<uint64_t>(aux_words, 2) * 8) != cudaSuccess) return PCR_E_CUDA;
     if (cudaMalloc(reinterpret_cast<void**>(&r->d_rec), len + 64) != cudaSuccess) { r->d_rec = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
+    if (cudaMalloc(reinterpret_cast<void**>(&r->d_ubuf), len + 64) != cudaSuccess) { r->d_ubuf = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
+    if (cudaMemset(r->d_ubuf, 0, len + 64) != cudaSuccess) return PCR_E_CUDA;
     if (cudaMalloc(reinterpret_cast<void**>(&r->d_planes), std::max<uint64_t>(blocks, 1) * 128) != cudaSuccess) { r->d_planes = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
     if (cudaMalloc(reinterpret_cast<void**>(&r->d_seg), (segs + 1) * 4) != cudaSuccess) { r->d_seg = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
     if (cudaMalloc(reinterpret_cast<void**>(&r->d_status), (size_t)N * 4) != cudaSuccess) { r->d_status = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
@@ -467,13 +481,13 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
     if (cudaMemsetAsync(rec->d_planes, 0, rec->total_blocks * 128, st) != cudaSuccess) return PCR_E_CUDA;
     mark("clear", 0);
     Params P;
-    P.rec = rec->d_rec; P.planes = rec->d_planes; P.script = rec->d_script; P.scans = rec->d_scans;
+    P.rec = rec->d_rec; P.ubuf = rec->d_ubuf; P.planes = rec->d_planes; P.script = rec->d_script; P.scans = rec->d_scans;
     P.saux = rec->d_saux; P.aux = rec->d_aux;
     P.imgs = rec->d_imgs; P.seg_start = rec->d_seg; P.items = rec->d_items; P.units = rec->d_units;
     P.qtab = rec->d_qtab; P.status = rec->d_status; P.N = rec->N;
     {
         uint32_t warps = (uint32_t)k * (uint32_t)rec->N;
-        seg_index_kernel<<<(warps + 7) / 8, 256, 0, st>>>(P, k);
+        unstuff_index_kernel<<<(warps + 7) / 8, 256, 0, st>>>(P, k);
         ++g_launches;
         mark("index", 1);
     }

@@ -64,7 +64,7 @@ struct Item {
     uint32_t si;          // scan * N + image
     uint32_t seg0;        // first restart interval of the item
     uint32_t count;       // restart intervals in the item (<= kSegsPerItem)
-    uint32_t rsvd;
+    uint32_t rsvd;        // 1: the item runs on into the first intervals of the next image
 };
 
 // Pixel work unit: a run of MCUs in one MCU row of one image.
@@ -75,6 +75,7 @@ struct Unit {
 
 struct Params {
     const uint8_t* rec;         // record bytes on the device
+    uint8_t* ubuf;              // entropy-coded bytes without stuffing, big-endian words
     int16_t* planes;            // coefficient planes, 64 int16 per block, zigzag order
     const ScanScript* script;   // [G]
     const ScanAux* saux;        // [G]
