@@ -66,18 +66,47 @@ __device__ __forceinline__ void build_hufftab(HuffTab& t, const uint8_t* __restr
 }
 
 // MSB-first bit reader over the unstuffed copy of the entropy-coded bytes (see
-// unstuff_index_kernel): the copy holds big-endian 32-bit words, so the next 32 bits at any
-// bit position are two aligned word loads and one funnel shift, and consuming bits is an add.
+// unstuff_index_kernel), which holds big-endian 32-bit words.  Each lane streams its restart
+// interval through registers: one 16-byte load per 128 bits, issued one step ahead of its use,
+// so the serial decode chain never waits on memory and every sector is fetched once (32 lanes
+// reading 32 different streams would otherwise thrash the small L1 left beside the tables).
 struct BitReader {
-    const uint32_t* w;   // word 0 of the (scan, image) chunk in the unstuffed copy
-    uint32_t pos;        // next bit, relative to w
-    uint32_t end;        // first bit past the restart interval
+    const uint4* base;   // 16-byte aligned start of the chunk's region in the copy
+    uint32_t q;          // next 16-byte group to fetch
+    uint4 cur, nxt;      // group being consumed, group already in flight
+    uint32_t wi;         // next word of cur
+    uint64_t buf;        // left-aligned bit buffer
+    int nbits;           // bits held in buf
+    uint32_t loaded;     // bits moved into buf so far
+    uint32_t limit;      // bits in the restart interval
 
-    __device__ __forceinline__ uint32_t peek() const {
-        const uint32_t i = pos >> 5;
-        return __funnelshift_l(__ldg(w + i + 1), __ldg(w + i), pos);
+    __device__ __forceinline__ void init(const uint8_t* ubuf, uint32_t bstart, uint32_t bend) {
+        base = reinterpret_cast<const uint4*>(ubuf);
+        q = bstart >> 4;
+        cur = __ldg(base + q);
+        nxt = __ldg(base + q + 1);
+        q += 2;
+        wi = (bstart >> 2) & 3u;
+        buf = 0; nbits = 0; loaded = 0;
+        limit = (bend - bstart) * 8u;
+        // the first word may start before the interval: drop those bytes
+        const uint32_t lead = 8u * (bstart & 3u);
+        refill();
+        buf <<= lead; nbits -= (int)lead; loaded -= lead;
     }
-    __device__ __forceinline__ bool overran() const { return pos > end; }
+    // afterwards at least 33 bits are held (call before every symbol and before every run of
+    // up to 32 raw bits)
+    __device__ __forceinline__ void refill() {
+        if (nbits <= 32) {
+            const uint32_t w = wi == 0 ? cur.x : (wi == 1 ? cur.y : (wi == 2 ? cur.z : cur.w));
+            buf |= (uint64_t)w << (32 - nbits);
+            nbits += 32; loaded += 32;
+            if (++wi == 4) { wi = 0; cur = nxt; nxt = __ldg(base + q); ++q; }
+        }
+    }
+    __device__ __forceinline__ uint32_t top32() const { return (uint32_t)(buf >> 32); }
+    __device__ __forceinline__ void skip(int n) { buf <<= n; nbits -= n; }
+    __device__ __forceinline__ bool overran() const { return (int)(loaded - (uint32_t)nbits) > (int)limit; }
 };
 
 // Huffman symbol at the top of the 32-bit window; returns (length << 8) | symbol, 0 if undefined
@@ -108,12 +137,12 @@ __device__ __forceinline__ uint32_t top_bits(uint32_t x, int n) { return n ? x >
 // interval j spans [seg[j], seg[j+1] - 2).  Lanes take 16-byte slices; positions come from a
 // warp prefix sum of the bytes each slice keeps.
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) unstuff_index_kernel(Params P, int nscans) {
+__global__ void __launch_bounds__(256) unstuff_index_kernel(Params P, int nscans, int img0, int nimg) {
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
-    if (warp >= nscans * P.N) return;
-    const ScanDesc sd = P.scans[warp];
-    const int img = warp % P.N;
+    if (warp >= nscans * nimg) return;
+    const int img = img0 + warp % nimg;
+    const ScanDesc sd = P.scans[(warp / nimg) * P.N + img];
     uint32_t* seg = P.seg_start + sd.seg_base;
     const uint32_t a = sd.data_off, b = sd.data_end;
     if (lane == 0) seg[0] = a;
@@ -194,6 +223,22 @@ __device__ __forceinline__ Geometry make_geometry(const ImgDesc& im) {
 
 __device__ __forceinline__ uint64_t low_mask(int p) { return p >= 64 ? ~0ull : ((1ull << p) - 1ull); }
 
+// position of the (r+1)-th set bit of z, or 64 if z has fewer: a fixed five-step search on
+// population counts, so lanes with different r stay converged
+__device__ __forceinline__ int select_bit(uint64_t z, int r) {
+    const uint32_t lo = (uint32_t)z, hi = (uint32_t)(z >> 32);
+    int c = __popc(lo), base = 0;
+    uint32_t x = lo;
+    if (r >= c) { r -= c; x = hi; base = 32; }
+    const bool none = r >= __popc(x);
+    c = __popc(x & 0xFFFFu); if (r >= c) { r -= c; x >>= 16; base += 16; }
+    c = __popc(x & 0xFFu);   if (r >= c) { r -= c; x >>= 8;  base += 8; }
+    c = __popc(x & 0xFu);    if (r >= c) { r -= c; x >>= 4;  base += 4; }
+    c = __popc(x & 0x3u);    if (r >= c) { r -= c; x >>= 2;  base += 2; }
+    if (r >= (int)(x & 1u)) base += 1;
+    return none ? 64 : base;
+}
+
 __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, uint32_t item_begin, uint32_t item_count) {
     __shared__ HuffTab tabs[kEntropyWarps][2];
     const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -237,10 +282,7 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
         return;
     }
     BitReader br;
-    const uint32_t wbase = sd.data_off & ~3u;
-    br.w = reinterpret_cast<const uint32_t*>(P.ubuf + wbase);
-    br.pos = (bstart - wbase) * 8;
-    br.end = (bend - wbase) * 8;
+    br.init(P.ubuf, bstart, bend);
     bool bad = false;
     const int Al = sc.Al, p1 = 1 << sc.Al;
 
@@ -257,19 +299,20 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
                     const uint64_t blk = g.coff[c] + (uint64_t)(mrow * hv + (sub >> (hv - 1))) * g.bw[c] + mcol * hv + (sub & (hv - 1));
                     int16_t* cf = P.planes + blk * 64;
                     if (br.overran()) { bad = true; break; }
-                    const uint32_t win = br.peek();
+                    br.refill();
+                    const uint32_t win = br.top32();
                     if (sc.Ah == 0) {
                         const uint32_t e = huff_lookup(tab, win);
                         const int len = (int)(e >> 8), sz = (int)(e & 255u);
                         if (e == 0 || sz > 15) { bad = true; break; }
                         const int d = extend_bits(top_bits(win << len, sz), sz);
-                        br.pos += len + sz;
+                        br.skip(len + sz);
                         int pv = (c == 0 ? pred0 : (c == 1 ? pred1 : pred2)) + d;
                         if (c == 0) pred0 = pv; else if (c == 1) pred1 = pv; else pred2 = pv;
                         cf[0] = (int16_t)(pv << Al);
                     } else {
                         if (win >> 31) cf[0] = (int16_t)(cf[0] | p1);
-                        br.pos += 1;
+                        br.skip(1);
                     }
                 }
                 if (bad) break;
@@ -293,7 +336,8 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
             uint64_t M = 0;
             while (m < m1) {
                 if (br.overran()) { bad = true; break; }
-                const uint32_t win = br.peek();
+                br.refill();
+                const uint32_t win = br.top32();
                 const uint32_t e = huff_lookup(tab, win);
                 if (e == 0) { bad = true; break; }
                 const int len = (int)(e >> 8), r = (int)(e >> 4) & 15, sz = (int)(e & 15u);
@@ -303,17 +347,17 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
                     k += r;
                     if (k > Se) { bad = true; break; }
                     plane[(uint64_t)bi * 64 + k] = (int16_t)(extend_bits(top_bits(rest, sz), sz) * p1);
-                    br.pos += len + sz;
+                    br.skip(len + sz);
                     M |= 1ull << k;
                     ++k;
                     done = k > Se;
                 } else if (r == 15) {
-                    br.pos += len;
+                    br.skip(len);
                     k += 16;
                     done = k > Se;
                 } else {
                     eobrun = (1u << r) + top_bits(rest, r) - 1u;
-                    br.pos += len + r;
+                    br.skip(len + r);
                     done = true;
                 }
                 if (done) {
@@ -362,7 +406,8 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
                 int r = 0, sz = 0;
                 uint32_t sign = 0;
                 if (!eob) {
-                    const uint32_t win = br.peek();
+                    br.refill();
+                    const uint32_t win = br.top32();
                     const uint32_t e = huff_lookup(tab, win);
                     if (e == 0) { bad = true; break; }
                     const int len = (int)(e >> 8);
@@ -371,29 +416,26 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
                     if (sz) {
                         if (sz != 1) { bad = true; break; }
                         sign = rest >> 31;
-                        br.pos += len + 1;
+                        br.skip(len + 1);
                     } else if (r < 15) {
                         eobrun = (1u << r) + top_bits(rest, r);
-                        br.pos += len + r;
+                        br.skip(len + r);
                         eob = true;
                     } else {
-                        br.pos += len;
+                        br.skip(len);
                     }
                 }
                 const uint64_t from = ~0ull << k;                      // k <= Se <= 63 here
                 int pos = Se + 1;
-                if (!eob) {
-                    uint64_t Z = ~H & band & from;                     // zero-valued positions still ahead
-                    for (; r > 0 && Z; --r) Z &= Z - 1;                // pass over r of them
-                    if (Z) pos = __ffsll((long long)Z) - 1;
-                }
+                if (!eob) pos = min(Se + 1, select_bit(~H & band & from, r));   // pass over r zero-valued positions
                 const uint64_t hist = H & from & low_mask(pos);        // non-zero positions passed: one correction bit each
                 const int n = __popcll(hist);
                 if (n) {
                     if (cn + n > 64) { bad = true; break; }
-                    uint64_t bits = top_bits(br.peek(), min(n, 32));
-                    br.pos += min(n, 32);
-                    if (n > 32) { bits = (bits << (n - 32)) | top_bits(br.peek(), n - 32); br.pos += n - 32; }
+                    br.refill();
+                    uint64_t bits = top_bits(br.top32(), min(n, 32));
+                    br.skip(min(n, 32));
+                    if (n > 32) { br.refill(); bits = (bits << (n - 32)) | top_bits(br.top32(), n - 32); br.skip(n - 32); }
                     cstr |= bits << (64 - cn - n);
                     cn += n;
                 }

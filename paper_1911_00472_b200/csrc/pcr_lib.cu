@@ -38,7 +38,15 @@ struct pcr_record {
     std::vector<ScanScript> script;
     std::vector<int> wave_of_scan;
     int n_waves = 0;
-    std::vector<uint32_t> scan_item_begin, scan_item_count;   // in the (wave, scan)-sorted item list
+    // images are cut into slices that run as independent pipelines on their own streams;
+    // items are sorted by (slice, wave, scan), units by image
+    int n_slices = 1;
+    std::vector<uint32_t> slice_img;                            // [n_slices + 1] first image of each slice
+    std::vector<uint32_t> slice_unit;                           // [n_slices + 1] first pixel unit of each slice
+    std::vector<uint32_t> item_begin, item_count;               // [n_slices][G]
+    std::vector<cudaStream_t> streams;                          // one per slice
+    cudaEvent_t ev_fork = nullptr;
+    std::vector<cudaEvent_t> ev_join;
     std::vector<std::vector<int>> wave_scans;
     uint32_t n_units = 0;
     // device state
@@ -201,6 +209,12 @@ int parse_chunk(const uint8_t* rec, uint64_t off, uint32_t len, bool first, Imag
 }
 
 void free_device(pcr_record* r) {
+    for (cudaStream_t q : r->streams) cudaStreamDestroy(q);
+    r->streams.clear();
+    if (r->ev_fork) cudaEventDestroy(r->ev_fork);
+    r->ev_fork = nullptr;
+    for (cudaEvent_t e : r->ev_join) cudaEventDestroy(e);
+    r->ev_join.clear();
     for (cudaEvent_t e : r->events) cudaEventDestroy(e);
     r->events.clear();
     cudaFree(r->d_rec); cudaFree(r->d_ubuf); cudaFree(r->d_planes); cudaFree(r->d_script); cudaFree(r->d_saux); cudaFree(r->d_aux); cudaFree(r->d_scans);
@@ -312,39 +326,53 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     }
     r->wave_scans.assign(r->n_waves, {});
     for (uint32_t s = 0; s < G; ++s) r->wave_scans[r->wave_of_scan[s]].push_back((int)s);
+    // slices: enough images each to fill the machine, few enough to keep launches cheap
+    {
+        int want = (int)std::min<uint32_t>(8, std::max<uint32_t>(1, N / 128));
+        if (const char* e = getenv("PCR_SLICES")) want = std::max(1, std::min(64, atoi(e)));
+        r->n_slices = (int)std::min<uint32_t>((uint32_t)want, N);
+        r->slice_img.resize(r->n_slices + 1);
+        for (int g = 0; g <= r->n_slices; ++g) r->slice_img[g] = (uint32_t)((uint64_t)N * g / r->n_slices);
+    }
     std::vector<Item> items;
-    r->scan_item_begin.assign(G, 0); r->scan_item_count.assign(G, 0);
-    for (int w = 0; w < r->n_waves; ++w)
-        for (int s : r->wave_scans[w]) {
-            r->scan_item_begin[s] = (uint32_t)items.size();
-            for (uint32_t i = 0; i < N; ++i) {
-                const ScanDesc& sd = scans[(size_t)s * N + i];
-                // full warps of 32 restart intervals; in AC scans the last warp of an image
-                // runs on into the first intervals of the next image (two tables per warp)
+    r->item_begin.assign((size_t)r->n_slices * G, 0); r->item_count.assign((size_t)r->n_slices * G, 0);
+    for (int g = 0; g < r->n_slices; ++g)
+        for (int w = 0; w < r->n_waves; ++w)
+            for (int s : r->wave_scans[w]) {
+                r->item_begin[(size_t)g * G + s] = (uint32_t)items.size();
                 const bool ac = r->script[s].Ss > 0;
-                uint32_t j = 0;
-                if (ac && !items.empty() && items.back().rsvd == 2) {     // continued from the previous image
-                    Item& prev = items.back();
-                    const uint32_t take = std::min<uint32_t>(kSegsPerItem - prev.count, sd.nseg);
-                    prev.count += take; prev.rsvd = 1;
-                    j = take;
+                for (uint32_t i = r->slice_img[g]; i < r->slice_img[g + 1]; ++i) {
+                    const ScanDesc& sd = scans[(size_t)s * N + i];
+                    // full warps of 32 restart intervals; in AC scans the last warp of an image
+                    // runs on into the first intervals of the next image (two tables per warp)
+                    uint32_t j = 0;
+                    if (ac && !items.empty() && items.back().rsvd == 2) {     // continued from the previous image
+                        Item& prev = items.back();
+                        const uint32_t take = std::min<uint32_t>(kSegsPerItem - prev.count, sd.nseg);
+                        prev.count += take; prev.rsvd = 1;
+                        j = take;
+                    }
+                    for (; j < sd.nseg; j += kSegsPerItem) {
+                        const uint32_t cnt = std::min<uint32_t>(kSegsPerItem, sd.nseg - j);
+                        // rsvd == 2 marks an unfilled last item that the next image may extend
+                        items.push_back(Item{(uint32_t)(s * N + i), j, cnt, (ac && cnt < (uint32_t)kSegsPerItem) ? 2u : 0u});
+                    }
                 }
-                for (; j < sd.nseg; j += kSegsPerItem) {
-                    const uint32_t cnt = std::min<uint32_t>(kSegsPerItem, sd.nseg - j);
-                    // rsvd == 2 marks an unfilled last item that the next image may extend
-                    items.push_back(Item{(uint32_t)(s * N + i), j, cnt, (ac && cnt < (uint32_t)kSegsPerItem && i + 1 < N) ? 2u : 0u});
-                }
+                if (!items.empty() && items.back().rsvd == 2) items.back().rsvd = 0;
+                r->item_count[(size_t)g * G + s] = (uint32_t)items.size() - r->item_begin[(size_t)g * G + s];
             }
-            if (!items.empty() && items.back().rsvd == 2) items.back().rsvd = 0;
-            r->scan_item_count[s] = (uint32_t)items.size() - r->scan_item_begin[s];
-        }
     std::vector<Unit> units;
-    for (uint32_t i = 0; i < N; ++i)
-        for (uint32_t row = 0; row < imgs[i].my; ++row)
-            for (uint32_t col = 0; col < imgs[i].mx; col += kPixMcus) {
-                if (imgs[i].my > 65535 || imgs[i].mx > 65535) return PCR_E_FORMAT;
-                units.push_back(Unit{i, (uint16_t)row, (uint16_t)col});
-            }
+    r->slice_unit.assign(r->n_slices + 1, 0);
+    for (int g = 0; g < r->n_slices; ++g) {
+        r->slice_unit[g] = (uint32_t)units.size();
+        for (uint32_t i = r->slice_img[g]; i < r->slice_img[g + 1]; ++i)
+            for (uint32_t row = 0; row < imgs[i].my; ++row)
+                for (uint32_t col = 0; col < imgs[i].mx; col += kPixMcus) {
+                    if (imgs[i].my > 65535 || imgs[i].mx > 65535) return PCR_E_FORMAT;
+                    units.push_back(Unit{i, (uint16_t)row, (uint16_t)col});
+                }
+    }
+    r->slice_unit[r->n_slices] = (uint32_t)units.size();
     r->n_units = (uint32_t)units.size();
 
     // side data of the AC scans: one word per block for a first pass, four for a refinement
@@ -405,6 +433,16 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     if ((rc = upload(&r->d_qtab, qtab))) return rc;
     r->h_status.assign(N, 0);
     r->resident = 0;
+    if (r->n_slices > 1) {
+        if (cudaEventCreateWithFlags(&r->ev_fork, cudaEventDisableTiming) != cudaSuccess) return PCR_E_CUDA;
+        for (int g = 0; g < r->n_slices; ++g) {
+            cudaStream_t q; cudaEvent_t e;
+            if (cudaStreamCreateWithFlags(&q, cudaStreamNonBlocking) != cudaSuccess) return PCR_E_CUDA;
+            r->streams.push_back(q);
+            if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return PCR_E_CUDA;
+            r->ev_join.push_back(e);
+        }
+    }
     return PCR_OK;
 }
 
@@ -478,60 +516,108 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
     }
     mark("h2d", 0);
     if (cudaMemsetAsync(rec->d_status, 0, (size_t)rec->N * 4, st) != cudaSuccess) return PCR_E_CUDA;
-    if (cudaMemsetAsync(rec->d_planes, 0, rec->total_blocks * 128, st) != cudaSuccess) return PCR_E_CUDA;
-    mark("clear", 0);
     Params P;
     P.rec = rec->d_rec; P.ubuf = rec->d_ubuf; P.planes = rec->d_planes; P.script = rec->d_script; P.scans = rec->d_scans;
     P.saux = rec->d_saux; P.aux = rec->d_aux;
     P.imgs = rec->d_imgs; P.seg_start = rec->d_seg; P.items = rec->d_items; P.units = rec->d_units;
     P.qtab = rec->d_qtab; P.status = rec->d_status; P.N = rec->N;
-    {
-        uint32_t warps = (uint32_t)k * (uint32_t)rec->N;
-        unstuff_index_kernel<<<(warps + 7) / 8, 256, 0, st>>>(P, k);
-        ++g_launches;
-        mark("index", 1);
-    }
-    for (int w = 0; w < rec->n_waves; ++w) {
-        uint32_t begin = 0, count = 0;
-        bool any = false;
-        for (int s : rec->wave_scans[w]) {
-            if (s >= k) break;   // scans of a wave are stored in ascending order
-            if (!any) { begin = rec->scan_item_begin[s]; any = true; }
-            count += rec->scan_item_count[s];
+    FinalizeList fl;
+    memset(&fl, 0, sizeof fl);
+    bool any_refine = false;
+    for (int s = 0; s < k; ++s) {
+        const ScanScript& sc = rec->script[s];
+        if (sc.Ss == 0 || sc.Ah == 0) continue;
+        const int c = sc.comp[0];
+        if (fl.n[c] < 4) {
+            fl.scan[c][fl.n[c]] = s;
+            fl.p1[c][fl.n[c]] = 1 << sc.Al;
+            fl.base[c][fl.n[c]] = rec->saux[s].base;
+            ++fl.n[c];
+            any_refine = true;
         }
-        if (!count) continue;
-        entropy_kernel<<<(count + kEntropyWarps - 1) / kEntropyWarps, 32 * kEntropyWarps, 0, st>>>(P, begin, count);
-        ++g_launches;
-        char name[24];
-        snprintf(name, sizeof name, "entropy%d", w);
-        mark(name, 1);
     }
-    {
-        FinalizeList fl;
-        memset(&fl, 0, sizeof fl);
-        bool any = false;
-        for (int s = 0; s < k; ++s) {
-            const ScanScript& sc = rec->script[s];
-            if (sc.Ss == 0 || sc.Ah == 0) continue;
-            int c = sc.comp[0];
-            if (fl.n[c] < 4) {
-                fl.scan[c][fl.n[c]] = s;
-                fl.p1[c][fl.n[c]] = 1 << sc.Al;
-                fl.base[c][fl.n[c]] = rec->saux[s].base;
-                ++fl.n[c];
-                any = true;
-            }
+    const int G = rec->G;
+    // the stages of one slice; stage numbers: 0 clear, 1 index, 2+w entropy wave w, 2+W finalize, 3+W pixels
+    const int W = rec->n_waves;
+    auto run_stage = [&](int stage, int g, cudaStream_t q) -> bool {
+        const uint32_t i0 = rec->slice_img[g], i1 = rec->slice_img[g + 1];
+        const uint32_t u0 = rec->slice_unit[g], nu = rec->slice_unit[g + 1] - u0;
+        if (stage == 0) {
+            const uint64_t b0 = rec->blk_base[i0], b1 = (i1 < (uint32_t)rec->N) ? rec->blk_base[i1] : rec->total_blocks;
+            return cudaMemsetAsync(rec->d_planes + b0 * 64, 0, (b1 - b0) * 128, q) == cudaSuccess;
         }
-        if (any) {
-            const uint64_t threads = (uint64_t)rec->n_units * 48;
-            finalize_kernel<<<(unsigned)((threads + kFinalizeThreads - 1) / kFinalizeThreads), kFinalizeThreads, 0, st>>>(P, fl, rec->n_units);
+        if (stage == 1) {
+            const uint32_t warps = (uint32_t)k * (i1 - i0);
+            unstuff_index_kernel<<<(warps + 7) / 8, 256, 0, q>>>(P, k, (int)i0, (int)(i1 - i0));
             ++g_launches;
-            mark("finalize", 1);
+            return true;
+        }
+        if (stage < 2 + W) {
+            const int w = stage - 2;
+            uint32_t begin = 0, count = 0;
+            bool any = false;
+            for (int s : rec->wave_scans[w]) {
+                if (s >= k) break;   // scans of a wave are stored in ascending order
+                if (!any) { begin = rec->item_begin[(size_t)g * G + s]; any = true; }
+                count += rec->item_count[(size_t)g * G + s];
+            }
+            if (!count) return true;
+            entropy_kernel<<<(count + kEntropyWarps - 1) / kEntropyWarps, 32 * kEntropyWarps, 0, q>>>(P, begin, count);
+            ++g_launches;
+            return true;
+        }
+        Params Q = P;
+        Q.units = P.units + u0;
+        if (stage == 2 + W) {
+            if (!any_refine || !nu) return true;
+            const uint64_t threads = (uint64_t)nu * 48;
+            finalize_kernel<<<(unsigned)((threads + kFinalizeThreads - 1) / kFinalizeThreads), kFinalizeThreads, 0, q>>>(Q, fl, nu);
+            ++g_launches;
+            return true;
+        }
+        if (nu) {
+            pixel_kernel<<<nu, kPixThreads, 0, q>>>(Q, static_cast<uint8_t*>(out));
+            ++g_launches;
+        }
+        return true;
+    };
+    auto launched_in = [&](int stage) -> int {      // kernel launches of a stage over all slices (for the profile)
+        if (stage == 0) return 0;
+        if (stage == 2 + W && !any_refine) return 0;
+        if (stage >= 2 && stage < 2 + W) {
+            bool any = false;
+            for (int s : rec->wave_scans[stage - 2]) if (s < k) any = true;
+            if (!any) return 0;
+        }
+        return rec->n_slices;
+    };
+    const int n_stages = 4 + W;
+    if (rec->n_slices == 1 || prof) {
+        // one stage after the other on the caller's stream (also the timed layout of the stage profile)
+        for (int stage = 0; stage < n_stages; ++stage) {
+            for (int g = 0; g < rec->n_slices; ++g)
+                if (!run_stage(stage, g, st)) return PCR_E_CUDA;
+            char name[24];
+            if (stage == 0) snprintf(name, sizeof name, "clear");
+            else if (stage == 1) snprintf(name, sizeof name, "index");
+            else if (stage < 2 + W) snprintf(name, sizeof name, "entropy%d", stage - 2);
+            else if (stage == 2 + W) snprintf(name, sizeof name, "finalize");
+            else snprintf(name, sizeof name, "pixels");
+            const int nl = launched_in(stage);
+            if (stage <= 1 || stage == n_stages - 1 || nl) mark(name, nl);
+        }
+    } else {
+        // every slice is its own pipeline on its own stream, forked from and joined to the caller's
+        if (cudaEventRecord(rec->ev_fork, st) != cudaSuccess) return PCR_E_CUDA;
+        for (int g = 0; g < rec->n_slices; ++g) {
+            cudaStream_t q = rec->streams[g];
+            if (cudaStreamWaitEvent(q, rec->ev_fork, 0) != cudaSuccess) return PCR_E_CUDA;
+            for (int stage = 0; stage < n_stages; ++stage)
+                if (!run_stage(stage, g, q)) return PCR_E_CUDA;
+            if (cudaEventRecord(rec->ev_join[g], q) != cudaSuccess) return PCR_E_CUDA;
+            if (cudaStreamWaitEvent(st, rec->ev_join[g], 0) != cudaSuccess) return PCR_E_CUDA;
         }
     }
-    pixel_kernel<<<rec->n_units, kPixThreads, 0, st>>>(P, static_cast<uint8_t*>(out));
-    ++g_launches;
-    mark("pixels", 1);
     if (cudaGetLastError() != cudaSuccess) return PCR_E_CUDA;
     return PCR_OK;
 }
