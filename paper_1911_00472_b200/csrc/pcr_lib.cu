@@ -593,10 +593,21 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
     };
     const int n_stages = 4 + W;
     if (rec->n_slices == 1 || prof) {
-        // one stage after the other on the caller's stream (also the timed layout of the stage profile)
+        // one stage after the other (also the timed layout of the stage profile); with several
+        // slices the slices of a stage run side by side on their streams, between two joins
         for (int stage = 0; stage < n_stages; ++stage) {
-            for (int g = 0; g < rec->n_slices; ++g)
-                if (!run_stage(stage, g, st)) return PCR_E_CUDA;
+            if (rec->n_slices == 1) {
+                if (!run_stage(stage, 0, st)) return PCR_E_CUDA;
+            } else {
+                if (cudaEventRecord(rec->ev_fork, st) != cudaSuccess) return PCR_E_CUDA;
+                for (int g = 0; g < rec->n_slices; ++g) {
+                    cudaStream_t q = rec->streams[g];
+                    if (cudaStreamWaitEvent(q, rec->ev_fork, 0) != cudaSuccess) return PCR_E_CUDA;
+                    if (!run_stage(stage, g, q)) return PCR_E_CUDA;
+                    if (cudaEventRecord(rec->ev_join[g], q) != cudaSuccess) return PCR_E_CUDA;
+                    if (cudaStreamWaitEvent(st, rec->ev_join[g], 0) != cudaSuccess) return PCR_E_CUDA;
+                }
+            }
             char name[24];
             if (stage == 0) snprintf(name, sizeof name, "clear");
             else if (stage == 1) snprintf(name, sizeof name, "index");

@@ -21,19 +21,16 @@ namespace pcr {
 
 constexpr int kPixMcus = 8;                   // MCUs per CTA
 constexpr int kPixBlocks = 6 * kPixMcus;      // 32 Y + 8 Cb + 8 Cr
-constexpr int kPixThreads = 8 * kPixBlocks;   // one thread per block column / row
-constexpr int kBlkPitch = 72;                 // words per block in shared memory: 8 rows of 9
-constexpr int kStagePitch = 3 * 16 * kPixMcus + 4;   // bytes per staged RGB row (+ one spare word)
+constexpr int kPixThreads = 64;               // one thread per block for the transform (48 used)
+constexpr int kStagePitch = 3 * 16 * kPixMcus + 16;   // bytes per staged RGB row (+ spare, keeps rows 16-byte aligned)
 
 // zigzag position -> natural index, by walking the anti-diagonals
 struct ZigzagTable {
     uint8_t nat[64];
-    uint8_t pad[64];   // position inside a 9-word-pitch block
-    constexpr ZigzagTable() : nat(), pad() {
+    constexpr ZigzagTable() : nat() {
         int r = 0, c = 0;
         for (int k = 0; k < 64; ++k) {
             nat[k] = (uint8_t)(r * 8 + c);
-            pad[k] = (uint8_t)(r * 9 + c);
             if (((r + c) & 1) == 0) {
                 if (c == 7) ++r; else if (r == 0) ++c; else { --r; ++c; }
             } else {
@@ -44,142 +41,161 @@ struct ZigzagTable {
 };
 __device__ constexpr ZigzagTable kZigzag{};
 
-__device__ __forceinline__ void idct8(const uint32_t x[8], int out[8], uint32_t rnd, int shift) {
+// One 8-point pass on the integer matrix M (see the header comment): out[n] = (sum_k M[n][k] x[k] + rnd) >> shift
+__device__ __forceinline__ void idct8(uint32_t& x0, uint32_t& x1, uint32_t& x2, uint32_t& x3, uint32_t& x4, uint32_t& x5,
+                                      uint32_t& x6, uint32_t& x7, uint32_t rnd, int shift) {
     constexpr uint32_t K1 = 8035, K2 = 7568, K3 = 6811, K4 = 5793, K5 = 4551, K6 = 3135, K7 = 1598;
-    uint32_t a0 = K4 * (x[0] + x[4]), a1 = K4 * (x[0] - x[4]);
-    uint32_t b0 = K2 * x[2] + K6 * x[6], b1 = K6 * x[2] - K2 * x[6];
-    uint32_t e0 = a0 + b0 + rnd, e3 = a0 - b0 + rnd, e1 = a1 + b1 + rnd, e2 = a1 - b1 + rnd;
-    uint32_t o0 = K1 * x[1] + K3 * x[3] + K5 * x[5] + K7 * x[7];
-    uint32_t o1 = K3 * x[1] - K7 * x[3] - K1 * x[5] - K5 * x[7];
-    uint32_t o2 = K5 * x[1] - K1 * x[3] + K7 * x[5] + K3 * x[7];
-    uint32_t o3 = K7 * x[1] - K5 * x[3] + K3 * x[5] - K1 * x[7];
-    out[0] = (int)(e0 + o0) >> shift; out[7] = (int)(e0 - o0) >> shift;
-    out[1] = (int)(e1 + o1) >> shift; out[6] = (int)(e1 - o1) >> shift;
-    out[2] = (int)(e2 + o2) >> shift; out[5] = (int)(e2 - o2) >> shift;
-    out[3] = (int)(e3 + o3) >> shift; out[4] = (int)(e3 - o3) >> shift;
+    const uint32_t a0 = K4 * (x0 + x4) + rnd, a1 = K4 * (x0 - x4) + rnd;
+    const uint32_t b0 = K2 * x2 + K6 * x6, b1 = K6 * x2 - K2 * x6;
+    const uint32_t e0 = a0 + b0, e3 = a0 - b0, e1 = a1 + b1, e2 = a1 - b1;
+    const uint32_t o0 = K1 * x1 + K3 * x3 + K5 * x5 + K7 * x7;
+    const uint32_t o1 = K3 * x1 - K7 * x3 - K1 * x5 - K5 * x7;
+    const uint32_t o2 = K5 * x1 - K1 * x3 + K7 * x5 + K3 * x7;
+    const uint32_t o3 = K7 * x1 - K5 * x3 + K3 * x5 - K1 * x7;
+    x0 = (uint32_t)((int)(e0 + o0) >> shift); x7 = (uint32_t)((int)(e0 - o0) >> shift);
+    x1 = (uint32_t)((int)(e1 + o1) >> shift); x6 = (uint32_t)((int)(e1 - o1) >> shift);
+    x2 = (uint32_t)((int)(e2 + o2) >> shift); x5 = (uint32_t)((int)(e2 - o2) >> shift);
+    x3 = (uint32_t)((int)(e3 + o3) >> shift); x4 = (uint32_t)((int)(e3 - o3) >> shift);
 }
 
-__device__ __forceinline__ uint32_t clamp255(int v) { return (uint32_t)min(max(v, 0), 255); }
+// bytes {clamp(v0), clamp(v1), clamp(v2), clamp(v3)} of a little-endian word, clamp to 0..255
+__device__ __forceinline__ uint32_t pack4_sat(int v0, int v1, int v2, int v3) {
+    uint32_t hi, w;
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(v3), "r"(v2), "r"(0));
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(v1), "r"(v0), "r"(hi));
+    return w;
+}
 
 __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, uint8_t* __restrict__ out) {
-    __shared__ __align__(16) uint32_t s_coef[kPixBlocks * kBlkPitch];
     __shared__ __align__(16) uint8_t s_y[16][16 * kPixMcus];
     __shared__ __align__(16) uint8_t s_c[2][8][8 * kPixMcus];
-    __shared__ uint8_t s_zpad[64];
+    __shared__ __align__(16) uint8_t s_stage[16 * kStagePitch];
+    __shared__ __align__(16) uint16_t s_q[3][64];
 
     const int tid = threadIdx.x;
     const Unit un = P.units[blockIdx.x];
     const ImgDesc im = P.imgs[un.img];
     const int nm = min((int)kPixMcus, (int)im.mx - (int)un.mcol0);   // MCUs in this unit
-    if (tid < 64) s_zpad[tid] = kZigzag.pad[tid];
+    for (int i = tid; i < 96; i += kPixThreads)
+        reinterpret_cast<uint32_t*>(&s_q[0][0])[i] = __ldg(reinterpret_cast<const uint32_t*>(P.qtab + (size_t)un.img * 192) + i);
     __syncthreads();
 
-    // ---- load + dequantise: shared block order is Y row 0 (16), Y row 1 (16), Cb (8), Cr (8)
-    const uint64_t ybase = im.blk_base, cbbase = im.blk_base + 4ull * im.mx * im.my, crbase = cbbase + (uint64_t)im.mx * im.my;
-    const uint16_t* q = P.qtab + (size_t)un.img * 192;
-    for (int idx = tid; idx < kPixBlocks * 32; idx += kPixThreads) {
-        int j = idx >> 5, w = idx & 31;
-        int comp, valid;
-        uint64_t blk;
+    // ---- transform: thread j owns block j; block order Y row 0 (16), Y row 1 (16), Cb (8), Cr (8)
+    {
+        const int j = tid;
+        int comp = 0;
+        bool valid = false;
+        uint64_t blk = 0;
         if (j < 32) {
-            int r = j >> 4, c = j & 15;
-            comp = 0; valid = c < 2 * nm;
-            blk = ybase + (uint64_t)(2 * un.mrow + r) * (2 * im.mx) + 2 * un.mcol0 + c;
-        } else {
-            int c = (j - 32) & 7;
-            comp = 1 + ((j - 32) >> 3); valid = c < nm;
-            blk = (comp == 1 ? cbbase : crbase) + (uint64_t)un.mrow * im.mx + un.mcol0 + c;
+            const int r = j >> 4, c = j & 15;
+            valid = c < 2 * nm;
+            blk = im.blk_base + (uint64_t)(2 * un.mrow + r) * (2 * im.mx) + 2 * un.mcol0 + c;
+        } else if (j < kPixBlocks) {
+            const int c = (j - 32) & 7;
+            comp = 1 + ((j - 32) >> 3);
+            valid = c < nm;
+            blk = im.blk_base + (comp == 1 ? 4ull : 5ull) * im.mx * im.my + (uint64_t)un.mrow * im.mx + un.mcol0 + c;
         }
         if (valid) {
-            uint32_t v = __ldg(reinterpret_cast<const uint32_t*>(P.planes + blk * 64) + w);
-            uint32_t qq = __ldg(reinterpret_cast<const uint32_t*>(q + comp * 64) + w);
-            int c0 = (int)(int16_t)(v & 0xFFFFu), c1 = (int)v >> 16;
-            s_coef[j * kBlkPitch + s_zpad[2 * w]] = (uint32_t)(c0 * (int)(qq & 0xFFFFu));
-            s_coef[j * kBlkPitch + s_zpad[2 * w + 1]] = (uint32_t)(c1 * (int)(qq >> 16));
-        }
-    }
-    __syncthreads();
-
-    const int j = tid >> 3, t8 = tid & 7;
-    bool valid;
-    if (j < 32) valid = (j & 15) < 2 * nm; else valid = ((j - 32) & 7) < nm;
-    uint32_t* blkp = s_coef + j * kBlkPitch;
-    // ---- pass 1: column t8
-    if (valid) {
-        uint32_t x[8]; int o[8];
+            const uint4* line = reinterpret_cast<const uint4*>(P.planes + blk * 64);
+            uint4 raw[8];
 #pragma unroll
-        for (int v = 0; v < 8; ++v) x[v] = blkp[v * 9 + t8];
-        idct8(x, o, 1u << 11, 12);
+            for (int q = 0; q < 8; ++q) raw[q] = __ldg(line + q);
+            const uint32_t* qw = reinterpret_cast<const uint32_t*>(&s_q[comp][0]);
+            uint32_t v[64];
 #pragma unroll
-        for (int v = 0; v < 8; ++v) blkp[v * 9 + t8] = (uint32_t)o[v];
-    }
-    __syncthreads();
-    // ---- pass 2: row t8
-    if (valid) {
-        uint32_t x[8]; int o[8];
+            for (int q = 0; q < 8; ++q) {
+                const uint32_t w4[4] = {raw[q].x, raw[q].y, raw[q].z, raw[q].w};
 #pragma unroll
-        for (int u = 0; u < 8; ++u) x[u] = blkp[t8 * 9 + u];
-        idct8(x, o, 1u << 15, 16);
-        uint32_t lo = clamp255(o[0] + 128) | (clamp255(o[1] + 128) << 8) | (clamp255(o[2] + 128) << 16) | (clamp255(o[3] + 128) << 24);
-        uint32_t hi = clamp255(o[4] + 128) | (clamp255(o[5] + 128) << 8) | (clamp255(o[6] + 128) << 16) | (clamp255(o[7] + 128) << 24);
-        uint2* dst;
-        if (j < 32) dst = reinterpret_cast<uint2*>(&s_y[(j >> 4) * 8 + t8][(j & 15) * 8]);
-        else dst = reinterpret_cast<uint2*>(&s_c[(j - 32) >> 3][t8][((j - 32) & 7) * 8]);
-        *dst = make_uint2(lo, hi);
-    }
-    __syncthreads();
-
-    // ---- colour: 4 pixels per step, staged as the output's byte layout (aliases s_coef)
-    uint8_t* stage = reinterpret_cast<uint8_t*>(s_coef);
-    for (int gi = tid; gi < 16 * 4 * kPixMcus; gi += kPixThreads) {
-        int row = gi / (4 * kPixMcus), gx = gi % (4 * kPixMcus);
-        if (gx >= 4 * nm) continue;
-        uint32_t yw = *reinterpret_cast<const uint32_t*>(&s_y[row][4 * gx]);
-        uint32_t cbw = *reinterpret_cast<const uint16_t*>(&s_c[0][row >> 1][2 * gx]);
-        uint32_t crw = *reinterpret_cast<const uint16_t*>(&s_c[1][row >> 1][2 * gx]);
-        uint32_t px[12];
+                for (int e = 0; e < 4; ++e) {
+                    const int k = 8 * q + 2 * e;                 // zigzag positions k, k + 1
+                    const uint32_t qq = qw[k >> 1];
+                    const int c0 = (int)(short)(w4[e] & 0xFFFFu), c1 = (int)w4[e] >> 16;
+                    v[kZigzag.nat[k]] = (uint32_t)(c0 * (int)(qq & 0xFFFFu));
+                    v[kZigzag.nat[k + 1]] = (uint32_t)(c1 * (int)(qq >> 16));
+                }
+            }
+            // pass 1: columns (two fraction bits kept)
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            int cb = (int)((cbw >> (8 * h)) & 255u) - 128, cr = (int)((crw >> (8 * h)) & 255u) - 128;
-            int dr = (91881 * cr + 32768) >> 16;
-            int dg = (-22553 * cb - 46802 * cr + 32768) >> 16;
-            int db = (116130 * cb + 32768) >> 16;
+            for (int u = 0; u < 8; ++u)
+                idct8(v[u], v[8 + u], v[16 + u], v[24 + u], v[32 + u], v[40 + u], v[48 + u], v[56 + u], 1u << 11, 12);
+            // pass 2: rows; the +128 level shift rides in the rounding constant
+            uint8_t* dst;
+            int pitch;
+            if (j < 32) { dst = &s_y[(j >> 4) * 8][(j & 15) * 8]; pitch = 16 * kPixMcus; }
+            else { dst = &s_c[(j - 32) >> 3][0][((j - 32) & 7) * 8]; pitch = 8 * kPixMcus; }
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                int Y = (int)((yw >> (8 * (2 * h + e))) & 255u);
-                px[(2 * h + e) * 3 + 0] = clamp255(Y + dr);
-                px[(2 * h + e) * 3 + 1] = clamp255(Y + dg);
-                px[(2 * h + e) * 3 + 2] = clamp255(Y + db);
+            for (int y = 0; y < 8; ++y) {
+                idct8(v[8 * y], v[8 * y + 1], v[8 * y + 2], v[8 * y + 3], v[8 * y + 4], v[8 * y + 5], v[8 * y + 6], v[8 * y + 7],
+                      (1u << 15) + (128u << 16), 16);
+                const uint32_t lo = pack4_sat((int)v[8 * y], (int)v[8 * y + 1], (int)v[8 * y + 2], (int)v[8 * y + 3]);
+                const uint32_t hi = pack4_sat((int)v[8 * y + 4], (int)v[8 * y + 5], (int)v[8 * y + 6], (int)v[8 * y + 7]);
+                *reinterpret_cast<uint2*>(dst + y * pitch) = make_uint2(lo, hi);
             }
         }
-        uint32_t* d = reinterpret_cast<uint32_t*>(stage + row * kStagePitch + 12 * gx);
-        d[0] = px[0] | (px[1] << 8) | (px[2] << 16) | (px[3] << 24);
-        d[1] = px[4] | (px[5] << 8) | (px[6] << 16) | (px[7] << 24);
-        d[2] = px[8] | (px[9] << 8) | (px[10] << 16) | (px[11] << 24);
     }
     __syncthreads();
 
-    // ---- store: each staged row is a contiguous byte run of the output; write aligned words
+    // ---- colour: 4 pixels per step, staged as the output's byte layout
+    for (int gi = tid; gi < 16 * 4 * kPixMcus; gi += kPixThreads) {
+        const int row = gi / (4 * kPixMcus), gx = gi % (4 * kPixMcus);
+        if (gx >= 4 * nm) continue;
+        const uint32_t yw = *reinterpret_cast<const uint32_t*>(&s_y[row][4 * gx]);
+        const uint32_t cbw = *reinterpret_cast<const uint16_t*>(&s_c[0][row >> 1][2 * gx]);
+        const uint32_t crw = *reinterpret_cast<const uint16_t*>(&s_c[1][row >> 1][2 * gx]);
+        int px[12];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int cb = (int)((cbw >> (8 * h)) & 255u) - 128, cr = (int)((crw >> (8 * h)) & 255u) - 128;
+            const int dr = (91881 * cr + 32768) >> 16;
+            const int dg = (-22553 * cb - 46802 * cr + 32768) >> 16;
+            const int db = (116130 * cb + 32768) >> 16;
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int Y = (int)((yw >> (8 * (2 * h + e))) & 255u);
+                px[(2 * h + e) * 3 + 0] = Y + dr;
+                px[(2 * h + e) * 3 + 1] = Y + dg;
+                px[(2 * h + e) * 3 + 2] = Y + db;
+            }
+        }
+        uint32_t* d = reinterpret_cast<uint32_t*>(s_stage + row * kStagePitch + 12 * gx);
+        d[0] = pack4_sat(px[0], px[1], px[2], px[3]);
+        d[1] = pack4_sat(px[4], px[5], px[6], px[7]);
+        d[2] = pack4_sat(px[8], px[9], px[10], px[11]);
+    }
+    __syncthreads();
+
+    // ---- store: each staged row is a contiguous byte run of the output
     const int x0 = 16 * (int)un.mcol0;
     const int npx = min(16 * nm, (int)im.W - x0);
     const int nrows = min(16, (int)im.H - 16 * (int)un.mrow);
     const int nbytes = 3 * npx;
-    const int wid = tid >> 5, lane = tid & 31;
-    for (int row = wid; row < nrows; row += kPixThreads / 32) {
-        uint64_t g0 = im.out_off + ((uint64_t)(16 * un.mrow + row) * im.W + x0) * 3;
-        uint8_t* gp = out + g0;
-        const int a = (int)(reinterpret_cast<uintptr_t>(gp) & 3u);
-        const uint8_t* srow = stage + row * kStagePitch;
-        const uint32_t* sw = reinterpret_cast<const uint32_t*>(srow);
-        const int nw = (a + nbytes + 3) >> 2;
-        for (int i = lane; i < nw; i += 32) {
-            int sb = 4 * i - a;                     // first staged byte of this output word
-            if (sb >= 0 && sb + 4 <= nbytes) {
-                uint32_t lo = sw[sb >> 2], hi = sw[(sb >> 2) + 1];   // the spare word keeps hi in bounds
-                uint32_t v = a ? __funnelshift_r(lo, hi, 8 * (sb & 3)) : lo;
-                *reinterpret_cast<uint32_t*>(gp + sb) = v;
-            } else {
-                for (int b = max(sb, 0); b < min(sb + 4, nbytes); ++b) gp[b] = srow[b];
+    uint8_t* gbase = out + im.out_off + ((uint64_t)(16 * un.mrow) * im.W + x0) * 3;
+    const size_t gpitch = (size_t)im.W * 3;
+    if (((reinterpret_cast<uintptr_t>(gbase) | gpitch | (uintptr_t)nbytes) & 15u) == 0) {
+        // rows start and end on 16-byte boundaries: whole 16-byte vectors
+        const int vec = nbytes >> 4;
+        for (int i = tid; i < nrows * vec; i += kPixThreads) {
+            const int row = i / vec, c = i % vec;
+            *reinterpret_cast<uint4*>(gbase + row * gpitch + 16 * c) = *reinterpret_cast<const uint4*>(s_stage + row * kStagePitch + 16 * c);
+        }
+    } else {
+        const int wid = tid >> 5, lane = tid & 31;
+        for (int row = wid; row < nrows; row += kPixThreads / 32) {
+            uint8_t* gp = gbase + row * gpitch;
+            const int a = (int)(reinterpret_cast<uintptr_t>(gp) & 3u);
+            const uint8_t* srow = s_stage + row * kStagePitch;
+            const uint32_t* sw = reinterpret_cast<const uint32_t*>(srow);
+            const int nw = (a + nbytes + 3) >> 2;
+            for (int i = lane; i < nw; i += 32) {
+                const int sb = 4 * i - a;                     // first staged byte of this output word
+                if (sb >= 0 && sb + 4 <= nbytes) {
+                    const uint32_t lo = sw[sb >> 2], hi = sw[(sb >> 2) + 1];   // the spare bytes keep hi in bounds
+                    const uint32_t v = a ? __funnelshift_r(lo, hi, 8 * (sb & 3)) : lo;
+                    *reinterpret_cast<uint32_t*>(gp + sb) = v;
+                } else {
+                    for (int b = max(sb, 0); b < min(sb + 4, nbytes); ++b) gp[b] = srow[b];
+                }
             }
         }
     }
