@@ -25,7 +25,7 @@ namespace pcr {
 constexpr int kErrCorrupt = -3;
 
 constexpr int kLutBits = 11;
-constexpr int kEntropyWarps = 4;
+constexpr int kEntropyWarps = 3;
 
 // Decoder tables of one Huffman table: a direct lookup on the next kLutBits bits for short
 // codes, and the canonical first-code / count / index triple per length for the rest.
@@ -66,47 +66,71 @@ __device__ __forceinline__ void build_hufftab(HuffTab& t, const uint8_t* __restr
 }
 
 // MSB-first bit reader over the unstuffed copy of the entropy-coded bytes (see
-// unstuff_index_kernel), which holds big-endian 32-bit words.  Each lane streams its restart
-// interval through registers: one 16-byte load per 128 bits, issued one step ahead of its use,
-// so the serial decode chain never waits on memory and every sector is fetched once (32 lanes
-// reading 32 different streams would otherwise thrash the small L1 left beside the tables).
-struct BitReader {
-    const uint4* base;   // 16-byte aligned start of the chunk's region in the copy
-    uint32_t q;          // next 16-byte group to fetch
-    uint4 cur, nxt;      // group being consumed, group already in flight
-    uint32_t wi;         // next word of cur
-    uint64_t buf;        // left-aligned bit buffer
-    int nbits;           // bits held in buf
-    uint32_t loaded;     // bits moved into buf so far
-    uint32_t limit;      // bits in the restart interval
+// unstuff_index_kernel), which holds big-endian 32-bit words.  Each lane owns one column of a
+// 16-word ring in shared memory.  All lanes of the warp top their rings up together
+// (16-byte global loads), then decode for a while reading single words from the ring: the
+// serial decode chain only ever waits on shared memory, and the latency of global memory is
+// paid once per top-up for the whole warp instead of once per lane and load.
+constexpr int kRingWords = 16;
 
-    __device__ __forceinline__ void init(const uint8_t* ubuf, uint32_t bstart, uint32_t bend) {
-        base = reinterpret_cast<const uint4*>(ubuf);
-        q = bstart >> 4;
-        cur = __ldg(base + q);
-        nxt = __ldg(base + q + 1);
-        q += 2;
-        wi = (bstart >> 2) & 3u;
-        buf = 0; nbits = 0; loaded = 0;
+struct BitReader {
+    uint32_t* col;        // this lane's ring column: word j lives at col[(j & 15) * 32]
+    const uint4* g4;      // the unstuffed copy as 16-byte groups
+    uint32_t rd, wr;      // next word to consume / to fetch (absolute word indices, wr a multiple of 4)
+    uint32_t rd0;         // first word of the restart interval
+    uint64_t buf;         // left-aligned bit buffer
+    int nbits;            // bits held in buf
+    uint32_t lead;        // bits of the first word that precede the interval
+    uint32_t limit;       // bits in the restart interval
+
+    __device__ __forceinline__ void init(uint32_t* ring_col, const uint8_t* ubuf, uint32_t bstart, uint32_t bend) {
+        col = ring_col;
+        g4 = reinterpret_cast<const uint4*>(ubuf);
+        rd = rd0 = bstart >> 2;
+        wr = rd & ~3u;
+        buf = 0; nbits = 0;
+        lead = 8u * (bstart & 3u);
         limit = (bend - bstart) * 8u;
-        // the first word may start before the interval: drop those bytes
-        const uint32_t lead = 8u * (bstart & 3u);
-        refill();
-        buf <<= lead; nbits -= (int)lead; loaded -= lead;
     }
-    // afterwards at least 33 bits are held (call before every symbol and before every run of
-    // up to 32 raw bits)
+    // fetch as many 16-byte groups as the ring has room for (all lanes call this together)
+    __device__ __forceinline__ void topup(bool on) {
+        const int room = on ? (int)(kRingWords - (wr - rd)) >> 2 : 0;
+        uint4 v0, v1, v2, v3;
+        if (room > 0) v0 = __ldg(g4 + (wr >> 2));
+        if (room > 1) v1 = __ldg(g4 + (wr >> 2) + 1);
+        if (room > 2) v2 = __ldg(g4 + (wr >> 2) + 2);
+        if (room > 3) v3 = __ldg(g4 + (wr >> 2) + 3);
+        if (room > 0) put(wr, v0);
+        if (room > 1) put(wr + 4, v1);
+        if (room > 2) put(wr + 8, v2);
+        if (room > 3) put(wr + 12, v3);
+        wr += 4u * (uint32_t)max(room, 0);
+    }
+    __device__ __forceinline__ void put(uint32_t w, const uint4& v) {
+        uint32_t* p = col + (w & (kRingWords - 1)) * 32;
+        p[0] = v.x; p[32] = v.y; p[64] = v.z; p[96] = v.w;
+    }
+    // enough words in the ring for one whole decode step (a code, its extra bits, 63 raw bits)
+    __device__ __forceinline__ bool ready() const { return wr - rd >= 3u; }
+    // once, after the first top-up: take the first word without the bytes that precede the interval
+    __device__ __forceinline__ void prime() {
+        const uint32_t w = col[(rd & (kRingWords - 1)) * 32] << lead;
+        buf = (uint64_t)w << 32;
+        nbits = 32 - (int)lead;
+        ++rd;
+    }
+    // afterwards at least 33 bits are held
     __device__ __forceinline__ void refill() {
         if (nbits <= 32) {
-            const uint32_t w = wi == 0 ? cur.x : (wi == 1 ? cur.y : (wi == 2 ? cur.z : cur.w));
+            const uint32_t w = col[(rd & (kRingWords - 1)) * 32];
             buf |= (uint64_t)w << (32 - nbits);
-            nbits += 32; loaded += 32;
-            if (++wi == 4) { wi = 0; cur = nxt; nxt = __ldg(base + q); ++q; }
+            nbits += 32;
+            ++rd;
         }
     }
     __device__ __forceinline__ uint32_t top32() const { return (uint32_t)(buf >> 32); }
     __device__ __forceinline__ void skip(int n) { buf <<= n; nbits -= n; }
-    __device__ __forceinline__ bool overran() const { return (int)(loaded - (uint32_t)nbits) > (int)limit; }
+    __device__ __forceinline__ bool overran() const { return (int)((rd - rd0) * 32u - lead) - nbits > (int)limit; }
 };
 
 // Huffman symbol at the top of the 32-bit window; returns (length << 8) | symbol, 0 if undefined
@@ -239,11 +263,15 @@ __device__ __forceinline__ int select_bit(uint64_t z, int r) {
     return none ? 64 : base;
 }
 
+constexpr int kDecodeSteps = 16;     // decode steps between two top-ups of the rings
+
 __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, uint32_t item_begin, uint32_t item_count) {
     __shared__ HuffTab tabs[kEntropyWarps][2];
+    __shared__ uint32_t s_ring[kEntropyWarps][kRingWords][32];
+    __shared__ uint64_t s_hq[kEntropyWarps][4][32];          // masks of the next blocks (AC refinement)
     const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t it = blockIdx.x * kEntropyWarps + wid;
-    if (it >= item_count) return;
+    if (it >= item_count) return;                             // whole warp
     const Item item = P.items[item_begin + it];
     const ScanDesc sd0 = P.scans[item.si];
     const int s = item.si / P.N;
@@ -257,13 +285,14 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
         if (two_images) build_hufftab(tabs[wid][1], P.rec + P.scans[item.si + 1].tab_off[0], lane);
         else if (sd0.tab_off[1]) build_hufftab(tabs[wid][1], P.rec + sd0.tab_off[1], lane);
     }
-    if ((uint32_t)lane >= item.count) return;
-    const uint32_t rem0 = sd0.nseg - item.seg0;           // restart intervals left in the first image
+    // From here on no lane leaves before the warp does: lanes without work just stay `done`.
+    bool done = (uint32_t)lane >= item.count;
+    const uint32_t rem0 = sd0.nseg - item.seg0;               // restart intervals left in the first image
     const int which = (two_images && (uint32_t)lane >= rem0) ? 1 : 0;
-    const uint32_t seg = which ? (uint32_t)lane - rem0 : item.seg0 + lane;
+    uint32_t seg = which ? (uint32_t)lane - rem0 : item.seg0 + lane;
     const ScanDesc sd = which ? P.scans[item.si + 1] : sd0;
     const int img = (int)(item.si % P.N) + which;
-    if (seg >= sd.nseg) return;
+    if (seg >= sd.nseg) { done = true; seg = 0; }
     const ImgDesc im = P.imgs[img];
     const Geometry g = make_geometry(im);
 
@@ -275,49 +304,65 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
     const uint32_t m0 = sd.ri ? seg * sd.ri : 0;
     const uint32_t m1 = sd.ri ? min(m0 + sd.ri, total) : total;
     const uint32_t* segtab = P.seg_start + sd.seg_base;
-    const uint32_t bstart = segtab[seg];
-    const uint32_t bend = segtab[seg + 1] - 2;
-    if (bstart < sd.data_off || bend > sd.data_end || bend < bstart) {   // a missing marker left a hole
-        atomicMin(&P.status[img], kErrCorrupt);
-        return;
-    }
-    BitReader br;
-    br.init(P.ubuf, bstart, bend);
+    uint32_t bstart = segtab[seg];
+    uint32_t bend = segtab[seg + 1] - 2;
     bool bad = false;
+    if (!done && (bstart < sd.data_off || bend > sd.data_end || bend < bstart)) {   // a missing marker left a hole
+        bad = true; done = true;
+    }
+    if (done) { bstart = sd.data_off; bend = sd.data_off; }
+    BitReader br;
+    br.init(&s_ring[wid][0][lane], P.ubuf, bstart, bend);
+    br.topup(!done);
+    br.prime();
     const int Al = sc.Al, p1 = 1 << sc.Al;
+    const unsigned full = 0xffffffffu;
 
     if (dc) {
-        // DC scans: every lane walks the same MCU structure, so the loop nest stays converged.
-        uint32_t mrow = m0 / mcu_w, mcol = m0 % mcu_w;
+        // ---- DC scans: one block per step
+        const int bpm = inter ? 6 : 1;                     // blocks per MCU
+        uint32_t m = m0, mrow = m0 / mcu_w, mcol = m0 % mcu_w;
+        int j = 0;                                         // block inside the MCU: Y00 Y01 Y10 Y11 Cb Cr
         int pred0 = 0, pred1 = 0, pred2 = 0;
-        for (uint32_t m = m0; m < m1 && !bad; ++m) {
-            for (int ci = 0; ci < sc.ncomp; ++ci) {
-                const int c = sc.comp[ci];
-                const int hv = (inter && c == 0) ? 2 : 1;
-                const HuffTab& tab = tabs[wid][(sd.slots >> (2 * ci)) & 1u];
-                for (int sub = 0; sub < hv * hv; ++sub) {
-                    const uint64_t blk = g.coff[c] + (uint64_t)(mrow * hv + (sub >> (hv - 1))) * g.bw[c] + mcol * hv + (sub & (hv - 1));
-                    int16_t* cf = P.planes + blk * 64;
-                    if (br.overran()) { bad = true; break; }
-                    br.refill();
-                    const uint32_t win = br.top32();
-                    if (sc.Ah == 0) {
-                        const uint32_t e = huff_lookup(tab, win);
-                        const int len = (int)(e >> 8), sz = (int)(e & 255u);
-                        if (e == 0 || sz > 15) { bad = true; break; }
-                        const int d = extend_bits(top_bits(win << len, sz), sz);
-                        br.skip(len + sz);
-                        int pv = (c == 0 ? pred0 : (c == 1 ? pred1 : pred2)) + d;
-                        if (c == 0) pred0 = pv; else if (c == 1) pred1 = pv; else pred2 = pv;
-                        cf[0] = (int16_t)(pv << Al);
-                    } else {
-                        if (win >> 31) cf[0] = (int16_t)(cf[0] | p1);
-                        br.skip(1);
-                    }
+        if (m >= m1) done = true;
+        for (;;) {
+            br.topup(!done);
+            __syncwarp(full);
+            if (__all_sync(full, done)) break;
+#pragma unroll 1
+            for (int t = 0; t < kDecodeSteps; ++t) {
+                if (done || !br.ready()) continue;
+                br.refill();
+                const uint32_t win = br.top32();
+                const int ci = inter ? (j < 4 ? 0 : j - 3) : 0;
+                const int c = inter ? ci : c0;
+                uint64_t blk;
+                if (inter && c == 0) blk = g.coff[0] + (uint64_t)(2 * mrow + (j >> 1)) * g.bw[0] + 2 * mcol + (j & 1);
+                else blk = g.coff[c] + (uint64_t)mrow * g.bw[c] + mcol;
+                int16_t* cf = P.planes + blk * 64;
+                if (sc.Ah == 0) {
+                    const HuffTab& tab = tabs[wid][(sd.slots >> (2 * ci)) & 1u];
+                    const uint32_t e = huff_lookup(tab, win);
+                    const int len = (int)(e >> 8), sz = (int)(e & 255u);
+                    if (e == 0 || sz > 15) { bad = true; done = true; continue; }
+                    const int d = extend_bits(top_bits(win << len, sz), sz);
+                    br.skip(len + sz);
+                    const int pv = (c == 0 ? pred0 : (c == 1 ? pred1 : pred2)) + d;
+                    if (c == 0) pred0 = pv; else if (c == 1) pred1 = pv; else pred2 = pv;
+                    cf[0] = (int16_t)(pv << Al);
+                } else {
+                    // coefficient 0 is the low half of the block's first word
+                    if (win >> 31) atomicOr(reinterpret_cast<unsigned int*>(cf), (unsigned int)p1);
+                    br.skip(1);
                 }
-                if (bad) break;
+                if (++j == bpm) {
+                    j = 0; ++m;
+                    if (++mcol == mcu_w) { mcol = 0; ++mrow; }
+                }
+                if (br.overran()) { bad = true; done = true; }
+                if (m >= m1) done = true;
             }
-            if (++mcol == mcu_w) { mcol = 0; ++mrow; }
+            __syncwarp(full);
         }
     } else {
         const HuffTab& tab = tabs[wid][which];
@@ -328,54 +373,67 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
         uint32_t m = m0, bcol = m0 % mcu_w;
         uint32_t bi = (m0 / mcu_w) * bw + bcol;            // block index inside the image's component
         uint32_t eobrun = 0;
-        int k = Ss;
+        if (m >= m1) done = true;
         if (sc.Ah == 0) {
-            // ---- AC first pass: one Huffman symbol per iteration
+            // ---- AC first pass: one Huffman symbol per step
             uint64_t* maskp = P.aux + ax.base + g.loff[c];
             int16_t* plane = P.planes + g.coff[c] * 64;
             uint64_t M = 0;
-            while (m < m1) {
-                if (br.overran()) { bad = true; break; }
-                br.refill();
-                const uint32_t win = br.top32();
-                const uint32_t e = huff_lookup(tab, win);
-                if (e == 0) { bad = true; break; }
-                const int len = (int)(e >> 8), r = (int)(e >> 4) & 15, sz = (int)(e & 15u);
-                const uint32_t rest = win << len;
-                bool done;
-                if (sz) {
-                    k += r;
-                    if (k > Se) { bad = true; break; }
-                    plane[(uint64_t)bi * 64 + k] = (int16_t)(extend_bits(top_bits(rest, sz), sz) * p1);
-                    br.skip(len + sz);
-                    M |= 1ull << k;
-                    ++k;
-                    done = k > Se;
-                } else if (r == 15) {
-                    br.skip(len);
-                    k += 16;
-                    done = k > Se;
-                } else {
-                    eobrun = (1u << r) + top_bits(rest, r) - 1u;
-                    br.skip(len + r);
-                    done = true;
-                }
-                if (done) {
-                    if (M) maskp[bi] = M;
-                    uint32_t adv = 1;
-                    if (eobrun) {                      // the following blocks of the run are empty
-                        const uint32_t extra = min(eobrun, m1 - (m + 1));
-                        eobrun -= extra;
-                        adv += extra;
+            int k = Ss;
+            for (;;) {
+                br.topup(!done);
+                __syncwarp(full);
+                if (__all_sync(full, done)) break;
+#pragma unroll 1
+                for (int t = 0; t < kDecodeSteps; ++t) {
+                    if (done || !br.ready()) continue;
+                    br.refill();
+                    const uint32_t win = br.top32();
+                    const uint32_t e = huff_lookup(tab, win);
+                    const int len = (int)(e >> 8), r = (int)(e >> 4) & 15, sz = (int)(e & 15u);
+                    const uint32_t rest = win << len;
+                    if (e == 0 || (sz && k + r > Se)) { bad = true; done = true; continue; }
+                    bool fin;
+                    if (sz) {
+                        k += r;
+                        plane[(uint64_t)bi * 64 + k] = (int16_t)(extend_bits(top_bits(rest, sz), sz) * p1);
+                        br.skip(len + sz);
+                        M |= 1ull << k;
+                        ++k;
+                        fin = k > Se;
+                    } else if (r == 15) {
+                        br.skip(len);
+                        k += 16;
+                        fin = k > Se;
+                    } else {
+                        eobrun = (1u << r) + top_bits(rest, r) - 1u;
+                        br.skip(len + r);
+                        fin = true;
                     }
-                    m += adv;
-                    if (adv == 1) { if (++bcol == mcu_w) { bcol = 0; bi += wrap; } else ++bi; }
-                    else { bcol = m % mcu_w; bi = (m / mcu_w) * bw + bcol; }
-                    k = Ss; M = 0;
+                    if (fin) {
+                        if (M) maskp[bi] = M;
+                        uint32_t adv = 1;
+                        if (eobrun) {                      // the following blocks of the run are empty
+                            const uint32_t extra = min(eobrun, m1 - (m + 1));
+                            eobrun -= extra;
+                            adv += extra;
+                        }
+                        m += adv;
+                        if (adv == 1) { if (++bcol == mcu_w) { bcol = 0; bi += wrap; } else ++bi; }
+                        else { bcol = m % mcu_w; bi = (m / mcu_w) * bw + bcol; }
+                        k = Ss; M = 0;
+                    }
+                    if (br.overran()) { bad = true; done = true; }
+                    if (m >= m1) done = true;
                 }
+                __syncwarp(full);
             }
         } else {
-            // ---- AC refinement: one Huffman symbol, or one block of an end-of-band run, per iteration
+            // ---- AC refinement: one Huffman symbol, or one block of an end-of-band run, per step.
+            // Hs holds the already-non-zero positions of the band from the current position k on
+            // (bit 0 = position k), rem the positions left.  Skipping r zero positions: the target
+            // sits at distance t = r + (non-zero positions up to t), found by iterating from t = r;
+            // the count reached is also the number of correction bits that follow the symbol.
             const uint64_t band = low_mask(Se + 1) & ~low_mask(Ss);
             const uint64_t* src0 = nullptr; const uint64_t* src1 = nullptr; const uint64_t* src2 = nullptr; const uint64_t* src3 = nullptr;
             uint32_t st0 = 0, st1 = 0, st2 = 0, st3 = 0;
@@ -387,76 +445,113 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
                 if (ax.nsrc > 3) { const ScanAux x = P.saux[ax.src[3]]; src3 = P.aux + x.base + g.loff[c] * x.stride; st3 = x.stride; }
             }
             uint64_t* outp = P.aux + ax.base + g.loff[c] * 4ull;
-            auto load_hist = [&](uint32_t b) -> uint64_t {
-                uint64_t h = src0[(uint64_t)b * st0];
-                if (src1) h |= src1[(uint64_t)b * st1];
-                if (src2) h |= src2[(uint64_t)b * st2];
-                if (src3) h |= src3[(uint64_t)b * st3];
-                return h & band;
-            };
-            uint64_t H = load_hist(bi);
-            uint32_t ncol = bcol + 1, nbi = bi + 1;
-            if (ncol == mcu_w) { ncol = 0; nbi = bi + wrap; }
-            uint64_t Hn = (m + 1 < m1) ? load_hist(nbi) : 0ull;      // the next block's mask is already in flight
-            uint64_t cstr = 0, Nw = 0, NS = 0;
-            int cn = 0;
-            while (m < m1) {
-                if (br.overran()) { bad = true; break; }
-                bool eob = eobrun > 0;
-                int r = 0, sz = 0;
-                uint32_t sign = 0;
-                if (!eob) {
+            uint64_t* hq = &s_hq[wid][0][lane];                       // slot j at hq[j * 32]
+            uint32_t hm = m, hcol = bcol, hbi = bi;                    // fetch cursor of the mask queue
+            uint64_t H = 0, Hs = 0, cstr = 0, Nw = 0, NS = 0;
+            int k = Ss, cn = 0;
+            uint32_t rem = 0;
+            bool newblk = true;
+            for (;;) {
+                br.topup(!done);
+                // masks of the next blocks, up to four ahead
+                {
+                    uint64_t h[4];
+                    const int want = done ? 0 : (int)min(4u - (hm - m), m1 - hm);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        if (q < want) {
+                            uint64_t v = src0[(uint64_t)hbi * st0];
+                            if (src1) v |= src1[(uint64_t)hbi * st1];
+                            if (src2) v |= src2[(uint64_t)hbi * st2];
+                            if (src3) v |= src3[(uint64_t)hbi * st3];
+                            h[q] = v & band;
+                            hq[((hm + q) & 3u) * 32] = h[q];
+                            if (++hcol == mcu_w) { hcol = 0; hbi += wrap; } else ++hbi;
+                        }
+                    }
+                    hm += (uint32_t)max(want, 0);
+                }
+                __syncwarp(full);
+                if (__all_sync(full, done)) break;
+#pragma unroll 1
+                for (int t = 0; t < kDecodeSteps; ++t) {
+                    if (done || !br.ready() || m >= hm) continue;
+                    if (newblk) {
+                        H = hq[(m & 3u) * 32];
+                        Hs = H >> Ss;
+                        k = Ss; rem = (uint32_t)(Se - Ss + 1);
+                        cstr = 0; Nw = 0; NS = 0; cn = 0;
+                        newblk = false;
+                    }
                     br.refill();
                     const uint32_t win = br.top32();
-                    const uint32_t e = huff_lookup(tab, win);
-                    if (e == 0) { bad = true; break; }
-                    const int len = (int)(e >> 8);
-                    r = (int)(e >> 4) & 15; sz = (int)(e & 15u);
-                    const uint32_t rest = win << len;
-                    if (sz) {
-                        if (sz != 1) { bad = true; break; }
-                        sign = rest >> 31;
-                        br.skip(len + 1);
-                    } else if (r < 15) {
-                        eobrun = (1u << r) + top_bits(rest, r);
-                        br.skip(len + r);
-                        eob = true;
-                    } else {
-                        br.skip(len);
+                    const bool run = eobrun > 0;                       // this block lies inside an end-of-band run
+                    uint32_t e = tab.lut[win >> (32 - kLutBits)];
+                    if (e == 0 && !run) e = huff_lookup(tab, win);
+                    const int len = (int)(e >> 8), r = (int)(e >> 4) & 15, sz = (int)(e & 15u);
+                    const bool is_new = !run && sz != 0;
+                    const bool is_eob = !run && sz == 0 && r < 15;
+                    if (!run && (e == 0 || sz > 1)) { bad = true; done = true; continue; }
+                    const int extra = is_new ? 1 : (is_eob ? r : 0);
+                    const uint32_t xbits = top_bits(win << len, extra);    // sign of a new coefficient / run length bits
+                    br.skip(run ? 0 : len + extra);
+                    if (is_eob) eobrun = (1u << r) + xbits;
+                    bool beyond = run || is_eob;                       // the rest of the band is passed over
+                    uint32_t dist = (uint32_t)r, cnt = 0;
+                    if (!beyond) {
+                        const uint32_t lo = (uint32_t)Hs;
+                        bool wide = false;
+                        for (;;) {
+                            if (dist >= rem) { beyond = true; break; }
+                            if (dist >= 32u) { wide = true; break; }
+                            cnt = __popc(lo & ((2u << dist) - 1u));
+                            const uint32_t nd = (uint32_t)r + cnt;
+                            if (nd == dist) break;
+                            dist = nd;
+                        }
+                        if (wide) {                                    // rare: the target lies in the upper half
+                            const int sel = select_bit(~Hs & low_mask((int)rem), r);
+                            if (sel >= 64) beyond = true;
+                            else { dist = (uint32_t)sel; cnt = (uint32_t)__popcll(Hs & low_mask(sel)); }
+                        }
                     }
+                    const int n = beyond ? __popcll(Hs) : (int)cnt;    // correction bits that follow
+                    const uint32_t adv = beyond ? rem : dist + 1u;
+                    if (cn + n > 64) { bad = true; done = true; continue; }
+                    if (n > 0) {
+                        br.refill();
+                        uint64_t bits = top_bits(br.top32(), min(n, 32));
+                        br.skip(min(n, 32));
+                        if (n > 32) { br.refill(); bits = (bits << (n - 32)) | top_bits(br.top32(), n - 32); br.skip(n - 32); }
+                        cstr |= bits << (64 - cn - n);
+                        cn += n;
+                    }
+                    if (is_new && !beyond) {
+                        const uint64_t bit = 1ull << (k + (int)dist);
+                        Nw |= bit;
+                        if (xbits) NS |= bit;
+                    }
+                    k += (int)adv;
+                    rem -= adv;
+                    Hs = adv >= 64u ? 0ull : Hs >> adv;
+                    if (run || is_eob) --eobrun;
+                    if (rem == 0) {                                    // block finished
+                        uint64_t* o = outp + (uint64_t)bi * 4;
+                        *reinterpret_cast<ulonglong2*>(o) = make_ulonglong2(H | Nw, cstr);
+                        *reinterpret_cast<ulonglong2*>(o + 2) = make_ulonglong2(Nw, NS);
+                        ++m;
+                        if (++bcol == mcu_w) { bcol = 0; bi += wrap; } else ++bi;
+                        newblk = true;
+                    }
+                    if (br.overran()) { bad = true; done = true; }
+                    if (m >= m1) done = true;
                 }
-                const uint64_t from = ~0ull << k;                      // k <= Se <= 63 here
-                int pos = Se + 1;
-                if (!eob) pos = min(Se + 1, select_bit(~H & band & from, r));   // pass over r zero-valued positions
-                const uint64_t hist = H & from & low_mask(pos);        // non-zero positions passed: one correction bit each
-                const int n = __popcll(hist);
-                if (n) {
-                    if (cn + n > 64) { bad = true; break; }
-                    br.refill();
-                    uint64_t bits = top_bits(br.top32(), min(n, 32));
-                    br.skip(min(n, 32));
-                    if (n > 32) { br.refill(); bits = (bits << (n - 32)) | top_bits(br.top32(), n - 32); br.skip(n - 32); }
-                    cstr |= bits << (64 - cn - n);
-                    cn += n;
-                }
-                if (sz && pos <= Se) { Nw |= 1ull << pos; NS |= (uint64_t)sign << pos; }
-                k = pos + 1;
-                if (eob) --eobrun;
-                if (k > Se) {                                          // block finished
-                    uint64_t* o = outp + (uint64_t)bi * 4;
-                    *reinterpret_cast<ulonglong2*>(o) = make_ulonglong2(H | Nw, cstr);
-                    *reinterpret_cast<ulonglong2*>(o + 2) = make_ulonglong2(Nw, NS);
-                    ++m;
-                    bi = nbi;
-                    H = Hn;
-                    if (++ncol == mcu_w) { ncol = 0; nbi += wrap; } else ++nbi;
-                    if (m + 1 < m1) Hn = load_hist(nbi);
-                    k = Ss; cstr = 0; Nw = 0; NS = 0; cn = 0;
-                }
+                __syncwarp(full);
             }
+
         }
     }
-    if (bad || br.overran()) atomicMin(&P.status[img], kErrCorrupt);
+    if (bad) atomicMin(&P.status[img], kErrCorrupt);
 }
 
 // ---------------------------------------------------------------------------------------

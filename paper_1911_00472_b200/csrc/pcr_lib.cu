@@ -417,8 +417,8 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     if (cudaMalloc(reinterpret_cast<void**>(&r->d_aux), std::max<uint64_t>(aux_words, 2) * 8) != cudaSuccess) { r->d_aux = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
     if (cudaMemset(r->d_aux, 0, std::max<uint64_t>(aux_words, 2) * 8) != cudaSuccess) return PCR_E_CUDA;
     if (cudaMalloc(reinterpret_cast<void**>(&r->d_rec), len + 64) != cudaSuccess) { r->d_rec = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
-    if (cudaMalloc(reinterpret_cast<void**>(&r->d_ubuf), len + 64) != cudaSuccess) { r->d_ubuf = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
-    if (cudaMemset(r->d_ubuf, 0, len + 64) != cudaSuccess) return PCR_E_CUDA;
+    if (cudaMalloc(reinterpret_cast<void**>(&r->d_ubuf), len + 256) != cudaSuccess) { r->d_ubuf = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
+    if (cudaMemset(r->d_ubuf, 0, len + 256) != cudaSuccess) return PCR_E_CUDA;
     if (cudaMalloc(reinterpret_cast<void**>(&r->d_planes), std::max<uint64_t>(blocks, 1) * 128) != cudaSuccess) { r->d_planes = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
     if (cudaMalloc(reinterpret_cast<void**>(&r->d_seg), (segs + 1) * 4) != cudaSuccess) { r->d_seg = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
     if (cudaMalloc(reinterpret_cast<void**>(&r->d_status), (size_t)N * 4) != cudaSuccess) { r->d_status = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
