@@ -76,9 +76,10 @@ def algorithmic_bytes(scans, infos, k: int):
     scans: [(ncomp, comp0, Ss, Se, Ah, wave, group_bytes)], infos: [(W, H)].
       index    : bytes of scan groups <= k, read once
       entropyW : compressed bytes of the wave's scans + 2 bytes per coefficient of every
-                 block a first pass visits (written once)
-      finalize : 2 bytes read + 2 bytes written per coefficient of every block a refinement
-                 scan visits (the in-place update of the planes)
+                 block the scan visits (written once by a first pass, read and written by a
+                 refinement).  The refinement's share is what the method has to move for that
+                 step; this implementation moves it in finalize_kernel, whose time therefore
+                 belongs to the refinement step and has no algorithmic bytes of its own.
       clear    : 128 bytes per block
       pixels   : 128 bytes per block read + 3 bytes per pixel written
     """
@@ -103,15 +104,33 @@ def algorithmic_bytes(scans, infos, k: int):
         band = Se - Ss + 1
         nb = blocks_pad if ncomp > 1 else blocks_unp[comp0]
         key = f"entropy{wave}"
-        out[key] = out.get(key, 0.0) + gbytes
-        if Ah and Ss > 0:
-            out["finalize"] = out.get("finalize", 0.0) + 4.0 * band * nb
-        elif Ah:
-            out[key] += 4.0 * band * nb
-        else:
-            out[key] += 2.0 * band * nb
+        out[key] = out.get(key, 0.0) + gbytes + 2.0 * band * nb * (2 if Ah else 1)
     out["total"] = sum(out.values())
     return out
+
+
+def source_hash() -> str:
+    """Hash of the CUDA sources: ncu counters are only quoted for the kernels they were taken on."""
+    import glob
+    import hashlib
+    h = hashlib.sha256()
+    for f in sorted(glob.glob(os.path.join(ROOT, "paper_1911_00472_b200", "csrc", "*"))):
+        with open(f, "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def measured_traffic(stage: str, k: int, n_images: int):
+    """dram__bytes_read + dram__bytes_write per launch of a stage's kernel from the committed ncu
+    capture (whole record, k = 10), or None when the kernels changed since or the case differs."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic_imagenet_shaped_k10.json")) as f:
+            t = json.load(f)
+        if t["source_sha256_16"] != source_hash() or k != 10 or n_images != 1024:
+            return None
+        return t["bytes_per_launch"].get(stage)
+    except Exception:
+        return None
 
 
 class ClockSampler:
@@ -381,9 +400,10 @@ def main():
     except Exception:
         pass
     achieved = model[dom] / (kernels[dom] * 1e-3) / 1e9
+    traffic = measured_traffic(dom, k, n_img)
     whole = model["total"] / (ms_max / args.steps * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None, "peak_source": peak_src, "kernel_ms": kernels[dom],
+                "traffic": traffic, "peak_source": peak_src, "kernel_ms": kernels[dom],
                 "algorithmic_bytes_per_launch": model[dom],
                 "whole_path": {"algorithmic_bytes_per_step": model["total"], "achieved": whole, "frac": whole / peak},
                 "stages_ms": stage_ms,
