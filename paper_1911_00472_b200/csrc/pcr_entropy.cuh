@@ -24,8 +24,14 @@ namespace pcr {
 
 constexpr int kErrCorrupt = -3;
 
-constexpr int kLutBits = 11;
-constexpr int kEntropyWarps = 3;
+#ifndef PCR_LUT_BITS
+#define PCR_LUT_BITS 11
+#endif
+#ifndef PCR_ENTROPY_WARPS
+#define PCR_ENTROPY_WARPS 3
+#endif
+constexpr int kLutBits = PCR_LUT_BITS;
+constexpr int kEntropyWarps = PCR_ENTROPY_WARPS;
 
 // Decoder tables of one Huffman table: a direct lookup on the next kLutBits bits for short
 // codes, and the canonical first-code / count / index triple per length for the rest.
