@@ -138,7 +138,8 @@ int pcr_get_scan(const pcr_record* rec, int s, pcr_scan_info* info);   /* s in 0
  * on its stream around each stage; after the stream has been synchronised pcr_get_profile
  * returns, for the last decode, up to `cap` entries {name, milliseconds, kernel launches}.
  * Stages: "h2d" (prefix copy), "clear" (status and plane clearing), "index" (restart-interval
- * index), "entropy0".."entropyW" (one per wave that ran), "pixels".  *n = entries written. */
+ * index and unstuffed copy), "entropy0".."entropyW" (one per wave that ran), "pixels" (in-place
+ * update of the planes from the refinement scans, then the pixel stage).  *n = entries written. */
 typedef struct {
     char name[24];
     float ms;

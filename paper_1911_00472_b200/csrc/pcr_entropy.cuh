@@ -12,8 +12,9 @@
 // AC scans leave that mask as side data; a refinement lane reads it, decodes with bit
 // operations (skipping r zero positions = dropping r set bits of the inverted mask; one
 // correction bit per set bit of the mask passed over) and leaves {new mask, correction bits,
-// new positions, their signs} as side data.  finalize_kernel then updates the planes in place,
-// one lane per coefficient pair, fully coalesced.
+// new positions, their signs} as side data.  The pixel kernel folds that side data into each
+// block before it transforms it and writes the updated block back, so the planes in device
+// memory end up holding the final coefficients.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -558,69 +559,6 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
         }
     }
     if (bad) atomicMin(&P.status[img], kErrCorrupt);
-}
-
-// ---------------------------------------------------------------------------------------
-// Fold the side data of the AC refinement scans into the coefficient planes, in scan order.
-// One thread per block; the work is proportional to the coefficients that actually change:
-// the thread walks the set bits of the "already non-zero" mask while correction bits equal to 1
-// remain (a correction moves the coefficient away from zero by 2^Al if its bit Al is still
-// clear), then the set bits of the "newly non-zero" mask (value +-2^Al).
-// ---------------------------------------------------------------------------------------
-constexpr int kFinalizeThreads = 192;      // four units of 48 blocks
-
-__global__ void __launch_bounds__(kFinalizeThreads) finalize_kernel(Params P, FinalizeList fl, uint32_t n_units) {
-    const uint32_t t = blockIdx.x * kFinalizeThreads + threadIdx.x;
-    const uint32_t unit = t / 48;
-    const int j = (int)(t % 48);
-    if (unit >= n_units) return;
-    const Unit un = P.units[unit];
-    const ImgDesc im = P.imgs[un.img];
-    const int nm = min(8, (int)im.mx - (int)un.mcol0);
-    const uint64_t mcus_before = im.blk_base / 6;
-    // same block order as the pixel kernel: Y row 0 (16), Y row 1 (16), Cb (8), Cr (8)
-    int c;
-    uint64_t local, blk;
-    if (j < 32) {
-        const int r = j >> 4, col = j & 15;
-        if (col >= 2 * nm) return;
-        c = 0;
-        local = (uint64_t)(2 * un.mrow + r) * (2 * im.mx) + 2 * un.mcol0 + col;
-        blk = im.blk_base + local;
-        local += 4 * mcus_before;
-    } else {
-        const int col = (j - 32) & 7;
-        if (col >= nm) return;
-        c = 1 + ((j - 32) >> 3);
-        local = (uint64_t)un.mrow * im.mx + un.mcol0 + col;
-        blk = im.blk_base + (c == 1 ? 4ull : 5ull) * im.mx * im.my + local;
-        local += mcus_before;
-    }
-    int16_t* cf = P.planes + blk * 64;
-    for (int i = 0; i < fl.n[c]; ++i) {
-        const int s = fl.scan[c][i];
-        const int p1 = fl.p1[c][i];
-        const ulonglong2* o = reinterpret_cast<const ulonglong2*>(P.aux + fl.base[c][i] + local * 4);
-        const ulonglong2 a = __ldg(o), b = __ldg(o + 1);       // {mask, corrections}, {new, signs}
-        (void)s;
-        uint64_t h = a.x & ~b.x, cc = a.y;
-        while (cc) {
-            const int pos = __ffsll((long long)h) - 1;
-            if (pos < 0) break;
-            h &= h - 1;
-            if (cc >> 63) {
-                const int v = cf[pos];
-                if ((v & p1) == 0) cf[pos] = (int16_t)(v >= 0 ? v + p1 : v - p1);
-            }
-            cc <<= 1;
-        }
-        uint64_t nw = b.x;
-        while (nw) {
-            const int pos = __ffsll((long long)nw) - 1;
-            nw &= nw - 1;
-            cf[pos] = (int16_t)(((b.y >> pos) & 1ull) ? p1 : -p1);
-        }
-    }
 }
 
 }  // namespace pcr

@@ -537,7 +537,8 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
         }
     }
     const int G = rec->G;
-    // the stages of one slice; stage numbers: 0 clear, 1 index, 2+w entropy wave w, 2+W finalize, 3+W pixels
+    // the stages of one slice; stage numbers: 0 clear, 1 index, 2+w entropy wave w, 2+W unused, 3+W pixels
+    // (the pixel kernel also folds the refinement side data into the planes)
     const int W = rec->n_waves;
     auto run_stage = [&](int stage, int g, cudaStream_t q) -> bool {
         const uint32_t i0 = rec->slice_img[g], i1 = rec->slice_img[g + 1];
@@ -568,22 +569,17 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
         }
         Params Q = P;
         Q.units = P.units + u0;
-        if (stage == 2 + W) {
-            if (!any_refine || !nu) return true;
-            const uint64_t threads = (uint64_t)nu * 48;
-            finalize_kernel<<<(unsigned)((threads + kFinalizeThreads - 1) / kFinalizeThreads), kFinalizeThreads, 0, q>>>(Q, fl, nu);
-            ++g_launches;
-            return true;
-        }
+        if (stage == 2 + W) return true;      // the refinement side data is folded in by the pixel kernel
         if (nu) {
-            pixel_kernel<<<nu, kPixThreads, 0, q>>>(Q, static_cast<uint8_t*>(out));
+            if (any_refine) pixel_kernel<true><<<nu, kPixThreads, 0, q>>>(Q, fl, static_cast<uint8_t*>(out));
+            else pixel_kernel<false><<<nu, kPixThreads, 0, q>>>(Q, fl, static_cast<uint8_t*>(out));
             ++g_launches;
         }
         return true;
     };
     auto launched_in = [&](int stage) -> int {      // kernel launches of a stage over all slices (for the profile)
         if (stage == 0) return 0;
-        if (stage == 2 + W && !any_refine) return 0;
+        if (stage == 2 + W) return 0;
         if (stage >= 2 && stage < 2 + W) {
             bool any = false;
             for (int s : rec->wave_scans[stage - 2]) if (s < k) any = true;
@@ -777,7 +773,9 @@ int pcr_pixels_noalloc(const int16_t* dev_coeffs, uint32_t width, uint32_t heigh
     memset(&P, 0, sizeof P);
     P.planes = const_cast<int16_t*>(dev_coeffs);     // read only by the pixel kernel
     P.imgs = &s->img; P.units = s->units; P.qtab = s->qtab; P.N = 1;
-    pixel_kernel<<<n_units, kPixThreads, 0, st>>>(P, dev_rgb);
+    FinalizeList none;
+    memset(&none, 0, sizeof none);
+    pixel_kernel<false><<<n_units, kPixThreads, 0, st>>>(P, none, dev_rgb);
     ++g_launches;
     if (cudaGetLastError() != cudaSuccess) return PCR_E_CUDA;
     return PCR_OK;

@@ -66,7 +66,15 @@ __device__ __forceinline__ uint32_t pack4_sat(int v0, int v1, int v2, int v3) {
     return w;
 }
 
-__global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, uint8_t* __restrict__ out) {
+// kRefine: first fold the side data of the AC refinement scans (see ScanAux) into the block, in
+// scan order, and write the updated 128-byte line back, so the planes in device memory hold the
+// final coefficients.  The thread parks its line in shared memory for that (word w of thread t
+// at [w][t]): the walk over the set bits of the masks addresses coefficients by position, which
+// registers cannot do.  A correction moves a non-zero coefficient away from zero by 2^Al if its
+// bit Al is still clear; a new coefficient is +-2^Al.
+template <bool kRefine>
+__global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeList fl, uint8_t* __restrict__ out) {
+    __shared__ __align__(16) uint32_t s_line[kRefine ? 32 * kPixThreads : 1];
     __shared__ __align__(16) uint8_t s_y[16][16 * kPixMcus];
     __shared__ __align__(16) uint8_t s_c[2][8][8 * kPixMcus];
     __shared__ __align__(16) uint8_t s_stage[16 * kStagePitch];
@@ -85,22 +93,70 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, uint8_t* _
         const int j = tid;
         int comp = 0;
         bool valid = false;
-        uint64_t blk = 0;
+        uint64_t blk = 0, local = 0;      // block number in the planes / inside its component
         if (j < 32) {
             const int r = j >> 4, c = j & 15;
             valid = c < 2 * nm;
-            blk = im.blk_base + (uint64_t)(2 * un.mrow + r) * (2 * im.mx) + 2 * un.mcol0 + c;
+            local = (uint64_t)(2 * un.mrow + r) * (2 * im.mx) + 2 * un.mcol0 + c;
+            blk = im.blk_base + local;
+            local += 4 * (im.blk_base / 6);
         } else if (j < kPixBlocks) {
             const int c = (j - 32) & 7;
             comp = 1 + ((j - 32) >> 3);
             valid = c < nm;
-            blk = im.blk_base + (comp == 1 ? 4ull : 5ull) * im.mx * im.my + (uint64_t)un.mrow * im.mx + un.mcol0 + c;
+            local = (uint64_t)un.mrow * im.mx + un.mcol0 + c;
+            blk = im.blk_base + (comp == 1 ? 4ull : 5ull) * im.mx * im.my + local;
+            local += im.blk_base / 6;
         }
         if (valid) {
-            const uint4* line = reinterpret_cast<const uint4*>(P.planes + blk * 64);
+            uint4* line = reinterpret_cast<uint4*>(P.planes + blk * 64);
             uint4 raw[8];
+            if (kRefine && fl.n[comp] > 0) {
 #pragma unroll
-            for (int q = 0; q < 8; ++q) raw[q] = __ldg(line + q);
+                for (int q = 0; q < 8; ++q) raw[q] = line[q];
+                uint32_t* col = s_line + tid;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    col[(4 * q) * kPixThreads] = raw[q].x; col[(4 * q + 1) * kPixThreads] = raw[q].y;
+                    col[(4 * q + 2) * kPixThreads] = raw[q].z; col[(4 * q + 3) * kPixThreads] = raw[q].w;
+                }
+                bool dirty = false;
+                for (int i = 0; i < fl.n[comp]; ++i) {
+                    const int p1 = fl.p1[comp][i];
+                    const ulonglong2* o = reinterpret_cast<const ulonglong2*>(P.aux + fl.base[comp][i] + local * 4);
+                    const ulonglong2 a = __ldg(o), b = __ldg(o + 1);       // {mask, corrections}, {new, signs}
+                    uint64_t h = a.x & ~b.x, cc = a.y;
+                    while (cc) {
+                        const int pos = __ffsll((long long)h) - 1;
+                        if (pos < 0) break;
+                        h &= h - 1;
+                        if (cc >> 63) {
+                            int16_t* e = reinterpret_cast<int16_t*>(col + (pos >> 1) * kPixThreads) + (pos & 1);
+                            const int v = *e;
+                            if ((v & p1) == 0) { *e = (int16_t)(v >= 0 ? v + p1 : v - p1); dirty = true; }
+                        }
+                        cc <<= 1;
+                    }
+                    uint64_t nw = b.x;
+                    while (nw) {
+                        const int pos = __ffsll((long long)nw) - 1;
+                        nw &= nw - 1;
+                        *(reinterpret_cast<int16_t*>(col + (pos >> 1) * kPixThreads) + (pos & 1)) = (int16_t)(((b.y >> pos) & 1ull) ? p1 : -p1);
+                        dirty = true;
+                    }
+                }
+                if (dirty) {
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        raw[q] = make_uint4(col[(4 * q) * kPixThreads], col[(4 * q + 1) * kPixThreads],
+                                            col[(4 * q + 2) * kPixThreads], col[(4 * q + 3) * kPixThreads]);
+                        line[q] = raw[q];
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int q = 0; q < 8; ++q) raw[q] = __ldg(line + q);
+            }
             const uint32_t* qw = reinterpret_cast<const uint32_t*>(&s_q[comp][0]);
             uint32_t v[64];
 #pragma unroll

@@ -17,7 +17,7 @@ struct ScanScript {
 //  - an AC refinement scan writes four words per block: {mask of non-zero positions of its band
 //    after the scan, correction bits in reading order (first bit at bit 63), mask of newly
 //    non-zero positions, mask of those that are positive}.  The coefficient planes are updated
-//    from these by the finalize kernel.
+//    from these by the pixel kernel.
 // A refinement scan finds the positions that were non-zero before it by OR-ing the masks of up
 // to four earlier scans (src), each read with its own stride.
 struct ScanAux {
