@@ -498,41 +498,50 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
                     const int len = (int)(e >> 8), r = (int)(e >> 4) & 15, sz = (int)(e & 15u);
                     const bool is_new = !run && sz != 0;
                     const bool is_eob = !run && sz == 0 && r < 15;
-                    if (!run && (e == 0 || sz > 1)) { bad = true; done = true; continue; }
+                    bool fail = !run && (e == 0 || sz > 1);
                     const int extra = is_new ? 1 : (is_eob ? r : 0);
                     const uint32_t xbits = top_bits(win << len, extra);    // sign of a new coefficient / run length bits
                     br.skip(run ? 0 : len + extra);
                     if (is_eob) eobrun = (1u << r) + xbits;
                     bool beyond = run || is_eob;                       // the rest of the band is passed over
-                    uint32_t dist = (uint32_t)r, cnt = 0;
-                    if (!beyond) {
-                        const uint32_t lo = (uint32_t)Hs;
-                        bool wide = false;
-                        for (;;) {
-                            if (dist >= rem) { beyond = true; break; }
-                            if (dist >= 32u) { wide = true; break; }
-                            cnt = __popc(lo & ((2u << dist) - 1u));
-                            const uint32_t nd = (uint32_t)r + cnt;
-                            if (nd == dist) break;
-                            dist = nd;
-                        }
-                        if (wide) {                                    // rare: the target lies in the upper half
+                    // three rounds of dist = r + (non-zero positions up to dist) settle all but rare
+                    // cases; those (and targets past bit 31) take the general search
+                    const uint32_t lo = (uint32_t)Hs;
+                    const uint32_t ur = (uint32_t)r;
+                    uint32_t dist, cnt;
+                    {
+                        const uint32_t c1 = __popc(lo & ((2u << ur) - 1u));                  // ur <= 15
+                        const uint32_t t1 = ur + c1;                                          // <= 31
+                        const uint32_t c2 = __popc(lo & ((2u << t1) - 1u));
+                        const uint32_t t2 = min(ur + c2, 31u);
+                        const uint32_t c3 = __popc(lo & ((2u << t2) - 1u));
+                        dist = ur + c3; cnt = c3;
+                        if (!beyond && (dist != ur + c2 || dist >= 32u) && dist < rem) {     // not settled
                             const int sel = select_bit(~Hs & low_mask((int)rem), r);
-                            if (sel >= 64) beyond = true;
+                            if (sel >= 64) dist = rem;
                             else { dist = (uint32_t)sel; cnt = (uint32_t)__popcll(Hs & low_mask(sel)); }
                         }
                     }
+                    beyond = beyond || dist >= rem;
                     const int n = beyond ? __popcll(Hs) : (int)cnt;    // correction bits that follow
                     const uint32_t adv = beyond ? rem : dist + 1u;
-                    if (cn + n > 64) { bad = true; done = true; continue; }
-                    if (n > 0) {
+                    fail = fail || cn + n > 64;
+                    if (n > 32) {                                      // rare: more than a word of correction bits
                         br.refill();
-                        uint64_t bits = top_bits(br.top32(), min(n, 32));
-                        br.skip(min(n, 32));
-                        if (n > 32) { br.refill(); bits = (bits << (n - 32)) | top_bits(br.top32(), n - 32); br.skip(n - 32); }
-                        cstr |= bits << (64 - cn - n);
-                        cn += n;
+                        uint64_t bits = br.top32();
+                        br.skip(32);
+                        br.refill();
+                        bits = (bits << (n - 32)) | top_bits(br.top32(), n - 32);
+                        br.skip(n - 32);
+                        if (!fail) cstr |= bits << (64 - cn - n);
+                    } else {
+                        if (br.nbits < n) br.refill();
+                        const uint64_t bits = top_bits(br.top32(), n);
+                        br.skip(n);
+                        if (!fail && n) cstr |= bits << (64 - cn - n);
                     }
+                    cn += n;
+                    if (fail) { bad = true; done = true; continue; }
                     if (is_new && !beyond) {
                         const uint64_t bit = 1ull << (k + (int)dist);
                         Nw |= bit;
