@@ -542,25 +542,31 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
                     }
                     cn += n;
                     if (fail) { bad = true; done = true; continue; }
-                    if (is_new && !beyond) {
-                        const uint64_t bit = 1ull << (k + (int)dist);
+                    {
+                        const uint64_t bit = (uint64_t)(is_new && !beyond) << ((k + (int)dist) & 63);
                         Nw |= bit;
-                        if (xbits) NS |= bit;
+                        NS |= xbits ? bit : 0ull;
                     }
                     k += (int)adv;
                     rem -= adv;
                     Hs = adv >= 64u ? 0ull : Hs >> adv;
-                    if (run || is_eob) --eobrun;
+                    eobrun -= (run || is_eob) ? 1u : 0u;
+                    fail = br.overran();
                     if (rem == 0) {                                    // block finished
                         uint64_t* o = outp + (uint64_t)bi * 4;
                         *reinterpret_cast<ulonglong2*>(o) = make_ulonglong2(H | Nw, cstr);
                         *reinterpret_cast<ulonglong2*>(o + 2) = make_ulonglong2(Nw, NS);
                         ++m;
                         if (++bcol == mcu_w) { bcol = 0; bi += wrap; } else ++bi;
-                        newblk = true;
+                        // the next block's mask is usually queued already
+                        newblk = m >= hm;
+                        H = hq[(m & 3u) * 32];
+                        Hs = H >> Ss;
+                        k = Ss; rem = (uint32_t)(Se - Ss + 1);
+                        cstr = 0; Nw = 0; NS = 0; cn = 0;
                     }
-                    if (br.overran()) { bad = true; done = true; }
-                    if (m >= m1) done = true;
+                    bad = bad || fail;
+                    done = fail || m >= m1;
                 }
                 __syncwarp(full);
             }
