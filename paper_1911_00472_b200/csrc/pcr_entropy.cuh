@@ -396,34 +396,30 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
                     if (done || !br.ready()) continue;
                     br.refill();
                     const uint32_t win = br.top32();
-                    const uint32_t e = huff_lookup(tab, win);
+                    uint32_t e = tab.lut[win >> (32 - kLutBits)];
+                    if (e == 0) e = huff_lookup(tab, win);
                     const int len = (int)(e >> 8), r = (int)(e >> 4) & 15, sz = (int)(e & 15u);
-                    const uint32_t rest = win << len;
-                    if (e == 0 || (sz && k + r > Se)) { bad = true; done = true; continue; }
-                    bool fin;
-                    if (sz) {
-                        k += r;
-                        plane[(uint64_t)bi * 64 + k] = (int16_t)(extend_bits(top_bits(rest, sz), sz) * p1);
-                        br.skip(len + sz);
-                        M |= 1ull << k;
-                        ++k;
-                        fin = k > Se;
-                    } else if (r == 15) {
-                        br.skip(len);
-                        k += 16;
-                        fin = k > Se;
-                    } else {
-                        eobrun = (1u << r) + top_bits(rest, r) - 1u;
-                        br.skip(len + r);
-                        fin = true;
+                    const bool is_coef = sz != 0, is_eob = sz == 0 && r < 15;
+                    const int kk = k + r;                                  // position of the coefficient
+                    const bool fail = e == 0 || (is_coef && kk > Se);
+                    const int extra = is_coef ? sz : (is_eob ? r : 0);
+                    const uint32_t xb = top_bits(win << len, extra);       // magnitude bits / run length bits
+                    br.skip(len + extra);
+                    if (is_coef && !fail) {
+                        plane[(uint64_t)bi * 64 + kk] = (int16_t)(extend_bits(xb, sz) * p1);
+                        M |= 1ull << kk;
                     }
+                    k = is_coef ? kk + 1 : (is_eob ? k : k + 16);
+                    if (is_eob) eobrun = (1u << r) + xb - 1u;
+                    const bool fin = is_eob || k > Se;
+                    if (fail) { bad = true; done = true; continue; }
                     if (fin) {
                         if (M) maskp[bi] = M;
                         uint32_t adv = 1;
                         if (eobrun) {                      // the following blocks of the run are empty
-                            const uint32_t extra = min(eobrun, m1 - (m + 1));
-                            eobrun -= extra;
-                            adv += extra;
+                            const uint32_t more = min(eobrun, m1 - (m + 1));
+                            eobrun -= more;
+                            adv += more;
                         }
                         m += adv;
                         if (adv == 1) { if (++bcol == mcu_w) { bcol = 0; bi += wrap; } else ++bi; }
