@@ -160,7 +160,7 @@ __device__ __forceinline__ int extend_bits(uint32_t v, int s) {
 __device__ __forceinline__ uint32_t top_bits(uint32_t x, int n) { return n ? x >> (32 - n) : 0u; }
 
 // ---------------------------------------------------------------------------------------
-// Restart-interval index and unstuffing, one warp per (scan < nscans, image).
+// Restart-interval index and unstuffing, one warp per (listed scan, image).
 // Copies the pair's entropy-coded bytes into P.ubuf with the zero byte after every 0xFF
 // removed, bytes of each aligned group of four stored in reverse (big-endian words), at the
 // same start offset as in the record.  Records, in offsets of that copy, the first byte of every
@@ -168,12 +168,14 @@ __device__ __forceinline__ uint32_t top_bits(uint32_t x, int n) { return n ? x >
 // interval j spans [seg[j], seg[j+1] - 2).  Lanes take 16-byte slices; positions come from a
 // warp prefix sum of the bytes each slice keeps.
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) unstuff_index_kernel(Params P, int nscans, int img0, int nimg) {
+struct ScanList { int32_t n; int32_t s[64]; };      // the scans one launch covers
+
+__global__ void __launch_bounds__(256) unstuff_index_kernel(Params P, ScanList sl, int img0, int nimg) {
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
-    if (warp >= nscans * nimg) return;
+    if (warp >= sl.n * nimg) return;
     const int img = img0 + warp % nimg;
-    const ScanDesc sd = P.scans[(warp / nimg) * P.N + img];
+    const ScanDesc sd = P.scans[sl.s[warp / nimg] * P.N + img];
     uint32_t* seg = P.seg_start + sd.seg_base;
     const uint32_t a = sd.data_off, b = sd.data_end;
     if (lane == 0) seg[0] = a;

@@ -46,6 +46,8 @@ struct pcr_record {
     std::vector<uint32_t> item_begin, item_count;               // [n_slices][G]
     std::vector<cudaStream_t> streams;                          // one per slice
     cudaEvent_t ev_fork = nullptr;
+    cudaStream_t copy_stream = nullptr;                         // host-to-device copies of later scan groups
+    std::vector<cudaEvent_t> ev_copy;                           // [n_waves] bytes of wave w have arrived
     std::vector<cudaEvent_t> ev_join;
     std::vector<std::vector<int>> wave_scans;
     uint32_t n_units = 0;
@@ -213,6 +215,10 @@ void free_device(pcr_record* r) {
     r->streams.clear();
     if (r->ev_fork) cudaEventDestroy(r->ev_fork);
     r->ev_fork = nullptr;
+    if (r->copy_stream) cudaStreamDestroy(r->copy_stream);
+    r->copy_stream = nullptr;
+    for (cudaEvent_t e : r->ev_copy) cudaEventDestroy(e);
+    r->ev_copy.clear();
     for (cudaEvent_t e : r->ev_join) cudaEventDestroy(e);
     r->ev_join.clear();
     for (cudaEvent_t e : r->events) cudaEventDestroy(e);
@@ -435,6 +441,12 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     r->resident = 0;
     if (r->n_slices > 1) {
         if (cudaEventCreateWithFlags(&r->ev_fork, cudaEventDisableTiming) != cudaSuccess) return PCR_E_CUDA;
+        if (cudaStreamCreateWithFlags(&r->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return PCR_E_CUDA;
+        for (int w = 0; w < r->n_waves; ++w) {
+            cudaEvent_t e;
+            if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return PCR_E_CUDA;
+            r->ev_copy.push_back(e);
+        }
         for (int g = 0; g < r->n_slices; ++g) {
             cudaStream_t q; cudaEvent_t e;
             if (cudaStreamCreateWithFlags(&q, cudaStreamNonBlocking) != cudaSuccess) return PCR_E_CUDA;
@@ -509,7 +521,8 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
         cudaEventRecord(rec->events[rec->stages.size()], st);
     };
     if (prof) cudaEventRecord(rec->events[0], st);
-    if (rec->resident < need) {
+    const bool pipelined = rec->n_slices > 1 && !prof;
+    if (!pipelined && rec->resident < need) {
         size_t from = rec->resident & ~(size_t)15;
         if (cudaMemcpyAsync(rec->d_rec + from, rec->host + from, need - from, cudaMemcpyHostToDevice, st) != cudaSuccess) return PCR_E_CUDA;
         rec->resident = need;
@@ -537,6 +550,7 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
         }
     }
     const int G = rec->G;
+    std::vector<char> copied(rec->n_waves, 0);      // wave w has to wait for its copy event
     // the stages of one slice; stage numbers: 0 clear, 1 index, 2+w entropy wave w, 2+W unused, 3+W pixels
     // (the pixel kernel also folds the refinement side data into the planes)
     const int W = rec->n_waves;
@@ -548,13 +562,28 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
             return cudaMemsetAsync(rec->d_planes + b0 * 64, 0, (b1 - b0) * 128, q) == cudaSuccess;
         }
         if (stage == 1) {
-            const uint32_t warps = (uint32_t)k * (i1 - i0);
-            unstuff_index_kernel<<<(warps + 7) / 8, 256, 0, q>>>(P, k, (int)i0, (int)(i1 - i0));
+            if (pipelined) return true;          // done wave by wave, as the bytes arrive
+            ScanList sl;
+            sl.n = 0;
+            for (int s = 0; s < k; ++s) sl.s[sl.n++] = s;
+            const uint32_t warps = (uint32_t)sl.n * (i1 - i0);
+            unstuff_index_kernel<<<(warps + 7) / 8, 256, 0, q>>>(P, sl, (int)i0, (int)(i1 - i0));
             ++g_launches;
             return true;
         }
         if (stage < 2 + W) {
             const int w = stage - 2;
+            if (pipelined) {
+                ScanList sl;
+                sl.n = 0;
+                for (int s : rec->wave_scans[w]) if (s < k) sl.s[sl.n++] = s;
+                if (sl.n) {
+                    if (copied[w] && cudaStreamWaitEvent(q, rec->ev_copy[w], 0) != cudaSuccess) return false;
+                    const uint32_t warps = (uint32_t)sl.n * (i1 - i0);
+                    unstuff_index_kernel<<<(warps + 7) / 8, 256, 0, q>>>(P, sl, (int)i0, (int)(i1 - i0));
+                    ++g_launches;
+                }
+            }
             uint32_t begin = 0, count = 0;
             bool any = false;
             for (int s : rec->wave_scans[w]) {
@@ -614,8 +643,27 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
             if (stage <= 1 || stage == n_stages - 1 || nl) mark(name, nl);
         }
     } else {
-        // every slice is its own pipeline on its own stream, forked from and joined to the caller's
+        // every slice is its own pipeline on its own stream, forked from and joined to the caller's;
+        // missing record bytes arrive on a copy stream, the scan groups of each wave behind an event
         if (cudaEventRecord(rec->ev_fork, st) != cudaSuccess) return PCR_E_CUDA;
+        if (rec->resident < need) {
+            if (cudaStreamWaitEvent(rec->copy_stream, rec->ev_fork, 0) != cudaSuccess) return PCR_E_CUDA;
+            bool any = false;
+            for (int w = 0; w < W; ++w) {
+                size_t upto = 0;
+                for (int s : rec->wave_scans[w]) if (s < k) upto = std::max(upto, (size_t)rec->group_end[s + 1]);
+                if (upto > rec->resident) {
+                    const size_t from = rec->resident & ~(size_t)15;
+                    if (cudaMemcpyAsync(rec->d_rec + from, rec->host + from, upto - from, cudaMemcpyHostToDevice, rec->copy_stream) != cudaSuccess) return PCR_E_CUDA;
+                    rec->resident = upto;
+                    any = true;
+                }
+                if (any) {
+                    if (cudaEventRecord(rec->ev_copy[w], rec->copy_stream) != cudaSuccess) return PCR_E_CUDA;
+                    copied[w] = true;
+                }
+            }
+        }
         for (int g = 0; g < rec->n_slices; ++g) {
             cudaStream_t q = rec->streams[g];
             if (cudaStreamWaitEvent(q, rec->ev_fork, 0) != cudaSuccess) return PCR_E_CUDA;
