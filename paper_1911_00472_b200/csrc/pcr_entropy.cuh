@@ -181,13 +181,33 @@ __global__ void __launch_bounds__(256) unstuff_index_kernel(Params P, ScanList s
     if (lane == 0) seg[0] = a;
     uint32_t found = 0;      // markers seen so far (warp uniform)
     uint32_t kept = 0;       // bytes written so far (warp uniform)
+    // the next tile's 16 bytes are loaded while the current tile is processed; the byte before
+    // and the byte after a lane's slice come from its neighbours by shuffle
+    const uint4 zero4 = make_uint4(0, 0, 0, 0);
+    uint4 ahead = zero4;
+    {
+        const uint32_t p = (a & ~15u) + 16u * lane;
+        if (p < b) ahead = __ldg(reinterpret_cast<const uint4*>(P.rec + p));   // chunks are padded to 16 bytes
+    }
+    uint32_t carry = 0;      // last byte of the previous tile
+    __shared__ __align__(16) uint8_t s_stage[8][528];
+    uint8_t* stage = s_stage[threadIdx.x >> 5];
+    uint32_t* out32 = reinterpret_cast<uint32_t*>(P.ubuf);
+    uint32_t gpos = a & ~3u;                 // position in the copy of stage[0]
+    uint32_t pend = a & 3u;                  // bytes already staged in front of the next tile's
+    if (lane < 4) stage[lane] = 0;
+    __syncwarp();
     for (uint32_t p0 = a & ~15u; p0 < b; p0 += 512) {
         const uint32_t p = p0 + 16u * lane;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        uint32_t nxt = 0, prev = 0;
-        if (p < b) v = __ldg(reinterpret_cast<const uint4*>(P.rec + p));   // chunks are padded to 16 bytes
-        if (p + 16 < b) nxt = __ldg(P.rec + p + 16);
-        if (p > a && p < b) prev = __ldg(P.rec + p - 1);
+        const uint4 v = ahead;
+        ahead = zero4;
+        if (p + 512 < b) ahead = __ldg(reinterpret_cast<const uint4*>(P.rec + p + 512));
+        const uint32_t first_next_tile = __shfl_sync(0xffffffffu, ahead.x & 255u, 0);
+        uint32_t nxt = __shfl_down_sync(0xffffffffu, v.x & 255u, 1);
+        if (lane == 31) nxt = first_next_tile;
+        uint32_t prev = __shfl_up_sync(0xffffffffu, v.w >> 24, 1);
+        if (lane == 0) prev = carry;
+        carry = __shfl_sync(0xffffffffu, v.w >> 24, 31);
         const uint32_t w[5] = {v.x, v.y, v.z, v.w, nxt};
         uint32_t keep = 0, mark = 0;
 #pragma unroll
@@ -207,21 +227,43 @@ __global__ void __launch_bounds__(256) unstuff_index_kernel(Params P, ScanList s
             const uint32_t ok = __shfl_up_sync(0xffffffffu, kin, d), om = __shfl_up_sync(0xffffffffu, min_, d);
             if (lane >= d) { kin += ok; min_ += om; }
         }
+        // kept bytes go to the warp's staging row (after the bytes left over from the last tile),
+        // from there to the copy as whole byte-reversed words
         const uint32_t obase = a + kept + kin - kc;
+        const uint32_t sbase = pend + kin - kc;
         uint32_t ord = found + min_ - mc;
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
             if ((keep >> j) & 1u) {
-                const uint32_t o = obase + __popc(keep & ((1u << j) - 1u));
-                P.ubuf[o ^ 3u] = (uint8_t)((w[j >> 2] >> (8 * (j & 3))) & 255u);
+                const uint32_t off = __popc(keep & ((1u << j) - 1u));
+                stage[sbase + off] = (uint8_t)((w[j >> 2] >> (8 * (j & 3))) & 255u);
                 if ((mark >> j) & 1u) {
                     ++ord;
-                    if (ord < sd.nseg) seg[ord] = o + 2;
+                    if (ord < sd.nseg) seg[ord] = obase + off + 2;
                 }
             }
         }
-        kept += __shfl_sync(0xffffffffu, kin, 31);
+        const uint32_t tile_kept = __shfl_sync(0xffffffffu, kin, 31);
+        __syncwarp();
+        const uint32_t total = pend + tile_kept, nwords = total >> 2;
+        for (uint32_t i = lane; i < nwords; i += 32)
+            out32[(gpos >> 2) + i] = __byte_perm(reinterpret_cast<const uint32_t*>(stage)[i], 0, 0x0123);
+        __syncwarp();
+        const uint32_t left = total & 3u;
+        uint32_t lb = 0;
+        if (lane < left) lb = stage[4 * nwords + lane];
+        __syncwarp();
+        if (lane < left) stage[lane] = (uint8_t)lb;
+        __syncwarp();
+        gpos += 4 * nwords;
+        pend = left;
+        kept += tile_kept;
         found += __shfl_sync(0xffffffffu, min_, 31);
+    }
+    if (pend && lane == 0) {                // the last, incomplete word (zero padded)
+        uint32_t wlast = 0;
+        for (uint32_t i = 0; i < pend; ++i) wlast |= (uint32_t)stage[i] << (8 * i);
+        out32[gpos >> 2] = __byte_perm(wlast, 0, 0x0123);
     }
     if (lane == 0) {
         seg[sd.nseg] = a + kept + 2;
