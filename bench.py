@@ -78,8 +78,8 @@ def algorithmic_bytes(scans, infos, k: int):
       entropyW : compressed bytes of the wave's scans + 2 bytes per coefficient of every
                  block the scan visits (written once by a first pass, read and written by a
                  refinement).  The refinement's share is what the method has to move for that
-                 step; this implementation moves it in finalize_kernel, whose time therefore
-                 belongs to the refinement step and has no algorithmic bytes of its own.
+                 step; this implementation moves it in the pixel kernel, which folds the
+                 refinement side data into the planes before it transforms a block.
       clear    : 128 bytes per block
       pixels   : 128 bytes per block read + 3 bytes per pixel written
     """
