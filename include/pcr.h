@@ -112,6 +112,9 @@ int pcr_evict(pcr_record* rec);
 int pcr_status(pcr_record* rec, int* first_bad_image, int* code);
 
 /* Test hook: the coefficient planes of the last decode, DEVICE memory owned by the record.
+ * Call it after the decode's stream has been synchronised: it completes the canonical layout
+ * (the decode keeps DC coefficients in a dense plane of their own; they are copied into the
+ * blocks here, with a small kernel on the default stream that this call waits for).
  * Layout: image after image (image i's first block = its blocks_offset), within an image
  * component Y, Cb, Cr, block rows then block columns of the MCU-padded grid, 64 int16 per
  * block in zigzag order (128 bytes per block).  *bytes = total size. */

@@ -390,7 +390,7 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
                 uint64_t blk;
                 if (inter && c == 0) blk = g.coff[0] + (uint64_t)(2 * mrow + (j >> 1)) * g.bw[0] + 2 * mcol + (j & 1);
                 else blk = g.coff[c] + (uint64_t)mrow * g.bw[c] + mcol;
-                int16_t* cf = P.planes + blk * 64;
+                int16_t* dcv = P.dcplane + blk;
                 if (sc.Ah == 0) {
                     const HuffTab& tab = tabs[wid][(sd.slots >> (2 * ci)) & 1u];
                     const uint32_t e = huff_lookup(tab, win);
@@ -400,10 +400,12 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
                     br.skip(len + sz);
                     const int pv = (c == 0 ? pred0 : (c == 1 ? pred1 : pred2)) + d;
                     if (c == 0) pred0 = pv; else if (c == 1) pred1 = pv; else pred2 = pv;
-                    cf[0] = (int16_t)(pv << Al);
+                    *dcv = (int16_t)(pv << Al);
                 } else {
-                    // coefficient 0 is the low half of the block's first word
-                    if (win >> 31) atomicOr(reinterpret_cast<unsigned int*>(cf), (unsigned int)p1);
+                    // two neighbouring blocks share a 32-bit word of the DC plane; the other block may
+                    // belong to another lane, so the bit is set atomically on the whole word
+                    if (win >> 31)
+                        atomicOr(reinterpret_cast<unsigned int*>(P.dcplane + (blk & ~1ull)), (unsigned int)p1 << (16 * (int)(blk & 1ull)));
                     br.skip(1);
                 }
                 if (++j == bpm) {

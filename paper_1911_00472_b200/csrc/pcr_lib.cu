@@ -57,6 +57,9 @@ struct pcr_record {
     uint8_t* d_ubuf = nullptr;
     size_t resident = 0;
     int16_t* d_planes = nullptr;
+    int16_t* d_dcplane = nullptr;
+    bool dc_merged = true;        // the planes hold the DC coefficients of the last decode
+    bool planes_cleared = true;   // ... and zeros wherever the last decode left no coefficient
     ScanScript* d_script = nullptr;
     ScanAux* d_saux = nullptr;
     uint64_t* d_aux = nullptr;
@@ -223,7 +226,7 @@ void free_device(pcr_record* r) {
     r->ev_join.clear();
     for (cudaEvent_t e : r->events) cudaEventDestroy(e);
     r->events.clear();
-    cudaFree(r->d_rec); cudaFree(r->d_ubuf); cudaFree(r->d_planes); cudaFree(r->d_script); cudaFree(r->d_saux); cudaFree(r->d_aux); cudaFree(r->d_scans);
+    cudaFree(r->d_rec); cudaFree(r->d_ubuf); cudaFree(r->d_planes); cudaFree(r->d_dcplane); cudaFree(r->d_script); cudaFree(r->d_saux); cudaFree(r->d_aux); cudaFree(r->d_scans);
     cudaFree(r->d_imgs); cudaFree(r->d_seg); cudaFree(r->d_items); cudaFree(r->d_units);
     cudaFree(r->d_qtab); cudaFree(r->d_status);
 }
@@ -426,6 +429,8 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     if (cudaMalloc(reinterpret_cast<void**>(&r->d_ubuf), len + 256) != cudaSuccess) { r->d_ubuf = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
     if (cudaMemset(r->d_ubuf, 0, len + 256) != cudaSuccess) return PCR_E_CUDA;
     if (cudaMalloc(reinterpret_cast<void**>(&r->d_planes), std::max<uint64_t>(blocks, 1) * 128) != cudaSuccess) { r->d_planes = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
+    if (cudaMalloc(reinterpret_cast<void**>(&r->d_dcplane), std::max<uint64_t>(blocks, 2) * 2 + 16) != cudaSuccess) { r->d_dcplane = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
+    if (cudaMemset(r->d_dcplane, 0, std::max<uint64_t>(blocks, 2) * 2 + 16) != cudaSuccess) return PCR_E_CUDA;
     if (cudaMalloc(reinterpret_cast<void**>(&r->d_seg), (segs + 1) * 4) != cudaSuccess) { r->d_seg = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
     if (cudaMalloc(reinterpret_cast<void**>(&r->d_status), (size_t)N * 4) != cudaSuccess) { r->d_status = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
     if (cudaMemset(r->d_seg, 0, (segs + 1) * 4) != cudaSuccess || cudaMemset(r->d_status, 0, (size_t)N * 4) != cudaSuccess) return PCR_E_CUDA;
@@ -530,7 +535,7 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
     mark("h2d", 0);
     if (cudaMemsetAsync(rec->d_status, 0, (size_t)rec->N * 4, st) != cudaSuccess) return PCR_E_CUDA;
     Params P;
-    P.rec = rec->d_rec; P.ubuf = rec->d_ubuf; P.planes = rec->d_planes; P.script = rec->d_script; P.scans = rec->d_scans;
+    P.rec = rec->d_rec; P.ubuf = rec->d_ubuf; P.planes = rec->d_planes; P.dcplane = rec->d_dcplane; P.script = rec->d_script; P.scans = rec->d_scans;
     P.saux = rec->d_saux; P.aux = rec->d_aux;
     P.imgs = rec->d_imgs; P.seg_start = rec->d_seg; P.items = rec->d_items; P.units = rec->d_units;
     P.qtab = rec->d_qtab; P.status = rec->d_status; P.N = rec->N;
@@ -549,6 +554,10 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
             any_refine = true;
         }
     }
+    bool dc_only = true;
+    for (int s = 0; s < k; ++s) if (rec->script[s].Ss > 0) dc_only = false;
+    rec->dc_merged = false;
+    rec->planes_cleared = !dc_only;
     const int G = rec->G;
     std::vector<char> copied(rec->n_waves, 0);      // wave w has to wait for its copy event
     // the stages of one slice; stage numbers: 0 clear, 1 index, 2+w entropy wave w, 2+W unused, 3+W pixels
@@ -559,6 +568,8 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
         const uint32_t u0 = rec->slice_unit[g], nu = rec->slice_unit[g + 1] - u0;
         if (stage == 0) {
             const uint64_t b0 = rec->blk_base[i0], b1 = (i1 < (uint32_t)rec->N) ? rec->blk_base[i1] : rec->total_blocks;
+            if (cudaMemsetAsync(rec->d_dcplane + b0, 0, (b1 - b0) * 2, q) != cudaSuccess) return false;
+            if (dc_only) return true;             // no AC scan: the planes are not touched at all
             return cudaMemsetAsync(rec->d_planes + b0 * 64, 0, (b1 - b0) * 128, q) == cudaSuccess;
         }
         if (stage == 1) {
@@ -600,8 +611,9 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
         Q.units = P.units + u0;
         if (stage == 2 + W) return true;      // the refinement side data is folded in by the pixel kernel
         if (nu) {
-            if (any_refine) pixel_kernel<true><<<nu, kPixThreads, 0, q>>>(Q, fl, static_cast<uint8_t*>(out));
-            else pixel_kernel<false><<<nu, kPixThreads, 0, q>>>(Q, fl, static_cast<uint8_t*>(out));
+            if (dc_only) pixel_kernel<false, 2><<<nu, kPixThreads, 0, q>>>(Q, fl, static_cast<uint8_t*>(out));
+            else if (any_refine) pixel_kernel<true, 1><<<nu, kPixThreads, 0, q>>>(Q, fl, static_cast<uint8_t*>(out));
+            else pixel_kernel<false, 1><<<nu, kPixThreads, 0, q>>>(Q, fl, static_cast<uint8_t*>(out));
             ++g_launches;
         }
         return true;
@@ -688,6 +700,21 @@ int pcr_status(pcr_record* rec, int* first_bad_image, int* code) {
 
 int pcr_coeffs(pcr_record* rec, const int16_t** dev_planes, size_t* bytes) {
     if (!rec || !dev_planes || !bytes) return PCR_E_ARG;
+    // the decode keeps the DC coefficients in a dense plane of their own (and leaves the planes
+    // alone when no AC scan was decoded): complete the canonical layout now
+    if (!rec->planes_cleared) {
+        if (cudaMemset(rec->d_planes, 0, rec->total_blocks * 128) != cudaSuccess) return PCR_E_CUDA;
+        rec->planes_cleared = true;
+    }
+    if (!rec->dc_merged && rec->total_blocks) {
+        Params P;
+        memset(&P, 0, sizeof P);
+        P.planes = rec->d_planes; P.dcplane = rec->d_dcplane;
+        merge_dc_kernel<<<(unsigned)((rec->total_blocks + 255) / 256), 256>>>(P, rec->total_blocks);
+        ++g_launches;
+        if (cudaDeviceSynchronize() != cudaSuccess) return PCR_E_CUDA;
+        rec->dc_merged = true;
+    }
     *dev_planes = rec->d_planes;
     *bytes = (size_t)rec->total_blocks * 128;
     return PCR_OK;
@@ -823,7 +850,7 @@ int pcr_pixels_noalloc(const int16_t* dev_coeffs, uint32_t width, uint32_t heigh
     P.imgs = &s->img; P.units = s->units; P.qtab = s->qtab; P.N = 1;
     FinalizeList none;
     memset(&none, 0, sizeof none);
-    pixel_kernel<false><<<n_units, kPixThreads, 0, st>>>(P, none, dev_rgb);
+    pixel_kernel<false, 0><<<n_units, kPixThreads, 0, st>>>(P, none, dev_rgb);
     ++g_launches;
     if (cudaGetLastError() != cudaSuccess) return PCR_E_CUDA;
     return PCR_OK;

@@ -72,7 +72,11 @@ __device__ __forceinline__ uint32_t pack4_sat(int v0, int v1, int v2, int v3) {
 // at [w][t]): the walk over the set bits of the masks addresses coefficients by position, which
 // registers cannot do.  A correction moves a non-zero coefficient away from zero by 2^Al if its
 // bit Al is still clear; a new coefficient is +-2^Al.
-template <bool kRefine>
+//
+// kDcMode: 0 = the DC coefficient sits in the block's line; 1 = it comes from the dense DC plane
+// (the line's first coefficient is ignored); 2 = the block has nothing but its DC coefficient (no
+// AC scan decoded): the line is not read at all and the transform collapses to one value.
+template <bool kRefine, int kDcMode>
 __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeList fl, uint8_t* __restrict__ out) {
     __shared__ __align__(16) uint32_t s_line[kRefine ? 32 * kPixThreads : 1];
     __shared__ __align__(16) uint8_t s_y[16][16 * kPixMcus];
@@ -108,7 +112,20 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
             blk = im.blk_base + (comp == 1 ? 4ull : 5ull) * im.mx * im.my + local;
             local += im.blk_base / 6;
         }
-        if (valid) {
+        if (valid && kDcMode == 2) {
+            // all AC zero: both passes keep only the k = 0 term, every sample of the block is equal
+            constexpr uint32_t K4 = 5793;
+            const int F = (int)P.dcplane[blk] * (int)s_q[comp][0];
+            const int T = (int)(K4 * (uint32_t)F + (1u << 11)) >> 12;
+            const int smp = (int)(K4 * (uint32_t)T + (1u << 15) + (128u << 16)) >> 16;
+            const uint32_t w = pack4_sat(smp, smp, smp, smp);
+            uint8_t* dst;
+            int pitch;
+            if (j < 32) { dst = &s_y[(j >> 4) * 8][(j & 15) * 8]; pitch = 16 * kPixMcus; }
+            else { dst = &s_c[(j - 32) >> 3][0][((j - 32) & 7) * 8]; pitch = 8 * kPixMcus; }
+#pragma unroll
+            for (int y = 0; y < 8; ++y) *reinterpret_cast<uint2*>(dst + y * pitch) = make_uint2(w, w);
+        } else if (valid) {
             uint4* line = reinterpret_cast<uint4*>(P.planes + blk * 64);
             uint4 raw[8];
             if (kRefine && fl.n[comp] > 0) {
@@ -157,6 +174,7 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
 #pragma unroll
                 for (int q = 0; q < 8; ++q) raw[q] = __ldg(line + q);
             }
+            if (kDcMode == 1) raw[0].x = (raw[0].x & 0xFFFF0000u) | (uint32_t)(uint16_t)P.dcplane[blk];
             const uint32_t* qw = reinterpret_cast<const uint32_t*>(&s_q[comp][0]);
             uint32_t v[64];
 #pragma unroll
@@ -255,6 +273,12 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
             }
         }
     }
+}
+
+// Copies the DC plane into coefficient 0 of every block (for readers of the full planes).
+__global__ void __launch_bounds__(256) merge_dc_kernel(Params P, uint64_t n_blocks) {
+    const uint64_t b = (uint64_t)blockIdx.x * 256 + threadIdx.x;
+    if (b < n_blocks) P.planes[b * 64] = P.dcplane[b];
 }
 
 }  // namespace pcr

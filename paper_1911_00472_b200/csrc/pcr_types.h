@@ -77,6 +77,9 @@ struct Params {
     const uint8_t* rec;         // record bytes on the device
     uint8_t* ubuf;              // entropy-coded bytes without stuffing, big-endian words
     int16_t* planes;            // coefficient planes, 64 int16 per block, zigzag order
+    int16_t* dcplane;           // DC coefficient of every block, dense (same block numbering); the DC
+                                // scans write here, so their stores fill whole sectors instead of
+                                // touching one 128-byte line per block
     const ScanScript* script;   // [G]
     const ScanAux* saux;        // [G]
     uint64_t* aux;              // side data of the AC scans
