@@ -47,6 +47,8 @@ struct pcr_record {
     std::vector<cudaStream_t> streams;                          // one per slice
     cudaEvent_t ev_fork = nullptr;
     cudaStream_t copy_stream = nullptr;                         // host-to-device copies of later scan groups
+    cudaStream_t clear_stream = nullptr;                        // zeroing of the planes, beside the index kernels
+    cudaEvent_t ev_clear = nullptr;
     std::vector<cudaEvent_t> ev_copy;                           // [n_waves] bytes of wave w have arrived
     std::vector<cudaEvent_t> ev_join;
     std::vector<std::vector<int>> wave_scans;
@@ -220,6 +222,10 @@ void free_device(pcr_record* r) {
     r->ev_fork = nullptr;
     if (r->copy_stream) cudaStreamDestroy(r->copy_stream);
     r->copy_stream = nullptr;
+    if (r->clear_stream) cudaStreamDestroy(r->clear_stream);
+    r->clear_stream = nullptr;
+    if (r->ev_clear) cudaEventDestroy(r->ev_clear);
+    r->ev_clear = nullptr;
     for (cudaEvent_t e : r->ev_copy) cudaEventDestroy(e);
     r->ev_copy.clear();
     for (cudaEvent_t e : r->ev_join) cudaEventDestroy(e);
@@ -447,6 +453,8 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     if (r->n_slices > 1) {
         if (cudaEventCreateWithFlags(&r->ev_fork, cudaEventDisableTiming) != cudaSuccess) return PCR_E_CUDA;
         if (cudaStreamCreateWithFlags(&r->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return PCR_E_CUDA;
+        if (cudaStreamCreateWithFlags(&r->clear_stream, cudaStreamNonBlocking) != cudaSuccess) return PCR_E_CUDA;
+        if (cudaEventCreateWithFlags(&r->ev_clear, cudaEventDisableTiming) != cudaSuccess) return PCR_E_CUDA;
         for (int w = 0; w < r->n_waves; ++w) {
             cudaEvent_t e;
             if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return PCR_E_CUDA;
@@ -567,6 +575,7 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
         const uint32_t i0 = rec->slice_img[g], i1 = rec->slice_img[g + 1];
         const uint32_t u0 = rec->slice_unit[g], nu = rec->slice_unit[g + 1] - u0;
         if (stage == 0) {
+            if (pipelined) return true;           // zeroed once for all slices on the clear stream
             const uint64_t b0 = rec->blk_base[i0], b1 = (i1 < (uint32_t)rec->N) ? rec->blk_base[i1] : rec->total_blocks;
             if (cudaMemsetAsync(rec->d_dcplane + b0, 0, (b1 - b0) * 2, q) != cudaSuccess) return false;
             if (dc_only) return true;             // no AC scan: the planes are not touched at all
@@ -594,6 +603,7 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
                     unstuff_index_kernel<<<(warps + 7) / 8, 256, 0, q>>>(P, sl, (int)i0, (int)(i1 - i0));
                     ++g_launches;
                 }
+                if (w == 0 && cudaStreamWaitEvent(q, rec->ev_clear, 0) != cudaSuccess) return false;
             }
             uint32_t begin = 0, count = 0;
             bool any = false;
@@ -658,6 +668,10 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
         // every slice is its own pipeline on its own stream, forked from and joined to the caller's;
         // missing record bytes arrive on a copy stream, the scan groups of each wave behind an event
         if (cudaEventRecord(rec->ev_fork, st) != cudaSuccess) return PCR_E_CUDA;
+        if (cudaStreamWaitEvent(rec->clear_stream, rec->ev_fork, 0) != cudaSuccess) return PCR_E_CUDA;
+        if (cudaMemsetAsync(rec->d_dcplane, 0, rec->total_blocks * 2, rec->clear_stream) != cudaSuccess) return PCR_E_CUDA;
+        if (!dc_only && cudaMemsetAsync(rec->d_planes, 0, rec->total_blocks * 128, rec->clear_stream) != cudaSuccess) return PCR_E_CUDA;
+        if (cudaEventRecord(rec->ev_clear, rec->clear_stream) != cudaSuccess) return PCR_E_CUDA;
         if (rec->resident < need) {
             if (cudaStreamWaitEvent(rec->copy_stream, rec->ev_fork, 0) != cudaSuccess) return PCR_E_CUDA;
             bool any = false;
