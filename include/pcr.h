@@ -101,6 +101,19 @@ size_t pcr_prefix_bytes(const pcr_record* rec, int k);
  * reported by pcr_status. */
 int pcr_decode(pcr_record* rec, int k, void* out, void* stream);
 
+/* Raise the fidelity of the last decode (Section 3: "a task then merely needs to read subsequent
+ * scan groups until the desired fidelity level is reached"; Section 4.3 switches fidelity while
+ * training).  The coefficient planes and the side data of scans 1..k_prev stay on the device
+ * after pcr_decode; this call copies the scan groups k_prev+1..k that are not yet resident,
+ * decodes only those scans on top of the resident state and produces the pixels of fidelity k.
+ * The result is identical to pcr_decode(rec, k, ...).
+ *   k : k_prev < k <= G, where k_prev is the fidelity of the last pcr_decode / pcr_decode_more
+ *       on this record (PCR_E_ARG otherwise, also when nothing has been decoded yet).
+ *   out, stream : as for pcr_decode.  The previous call's work must be complete or ordered
+ *       before this one (same stream, or synchronised).
+ * Status words accumulate: an error flagged by the earlier decode stays set. */
+int pcr_decode_more(pcr_record* rec, int k, void* out, void* stream);
+
 /* Forget which record bytes are resident on the device: the next pcr_decode copies its whole
  * prefix again (what a loader that streams each record once from host memory pays). */
 int pcr_evict(pcr_record* rec);

@@ -17,7 +17,7 @@ PCR_E_ARG, PCR_E_FORMAT, PCR_E_CORRUPT, PCR_E_TIMEOUT, PCR_E_CUDA, PCR_E_NOMEM =
 EXPORTS = ("pcr_open", "pcr_num_images", "pcr_num_groups", "pcr_get_image", "pcr_out_bytes", "pcr_prefix_bytes",
            "pcr_decode", "pcr_evict", "pcr_status", "pcr_coeffs", "pcr_image_blocks", "pcr_launch_count",
            "pcr_strerror", "pcr_close", "pcr_get_scan", "pcr_set_profiling", "pcr_get_profile",
-           "pcr_pixels_noalloc")
+           "pcr_pixels_noalloc", "pcr_decode_more")
 
 
 class ImageInfo(C.Structure):
@@ -60,6 +60,7 @@ def lib():
         L.pcr_prefix_bytes.restype = C.c_size_t
         L.pcr_prefix_bytes.argtypes = [vp, C.c_int]
         L.pcr_decode.argtypes = [vp, C.c_int, vp, vp]
+        L.pcr_decode_more.argtypes = [vp, C.c_int, vp, vp]
         L.pcr_evict.argtypes = [vp]
         L.pcr_status.argtypes = [vp, C.POINTER(C.c_int), C.POINTER(C.c_int)]
         L.pcr_coeffs.argtypes = [vp, C.POINTER(vp), C.POINTER(C.c_size_t)]
@@ -121,6 +122,10 @@ def pcr_prefix_bytes(handle: int, k: int) -> int:
 
 def pcr_decode(handle: int, k: int, out_dev_ptr: int, stream: int = 0) -> None:
     _chk(lib().pcr_decode(handle, k, out_dev_ptr, stream), "pcr_decode")
+
+
+def pcr_decode_more(handle: int, k: int, out_dev_ptr: int, stream: int = 0) -> None:
+    _chk(lib().pcr_decode_more(handle, k, out_dev_ptr, stream), "pcr_decode_more")
 
 
 def pcr_evict(handle: int) -> None:

@@ -60,6 +60,7 @@ struct pcr_record {
     size_t resident = 0;
     int16_t* d_planes = nullptr;
     int16_t* d_dcplane = nullptr;
+    int decoded_k = 0;            // fidelity of the state the planes and side data hold (0: none)
     bool dc_merged = true;        // the planes hold the DC coefficients of the last decode
     bool planes_cleared = true;   // ... and zeros wherever the last decode left no coefficient
     ScanScript* d_script = nullptr;
@@ -517,9 +518,11 @@ int pcr_evict(pcr_record* rec) {
     return PCR_OK;
 }
 
-int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
-    if (!rec || !out || k < 1 || k > rec->G) return PCR_E_ARG;
-    if (reinterpret_cast<uintptr_t>(out) & 15u) return PCR_E_ARG;
+}  // extern "C"
+
+// Decode scans k0 .. k-1 on top of the state scans 0 .. k0-1 left behind (k0 = 0: from scratch),
+// then produce the pixels of fidelity k.
+static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream) {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t need = (size_t)rec->group_end[k];
     const bool prof = rec->profiling;
@@ -541,7 +544,7 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
         rec->resident = need;
     }
     mark("h2d", 0);
-    if (cudaMemsetAsync(rec->d_status, 0, (size_t)rec->N * 4, st) != cudaSuccess) return PCR_E_CUDA;
+    if (k0 == 0 && cudaMemsetAsync(rec->d_status, 0, (size_t)rec->N * 4, st) != cudaSuccess) return PCR_E_CUDA;
     Params P;
     P.rec = rec->d_rec; P.ubuf = rec->d_ubuf; P.planes = rec->d_planes; P.dcplane = rec->d_dcplane; P.script = rec->d_script; P.scans = rec->d_scans;
     P.saux = rec->d_saux; P.aux = rec->d_aux;
@@ -550,7 +553,7 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
     FinalizeList fl;
     memset(&fl, 0, sizeof fl);
     bool any_refine = false;
-    for (int s = 0; s < k; ++s) {
+    for (int s = k0; s < k; ++s) {
         const ScanScript& sc = rec->script[s];
         if (sc.Ss == 0 || sc.Ah == 0) continue;
         const int c = sc.comp[0];
@@ -565,7 +568,12 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
     bool dc_only = true;
     for (int s = 0; s < k; ++s) if (rec->script[s].Ss > 0) dc_only = false;
     rec->dc_merged = false;
-    rec->planes_cleared = !dc_only;
+    // the planes must be zero before the first AC scan writes into them
+    const bool clear_planes = !dc_only && (k0 == 0 || !rec->planes_cleared);
+    const bool clear_dc = k0 == 0;
+    if (k0 == 0) rec->planes_cleared = false;
+    if (clear_planes) rec->planes_cleared = true;
+    rec->decoded_k = k;
     const int G = rec->G;
     std::vector<char> copied(rec->n_waves, 0);      // wave w has to wait for its copy event
     // the stages of one slice; stage numbers: 0 clear, 1 index, 2+w entropy wave w, 2+W unused, 3+W pixels
@@ -577,15 +585,15 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
         if (stage == 0) {
             if (pipelined) return true;           // zeroed once for all slices on the clear stream
             const uint64_t b0 = rec->blk_base[i0], b1 = (i1 < (uint32_t)rec->N) ? rec->blk_base[i1] : rec->total_blocks;
-            if (cudaMemsetAsync(rec->d_dcplane + b0, 0, (b1 - b0) * 2, q) != cudaSuccess) return false;
-            if (dc_only) return true;             // no AC scan: the planes are not touched at all
+            if (clear_dc && cudaMemsetAsync(rec->d_dcplane + b0, 0, (b1 - b0) * 2, q) != cudaSuccess) return false;
+            if (!clear_planes) return true;       // no AC scan yet, or already zeroed by the decode this one continues
             return cudaMemsetAsync(rec->d_planes + b0 * 64, 0, (b1 - b0) * 128, q) == cudaSuccess;
         }
         if (stage == 1) {
             if (pipelined) return true;          // done wave by wave, as the bytes arrive
             ScanList sl;
             sl.n = 0;
-            for (int s = 0; s < k; ++s) sl.s[sl.n++] = s;
+            for (int s = k0; s < k; ++s) sl.s[sl.n++] = s;
             const uint32_t warps = (uint32_t)sl.n * (i1 - i0);
             unstuff_index_kernel<<<(warps + 7) / 8, 256, 0, q>>>(P, sl, (int)i0, (int)(i1 - i0));
             ++g_launches;
@@ -596,7 +604,7 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
             if (pipelined) {
                 ScanList sl;
                 sl.n = 0;
-                for (int s : rec->wave_scans[w]) if (s < k) sl.s[sl.n++] = s;
+                for (int s : rec->wave_scans[w]) if (s >= k0 && s < k) sl.s[sl.n++] = s;
                 if (sl.n) {
                     if (copied[w] && cudaStreamWaitEvent(q, rec->ev_copy[w], 0) != cudaSuccess) return false;
                     const uint32_t warps = (uint32_t)sl.n * (i1 - i0);
@@ -609,6 +617,7 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
             bool any = false;
             for (int s : rec->wave_scans[w]) {
                 if (s >= k) break;   // scans of a wave are stored in ascending order
+                if (s < k0) continue;
                 if (!any) { begin = rec->item_begin[(size_t)g * G + s]; any = true; }
                 count += rec->item_count[(size_t)g * G + s];
             }
@@ -633,7 +642,7 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
         if (stage == 2 + W) return 0;
         if (stage >= 2 && stage < 2 + W) {
             bool any = false;
-            for (int s : rec->wave_scans[stage - 2]) if (s < k) any = true;
+            for (int s : rec->wave_scans[stage - 2]) if (s >= k0 && s < k) any = true;
             if (!any) return 0;
         }
         return rec->n_slices;
@@ -669,8 +678,8 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
         // missing record bytes arrive on a copy stream, the scan groups of each wave behind an event
         if (cudaEventRecord(rec->ev_fork, st) != cudaSuccess) return PCR_E_CUDA;
         if (cudaStreamWaitEvent(rec->clear_stream, rec->ev_fork, 0) != cudaSuccess) return PCR_E_CUDA;
-        if (cudaMemsetAsync(rec->d_dcplane, 0, rec->total_blocks * 2, rec->clear_stream) != cudaSuccess) return PCR_E_CUDA;
-        if (!dc_only && cudaMemsetAsync(rec->d_planes, 0, rec->total_blocks * 128, rec->clear_stream) != cudaSuccess) return PCR_E_CUDA;
+        if (clear_dc && cudaMemsetAsync(rec->d_dcplane, 0, rec->total_blocks * 2, rec->clear_stream) != cudaSuccess) return PCR_E_CUDA;
+        if (clear_planes && cudaMemsetAsync(rec->d_planes, 0, rec->total_blocks * 128, rec->clear_stream) != cudaSuccess) return PCR_E_CUDA;
         if (cudaEventRecord(rec->ev_clear, rec->clear_stream) != cudaSuccess) return PCR_E_CUDA;
         if (rec->resident < need) {
             if (cudaStreamWaitEvent(rec->copy_stream, rec->ev_fork, 0) != cudaSuccess) return PCR_E_CUDA;
@@ -701,6 +710,21 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
     }
     if (cudaGetLastError() != cudaSuccess) return PCR_E_CUDA;
     return PCR_OK;
+}
+
+extern "C" {
+
+int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
+    if (!rec || !out || k < 1 || k > rec->G) return PCR_E_ARG;
+    if (reinterpret_cast<uintptr_t>(out) & 15u) return PCR_E_ARG;
+    return decode_range(rec, 0, k, out, stream);
+}
+
+int pcr_decode_more(pcr_record* rec, int k, void* out, void* stream) {
+    if (!rec || !out || k < 1 || k > rec->G) return PCR_E_ARG;
+    if (reinterpret_cast<uintptr_t>(out) & 15u) return PCR_E_ARG;
+    if (rec->decoded_k < 1 || k <= rec->decoded_k) return PCR_E_ARG;
+    return decode_range(rec, rec->decoded_k, k, out, stream);
 }
 
 int pcr_status(pcr_record* rec, int* first_bad_image, int* code) {

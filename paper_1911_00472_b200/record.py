@@ -46,6 +46,17 @@ class Decoder:
             B.pcr_decode(self.handle, k, out.data_ptr(), s.cuda_stream)
         return out
 
+    def decode_more(self, k: int, out: torch.Tensor | None = None, stream: torch.cuda.Stream | None = None) -> torch.Tensor:
+        """Raise the fidelity of the last decode to k: only the scans not yet decoded are processed."""
+        if out is None:
+            if self.out is None:
+                self.out = self.alloc_out()
+            out = self.out
+        s = stream if stream is not None else torch.cuda.current_stream(self.device)
+        with torch.cuda.device(self.device):
+            B.pcr_decode_more(self.handle, k, out.data_ptr(), s.cuda_stream)
+        return out
+
     def evict(self) -> None:
         B.pcr_evict(self.handle)
 
