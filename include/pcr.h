@@ -201,8 +201,15 @@ uint64_t pcr_launch_count(void);
 /* Text for a status code. */
 const char* pcr_strerror(int code);
 
-/* Frees host and device state.  NULL is allowed.  The borrowed bytes are not touched. */
+/* Frees the record's host state and gives its device buffers up.  Waits for the last decode
+ * enqueued on this record (not for the whole device).  NULL is allowed.  The borrowed bytes are
+ * not touched.  The device buffers are kept in a per-process cache (up to 24 GiB) and handed to
+ * later pcr_open calls, so that a loader that opens and closes record after record does not pay
+ * cudaMalloc/cudaFree each time. */
 void pcr_close(pcr_record* rec);
+
+/* Returns the cached device buffers of closed records to the driver. */
+void pcr_release_cached_memory(void);
 
 #ifdef __cplusplus
 }

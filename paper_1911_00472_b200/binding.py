@@ -17,7 +17,7 @@ PCR_E_ARG, PCR_E_FORMAT, PCR_E_CORRUPT, PCR_E_TIMEOUT, PCR_E_CUDA, PCR_E_NOMEM =
 EXPORTS = ("pcr_open", "pcr_num_images", "pcr_num_groups", "pcr_get_image", "pcr_out_bytes", "pcr_prefix_bytes",
            "pcr_decode", "pcr_evict", "pcr_status", "pcr_coeffs", "pcr_image_blocks", "pcr_launch_count",
            "pcr_strerror", "pcr_close", "pcr_get_scan", "pcr_set_profiling", "pcr_get_profile",
-           "pcr_pixels_noalloc", "pcr_decode_more")
+           "pcr_pixels_noalloc", "pcr_decode_more", "pcr_release_cached_memory")
 
 
 class ImageInfo(C.Structure):
@@ -73,6 +73,8 @@ def lib():
         L.pcr_launch_count.argtypes = []
         L.pcr_strerror.restype = C.c_char_p
         L.pcr_strerror.argtypes = [C.c_int]
+        L.pcr_release_cached_memory.restype = None
+        L.pcr_release_cached_memory.argtypes = []
         L.pcr_close.restype = None
         L.pcr_close.argtypes = [vp]
         _lib = L
@@ -178,3 +180,7 @@ def pcr_pixels_noalloc(dev_coeffs_ptr: int, width: int, height: int, host_qtab_p
     device coefficients + host quantisers -> device RGB, enqueued on `stream`."""
     _chk(lib().pcr_pixels_noalloc(dev_coeffs_ptr, width, height, host_qtab_ptr, dev_rgb_ptr, stream),
          "pcr_pixels_noalloc")
+
+
+def pcr_release_cached_memory() -> None:
+    lib().pcr_release_cached_memory()

@@ -13,7 +13,10 @@
 
 #include <algorithm>
 #include <atomic>
+#include <map>
+#include <mutex>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "../../include/pcr.h"
@@ -24,6 +27,64 @@
 using namespace pcr;
 
 static std::atomic<uint64_t> g_launches{0};
+
+// Device buffers of closed records are kept for the next pcr_open instead of going back to the
+// driver: cudaMalloc and cudaFree cost milliseconds and cudaFree waits for the whole device, which
+// a loader that opens and closes one record after the other cannot afford.  Sizes are rounded up
+// to classes with three mantissa bits (at most 12.5 % slack) so that records of similar size
+// reuse each other's buffers.
+namespace {
+struct DeviceCache {
+    std::mutex mu;
+    std::multimap<std::pair<int, size_t>, void*> free_;
+    size_t cached = 0;
+    static constexpr size_t kLimit = 24ull << 30;
+} g_cache;
+
+size_t size_class(size_t n) {
+    if (n < 4096) return 4096;
+    int top = 63 - __builtin_clzll((unsigned long long)n);
+    const size_t step = (size_t)1 << (top - 3);
+    return (n + step - 1) & ~(step - 1);
+}
+
+void* dev_alloc(size_t n, int device) {
+    const size_t cls = size_class(n);
+    {
+        std::lock_guard<std::mutex> lk(g_cache.mu);
+        auto it = g_cache.free_.find({device, cls});
+        if (it != g_cache.free_.end()) {
+            void* p = it->second;
+            g_cache.free_.erase(it);
+            g_cache.cached -= cls;
+            return p;
+        }
+    }
+    void* p = nullptr;
+    if (cudaMalloc(&p, cls) != cudaSuccess) {
+        cudaGetLastError();
+        // give cached buffers back and try once more
+        std::lock_guard<std::mutex> lk(g_cache.mu);
+        for (auto& kv : g_cache.free_) cudaFree(kv.second);
+        g_cache.free_.clear();
+        g_cache.cached = 0;
+        if (cudaMalloc(&p, cls) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    }
+    return p;
+}
+
+void dev_release(void* p, size_t n, int device) {
+    if (!p) return;
+    const size_t cls = size_class(n);
+    std::lock_guard<std::mutex> lk(g_cache.mu);
+    if (g_cache.cached + cls <= DeviceCache::kLimit) {
+        g_cache.free_.insert({{device, cls}, p});
+        g_cache.cached += cls;
+    } else {
+        cudaFree(p);
+    }
+}
+}  // namespace
 
 struct pcr_record {
     const uint8_t* host = nullptr;
@@ -75,6 +136,9 @@ struct pcr_record {
     uint16_t* d_qtab = nullptr;
     int* d_status = nullptr;
     std::vector<int> h_status;
+    std::vector<std::pair<void*, size_t>> bufs;   // every device buffer of the record with its size
+    cudaEvent_t ev_done = nullptr;                // end of the last decode enqueued
+    bool decode_enqueued = false;
     // optional stage timing
     bool profiling = false;
     std::vector<cudaEvent_t> events;
@@ -233,15 +297,28 @@ void free_device(pcr_record* r) {
     r->ev_join.clear();
     for (cudaEvent_t e : r->events) cudaEventDestroy(e);
     r->events.clear();
-    cudaFree(r->d_rec); cudaFree(r->d_ubuf); cudaFree(r->d_planes); cudaFree(r->d_dcplane); cudaFree(r->d_script); cudaFree(r->d_saux); cudaFree(r->d_aux); cudaFree(r->d_scans);
-    cudaFree(r->d_imgs); cudaFree(r->d_seg); cudaFree(r->d_items); cudaFree(r->d_units);
-    cudaFree(r->d_qtab); cudaFree(r->d_status);
+    // buffers go back to the cache once the record's last decode has finished
+    if (r->ev_done) {
+        if (r->decode_enqueued) cudaEventSynchronize(r->ev_done);
+        cudaEventDestroy(r->ev_done);
+        r->ev_done = nullptr;
+    }
+    for (auto& b : r->bufs) dev_release(b.first, b.second, r->device);
+    r->bufs.clear();
 }
 
 template <class T>
-int upload(T** dst, const std::vector<T>& v) {
+int take(pcr_record* r, T** dst, size_t bytes) {
+    *dst = static_cast<T*>(dev_alloc(bytes, r->device));
+    if (!*dst) return PCR_E_NOMEM;
+    r->bufs.push_back({*dst, bytes});
+    return PCR_OK;
+}
+
+template <class T>
+int upload(pcr_record* r, T** dst, const std::vector<T>& v) {
     size_t n = std::max<size_t>(v.size(), 1) * sizeof(T);
-    if (cudaMalloc(reinterpret_cast<void**>(dst), n) != cudaSuccess) { *dst = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
+    if (int rc = take(r, dst, n)) return rc;
     if (!v.empty() && cudaMemcpy(*dst, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice) != cudaSuccess) return PCR_E_CUDA;
     return PCR_OK;
 }
@@ -430,27 +507,30 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
 
     // device state
     if (cudaGetDevice(&r->device) != cudaSuccess) return PCR_E_CUDA;
-    if (cudaMalloc(reinterpret_cast<void**>(&r->d_aux), std::max<uint64_t>(aux_words, 2) * 8) != cudaSuccess) { r->d_aux = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
+    if (int rc = take(r, &r->d_aux, (size_t)(std::max<uint64_t>(aux_words, 2) * 8))) return rc;
     if (cudaMemset(r->d_aux, 0, std::max<uint64_t>(aux_words, 2) * 8) != cudaSuccess) return PCR_E_CUDA;
-    if (cudaMalloc(reinterpret_cast<void**>(&r->d_rec), len + 64) != cudaSuccess) { r->d_rec = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
-    if (cudaMalloc(reinterpret_cast<void**>(&r->d_ubuf), len + 256) != cudaSuccess) { r->d_ubuf = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
+    if (int rc = take(r, &r->d_rec, (size_t)(len + 64))) return rc;
+    if (int rc = take(r, &r->d_ubuf, (size_t)(len + 256))) return rc;
     if (cudaMemset(r->d_ubuf, 0, len + 256) != cudaSuccess) return PCR_E_CUDA;
-    if (cudaMalloc(reinterpret_cast<void**>(&r->d_planes), std::max<uint64_t>(blocks, 1) * 128) != cudaSuccess) { r->d_planes = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
-    if (cudaMalloc(reinterpret_cast<void**>(&r->d_dcplane), std::max<uint64_t>(blocks, 2) * 2 + 16) != cudaSuccess) { r->d_dcplane = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
+    if (int rc = take(r, &r->d_planes, (size_t)(std::max<uint64_t>(blocks, 1) * 128))) return rc;
+    if (int rc = take(r, &r->d_dcplane, (size_t)(std::max<uint64_t>(blocks, 2) * 2 + 16))) return rc;
     if (cudaMemset(r->d_dcplane, 0, std::max<uint64_t>(blocks, 2) * 2 + 16) != cudaSuccess) return PCR_E_CUDA;
-    if (cudaMalloc(reinterpret_cast<void**>(&r->d_seg), (segs + 1) * 4) != cudaSuccess) { r->d_seg = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
-    if (cudaMalloc(reinterpret_cast<void**>(&r->d_status), (size_t)N * 4) != cudaSuccess) { r->d_status = nullptr; cudaGetLastError(); return PCR_E_NOMEM; }
+    if (int rc = take(r, &r->d_seg, (size_t)((segs + 1) * 4))) return rc;
+    if (int rc = take(r, &r->d_status, (size_t)((size_t)N * 4))) return rc;
     if (cudaMemset(r->d_seg, 0, (segs + 1) * 4) != cudaSuccess || cudaMemset(r->d_status, 0, (size_t)N * 4) != cudaSuccess) return PCR_E_CUDA;
     int rc;
-    if ((rc = upload(&r->d_script, r->script))) return rc;
-    if ((rc = upload(&r->d_saux, r->saux))) return rc;
-    if ((rc = upload(&r->d_scans, scans))) return rc;
-    if ((rc = upload(&r->d_imgs, imgs))) return rc;
-    if ((rc = upload(&r->d_items, items))) return rc;
-    if ((rc = upload(&r->d_units, units))) return rc;
-    if ((rc = upload(&r->d_qtab, qtab))) return rc;
+    if ((rc = upload(r, &r->d_script, r->script))) return rc;
+    if ((rc = upload(r, &r->d_saux, r->saux))) return rc;
+    if ((rc = upload(r, &r->d_scans, scans))) return rc;
+    if ((rc = upload(r, &r->d_imgs, imgs))) return rc;
+    if ((rc = upload(r, &r->d_items, items))) return rc;
+    if ((rc = upload(r, &r->d_units, units))) return rc;
+    if ((rc = upload(r, &r->d_qtab, qtab))) return rc;
     r->h_status.assign(N, 0);
     r->resident = 0;
+    if (cudaEventCreateWithFlags(&r->ev_done, cudaEventDisableTiming) != cudaSuccess) return PCR_E_CUDA;
+    // the zeroing above ran on the default stream; decodes may run on streams that do not wait for it
+    if (cudaStreamSynchronize(cudaStreamLegacy) != cudaSuccess) return PCR_E_CUDA;
     if (r->n_slices > 1) {
         if (cudaEventCreateWithFlags(&r->ev_fork, cudaEventDisableTiming) != cudaSuccess) return PCR_E_CUDA;
         if (cudaStreamCreateWithFlags(&r->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return PCR_E_CUDA;
@@ -708,11 +788,20 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream)
             if (cudaStreamWaitEvent(st, rec->ev_join[g], 0) != cudaSuccess) return PCR_E_CUDA;
         }
     }
+    if (cudaEventRecord(rec->ev_done, st) != cudaSuccess) return PCR_E_CUDA;
+    rec->decode_enqueued = true;
     if (cudaGetLastError() != cudaSuccess) return PCR_E_CUDA;
     return PCR_OK;
 }
 
 extern "C" {
+
+void pcr_release_cached_memory(void) {
+    std::lock_guard<std::mutex> lk(g_cache.mu);
+    for (auto& kv : g_cache.free_) cudaFree(kv.second);
+    g_cache.free_.clear();
+    g_cache.cached = 0;
+}
 
 int pcr_decode(pcr_record* rec, int k, void* out, void* stream) {
     if (!rec || !out || k < 1 || k > rec->G) return PCR_E_ARG;
