@@ -73,6 +73,44 @@ void* dev_alloc(size_t n, int device) {
     return p;
 }
 
+// internal streams and (non-timing) events are pooled the same way
+struct HandlePool {
+    std::mutex mu;
+    std::multimap<int, cudaStream_t> streams;
+    std::multimap<int, cudaEvent_t> events;
+} g_handles;
+
+cudaStream_t pool_stream_get(int device) {
+    {
+        std::lock_guard<std::mutex> lk(g_handles.mu);
+        auto it = g_handles.streams.find(device);
+        if (it != g_handles.streams.end()) { cudaStream_t q = it->second; g_handles.streams.erase(it); return q; }
+    }
+    cudaStream_t q = nullptr;
+    if (cudaStreamCreateWithFlags(&q, cudaStreamNonBlocking) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    return q;
+}
+void pool_stream_put(cudaStream_t q, int device) {
+    if (!q) return;
+    std::lock_guard<std::mutex> lk(g_handles.mu);
+    g_handles.streams.insert({device, q});
+}
+cudaEvent_t pool_event_get(int device) {
+    {
+        std::lock_guard<std::mutex> lk(g_handles.mu);
+        auto it = g_handles.events.find(device);
+        if (it != g_handles.events.end()) { cudaEvent_t e = it->second; g_handles.events.erase(it); return e; }
+    }
+    cudaEvent_t e = nullptr;
+    if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    return e;
+}
+void pool_event_put(cudaEvent_t e, int device) {
+    if (!e) return;
+    std::lock_guard<std::mutex> lk(g_handles.mu);
+    g_handles.events.insert({device, e});
+}
+
 void dev_release(void* p, size_t n, int device) {
     if (!p) return;
     const size_t cls = size_class(n);
@@ -281,26 +319,29 @@ int parse_chunk(const uint8_t* rec, uint64_t off, uint32_t len, bool first, Imag
 }
 
 void free_device(pcr_record* r) {
-    for (cudaStream_t q : r->streams) cudaStreamDestroy(q);
+    // nothing is handed on before the record's last decode has finished
+    if (r->ev_done && r->decode_enqueued) cudaEventSynchronize(r->ev_done);
+    r->decode_enqueued = false;
+    for (cudaStream_t q : r->streams) pool_stream_put(q, r->device);
     r->streams.clear();
-    if (r->ev_fork) cudaEventDestroy(r->ev_fork);
+    if (r->ev_fork) pool_event_put(r->ev_fork, r->device);
     r->ev_fork = nullptr;
-    if (r->copy_stream) cudaStreamDestroy(r->copy_stream);
+    if (r->copy_stream) pool_stream_put(r->copy_stream, r->device);
     r->copy_stream = nullptr;
-    if (r->clear_stream) cudaStreamDestroy(r->clear_stream);
+    if (r->clear_stream) pool_stream_put(r->clear_stream, r->device);
     r->clear_stream = nullptr;
-    if (r->ev_clear) cudaEventDestroy(r->ev_clear);
+    if (r->ev_clear) pool_event_put(r->ev_clear, r->device);
     r->ev_clear = nullptr;
-    for (cudaEvent_t e : r->ev_copy) cudaEventDestroy(e);
+    for (cudaEvent_t e : r->ev_copy) pool_event_put(e, r->device);
     r->ev_copy.clear();
-    for (cudaEvent_t e : r->ev_join) cudaEventDestroy(e);
+    for (cudaEvent_t e : r->ev_join) pool_event_put(e, r->device);
     r->ev_join.clear();
     for (cudaEvent_t e : r->events) cudaEventDestroy(e);
     r->events.clear();
     // buffers go back to the cache once the record's last decode has finished
     if (r->ev_done) {
         if (r->decode_enqueued) cudaEventSynchronize(r->ev_done);
-        cudaEventDestroy(r->ev_done);
+        pool_event_put(r->ev_done, r->device);
         r->ev_done = nullptr;
     }
     for (auto& b : r->bufs) dev_release(b.first, b.second, r->device);
@@ -528,24 +569,24 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     if ((rc = upload(r, &r->d_qtab, qtab))) return rc;
     r->h_status.assign(N, 0);
     r->resident = 0;
-    if (cudaEventCreateWithFlags(&r->ev_done, cudaEventDisableTiming) != cudaSuccess) return PCR_E_CUDA;
+    if (!(r->ev_done = pool_event_get(r->device))) return PCR_E_CUDA;
     // the zeroing above ran on the default stream; decodes may run on streams that do not wait for it
     if (cudaStreamSynchronize(cudaStreamLegacy) != cudaSuccess) return PCR_E_CUDA;
     if (r->n_slices > 1) {
-        if (cudaEventCreateWithFlags(&r->ev_fork, cudaEventDisableTiming) != cudaSuccess) return PCR_E_CUDA;
-        if (cudaStreamCreateWithFlags(&r->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return PCR_E_CUDA;
-        if (cudaStreamCreateWithFlags(&r->clear_stream, cudaStreamNonBlocking) != cudaSuccess) return PCR_E_CUDA;
-        if (cudaEventCreateWithFlags(&r->ev_clear, cudaEventDisableTiming) != cudaSuccess) return PCR_E_CUDA;
+        if (!(r->ev_fork = pool_event_get(r->device))) return PCR_E_CUDA;
+        if (!(r->copy_stream = pool_stream_get(r->device))) return PCR_E_CUDA;
+        if (!(r->clear_stream = pool_stream_get(r->device))) return PCR_E_CUDA;
+        if (!(r->ev_clear = pool_event_get(r->device))) return PCR_E_CUDA;
         for (int w = 0; w < r->n_waves; ++w) {
             cudaEvent_t e;
-            if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return PCR_E_CUDA;
+            if (!(e = pool_event_get(r->device))) return PCR_E_CUDA;
             r->ev_copy.push_back(e);
         }
         for (int g = 0; g < r->n_slices; ++g) {
             cudaStream_t q; cudaEvent_t e;
-            if (cudaStreamCreateWithFlags(&q, cudaStreamNonBlocking) != cudaSuccess) return PCR_E_CUDA;
+            if (!(q = pool_stream_get(r->device))) return PCR_E_CUDA;
             r->streams.push_back(q);
-            if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return PCR_E_CUDA;
+            if (!(e = pool_event_get(r->device))) return PCR_E_CUDA;
             r->ev_join.push_back(e);
         }
     }
