@@ -16,6 +16,7 @@
 #include <map>
 #include <mutex>
 #include <new>
+#include <thread>
 #include <utility>
 #include <vector>
 
@@ -387,8 +388,10 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     std::vector<uint16_t> qtab((size_t)N * 192);
     r->info.resize(N); r->blk_base.resize(N); r->nblk.resize(N);
     r->script.resize(G);
-    uint64_t blocks = 0, out_off = 0, segs = 0;
-    for (uint32_t i = 0; i < N; ++i) {
+    // every image's chunks are walked independently (a few host threads for large records); the
+    // running sums over images follow in one serial pass
+    std::vector<ScanScript> scripts((size_t)N * G);
+    auto parse_image = [&](uint32_t i) -> int {
         ImageParse im;
         const uint8_t* m = rec + meta_off + 16ull * i;
         for (uint32_t g = 0; g < G; ++g) {
@@ -400,8 +403,7 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
             ScanParse sp;
             int rc = parse_chunk(rec, off, clen, g == 0, im, sp);
             if (rc) return rc;
-            if (i == 0) r->script[g] = sp.sc;
-            else if (memcmp(&r->script[g], &sp.sc, sizeof(ScanScript)) != 0) return PCR_E_FORMAT;   // one script per record
+            scripts[(size_t)i * G + g] = sp.sc;
             ScanDesc& sd = scans[(size_t)g * N + i];
             sd.data_off = sp.data_off; sd.data_end = sp.data_end; sd.ri = sp.ri;
             // up to two distinct tables per scan
@@ -420,9 +422,6 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
                 total_mcu = (uint64_t)((wc + 7) / 8) * ((hc + 7) / 8);
             }
             sd.nseg = sd.ri ? (uint32_t)((total_mcu + sd.ri - 1) / sd.ri) : 1u;
-            sd.seg_base = (uint32_t)segs;
-            segs += sd.nseg + 1;                      // one closing entry per (scan, image)
-            if (segs >= (1ull << 32)) return PCR_E_FORMAT;
         }
         if (!im.have_frame) return PCR_E_FORMAT;
         if (rd32(m + 4) != im.W || rd32(m + 8) != im.H) return PCR_E_FORMAT;   // metadata and frame header agree
@@ -430,13 +429,42 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
             if (!im.qdef[im.tq[c]]) return PCR_E_FORMAT;
             memcpy(&qtab[(size_t)i * 192 + 64 * c], im.q[im.tq[c]], 128);
         }
-        uint32_t mx = (im.W + 15) / 16, my = (im.H + 15) / 16;
         pcr_image_info& inf = r->info[i];
         inf.width = im.W; inf.height = im.H; inf.label = (int32_t)rd32(m); inf.rsvd = 0;
-        inf.out_offset = out_off; inf.out_bytes = 3ull * im.W * im.H;
+        inf.out_bytes = 3ull * im.W * im.H;
+        imgs[i].W = im.W; imgs[i].H = im.H; imgs[i].mx = (im.W + 15) / 16; imgs[i].my = (im.H + 15) / 16;
+        return PCR_OK;
+    };
+    {
+        const unsigned hw = std::max(1u, std::thread::hardware_concurrency());
+        const unsigned nthreads = N >= 256 ? std::min(4u, hw) : 1u;
+        std::vector<int> rcs(nthreads, PCR_OK);
+        auto work = [&](unsigned t) {
+            for (uint32_t i = t; i < N; i += nthreads) {
+                const int rc = parse_image(i);
+                if (rc != PCR_OK) { rcs[t] = rc; return; }
+            }
+        };
+        std::vector<std::thread> pool;
+        for (unsigned t = 1; t < nthreads; ++t) pool.emplace_back(work, t);
+        work(0);
+        for (auto& th : pool) th.join();
+        for (int rc : rcs) if (rc != PCR_OK) return rc;
+    }
+    uint64_t blocks = 0, out_off = 0, segs = 0;
+    for (uint32_t g = 0; g < G; ++g) r->script[g] = scripts[g];
+    for (uint32_t i = 0; i < N; ++i) {
+        if (i && memcmp(&scripts[(size_t)i * G], &scripts[0], sizeof(ScanScript) * G) != 0) return PCR_E_FORMAT;   // one script per record
+        for (uint32_t g = 0; g < G; ++g) {
+            ScanDesc& sd = scans[(size_t)g * N + i];
+            sd.seg_base = (uint32_t)segs;
+            segs += sd.nseg + 1;                      // one closing entry per (scan, image)
+            if (segs >= (1ull << 32)) return PCR_E_FORMAT;
+        }
+        pcr_image_info& inf = r->info[i];
+        inf.out_offset = out_off;
         out_off += (inf.out_bytes + 127) & ~127ull;
-        r->blk_base[i] = blocks; r->nblk[i] = 6ull * mx * my;
-        imgs[i].W = im.W; imgs[i].H = im.H; imgs[i].mx = mx; imgs[i].my = my;
+        r->blk_base[i] = blocks; r->nblk[i] = 6ull * imgs[i].mx * imgs[i].my;
         imgs[i].blk_base = blocks; imgs[i].out_off = inf.out_offset;
         blocks += r->nblk[i];
     }
@@ -469,6 +497,7 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
         for (int g = 0; g <= r->n_slices; ++g) r->slice_img[g] = (uint32_t)((uint64_t)N * g / r->n_slices);
     }
     std::vector<Item> items;
+    items.reserve((size_t)(segs / 24 + (uint64_t)N * G));
     r->item_begin.assign((size_t)r->n_slices * G, 0); r->item_count.assign((size_t)r->n_slices * G, 0);
     for (int g = 0; g < r->n_slices; ++g)
         for (int w = 0; w < r->n_waves; ++w)
@@ -496,6 +525,7 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
                 r->item_count[(size_t)g * G + s] = (uint32_t)items.size() - r->item_begin[(size_t)g * G + s];
             }
     std::vector<Unit> units;
+    units.reserve((size_t)(blocks / 24 + N));
     r->slice_unit.assign(r->n_slices + 1, 0);
     for (int g = 0; g < r->n_slices; ++g) {
         r->slice_unit[g] = (uint32_t)units.size();
