@@ -390,7 +390,7 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
                 uint64_t blk;
                 if (inter && c == 0) blk = g.coff[0] + (uint64_t)(2 * mrow + (j >> 1)) * g.bw[0] + 2 * mcol + (j & 1);
                 else blk = g.coff[c] + (uint64_t)mrow * g.bw[c] + mcol;
-                int16_t* dcv = P.dcplane + blk;
+                int16_t* dcv = P.head + blk * 8;
                 if (sc.Ah == 0) {
                     const HuffTab& tab = tabs[wid][(sd.slots >> (2 * ci)) & 1u];
                     const uint32_t e = huff_lookup(tab, win);
@@ -402,10 +402,9 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
                     if (c == 0) pred0 = pv; else if (c == 1) pred1 = pv; else pred2 = pv;
                     *dcv = (int16_t)(pv << Al);
                 } else {
-                    // two neighbouring blocks share a 32-bit word of the DC plane; the other block may
-                    // belong to another lane, so the bit is set atomically on the whole word
-                    if (win >> 31)
-                        atomicOr(reinterpret_cast<unsigned int*>(P.dcplane + (blk & ~1ull)), (unsigned int)p1 << (16 * (int)(blk & 1ull)));
+                    // coefficient 0 is the low half of the block's first head word; position 1 in the
+                    // upper half may be written by an AC scan of the same wave, hence the atomic
+                    if (win >> 31) atomicOr(reinterpret_cast<unsigned int*>(dcv), (unsigned int)p1);
                     br.skip(1);
                 }
                 if (++j == bpm) {
@@ -431,6 +430,7 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
             // ---- AC first pass: one Huffman symbol per step
             uint64_t* maskp = P.aux + ax.base + g.loff[c];
             int16_t* plane = P.planes + g.coff[c] * 64;
+            int16_t* headp = P.head + g.coff[c] * 8;
             uint64_t M = 0;
             int k = Ss;
             for (;;) {
@@ -452,7 +452,9 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
                     const uint32_t xb = top_bits(win << len, extra);       // magnitude bits / run length bits
                     br.skip(len + extra);
                     if (is_coef && !fail) {
-                        plane[(uint64_t)bi * 64 + kk] = (int16_t)(extend_bits(xb, sz) * p1);
+                        const int16_t val = (int16_t)(extend_bits(xb, sz) * p1);
+                        if (kk < 8) headp[(uint64_t)bi * 8 + kk] = val;
+                        else plane[(uint64_t)bi * 64 + kk] = val;
                         M |= 1ull << kk;
                     }
                     k = is_coef ? kk + 1 : (is_eob ? k : k + 16);

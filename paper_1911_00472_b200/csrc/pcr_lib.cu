@@ -159,7 +159,7 @@ struct pcr_record {
     uint8_t* d_ubuf = nullptr;
     size_t resident = 0;
     int16_t* d_planes = nullptr;
-    int16_t* d_dcplane = nullptr;
+    int16_t* d_head = nullptr;
     int decoded_k = 0;            // fidelity of the state the planes and side data hold (0: none)
     bool dc_merged = true;        // the planes hold the DC coefficients of the last decode
     bool planes_cleared = true;   // ... and zeros wherever the last decode left no coefficient
@@ -584,8 +584,8 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     if (int rc = take(r, &r->d_ubuf, (size_t)(len + 256))) return rc;
     if (cudaMemset(r->d_ubuf, 0, len + 256) != cudaSuccess) return PCR_E_CUDA;
     if (int rc = take(r, &r->d_planes, (size_t)(std::max<uint64_t>(blocks, 1) * 128))) return rc;
-    if (int rc = take(r, &r->d_dcplane, (size_t)(std::max<uint64_t>(blocks, 2) * 2 + 16))) return rc;
-    if (cudaMemset(r->d_dcplane, 0, std::max<uint64_t>(blocks, 2) * 2 + 16) != cudaSuccess) return PCR_E_CUDA;
+    if (int rc = take(r, &r->d_head, (size_t)(std::max<uint64_t>(blocks, 1) * 16))) return rc;
+    if (cudaMemset(r->d_head, 0, std::max<uint64_t>(blocks, 1) * 16) != cudaSuccess) return PCR_E_CUDA;
     if (int rc = take(r, &r->d_seg, (size_t)((segs + 1) * 4))) return rc;
     if (int rc = take(r, &r->d_status, (size_t)((size_t)N * 4))) return rc;
     if (cudaMemset(r->d_seg, 0, (segs + 1) * 4) != cudaSuccess || cudaMemset(r->d_status, 0, (size_t)N * 4) != cudaSuccess) return PCR_E_CUDA;
@@ -697,7 +697,7 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream)
     mark("h2d", 0);
     if (k0 == 0 && cudaMemsetAsync(rec->d_status, 0, (size_t)rec->N * 4, st) != cudaSuccess) return PCR_E_CUDA;
     Params P;
-    P.rec = rec->d_rec; P.ubuf = rec->d_ubuf; P.planes = rec->d_planes; P.dcplane = rec->d_dcplane; P.script = rec->d_script; P.scans = rec->d_scans;
+    P.rec = rec->d_rec; P.ubuf = rec->d_ubuf; P.planes = rec->d_planes; P.head = rec->d_head; P.script = rec->d_script; P.scans = rec->d_scans;
     P.saux = rec->d_saux; P.aux = rec->d_aux;
     P.imgs = rec->d_imgs; P.seg_start = rec->d_seg; P.items = rec->d_items; P.units = rec->d_units;
     P.qtab = rec->d_qtab; P.status = rec->d_status; P.N = rec->N;
@@ -716,11 +716,14 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream)
             any_refine = true;
         }
     }
-    bool dc_only = true;
-    for (int s = 0; s < k; ++s) if (rec->script[s].Ss > 0) dc_only = false;
+    bool dc_only = true, head_only = true;      // no AC scan at all / no scan beyond zigzag position 7
+    for (int s = 0; s < k; ++s) {
+        if (rec->script[s].Ss > 0) dc_only = false;
+        if (rec->script[s].Se > 7) head_only = false;
+    }
     rec->dc_merged = false;
     // the planes must be zero before the first AC scan writes into them
-    const bool clear_planes = !dc_only && (k0 == 0 || !rec->planes_cleared);
+    const bool clear_planes = !head_only && (k0 == 0 || !rec->planes_cleared);
     const bool clear_dc = k0 == 0;
     if (k0 == 0) rec->planes_cleared = false;
     if (clear_planes) rec->planes_cleared = true;
@@ -736,7 +739,7 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream)
         if (stage == 0) {
             if (pipelined) return true;           // zeroed once for all slices on the clear stream
             const uint64_t b0 = rec->blk_base[i0], b1 = (i1 < (uint32_t)rec->N) ? rec->blk_base[i1] : rec->total_blocks;
-            if (clear_dc && cudaMemsetAsync(rec->d_dcplane + b0, 0, (b1 - b0) * 2, q) != cudaSuccess) return false;
+            if (clear_dc && cudaMemsetAsync(rec->d_head + b0 * 8, 0, (b1 - b0) * 16, q) != cudaSuccess) return false;
             if (!clear_planes) return true;       // no AC scan yet, or already zeroed by the decode this one continues
             return cudaMemsetAsync(rec->d_planes + b0 * 64, 0, (b1 - b0) * 128, q) == cudaSuccess;
         }
@@ -782,6 +785,8 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream)
         if (stage == 2 + W) return true;      // the refinement side data is folded in by the pixel kernel
         if (nu) {
             if (dc_only) pixel_kernel<false, 2><<<nu, kPixThreads, 0, q>>>(Q, fl, static_cast<uint8_t*>(out));
+            else if (head_only && any_refine) pixel_kernel<true, 3><<<nu, kPixThreads, 0, q>>>(Q, fl, static_cast<uint8_t*>(out));
+            else if (head_only) pixel_kernel<false, 3><<<nu, kPixThreads, 0, q>>>(Q, fl, static_cast<uint8_t*>(out));
             else if (any_refine) pixel_kernel<true, 1><<<nu, kPixThreads, 0, q>>>(Q, fl, static_cast<uint8_t*>(out));
             else pixel_kernel<false, 1><<<nu, kPixThreads, 0, q>>>(Q, fl, static_cast<uint8_t*>(out));
             ++g_launches;
@@ -829,7 +834,7 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream)
         // missing record bytes arrive on a copy stream, the scan groups of each wave behind an event
         if (cudaEventRecord(rec->ev_fork, st) != cudaSuccess) return PCR_E_CUDA;
         if (cudaStreamWaitEvent(rec->clear_stream, rec->ev_fork, 0) != cudaSuccess) return PCR_E_CUDA;
-        if (clear_dc && cudaMemsetAsync(rec->d_dcplane, 0, rec->total_blocks * 2, rec->clear_stream) != cudaSuccess) return PCR_E_CUDA;
+        if (clear_dc && cudaMemsetAsync(rec->d_head, 0, rec->total_blocks * 16, rec->clear_stream) != cudaSuccess) return PCR_E_CUDA;
         if (clear_planes && cudaMemsetAsync(rec->d_planes, 0, rec->total_blocks * 128, rec->clear_stream) != cudaSuccess) return PCR_E_CUDA;
         if (cudaEventRecord(rec->ev_clear, rec->clear_stream) != cudaSuccess) return PCR_E_CUDA;
         if (rec->resident < need) {
@@ -907,8 +912,8 @@ int pcr_coeffs(pcr_record* rec, const int16_t** dev_planes, size_t* bytes) {
     if (!rec->dc_merged && rec->total_blocks) {
         Params P;
         memset(&P, 0, sizeof P);
-        P.planes = rec->d_planes; P.dcplane = rec->d_dcplane;
-        merge_dc_kernel<<<(unsigned)((rec->total_blocks + 255) / 256), 256>>>(P, rec->total_blocks);
+        P.planes = rec->d_planes; P.head = rec->d_head;
+        merge_head_kernel<<<(unsigned)((rec->total_blocks + 255) / 256), 256>>>(P, rec->total_blocks);
         ++g_launches;
         if (cudaDeviceSynchronize() != cudaSuccess) return PCR_E_CUDA;
         rec->dc_merged = true;

@@ -73,9 +73,10 @@ __device__ __forceinline__ uint32_t pack4_sat(int v0, int v1, int v2, int v3) {
 // registers cannot do.  A correction moves a non-zero coefficient away from zero by 2^Al if its
 // bit Al is still clear; a new coefficient is +-2^Al.
 //
-// kDcMode: 0 = the DC coefficient sits in the block's line; 1 = it comes from the dense DC plane
-// (the line's first coefficient is ignored); 2 = the block has nothing but its DC coefficient (no
-// AC scan decoded): the line is not read at all and the transform collapses to one value.
+// kDcMode: 0 = all 64 coefficients sit in the block's line; 1 = positions 0..7 come from the dense
+// head plane (the line's first 16 bytes are ignored); 2 = the block has nothing but its DC
+// coefficient (no AC scan decoded): only the head plane is read and the transform collapses to
+// one value; 3 = no decoded scan reaches beyond position 7: the lines are not read at all.
 template <bool kRefine, int kDcMode>
 __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeList fl, uint8_t* __restrict__ out) {
     __shared__ __align__(16) uint32_t s_line[kRefine ? 32 * kPixThreads : 1];
@@ -115,7 +116,7 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
         if (valid && kDcMode == 2) {
             // all AC zero: both passes keep only the k = 0 term, every sample of the block is equal
             constexpr uint32_t K4 = 5793;
-            const int F = (int)P.dcplane[blk] * (int)s_q[comp][0];
+            const int F = (int)P.head[blk * 8] * (int)s_q[comp][0];
             const int T = (int)(K4 * (uint32_t)F + (1u << 11)) >> 12;
             const int smp = (int)(K4 * (uint32_t)T + (1u << 15) + (128u << 16)) >> 16;
             const uint32_t w = pack4_sat(smp, smp, smp, smp);
@@ -128,9 +129,16 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
         } else if (valid) {
             uint4* line = reinterpret_cast<uint4*>(P.planes + blk * 64);
             uint4 raw[8];
+            const uint4* headv = reinterpret_cast<const uint4*>(P.head + blk * 8);
             if (kRefine && fl.n[comp] > 0) {
+                if (kDcMode == 3) {
 #pragma unroll
-                for (int q = 0; q < 8; ++q) raw[q] = line[q];
+                    for (int q = 1; q < 8; ++q) raw[q] = make_uint4(0, 0, 0, 0);
+                } else {
+#pragma unroll
+                    for (int q = (kDcMode == 0 ? 0 : 1); q < 8; ++q) raw[q] = line[q];
+                }
+                if (kDcMode != 0) raw[0] = *headv;
                 uint32_t* col = s_line + tid;
 #pragma unroll
                 for (int q = 0; q < 8; ++q) {
@@ -167,14 +175,20 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
                     for (int q = 0; q < 8; ++q) {
                         raw[q] = make_uint4(col[(4 * q) * kPixThreads], col[(4 * q + 1) * kPixThreads],
                                             col[(4 * q + 2) * kPixThreads], col[(4 * q + 3) * kPixThreads]);
-                        line[q] = raw[q];
+                        if (q == 0 && kDcMode != 0) *reinterpret_cast<uint4*>(P.head + blk * 8) = raw[0];
+                        else if (kDcMode != 3) line[q] = raw[q];
                     }
                 }
             } else {
+                if (kDcMode == 3) {
 #pragma unroll
-                for (int q = 0; q < 8; ++q) raw[q] = __ldg(line + q);
+                    for (int q = 1; q < 8; ++q) raw[q] = make_uint4(0, 0, 0, 0);
+                } else {
+#pragma unroll
+                    for (int q = (kDcMode == 0 ? 0 : 1); q < 8; ++q) raw[q] = __ldg(line + q);
+                }
+                if (kDcMode != 0) raw[0] = __ldg(headv);
             }
-            if (kDcMode == 1) raw[0].x = (raw[0].x & 0xFFFF0000u) | (uint32_t)(uint16_t)P.dcplane[blk];
             const uint32_t* qw = reinterpret_cast<const uint32_t*>(&s_q[comp][0]);
             uint32_t v[64];
 #pragma unroll
@@ -275,10 +289,10 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
     }
 }
 
-// Copies the DC plane into coefficient 0 of every block (for readers of the full planes).
-__global__ void __launch_bounds__(256) merge_dc_kernel(Params P, uint64_t n_blocks) {
+// Copies the head plane into positions 0..7 of every block (for readers of the full planes).
+__global__ void __launch_bounds__(256) merge_head_kernel(Params P, uint64_t n_blocks) {
     const uint64_t b = (uint64_t)blockIdx.x * 256 + threadIdx.x;
-    if (b < n_blocks) P.planes[b * 64] = P.dcplane[b];
+    if (b < n_blocks) *reinterpret_cast<uint4*>(P.planes + b * 64) = *reinterpret_cast<const uint4*>(P.head + b * 8);
 }
 
 }  // namespace pcr

@@ -77,9 +77,11 @@ struct Params {
     const uint8_t* rec;         // record bytes on the device
     uint8_t* ubuf;              // entropy-coded bytes without stuffing, big-endian words
     int16_t* planes;            // coefficient planes, 64 int16 per block, zigzag order
-    int16_t* dcplane;           // DC coefficient of every block, dense (same block numbering); the DC
-                                // scans write here, so their stores fill whole sectors instead of
-                                // touching one 128-byte line per block
+    int16_t* head;              // zigzag positions 0..7 of every block, dense (8 int16 = 16 bytes per
+                                // block, same block numbering).  First passes store these positions
+                                // here and only positions 8..63 in the 128-byte line: the dense
+                                // plane stays in L2 while it is written, instead of one cold
+                                // 128-byte line being read and written back per coefficient
     const ScanScript* script;   // [G]
     const ScanAux* saux;        // [G]
     uint64_t* aux;              // side data of the AC scans
