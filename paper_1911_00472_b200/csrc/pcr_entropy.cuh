@@ -174,7 +174,7 @@ __global__ void __launch_bounds__(256) unstuff_index_kernel(Params P, ScanList s
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (warp >= sl.n * nimg) return;
-    const int img = img0 + warp % nimg;
+    const int img = (int)P.order[img0 + warp % nimg];      // img0, nimg: a run of the processing order
     const ScanDesc sd = P.scans[sl.s[warp / nimg] * P.N + img];
     uint32_t* seg = P.seg_start + sd.seg_base;
     const uint32_t a = sd.data_off, b = sd.data_end;
@@ -330,10 +330,11 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
     const bool dc = sc.Ss == 0;
     const bool huff = !(dc && sc.Ah != 0);
     // tables: a DC scan may use two tables of one image; an AC item may span two images
-    const bool two_images = item.rsvd != 0;
+    const bool two_images = item.next != 0;
+    const uint32_t si1 = two_images ? item.next - 1u : item.si;
     if (huff) {
         build_hufftab(tabs[wid][0], P.rec + sd0.tab_off[0], lane);
-        if (two_images) build_hufftab(tabs[wid][1], P.rec + P.scans[item.si + 1].tab_off[0], lane);
+        if (two_images) build_hufftab(tabs[wid][1], P.rec + P.scans[si1].tab_off[0], lane);
         else if (sd0.tab_off[1]) build_hufftab(tabs[wid][1], P.rec + sd0.tab_off[1], lane);
     }
     // From here on no lane leaves before the warp does: lanes without work just stay `done`.
@@ -341,8 +342,8 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
     const uint32_t rem0 = sd0.nseg - item.seg0;               // restart intervals left in the first image
     const int which = (two_images && (uint32_t)lane >= rem0) ? 1 : 0;
     uint32_t seg = which ? (uint32_t)lane - rem0 : item.seg0 + lane;
-    const ScanDesc sd = which ? P.scans[item.si + 1] : sd0;
-    const int img = (int)(item.si % P.N) + which;
+    const ScanDesc sd = which ? P.scans[si1] : sd0;
+    const int img = (int)((which ? si1 : item.si) % (uint32_t)P.N);
     if (seg >= sd.nseg) { done = true; seg = 0; }
     const ImgDesc im = P.imgs[img];
     const Geometry g = make_geometry(im);

@@ -145,6 +145,8 @@ struct pcr_record {
     std::vector<uint32_t> slice_unit;                           // [n_slices + 1] first pixel unit of each slice
     std::vector<uint32_t> item_begin, item_count;               // [n_slices][G]
     std::vector<cudaStream_t> streams;                          // one per slice
+    std::vector<cudaEvent_t> ev_index;                          // [n_waves] index of wave w done (side stream)
+    cudaEvent_t ev_start = nullptr;                             // index of the first wave done
     cudaEvent_t ev_fork = nullptr;
     cudaStream_t copy_stream = nullptr;                         // host-to-device copies of later scan groups
     cudaStream_t clear_stream = nullptr;                        // zeroing of the planes, beside the index kernels
@@ -173,6 +175,7 @@ struct pcr_record {
     Item* d_items = nullptr;
     Unit* d_units = nullptr;
     uint16_t* d_qtab = nullptr;
+    uint32_t* d_order = nullptr;  // processing order of the images (slices are runs of it)
     int* d_status = nullptr;
     std::vector<int> h_status;
     std::vector<std::pair<void*, size_t>> bufs;   // every device buffer of the record with its size
@@ -325,6 +328,10 @@ void free_device(pcr_record* r) {
     r->decode_enqueued = false;
     for (cudaStream_t q : r->streams) pool_stream_put(q, r->device);
     r->streams.clear();
+    if (r->ev_start) pool_event_put(r->ev_start, r->device);
+    r->ev_start = nullptr;
+    for (cudaEvent_t e : r->ev_index) pool_event_put(e, r->device);
+    r->ev_index.clear();
     if (r->ev_fork) pool_event_put(r->ev_fork, r->device);
     r->ev_fork = nullptr;
     if (r->copy_stream) pool_stream_put(r->copy_stream, r->device);
@@ -496,6 +503,17 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
         r->slice_img.resize(r->n_slices + 1);
         for (int g = 0; g <= r->n_slices; ++g) r->slice_img[g] = (uint32_t)((uint64_t)N * g / r->n_slices);
     }
+    // Processing order of the images: a slice is a run of this order.  The time a slice needs for
+    // its entropy waves is set by its longest restart interval, i.e. by its widest image, so the
+    // images are sorted by decreasing width: slices of narrow images finish their waves early and
+    // their pixel stage overlaps the waves of the wide ones.
+    std::vector<uint32_t> order(N);
+    for (uint32_t i = 0; i < N; ++i) order[i] = i;
+    if (r->n_slices > 1)
+        std::stable_sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) {
+            if (imgs[a].mx != imgs[b].mx) return imgs[a].mx > imgs[b].mx;
+            return imgs[a].my > imgs[b].my;
+        });
     std::vector<Item> items;
     items.reserve((size_t)(segs / 24 + (uint64_t)N * G));
     r->item_begin.assign((size_t)r->n_slices * G, 0); r->item_count.assign((size_t)r->n_slices * G, 0);
@@ -504,24 +522,25 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
             for (int s : r->wave_scans[w]) {
                 r->item_begin[(size_t)g * G + s] = (uint32_t)items.size();
                 const bool ac = r->script[s].Ss > 0;
-                for (uint32_t i = r->slice_img[g]; i < r->slice_img[g + 1]; ++i) {
+                for (uint32_t pos = r->slice_img[g]; pos < r->slice_img[g + 1]; ++pos) {
+                    const uint32_t i = order[pos];
                     const ScanDesc& sd = scans[(size_t)s * N + i];
                     // full warps of 32 restart intervals; in AC scans the last warp of an image
                     // runs on into the first intervals of the next image (two tables per warp)
                     uint32_t j = 0;
-                    if (ac && !items.empty() && items.back().rsvd == 2) {     // continued from the previous image
+                    if (ac && !items.empty() && items.back().next == kItemOpen) {     // continued from the previous image
                         Item& prev = items.back();
                         const uint32_t take = std::min<uint32_t>(kSegsPerItem - prev.count, sd.nseg);
-                        prev.count += take; prev.rsvd = 1;
+                        prev.count += take; prev.next = (uint32_t)(s * N + i) + 1u;
                         j = take;
                     }
                     for (; j < sd.nseg; j += kSegsPerItem) {
                         const uint32_t cnt = std::min<uint32_t>(kSegsPerItem, sd.nseg - j);
-                        // rsvd == 2 marks an unfilled last item that the next image may extend
-                        items.push_back(Item{(uint32_t)(s * N + i), j, cnt, (ac && cnt < (uint32_t)kSegsPerItem) ? 2u : 0u});
+                        // kItemOpen marks an unfilled last item that the next image may extend
+                        items.push_back(Item{(uint32_t)(s * N + i), j, cnt, (ac && cnt < (uint32_t)kSegsPerItem) ? kItemOpen : 0u});
                     }
                 }
-                if (!items.empty() && items.back().rsvd == 2) items.back().rsvd = 0;
+                if (!items.empty() && items.back().next == kItemOpen) items.back().next = 0;
                 r->item_count[(size_t)g * G + s] = (uint32_t)items.size() - r->item_begin[(size_t)g * G + s];
             }
     std::vector<Unit> units;
@@ -529,8 +548,8 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     r->slice_unit.assign(r->n_slices + 1, 0);
     for (int g = 0; g < r->n_slices; ++g) {
         r->slice_unit[g] = (uint32_t)units.size();
-        for (uint32_t i = r->slice_img[g]; i < r->slice_img[g + 1]; ++i)
-            for (uint32_t row = 0; row < imgs[i].my; ++row)
+        for (uint32_t pos = r->slice_img[g]; pos < r->slice_img[g + 1]; ++pos)
+            for (uint32_t i = order[pos], row = 0; row < imgs[i].my; ++row)
                 for (uint32_t col = 0; col < imgs[i].mx; col += kPixMcus) {
                     if (imgs[i].my > 65535 || imgs[i].mx > 65535) return PCR_E_FORMAT;
                     units.push_back(Unit{i, (uint16_t)row, (uint16_t)col});
@@ -597,6 +616,7 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     if ((rc = upload(r, &r->d_items, items))) return rc;
     if ((rc = upload(r, &r->d_units, units))) return rc;
     if ((rc = upload(r, &r->d_qtab, qtab))) return rc;
+    if ((rc = upload(r, &r->d_order, order))) return rc;
     r->h_status.assign(N, 0);
     r->resident = 0;
     if (!(r->ev_done = pool_event_get(r->device))) return PCR_E_CUDA;
@@ -607,10 +627,13 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
         if (!(r->copy_stream = pool_stream_get(r->device))) return PCR_E_CUDA;
         if (!(r->clear_stream = pool_stream_get(r->device))) return PCR_E_CUDA;
         if (!(r->ev_clear = pool_event_get(r->device))) return PCR_E_CUDA;
+        if (!(r->ev_start = pool_event_get(r->device))) return PCR_E_CUDA;
         for (int w = 0; w < r->n_waves; ++w) {
             cudaEvent_t e;
             if (!(e = pool_event_get(r->device))) return PCR_E_CUDA;
             r->ev_copy.push_back(e);
+            if (!(e = pool_event_get(r->device))) return PCR_E_CUDA;
+            r->ev_index.push_back(e);
         }
         for (int g = 0; g < r->n_slices; ++g) {
             cudaStream_t q; cudaEvent_t e;
@@ -618,6 +641,7 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
             r->streams.push_back(q);
             if (!(e = pool_event_get(r->device))) return PCR_E_CUDA;
             r->ev_join.push_back(e);
+
         }
     }
     return PCR_OK;
@@ -700,7 +724,7 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream)
     P.rec = rec->d_rec; P.ubuf = rec->d_ubuf; P.planes = rec->d_planes; P.head = rec->d_head; P.script = rec->d_script; P.scans = rec->d_scans;
     P.saux = rec->d_saux; P.aux = rec->d_aux;
     P.imgs = rec->d_imgs; P.seg_start = rec->d_seg; P.items = rec->d_items; P.units = rec->d_units;
-    P.qtab = rec->d_qtab; P.status = rec->d_status; P.N = rec->N;
+    P.qtab = rec->d_qtab; P.order = rec->d_order; P.status = rec->d_status; P.N = rec->N;
     FinalizeList fl;
     memset(&fl, 0, sizeof fl);
     bool any_refine = false;
@@ -733,15 +757,29 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream)
     // the stages of one slice; stage numbers: 0 clear, 1 index, 2+w entropy wave w, 2+W unused, 3+W pixels
     // (the pixel kernel also folds the refinement side data into the planes)
     const int W = rec->n_waves;
+    std::vector<char> indexed(rec->n_waves, 0);     // wave w of the current slice has an index launch to wait for
+    // restart-interval index of wave w of slice g on stream q: 1 launched, 0 nothing to do, -1 error
+    auto launch_index = [&](int w, cudaStream_t q) -> int {
+        ScanList sl;
+        sl.n = 0;
+        for (int s : rec->wave_scans[w]) if (s >= k0 && s < k) sl.s[sl.n++] = s;
+        if (!sl.n) return 0;
+        const uint32_t i0 = 0, i1 = (uint32_t)rec->N;      // one launch covers every slice
+        if (copied[w] && cudaStreamWaitEvent(q, rec->ev_copy[w], 0) != cudaSuccess) return -1;
+        const uint32_t warps = (uint32_t)sl.n * (i1 - i0);
+        unstuff_index_kernel<<<(warps + 7) / 8, 256, 0, q>>>(P, sl, (int)i0, (int)(i1 - i0));
+        ++g_launches;
+        return 1;
+    };
     auto run_stage = [&](int stage, int g, cudaStream_t q) -> bool {
         const uint32_t i0 = rec->slice_img[g], i1 = rec->slice_img[g + 1];
         const uint32_t u0 = rec->slice_unit[g], nu = rec->slice_unit[g + 1] - u0;
         if (stage == 0) {
             if (pipelined) return true;           // zeroed once for all slices on the clear stream
-            const uint64_t b0 = rec->blk_base[i0], b1 = (i1 < (uint32_t)rec->N) ? rec->blk_base[i1] : rec->total_blocks;
-            if (clear_dc && cudaMemsetAsync(rec->d_head + b0 * 8, 0, (b1 - b0) * 16, q) != cudaSuccess) return false;
+            if (g != 0) return true;              // the first slice zeroes for all (a slice's blocks are not contiguous)
+            if (clear_dc && cudaMemsetAsync(rec->d_head, 0, rec->total_blocks * 16, q) != cudaSuccess) return false;
             if (!clear_planes) return true;       // no AC scan yet, or already zeroed by the decode this one continues
-            return cudaMemsetAsync(rec->d_planes + b0 * 64, 0, (b1 - b0) * 128, q) == cudaSuccess;
+            return cudaMemsetAsync(rec->d_planes, 0, rec->total_blocks * 128, q) == cudaSuccess;
         }
         if (stage == 1) {
             if (pipelined) return true;          // done wave by wave, as the bytes arrive
@@ -756,16 +794,12 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream)
         if (stage < 2 + W) {
             const int w = stage - 2;
             if (pipelined) {
-                ScanList sl;
-                sl.n = 0;
-                for (int s : rec->wave_scans[w]) if (s >= k0 && s < k) sl.s[sl.n++] = s;
-                if (sl.n) {
-                    if (copied[w] && cudaStreamWaitEvent(q, rec->ev_copy[w], 0) != cudaSuccess) return false;
-                    const uint32_t warps = (uint32_t)sl.n * (i1 - i0);
-                    unstuff_index_kernel<<<(warps + 7) / 8, 256, 0, q>>>(P, sl, (int)i0, (int)(i1 - i0));
-                    ++g_launches;
+                if (w == 0) {
+                    if (cudaStreamWaitEvent(q, rec->ev_clear, 0) != cudaSuccess) return false;
+                } else if (indexed[w]) {
+                    // the later waves were indexed on the side stream, beside the first wave
+                    if (cudaStreamWaitEvent(q, rec->ev_index[w], 0) != cudaSuccess) return false;
                 }
-                if (w == 0 && cudaStreamWaitEvent(q, rec->ev_clear, 0) != cudaSuccess) return false;
             }
             uint32_t begin = 0, count = 0;
             bool any = false;
@@ -855,14 +889,29 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream)
                 }
             }
         }
+        // restart-interval index, one launch per wave for all slices: the first wave's on the caller's
+        // stream, the later waves' on the side stream behind the memsets, beside the first entropy wave
+        if (launch_index(0, st) < 0) return PCR_E_CUDA;
+        if (cudaEventRecord(rec->ev_start, st) != cudaSuccess) return PCR_E_CUDA;
+        for (int w = 1; w < W; ++w) {
+            const int li = launch_index(w, rec->clear_stream);
+            if (li < 0) return PCR_E_CUDA;
+            indexed[w] = li > 0;
+            if (li > 0 && cudaEventRecord(rec->ev_index[w], rec->clear_stream) != cudaSuccess) return PCR_E_CUDA;
+        }
         for (int g = 0; g < rec->n_slices; ++g) {
             cudaStream_t q = rec->streams[g];
-            if (cudaStreamWaitEvent(q, rec->ev_fork, 0) != cudaSuccess) return PCR_E_CUDA;
+            if (cudaStreamWaitEvent(q, rec->ev_start, 0) != cudaSuccess) return PCR_E_CUDA;
             for (int stage = 0; stage < n_stages; ++stage)
                 if (!run_stage(stage, g, q)) return PCR_E_CUDA;
             if (cudaEventRecord(rec->ev_join[g], q) != cudaSuccess) return PCR_E_CUDA;
             if (cudaStreamWaitEvent(st, rec->ev_join[g], 0) != cudaSuccess) return PCR_E_CUDA;
         }
+        // the side and copy streams rejoin the caller's stream too (implied by the slices' waits
+        // whenever they carried work; stated so that every fork is joined)
+        if (cudaEventRecord(rec->ev_clear, rec->clear_stream) != cudaSuccess) return PCR_E_CUDA;
+        if (cudaStreamWaitEvent(st, rec->ev_clear, 0) != cudaSuccess) return PCR_E_CUDA;
+        if (copied[W - 1] && cudaStreamWaitEvent(st, rec->ev_copy[W - 1], 0) != cudaSuccess) return PCR_E_CUDA;
     }
     if (cudaEventRecord(rec->ev_done, st) != cudaSuccess) return PCR_E_CUDA;
     rec->decode_enqueued = true;

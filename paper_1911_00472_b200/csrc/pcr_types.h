@@ -64,8 +64,9 @@ struct Item {
     uint32_t si;          // scan * N + image
     uint32_t seg0;        // first restart interval of the item
     uint32_t count;       // restart intervals in the item (<= kSegsPerItem)
-    uint32_t rsvd;        // 1: the item runs on into the first intervals of the next image
+    uint32_t next;        // 0, or 1 + (scan * N + image) of the image whose first intervals the item runs on into
 };
+constexpr uint32_t kItemOpen = 0xFFFFFFFFu;   // host only, while the list is built: the item may still be extended
 
 // Pixel work unit: a run of MCUs in one MCU row of one image.
 struct Unit {
@@ -91,6 +92,7 @@ struct Params {
     const Item* items;
     const Unit* units;
     const uint16_t* qtab;       // [N][3][64] quantisers, zigzag order
+    const uint32_t* order;      // [N] processing order of the images
     int* status;                // [N]
     int32_t N;
 };
