@@ -197,3 +197,43 @@ def _pool_worker(args):
         _, rgb = decode_image(rec, i, k, True)
         npx += rgb.shape[0] * rgb.shape[1]
     return hi - lo, npx
+
+
+# --------------------------------------------------------------------------------------
+# Training-tensor epilogue (Section 6 of the paper, experimental setup: resizing, crop and
+# horizontal-flip augmentations, after which all inputs have the same size; 224x224 in the
+# main experiments, 160x160 crops in the appendix's second pipeline).  The paper leaves
+# the resampling filter to its frameworks; the reading taken here: plain bilinear
+# interpolation with half-pixel centres inside the crop rectangle, edge pixels of the crop
+# repeated, no low-pass filter, then (v / 255 - mean_c) / std_c per channel, planar layout.
+# Evaluated in float64 by the definition, one output pixel = four taps.
+# --------------------------------------------------------------------------------------
+def training_tensor(rgb: np.ndarray, crop, size: int, mean, std, dtype=np.float16) -> np.ndarray:
+    """rgb: (H, W, 3) uint8.  crop = (x0, y0, w, h, flip) in pixels of that image.
+    Returns (3, size, size) of `dtype`: out[c, oy, ox] for output column ox taken from the
+    crop's column u = size-1-ox when flip is set, else u = ox."""
+    x0, y0, cw, ch, flip = (int(v) for v in crop)
+    H, W, _ = rgb.shape
+    if cw < 1 or ch < 1 or x0 < 0 or y0 < 0 or x0 + cw > W or y0 + ch > H:
+        raise ValueError("crop outside the image")
+    region = rgb[y0:y0 + ch, x0:x0 + cw, :].astype(np.float64)
+    out = np.empty((3, size, size), dtype=np.float64)
+    for oy in range(size):
+        fy = (oy + 0.5) * ch / size - 0.5
+        fy = min(max(fy, 0.0), ch - 1.0)
+        iy = int(np.floor(fy))
+        ay = fy - iy
+        iy1 = min(iy + 1, ch - 1)
+        for ox in range(size):
+            u = size - 1 - ox if flip else ox
+            fx = (u + 0.5) * cw / size - 0.5
+            fx = min(max(fx, 0.0), cw - 1.0)
+            ix = int(np.floor(fx))
+            ax = fx - ix
+            ix1 = min(ix + 1, cw - 1)
+            top = (1.0 - ax) * region[iy, ix] + ax * region[iy, ix1]
+            bot = (1.0 - ax) * region[iy1, ix] + ax * region[iy1, ix1]
+            out[:, oy, ox] = (1.0 - ay) * top + ay * bot
+    m = np.asarray(mean, dtype=np.float64).reshape(3, 1, 1)
+    s = np.asarray(std, dtype=np.float64).reshape(3, 1, 1)
+    return ((out / 255.0 - m) / s).astype(dtype)

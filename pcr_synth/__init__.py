@@ -275,3 +275,34 @@ def block_grids(W: int, H: int):
     unp = [((W + 7) // 8, (H + 7) // 8), ((cw + 7) // 8, (ch + 7) // 8), ((cw + 7) // 8, (ch + 7) // 8)]
     off = [0, padded[0][0] * padded[0][1], padded[0][0] * padded[0][1] + mx * my]
     return padded, unp, off
+
+
+def random_resized_crops(dims, seed: int, scale=(0.08, 1.0), ratio=(3.0 / 4.0, 4.0 / 3.0)) -> np.ndarray:
+    """Seeded crop rectangles and flip flags, one per image: (N, 5) uint32 rows x0, y0, w, h, flip.
+
+    The usual ImageNet training augmentation draws: area fraction uniform in `scale`, aspect
+    ratio log-uniform in `ratio`, position uniform, ten attempts then the whole image; flip
+    with probability one half.  These are inputs of the decode path (the random numbers are
+    drawn here, never inside it)."""
+    import math
+    out = np.zeros((len(dims), 5), dtype=np.uint32)
+    for i, (W, H) in enumerate(dims):
+        st = splitmix64((seed * 0x9E3779B97F4A7C15 + i + 1) & _M64)
+        def u():
+            nonlocal st
+            st = splitmix64(st)
+            return _unit(st)
+        rect = (0, 0, int(W), int(H))
+        for _ in range(10):
+            area = W * H * (scale[0] + (scale[1] - scale[0]) * u())
+            ar = math.exp(math.log(ratio[0]) + (math.log(ratio[1]) - math.log(ratio[0])) * u())
+            w = int(round(math.sqrt(area * ar)))
+            h = int(round(math.sqrt(area / ar)))
+            if 0 < w <= W and 0 < h <= H:
+                x0 = int(u() * (W - w + 1))
+                y0 = int(u() * (H - h + 1))
+                rect = (min(x0, W - w), min(y0, H - h), w, h)
+                break
+        out[i, :4] = rect
+        out[i, 4] = 1 if u() < 0.5 else 0
+    return out
