@@ -114,6 +114,34 @@ int pcr_decode(pcr_record* rec, int k, void* out, void* stream);
  * Status words accumulate: an error flagged by the earlier decode stays set. */
 int pcr_decode_more(pcr_record* rec, int k, void* out, void* stream);
 
+/* Decode at fidelity k straight to a training batch (Section 6, experimental setup: the
+ * experiments use resizing, crop and horizontal-flip augmentations, after which all inputs have
+ * the same size: 224x224, or 160x160 crops in the appendix's second pipeline).  The decode is
+ * pcr_decode's; the pixel stage transforms only the 16x16 MCUs that touch an image's crop
+ * rectangle, and an epilogue kernel resamples the crop to size x size and writes the tensor:
+ *   for output pixel (ox, oy): u = flip ? size-1-ox : ox;
+ *   fx = clamp((u + 0.5) * w / size - 0.5, 0, w - 1), fy likewise with h (half-pixel centres,
+ *   the crop's edge pixels repeated, no low-pass filter); v = bilinear interpolation of the four
+ *   pixels around (x0 + fx, y0 + fy); tensor[i][c][oy][ox] = (v_c / 255 - mean[c]) / std[c],
+ *   evaluated in single precision, stored as dtype (half: round to nearest even).
+ *   crops  : HOST array of pcr_num_images entries (read before the call returns); every
+ *            rectangle must lie inside its image, w, h >= 1, flip 0 or 1 (else PCR_E_ARG).
+ *            The random draws of an augmentation policy are the caller's.
+ *   size   : 1..4096.   mean, std : HOST, three floats each, std > 0.   dtype : PCR_F16 / PCR_F32.
+ *   rgb    : DEVICE scratch as pcr_decode's `out` (same size and alignment); afterwards it holds
+ *            the decoded pixels of the transformed MCUs, other bytes are left as they were.
+ *   tensor : DEVICE, pcr_num_images * 3 * size * size elements of dtype, image i at index i.
+ * Enqueues on `stream` and returns; errors as pcr_decode.  The first call on a record allocates
+ * a small device array for the rectangles. */
+#define PCR_F16 0
+#define PCR_F32 1
+typedef struct {
+    uint32_t x0, y0, w, h; /* crop rectangle in pixels of the decoded image */
+    uint32_t flip;         /* 1: mirror the columns                         */
+} pcr_crop;
+int pcr_decode_tensor(pcr_record* rec, int k, const pcr_crop* crops, int size, const float* mean, const float* std,
+                      int dtype, void* rgb, void* tensor, void* stream);
+
 /* Forget which record bytes are resident on the device: the next pcr_decode copies its whole
  * prefix again (what a loader that streams each record once from host memory pays). */
 int pcr_evict(pcr_record* rec);

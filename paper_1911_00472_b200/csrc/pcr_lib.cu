@@ -176,6 +176,7 @@ struct pcr_record {
     Unit* d_units = nullptr;
     uint16_t* d_qtab = nullptr;
     uint32_t* d_order = nullptr;  // processing order of the images (slices are runs of it)
+    CropRect* d_crops = nullptr;  // crop rectangles of the last pcr_decode_tensor (allocated on first use)
     int* d_status = nullptr;
     std::vector<int> h_status;
     std::vector<std::pair<void*, size_t>> bufs;   // every device buffer of the record with its size
@@ -697,7 +698,7 @@ int pcr_evict(pcr_record* rec) {
 
 // Decode scans k0 .. k-1 on top of the state scans 0 .. k0-1 left behind (k0 = 0: from scratch),
 // then produce the pixels of fidelity k.
-static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream) {
+static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream, const TensorArgs* targs = nullptr) {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t need = (size_t)rec->group_end[k];
     const bool prof = rec->profiling;
@@ -725,6 +726,7 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream)
     P.saux = rec->d_saux; P.aux = rec->d_aux;
     P.imgs = rec->d_imgs; P.seg_start = rec->d_seg; P.items = rec->d_items; P.units = rec->d_units;
     P.qtab = rec->d_qtab; P.order = rec->d_order; P.status = rec->d_status; P.N = rec->N;
+    P.roi = targs ? targs->crops : nullptr;
     FinalizeList fl;
     memset(&fl, 0, sizeof fl);
     bool any_refine = false;
@@ -824,6 +826,11 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream)
             else if (any_refine) pixel_kernel<true, 1><<<nu, kPixThreads, 0, q>>>(Q, fl, static_cast<uint8_t*>(out));
             else pixel_kernel<false, 1><<<nu, kPixThreads, 0, q>>>(Q, fl, static_cast<uint8_t*>(out));
             ++g_launches;
+            if (targs && i1 > i0) {
+                const unsigned tiles = (unsigned)((targs->size * targs->size + 255) / 256);
+                tensor_kernel<<<dim3(tiles, i1 - i0), 256, 0, q>>>(P, *targs, static_cast<const uint8_t*>(out), i0);
+                ++g_launches;
+            }
         }
         return true;
     };
@@ -939,6 +946,31 @@ int pcr_decode_more(pcr_record* rec, int k, void* out, void* stream) {
     if (reinterpret_cast<uintptr_t>(out) & 15u) return PCR_E_ARG;
     if (rec->decoded_k < 1 || k <= rec->decoded_k) return PCR_E_ARG;
     return decode_range(rec, rec->decoded_k, k, out, stream);
+}
+
+int pcr_decode_tensor(pcr_record* rec, int k, const pcr_crop* crops, int size, const float* mean, const float* std_,
+                      int dtype, void* rgb, void* tensor, void* stream) {
+    if (!rec || !crops || !mean || !std_ || !rgb || !tensor || k < 1 || k > rec->G) return PCR_E_ARG;
+    if (size < 1 || size > 4096 || (dtype != PCR_F16 && dtype != PCR_F32)) return PCR_E_ARG;
+    if (reinterpret_cast<uintptr_t>(rgb) & 15u) return PCR_E_ARG;
+    if (reinterpret_cast<uintptr_t>(tensor) & (dtype == PCR_F32 ? 3u : 1u)) return PCR_E_ARG;
+    static_assert(sizeof(pcr_crop) == sizeof(CropRect), "pcr_crop and CropRect have the same layout");
+    for (int i = 0; i < rec->N; ++i) {
+        const pcr_crop& c = crops[i];
+        const pcr_image_info& inf = rec->info[i];
+        if (c.w < 1 || c.h < 1 || c.flip > 1 || c.x0 > inf.width || c.y0 > inf.height || c.w > inf.width - c.x0 ||
+            c.h > inf.height - c.y0) return PCR_E_ARG;
+        if (!(std_[0] > 0.f) || !(std_[1] > 0.f) || !(std_[2] > 0.f)) return PCR_E_ARG;
+    }
+    if (!rec->d_crops) {
+        if (int rc = take(rec, &rec->d_crops, (size_t)rec->N * sizeof(CropRect))) return rc;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(rec->d_crops, crops, (size_t)rec->N * sizeof(CropRect), cudaMemcpyHostToDevice, st) != cudaSuccess) return PCR_E_CUDA;
+    TensorArgs T;
+    T.crops = rec->d_crops; T.out = tensor; T.size = size; T.f32 = dtype == PCR_F32 ? 1 : 0;
+    for (int c = 0; c < 3; ++c) { T.mean[c] = mean[c]; T.inv_std[c] = 1.0f / std_[c]; }
+    return decode_range(rec, 0, k, rgb, stream, &T);
 }
 
 int pcr_status(pcr_record* rec, int* first_bad_image, int* code) {

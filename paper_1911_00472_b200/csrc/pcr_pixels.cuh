@@ -12,6 +12,7 @@
 //   R = clamp(Y + ((91881 cr + 32768) >> 16)), G = clamp(Y + ((-22553 cb - 46802 cr + 32768) >> 16)),
 //   B = clamp(Y + ((116130 cb + 32768) >> 16)) with cb, cr = sample - 128 of chroma (x>>1, y>>1).
 #pragma once
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -89,6 +90,11 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
     const Unit un = P.units[blockIdx.x];
     const ImgDesc im = P.imgs[un.img];
     const int nm = min((int)kPixMcus, (int)im.mx - (int)un.mcol0);   // MCUs in this unit
+    if (P.roi) {                                                      // whole CTA: nothing of this unit is wanted
+        const CropRect r = P.roi[un.img];
+        const uint32_t ux0 = 16u * un.mcol0, uy0 = 16u * un.mrow;
+        if (ux0 >= r.x0 + r.w || ux0 + 16u * (uint32_t)nm <= r.x0 || uy0 >= r.y0 + r.h || uy0 + 16u <= r.y0) return;
+    }
     for (int i = tid; i < 96; i += kPixThreads)
         reinterpret_cast<uint32_t*>(&s_q[0][0])[i] = __ldg(reinterpret_cast<const uint32_t*>(P.qtab + (size_t)un.img * 192) + i);
     __syncthreads();
@@ -286,6 +292,56 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
                 }
             }
         }
+    }
+}
+
+// Training-tensor epilogue: crop, optional mirror, bilinear resize to size x size with half-pixel
+// centres (the crop's edge pixels repeated, no low-pass filter), (v / 255 - mean) / std, planar
+// output [image][channel][row][column].  One thread per output pixel, all three channels.
+// Images pos0 .. pos0 + gridDim.y - 1 of the processing order.
+struct TensorArgs {
+    const CropRect* crops;     // [N], by image index
+    void* out;                 // [N][3][size][size]
+    int32_t size;
+    int32_t f32;               // 0: half precision output, 1: single precision
+    float mean[3], inv_std[3];
+};
+
+__device__ __forceinline__ void tensor_store(void* out, size_t idx, float v, int f32) {
+    if (f32) static_cast<float*>(out)[idx] = v;
+    else static_cast<__half*>(out)[idx] = __float2half_rn(v);
+}
+
+__global__ void __launch_bounds__(256) tensor_kernel(Params P, TensorArgs T, const uint8_t* __restrict__ rgb, uint32_t pos0) {
+    const uint32_t img = P.order[pos0 + blockIdx.y];
+    const int S = T.size;
+    const int p = blockIdx.x * 256 + threadIdx.x;
+    if (p >= S * S) return;
+    const int oy = p / S, ox = p - oy * S;
+    const ImgDesc im = P.imgs[img];
+    const CropRect r = T.crops[img];
+    const int u = r.flip ? S - 1 - ox : ox;
+    const float sx = (float)r.w / (float)S, sy = (float)r.h / (float)S;
+    float fx = ((float)u + 0.5f) * sx - 0.5f, fy = ((float)oy + 0.5f) * sy - 0.5f;
+    fx = fminf(fmaxf(fx, 0.f), (float)(r.w - 1));
+    fy = fminf(fmaxf(fy, 0.f), (float)(r.h - 1));
+    const int ix = (int)floorf(fx), iy = (int)floorf(fy);
+    const float ax = fx - (float)ix, ay = fy - (float)iy;
+    const int ix1 = min(ix + 1, (int)r.w - 1), iy1 = min(iy + 1, (int)r.h - 1);
+    const uint8_t* base = rgb + im.out_off;
+    const size_t pitch = (size_t)im.W * 3;
+    const uint8_t* p00 = base + (size_t)(r.y0 + iy) * pitch + (size_t)(r.x0 + ix) * 3;
+    const uint8_t* p01 = base + (size_t)(r.y0 + iy) * pitch + (size_t)(r.x0 + ix1) * 3;
+    const uint8_t* p10 = base + (size_t)(r.y0 + iy1) * pitch + (size_t)(r.x0 + ix) * 3;
+    const uint8_t* p11 = base + (size_t)(r.y0 + iy1) * pitch + (size_t)(r.x0 + ix1) * 3;
+    const size_t plane = (size_t)S * S;
+    const size_t o = (size_t)img * 3 * plane + (size_t)oy * S + ox;
+#pragma unroll
+    for (int c = 0; c < 3; ++c) {
+        const float top = (1.f - ax) * (float)p00[c] + ax * (float)p01[c];
+        const float bot = (1.f - ax) * (float)p10[c] + ax * (float)p11[c];
+        const float v = (1.f - ay) * top + ay * bot;
+        tensor_store(T.out, o + c * plane, (v * (1.f / 255.f) - T.mean[c]) * T.inv_std[c], T.f32);
     }
 }
 

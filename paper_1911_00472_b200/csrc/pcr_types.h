@@ -68,6 +68,12 @@ struct Item {
 };
 constexpr uint32_t kItemOpen = 0xFFFFFFFFu;   // host only, while the list is built: the item may still be extended
 
+// Crop rectangle of one image (pixels) and whether its columns are mirrored; the pixel kernel
+// skips work units that lie outside it when one is given.
+struct CropRect {
+    uint32_t x0, y0, w, h, flip;
+};
+
 // Pixel work unit: a run of MCUs in one MCU row of one image.
 struct Unit {
     uint32_t img;
@@ -93,6 +99,7 @@ struct Params {
     const Unit* units;
     const uint16_t* qtab;       // [N][3][64] quantisers, zigzag order
     const uint32_t* order;      // [N] processing order of the images
+    const CropRect* roi;        // [N] or null: only work units that touch the image's rectangle are transformed
     int* status;                // [N]
     int32_t N;
 };

@@ -57,6 +57,31 @@ class Decoder:
             B.pcr_decode_more(self.handle, k, out.data_ptr(), s.cuda_stream)
         return out
 
+    def decode_tensor(self, k: int, crops: np.ndarray, size: int, mean, std, dtype: torch.dtype = torch.float16,
+                      rgb: torch.Tensor | None = None, tensor: torch.Tensor | None = None,
+                      stream: torch.cuda.Stream | None = None) -> torch.Tensor:
+        """Decode at fidelity k to a (N, 3, size, size) training batch: crops is an (N, 5) array of
+        x0, y0, w, h, flip per image.  Argument marshalling only; the work is pcr_decode_tensor's."""
+        crops = np.ascontiguousarray(crops, dtype=np.uint32)
+        if crops.shape != (self.n_images, 5):
+            raise ValueError("crops must have shape (n_images, 5)")
+        if dtype not in (torch.float16, torch.float32):
+            raise ValueError("dtype must be torch.float16 or torch.float32")
+        m = np.ascontiguousarray(mean, dtype=np.float32)
+        sd = np.ascontiguousarray(std, dtype=np.float32)
+        if rgb is None:
+            if self.out is None:
+                self.out = self.alloc_out()
+            rgb = self.out
+        if tensor is None:
+            tensor = torch.empty((self.n_images, 3, size, size), dtype=dtype, device=self.device)
+        s = stream if stream is not None else torch.cuda.current_stream(self.device)
+        with torch.cuda.device(self.device):
+            B.pcr_decode_tensor(self.handle, k, crops.ctypes.data, size, m.ctypes.data, sd.ctypes.data,
+                                B.PCR_F16 if dtype == torch.float16 else B.PCR_F32, rgb.data_ptr(), tensor.data_ptr(),
+                                s.cuda_stream)
+        return tensor
+
     def evict(self) -> None:
         B.pcr_evict(self.handle)
 
