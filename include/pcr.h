@@ -125,7 +125,8 @@ int pcr_decode_more(pcr_record* rec, int k, void* out, void* stream);
  *   pixels around (x0 + fx, y0 + fy); tensor[i][c][oy][ox] = (v_c / 255 - mean[c]) / std[c],
  *   evaluated in single precision, stored as dtype (half: round to nearest even).
  *   crops  : HOST array of pcr_num_images entries (read before the call returns); every
- *            rectangle must lie inside its image, w, h >= 1, flip 0 or 1 (else PCR_E_ARG).
+ *            rectangle must lie inside its image, w, h >= 1, flip 0 or 1 (else PCR_E_ARG; also
+ *            when an image has 2 GiB of pixels or more).
  *            The random draws of an augmentation policy are the caller's.
  *   size   : 1..4096.   mean, std : HOST, three floats each, std > 0.   dtype : PCR_F16 / PCR_F32.
  *   rgb    : DEVICE scratch as pcr_decode's `out` (same size and alignment); afterwards it holds

@@ -820,15 +820,26 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
         Q.units = P.units + u0;
         if (stage == 2 + W) return true;      // the refinement side data is folded in by the pixel kernel
         if (nu) {
-            if (dc_only) pixel_kernel<false, 2><<<nu, kPixThreads, 0, q>>>(Q, fl, static_cast<uint8_t*>(out));
-            else if (head_only && any_refine) pixel_kernel<true, 3><<<nu, kPixThreads, 0, q>>>(Q, fl, static_cast<uint8_t*>(out));
-            else if (head_only) pixel_kernel<false, 3><<<nu, kPixThreads, 0, q>>>(Q, fl, static_cast<uint8_t*>(out));
-            else if (any_refine) pixel_kernel<true, 1><<<nu, kPixThreads, 0, q>>>(Q, fl, static_cast<uint8_t*>(out));
-            else pixel_kernel<false, 1><<<nu, kPixThreads, 0, q>>>(Q, fl, static_cast<uint8_t*>(out));
+            const unsigned grid = nu;
+            uint8_t* o8 = static_cast<uint8_t*>(out);
+            if (!targs) {
+                if (dc_only) pixel_kernel<false, 2><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+                else if (head_only && any_refine) pixel_kernel<true, 3><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+                else if (head_only) pixel_kernel<false, 3><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+                else if (any_refine) pixel_kernel<true, 1><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+                else pixel_kernel<false, 1><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+            } else {
+                if (dc_only) pixel_kernel<false, 2, true><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+                else if (head_only && any_refine) pixel_kernel<true, 3, true><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+                else if (head_only) pixel_kernel<false, 3, true><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+                else if (any_refine) pixel_kernel<true, 1, true><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+                else pixel_kernel<false, 1, true><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+            }
             ++g_launches;
             if (targs && i1 > i0) {
-                const unsigned tiles = (unsigned)((targs->size * targs->size + 255) / 256);
-                tensor_kernel<<<dim3(tiles, i1 - i0), 256, 0, q>>>(P, *targs, static_cast<const uint8_t*>(out), i0);
+                const dim3 tg((unsigned)((targs->size + kTensorRows - 1) / kTensorRows), i1 - i0);
+                if (targs->f32) tensor_kernel<float><<<tg, 256, 0, q>>>(P, *targs, static_cast<const uint8_t*>(out), i0);
+                else tensor_kernel<__half><<<tg, 256, 0, q>>>(P, *targs, static_cast<const uint8_t*>(out), i0);
                 ++g_launches;
             }
         }
@@ -958,6 +969,7 @@ int pcr_decode_tensor(pcr_record* rec, int k, const pcr_crop* crops, int size, c
     for (int i = 0; i < rec->N; ++i) {
         const pcr_crop& c = crops[i];
         const pcr_image_info& inf = rec->info[i];
+        if (inf.out_bytes >= (1ull << 31)) return PCR_E_ARG;      // the epilogue indexes an image's bytes with 32 bits
         if (c.w < 1 || c.h < 1 || c.flip > 1 || c.x0 > inf.width || c.y0 > inf.height || c.w > inf.width - c.x0 ||
             c.h > inf.height - c.y0) return PCR_E_ARG;
         if (!(std_[0] > 0.f) || !(std_[1] > 0.f) || !(std_[2] > 0.f)) return PCR_E_ARG;

@@ -78,7 +78,8 @@ __device__ __forceinline__ uint32_t pack4_sat(int v0, int v1, int v2, int v3) {
 // head plane (the line's first 16 bytes are ignored); 2 = the block has nothing but its DC
 // coefficient (no AC scan decoded): only the head plane is read and the transform collapses to
 // one value; 3 = no decoded scan reaches beyond position 7: the lines are not read at all.
-template <bool kRefine, int kDcMode>
+// kRoi: only work units that touch their image's crop rectangle (P.roi) are processed.
+template <bool kRefine, int kDcMode, bool kRoi = false>
 __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeList fl, uint8_t* __restrict__ out) {
     __shared__ __align__(16) uint32_t s_line[kRefine ? 32 * kPixThreads : 1];
     __shared__ __align__(16) uint8_t s_y[16][16 * kPixMcus];
@@ -90,7 +91,7 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
     const Unit un = P.units[blockIdx.x];
     const ImgDesc im = P.imgs[un.img];
     const int nm = min((int)kPixMcus, (int)im.mx - (int)un.mcol0);   // MCUs in this unit
-    if (P.roi) {                                                      // whole CTA: nothing of this unit is wanted
+    if (kRoi) {                                                       // whole CTA: nothing of this unit is wanted
         const CropRect r = P.roi[un.img];
         const uint32_t ux0 = 16u * un.mcol0, uy0 = 16u * un.mrow;
         if (ux0 >= r.x0 + r.w || ux0 + 16u * (uint32_t)nm <= r.x0 || uy0 >= r.y0 + r.h || uy0 + 16u <= r.y0) return;
@@ -297,8 +298,7 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
 
 // Training-tensor epilogue: crop, optional mirror, bilinear resize to size x size with half-pixel
 // centres (the crop's edge pixels repeated, no low-pass filter), (v / 255 - mean) / std, planar
-// output [image][channel][row][column].  One thread per output pixel, all three channels.
-// Images pos0 .. pos0 + gridDim.y - 1 of the processing order.
+// output [image][channel][row][column].  Images pos0 .. pos0 + gridDim.y - 1 of the processing order.
 struct TensorArgs {
     const CropRect* crops;     // [N], by image index
     void* out;                 // [N][3][size][size]
@@ -307,41 +307,112 @@ struct TensorArgs {
     float mean[3], inv_std[3];
 };
 
-__device__ __forceinline__ void tensor_store(void* out, size_t idx, float v, int f32) {
-    if (f32) static_cast<float*>(out)[idx] = v;
-    else static_cast<__half*>(out)[idx] = __float2half_rn(v);
+__device__ __forceinline__ void tensor_store(float* p, float v) { *p = v; }
+__device__ __forceinline__ void tensor_store(__half* p, float v) { *p = __float2half_rn(v); }
+
+// the three bytes at byte offset `off` of a 4-byte-aligned shared buffer, as floats: two aligned
+// words, a funnel shift, and per byte a permute into the mantissa of 2^23 (exact for 0..255)
+__device__ __forceinline__ void load_rgb(const uint8_t* buf, int off, float& r, float& g, float& b) {
+    const uint32_t* w = reinterpret_cast<const uint32_t*>(buf + (off & ~3));
+    const uint32_t v = __funnelshift_r(w[0], w[1], 8 * (off & 3));
+    r = __uint_as_float(__byte_perm(v, 0x4B000000u, 0x7540)) - 8388608.f;
+    g = __uint_as_float(__byte_perm(v, 0x4B000000u, 0x7541)) - 8388608.f;
+    b = __uint_as_float(__byte_perm(v, 0x4B000000u, 0x7542)) - 8388608.f;
 }
 
+constexpr int kTensorRows = 8;                  // output rows per CTA
+constexpr int kTensorStage = 40 * 1024;         // bytes of source rows a CTA can stage
+
+// One CTA per band of kTensorRows output rows of one image: the source rows the band interpolates
+// between are staged in shared memory with aligned word loads (the crop's first byte sits at any
+// alignment), then every thread produces the band's pixels of its output columns from the staged
+// bytes.  Bands whose source rows do not fit read their taps from global memory directly.
+template <typename OutT>
 __global__ void __launch_bounds__(256) tensor_kernel(Params P, TensorArgs T, const uint8_t* __restrict__ rgb, uint32_t pos0) {
+    __shared__ __align__(16) uint8_t s_src[kTensorStage];
+    __shared__ int s_off0[kTensorRows], s_off1[kTensorRows];       // byte offsets of a row's upper / lower source row
+    __shared__ float s_ay[kTensorRows];
     const uint32_t img = P.order[pos0 + blockIdx.y];
     const int S = T.size;
-    const int p = blockIdx.x * 256 + threadIdx.x;
-    if (p >= S * S) return;
-    const int oy = p / S, ox = p - oy * S;
+    const int oy0 = blockIdx.x * kTensorRows;
+    const int nrows = min(kTensorRows, S - oy0);
     const ImgDesc im = P.imgs[img];
     const CropRect r = T.crops[img];
-    const int u = r.flip ? S - 1 - ox : ox;
     const float sx = (float)r.w / (float)S, sy = (float)r.h / (float)S;
-    float fx = ((float)u + 0.5f) * sx - 0.5f, fy = ((float)oy + 0.5f) * sy - 0.5f;
-    fx = fminf(fmaxf(fx, 0.f), (float)(r.w - 1));
-    fy = fminf(fmaxf(fy, 0.f), (float)(r.h - 1));
-    const int ix = (int)floorf(fx), iy = (int)floorf(fy);
-    const float ax = fx - (float)ix, ay = fy - (float)iy;
-    const int ix1 = min(ix + 1, (int)r.w - 1), iy1 = min(iy + 1, (int)r.h - 1);
-    const uint8_t* base = rgb + im.out_off;
-    const size_t pitch = (size_t)im.W * 3;
-    const uint8_t* p00 = base + (size_t)(r.y0 + iy) * pitch + (size_t)(r.x0 + ix) * 3;
-    const uint8_t* p01 = base + (size_t)(r.y0 + iy) * pitch + (size_t)(r.x0 + ix1) * 3;
-    const uint8_t* p10 = base + (size_t)(r.y0 + iy1) * pitch + (size_t)(r.x0 + ix) * 3;
-    const uint8_t* p11 = base + (size_t)(r.y0 + iy1) * pitch + (size_t)(r.x0 + ix1) * 3;
-    const size_t plane = (size_t)S * S;
-    const size_t o = (size_t)img * 3 * plane + (size_t)oy * S + ox;
-#pragma unroll
-    for (int c = 0; c < 3; ++c) {
-        const float top = (1.f - ax) * (float)p00[c] + ax * (float)p01[c];
-        const float bot = (1.f - ax) * (float)p10[c] + ax * (float)p11[c];
-        const float v = (1.f - ay) * top + ay * bot;
-        tensor_store(T.out, o + c * plane, (v * (1.f / 255.f) - T.mean[c]) * T.inv_std[c], T.f32);
+    const uint32_t pitch = im.W * 3u;
+    const uint8_t* crop0 = rgb + im.out_off + (size_t)r.y0 * pitch + (size_t)r.x0 * 3;   // first byte of the crop
+    const int nbytes = 3 * (int)r.w;
+    // source rows of the band: from the upper tap of its first row to the lower tap of its last
+    float fyA = ((float)oy0 + 0.5f) * sy - 0.5f, fyB = ((float)(oy0 + nrows - 1) + 0.5f) * sy - 0.5f;
+    fyA = fminf(fmaxf(fyA, 0.f), (float)(r.h - 1));
+    fyB = fminf(fmaxf(fyB, 0.f), (float)(r.h - 1));
+    const int ys = (int)floorf(fyA), ye = min((int)floorf(fyB) + 1, (int)r.h - 1);
+    const int stride = (nbytes + 3 + 7 + 15) & ~15;                   // staged row: alignment slack in front, a spare word behind
+    const bool staged = (ye - ys + 1) * stride <= kTensorStage;       // same for the whole CTA
+    if (staged) {
+        for (int y = ys; y <= ye; ++y) {
+            const uint8_t* src = crop0 + (size_t)y * pitch;
+            const int a = (int)(reinterpret_cast<uintptr_t>(src) & 3u);
+            const uint32_t* w = reinterpret_cast<const uint32_t*>(src - a);
+            const int nw = (a + nbytes + 3) >> 2;      // ends at the next word boundary, inside the image's rounded-up area
+            uint32_t* d = reinterpret_cast<uint32_t*>(s_src + (y - ys) * stride);
+            for (int i = threadIdx.x; i < nw; i += 256) d[i] = __ldg(w + i);
+        }
+    }
+    if ((int)threadIdx.x < nrows) {
+        float fy = ((float)(oy0 + (int)threadIdx.x) + 0.5f) * sy - 0.5f;
+        fy = fminf(fmaxf(fy, 0.f), (float)(r.h - 1));
+        const int iy = (int)floorf(fy), iy1 = min(iy + 1, (int)r.h - 1);
+        s_ay[threadIdx.x] = fy - (float)iy;
+        if (staged) {
+            s_off0[threadIdx.x] = (iy - ys) * stride + (int)(reinterpret_cast<uintptr_t>(crop0 + (size_t)iy * pitch) & 3u);
+            s_off1[threadIdx.x] = (iy1 - ys) * stride + (int)(reinterpret_cast<uintptr_t>(crop0 + (size_t)iy1 * pitch) & 3u);
+        } else {
+            s_off0[threadIdx.x] = iy * (int)pitch; s_off1[threadIdx.x] = iy1 * (int)pitch;   // records are below 4 GiB
+        }
+    }
+    __syncthreads();
+    const uint32_t plane = (uint32_t)S * (uint32_t)S;
+    const float k255 = 1.f / 255.f;
+    const float m0 = T.mean[0], m1 = T.mean[1], m2 = T.mean[2], i0 = T.inv_std[0], i1 = T.inv_std[1], i2 = T.inv_std[2];
+    OutT* const obase = static_cast<OutT*>(T.out) + (size_t)img * 3 * plane + (size_t)oy0 * S;
+    for (int ox = threadIdx.x; ox < S; ox += 256) {
+        const int u = r.flip ? S - 1 - ox : ox;
+        float fx = ((float)u + 0.5f) * sx - 0.5f;
+        fx = fminf(fmaxf(fx, 0.f), (float)(r.w - 1));
+        const int ix = (int)floorf(fx);
+        const float ax = fx - (float)ix, bx = 1.f - ax;
+        const int c0 = 3 * ix, c1 = 3 * min(ix + 1, (int)r.w - 1);
+        OutT* o = obase + ox;
+        if (staged) {
+            for (int dy = 0; dy < nrows; ++dy, o += S) {
+                const int q0 = s_off0[dy], q1 = s_off1[dy];
+                const float ay = s_ay[dy], by = 1.f - ay;
+                float r00, g00, b00, r01, g01, b01, r10, g10, b10, r11, g11, b11;
+                load_rgb(s_src, q0 + c0, r00, g00, b00);
+                load_rgb(s_src, q0 + c1, r01, g01, b01);
+                load_rgb(s_src, q1 + c0, r10, g10, b10);
+                load_rgb(s_src, q1 + c1, r11, g11, b11);
+                const float r_ = by * (bx * r00 + ax * r01) + ay * (bx * r10 + ax * r11);
+                const float g_ = by * (bx * g00 + ax * g01) + ay * (bx * g10 + ax * g11);
+                const float b_ = by * (bx * b00 + ax * b01) + ay * (bx * b10 + ax * b11);
+                tensor_store(o, (r_ * k255 - m0) * i0);
+                tensor_store(o + plane, (g_ * k255 - m1) * i1);
+                tensor_store(o + 2 * plane, (b_ * k255 - m2) * i2);
+            }
+        } else {
+            for (int dy = 0; dy < nrows; ++dy, o += S) {
+                const uint8_t* t0 = crop0 + s_off0[dy];
+                const uint8_t* t1 = crop0 + s_off1[dy];
+                const float ay = s_ay[dy], by = 1.f - ay;
+                const float r_ = by * (bx * (float)__ldg(t0 + c0) + ax * (float)__ldg(t0 + c1)) + ay * (bx * (float)__ldg(t1 + c0) + ax * (float)__ldg(t1 + c1));
+                const float g_ = by * (bx * (float)__ldg(t0 + c0 + 1) + ax * (float)__ldg(t0 + c1 + 1)) + ay * (bx * (float)__ldg(t1 + c0 + 1) + ax * (float)__ldg(t1 + c1 + 1));
+                const float b_ = by * (bx * (float)__ldg(t0 + c0 + 2) + ax * (float)__ldg(t0 + c1 + 2)) + ay * (bx * (float)__ldg(t1 + c0 + 2) + ax * (float)__ldg(t1 + c1 + 2));
+                tensor_store(o, (r_ * k255 - m0) * i0);
+                tensor_store(o + plane, (g_ * k255 - m1) * i1);
+                tensor_store(o + 2 * plane, (b_ * k255 - m2) * i2);
+            }
+        }
     }
 }
 

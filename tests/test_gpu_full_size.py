@@ -56,3 +56,32 @@ def test_celeba_shaped_full_record_every_k():
 
 def test_ham_shaped_full_record_no_restart_markers():
     _check(3, (1, 5, 10), 6)
+
+
+def test_imagenet_shaped_full_record_training_tensor():
+    """The fixed-size training batch at full record size, in the benchmark's configuration:
+    sampled images against the oracle, and for every image the mirror property (the same crop
+    with the flip flag toggled gives the column-reversed tensor, bit for bit)."""
+    import torch
+    from paper_1911_00472_b200 import Decoder
+    rec = pcr_synth.make_record(1, 0)
+    dec = Decoder(rec.bytes)
+    mean, std = (0.485, 0.456, 0.406), (0.229, 0.224, 0.225)
+    crops = pcr_synth.random_resized_crops([(int(w), int(h)) for w, h in rec.dims], 21)
+    try:
+        for k, size in ((10, 224), (2, 160)):
+            t = dec.decode_tensor(k, crops, size, mean, std).clone()
+            torch.cuda.synchronize()
+            assert dec.status() == (-1, 0)
+            flipped = crops.copy()
+            flipped[:, 4] ^= 1
+            t2 = dec.decode_tensor(k, flipped, size, mean, std)
+            torch.cuda.synchronize()
+            assert torch.equal(t2, torch.flip(t, dims=[3]))
+            got = t.cpu().numpy().astype(np.float64)
+            for i in (0, 511, rec.n_images - 1):
+                _, rgb = O.decode_image(rec.bytes, i, k)
+                want = O.training_tensor(rgb, crops[i], size, mean, std).astype(np.float64)
+                assert np.abs(got[i] - want).max() <= 2.0 ** -9, (k, i)
+    finally:
+        dec.close()
