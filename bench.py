@@ -560,6 +560,9 @@ def main():
                         "one_core": v1}
         tmpdir.cleanup()
 
+    # Theorem 1 of the paper: a data-bound pipeline speeds up by the ratio of mean sample sizes;
+    # here full-fidelity bytes over the bytes of the record prefix that fidelity k reads
+    io_speedup = {str(kk): dec.prefix_bytes(dec.n_groups) / dec.prefix_bytes(kk) for kk in range(1, dec.n_groups + 1)}
     if rank == 0:
         comp = [s[6] for s in scans]
         print(json.dumps({
@@ -572,7 +575,7 @@ def main():
                        "mean_compressed_bytes_per_image_by_scan": [c / n_img for c in comp]},
             "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
             "cpu_baseline": cpu_baseline, "images_per_s_by_k": per_k, "raise_fidelity_ms_per_record": raise_ms,
-            "training_tensor": training_tensor,
+            "training_tensor": training_tensor, "predicted_io_speedup_by_k": io_speedup,
         }))
     dec.close()
     if world > 1:

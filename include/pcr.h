@@ -132,6 +132,10 @@ int pcr_decode_more(pcr_record* rec, int k, void* out, void* stream);
  *   rgb    : DEVICE scratch as pcr_decode's `out` (same size and alignment); afterwards it holds
  *            the decoded pixels of the transformed MCUs, other bytes are left as they were.
  *   tensor : DEVICE, pcr_num_images * 3 * size * size elements of dtype, image i at index i.
+ * Restart intervals whose MCU rows lie outside the MCU rows an image's rectangle touches are not
+ * entropy-decoded either, so afterwards the coefficient planes are incomplete: pcr_decode_more
+ * refuses to continue from this call (PCR_E_ARG) and pcr_coeffs is meaningful only for the
+ * decoded rows.
  * Enqueues on `stream` and returns; errors as pcr_decode.  The first call on a record allocates
  * a small device array for the rectangles. */
 #define PCR_F16 0

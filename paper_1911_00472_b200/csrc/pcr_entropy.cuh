@@ -316,6 +316,9 @@ __device__ __forceinline__ int select_bit(uint64_t z, int r) {
 
 constexpr int kDecodeSteps = 16;     // decode steps between two top-ups of the rings
 
+// kRoi: restart intervals whose MCU rows lie wholly outside the MCU rows that the image's crop
+// rectangle (P.roi) touches are not decoded (their blocks are never transformed).
+template <bool kRoi>
 __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, uint32_t item_begin, uint32_t item_count) {
     __shared__ HuffTab tabs[kEntropyWarps][2];
     __shared__ uint32_t s_ring[kEntropyWarps][kRingWords][32];
@@ -332,11 +335,6 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
     // tables: a DC scan may use two tables of one image; an AC item may span two images
     const bool two_images = item.next != 0;
     const uint32_t si1 = two_images ? item.next - 1u : item.si;
-    if (huff) {
-        build_hufftab(tabs[wid][0], P.rec + sd0.tab_off[0], lane);
-        if (two_images) build_hufftab(tabs[wid][1], P.rec + P.scans[si1].tab_off[0], lane);
-        else if (sd0.tab_off[1]) build_hufftab(tabs[wid][1], P.rec + sd0.tab_off[1], lane);
-    }
     // From here on no lane leaves before the warp does: lanes without work just stay `done`.
     bool done = (uint32_t)lane >= item.count;
     const uint32_t rem0 = sd0.nseg - item.seg0;               // restart intervals left in the first image
@@ -355,6 +353,22 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
     const uint32_t total = mcu_w * mcu_h;
     const uint32_t m0 = sd.ri ? seg * sd.ri : 0;
     const uint32_t m1 = sd.ri ? min(m0 + sd.ri, total) : total;
+    const unsigned full = 0xffffffffu;
+    if (kRoi) {
+        if (!done && m1 > m0) {
+            const CropRect rc = P.roi[img];
+            const uint32_t ph = (inter || c0 != 0) ? 16u : 8u;             // pixel rows per MCU row of this scan
+            const uint32_t lo = 16u * (rc.y0 >> 4), hi = 16u * ((rc.y0 + rc.h + 15u) >> 4);
+            const uint32_t r0 = m0 / mcu_w, r1 = (m1 - 1u) / mcu_w;
+            if ((r1 + 1u) * ph <= lo || r0 * ph >= hi) done = true;
+        }
+        if (__all_sync(full, done)) return;                               // nothing of this item is wanted
+    }
+    if (huff) {
+        build_hufftab(tabs[wid][0], P.rec + sd0.tab_off[0], lane);
+        if (two_images) build_hufftab(tabs[wid][1], P.rec + P.scans[si1].tab_off[0], lane);
+        else if (sd0.tab_off[1]) build_hufftab(tabs[wid][1], P.rec + sd0.tab_off[1], lane);
+    }
     const uint32_t* segtab = P.seg_start + sd.seg_base;
     uint32_t bstart = segtab[seg];
     uint32_t bend = segtab[seg + 1] - 2;
@@ -368,7 +382,6 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
     br.topup(!done);
     br.prime();
     const int Al = sc.Al, p1 = 1 << sc.Al;
-    const unsigned full = 0xffffffffu;
 
     if (dc) {
         // ---- DC scans: one block per step

@@ -812,7 +812,8 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
                 count += rec->item_count[(size_t)g * G + s];
             }
             if (!count) return true;
-            entropy_kernel<<<(count + kEntropyWarps - 1) / kEntropyWarps, 32 * kEntropyWarps, 0, q>>>(P, begin, count);
+            if (targs) entropy_kernel<true><<<(count + kEntropyWarps - 1) / kEntropyWarps, 32 * kEntropyWarps, 0, q>>>(P, begin, count);
+            else entropy_kernel<false><<<(count + kEntropyWarps - 1) / kEntropyWarps, 32 * kEntropyWarps, 0, q>>>(P, begin, count);
             ++g_launches;
             return true;
         }
@@ -982,7 +983,9 @@ int pcr_decode_tensor(pcr_record* rec, int k, const pcr_crop* crops, int size, c
     TensorArgs T;
     T.crops = rec->d_crops; T.out = tensor; T.size = size; T.f32 = dtype == PCR_F32 ? 1 : 0;
     for (int c = 0; c < 3; ++c) { T.mean[c] = mean[c]; T.inv_std[c] = 1.0f / std_[c]; }
-    return decode_range(rec, 0, k, rgb, stream, &T);
+    const int rc = decode_range(rec, 0, k, rgb, stream, &T);
+    rec->decoded_k = 0;          // rows outside the crops were not decoded: nothing to raise the fidelity of
+    return rc;
 }
 
 int pcr_status(pcr_record* rec, int* first_bad_image, int* code) {

@@ -96,6 +96,16 @@ def test_bad_arguments_are_rejected(rec0):
             dec.decode_tensor(10, crops, 8, MEAN, (0.2, 0.0, 0.2))
         with pytest.raises(PcrError):
             dec.decode_tensor(11, crops, 8, MEAN, STD)
+        # rows outside the crops are not decoded: the fidelity of such a decode cannot be raised
+        dec.decode_tensor(5, crops, 8, MEAN, STD)
+        with pytest.raises(PcrError):
+            dec.decode_more(10)
+        # a plain decode afterwards is complete again
+        out = dec.decode(10)
+        torch.cuda.synchronize()
+        want_c, want = O.decode_image(rec0.bytes, 7, 10)
+        assert np.array_equal(dec.image(out, 7).cpu().numpy(), want)
+        assert np.array_equal(dec.coeffs(7).cpu().numpy(), want_c)
         torch.cuda.synchronize()
     finally:
         dec.close()
