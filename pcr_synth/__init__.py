@@ -69,6 +69,7 @@ def _load():
             lib.synth_num_blocks.restype = C.c_size_t
             lib.synth_num_blocks.argtypes = [C.c_uint32, C.c_uint32]
             lib.synth_zigzag.argtypes = [C.c_void_p]
+            lib.synth_set_script.argtypes = [C.c_void_p, C.c_int]
             lib.synth_rgb_to_coeffs.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
             _lib = lib
     return _lib
@@ -306,3 +307,44 @@ def random_resized_crops(dims, seed: int, scale=(0.08, 1.0), ratio=(3.0 / 4.0, 4
         out[i, :4] = rect
         out[i, 4] = 1 if u() < 0.5 else 0
     return out
+
+
+# --------------------------------------------------------------------------------------
+# other scan scripts (the paper, Section 4.2: unused scans can be dropped; any script that
+# progressive JPEG allows makes a record, one scan per group)
+# --------------------------------------------------------------------------------------
+# (components, Ss, Se, Ah, Al); components: (0, 1, 2) = interleaved Y, Cb, Cr
+SCRIPT_DEFAULT = None
+SCRIPT_SPECTRAL_4 = [((0, 1, 2), 0, 0, 0, 0), ((0,), 1, 63, 0, 0), ((1,), 1, 63, 0, 0), ((2,), 1, 63, 0, 0)]
+SCRIPT_MIXED_6 = [((0, 1, 2), 0, 0, 0, 1), ((0,), 1, 63, 0, 1), ((1,), 1, 63, 0, 0), ((2,), 1, 63, 0, 0),
+                  ((0, 1, 2), 0, 0, 1, 0), ((0,), 1, 63, 1, 0)]
+SCRIPT_DEEP_14 = [((0, 1, 2), 0, 0, 0, 2), ((0,), 1, 9, 0, 3), ((0,), 10, 63, 0, 3), ((1,), 1, 63, 0, 2),
+                  ((2,), 1, 63, 0, 2), ((0,), 1, 63, 3, 2), ((0, 1, 2), 0, 0, 2, 1), ((0,), 1, 63, 2, 1),
+                  ((1,), 1, 63, 2, 1), ((2,), 1, 63, 2, 1), ((0, 1, 2), 0, 0, 1, 0), ((0,), 1, 63, 1, 0),
+                  ((1,), 1, 63, 1, 0), ((2,), 1, 63, 1, 0)]
+
+
+class scan_script:
+    """Context manager: records made inside use `script` (a list of (components, Ss, Se, Ah, Al),
+    at most 16 scans) instead of the ten-scan default.  Not thread safe (a process-wide setting)."""
+
+    def __init__(self, script):
+        self.script = script
+
+    def __enter__(self):
+        lib = _load()
+        if self.script is None:
+            lib.synth_set_script(None, 0)
+            return self
+        flat = []
+        for comps, Ss, Se, Ah, Al in self.script:
+            cs = list(comps) + [0] * (3 - len(comps))
+            flat += [len(comps)] + cs + [Ss, Se, Ah, Al]
+        arr = (C.c_int * len(flat))(*flat)
+        if lib.synth_set_script(arr, len(self.script)) != 0:
+            raise ValueError("scan script too long")
+        return self
+
+    def __exit__(self, *exc):
+        _load().synth_set_script(None, 0)
+        return False

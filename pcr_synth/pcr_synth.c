@@ -320,6 +320,27 @@ static const scan_spec SCRIPT10[10] = {
     {3, {0, 1, 2}, 0, 0, 1, 0}, {1, {2, 0, 0}, 1, 63, 1, 0},  {1, {1, 0, 0}, 1, 63, 1, 0},
     {1, {0, 0, 0}, 1, 63, 1, 0}};
 
+/* The script in force (default: the ten-scan one).  synth_set_script replaces it for the records
+ * made afterwards; n = 0 restores the default.  flat: 8 ints per scan (ncomp, comp[3], Ss, Se, Ah, Al). */
+#define MAX_SCANS 16
+static scan_spec g_script[MAX_SCANS];
+static int g_nscans = 0;
+static const scan_spec* cur_script(int* n) {
+    if (g_nscans > 0) { *n = g_nscans; return g_script; }
+    *n = 10; return SCRIPT10;
+}
+int synth_set_script(const int* flat, int n) {
+    if (n < 0 || n > MAX_SCANS) return -1;
+    for (int s = 0; s < n; ++s) {
+        scan_spec* sc = &g_script[s];
+        sc->ncomp = flat[8 * s];
+        for (int c = 0; c < 3; ++c) sc->comp[c] = flat[8 * s + 1 + c];
+        sc->Ss = flat[8 * s + 4]; sc->Se = flat[8 * s + 5]; sc->Ah = flat[8 * s + 6]; sc->Al = flat[8 * s + 7];
+    }
+    g_nscans = n;
+    return 0;
+}
+
 #define TOK_SYM 0u   /* [9:8] table slot, [7:0] symbol */
 #define TOK_BITS 1u  /* [28:24] count, [23:0] value     */
 #define TOK_RST 2u   /* [2:0] marker index              */
@@ -554,7 +575,7 @@ static void encode_scan(enc_state* st, const geom_t* g, const int16_t* coef, con
  * restart_fixed > 0 overrides with a fixed interval in MCUs.
  * scan_end[s] = offset just past scan s's entropy data (EOI follows the last). */
 static void encode_image(enc_state* st, const geom_t* g, const int16_t* coef, const uint8_t qy[64],
-                         const uint8_t qc[64], int restart_rows, int restart_fixed, bytebuf* out, size_t scan_end[10]) {
+                         const uint8_t qc[64], int restart_rows, int restart_fixed, bytebuf* out, size_t scan_end[MAX_SCANS]) {
     st->cur_ri = 0;
     bb_put16(out, 0xFFD8);
     static const uint8_t jfif[] = {0xFF, 0xE0, 0, 16, 'J', 'F', 'I', 'F', 0, 1, 1, 0, 0, 1, 0, 1, 0, 0};
@@ -569,8 +590,10 @@ static void encode_image(enc_state* st, const geom_t* g, const int16_t* coef, co
     bb_put(out, 1); bb_put(out, 0x22); bb_put(out, 0);
     bb_put(out, 2); bb_put(out, 0x11); bb_put(out, 1);
     bb_put(out, 3); bb_put(out, 0x11); bb_put(out, 1);
-    for (int s = 0; s < 10; ++s) {
-        encode_scan(st, g, coef, &SCRIPT10[s], restart_rows, restart_fixed, out);
+    int ns;
+    const scan_spec* script = cur_script(&ns);
+    for (int s = 0; s < ns; ++s) {
+        encode_scan(st, g, coef, &script[s], restart_rows, restart_fixed, out);
         scan_end[s] = out->n;
     }
     bb_put16(out, 0xFFD9);
@@ -590,9 +613,9 @@ typedef struct synth_record {
 static void put32(uint8_t* p, uint32_t v) { p[0] = v; p[1] = v >> 8; p[2] = v >> 16; p[3] = v >> 24; }
 static void put64(uint8_t* p, uint64_t v) { put32(p, (uint32_t)v); put32(p + 4, (uint32_t)(v >> 32)); }
 
-#define PCR_G 10
-static void assemble_record(synth_record* r, const int32_t* labels, size_t (*scan_end)[10]) {
-    int N = r->n, G = PCR_G;
+static void assemble_record(synth_record* r, const int32_t* labels, size_t (*scan_end)[MAX_SCANS]) {
+    int N = r->n, G;
+    (void)cur_script(&G);                 /* one scan per group */
     size_t meta_off = 64;
     size_t index_off = meta_off + 16 * (size_t)N;
     size_t data_off = index_off + 8 * (size_t)(G + 1) + 16 * (size_t)G * N;
@@ -644,7 +667,7 @@ synth_record* synth_record_from_coeffs(int n, const uint32_t* W, const uint32_t*
     r->truth = (int16_t**)calloc((size_t)n, sizeof(void*)); r->truth_n = (size_t*)calloc((size_t)n, sizeof(size_t));
     r->jpeg = (uint8_t**)calloc((size_t)n, sizeof(void*)); r->jpeg_n = (size_t*)calloc((size_t)n, sizeof(size_t));
     r->W = (uint32_t*)calloc((size_t)n, 4); r->H = (uint32_t*)calloc((size_t)n, 4);
-    size_t (*scan_end)[10] = (size_t(*)[10])calloc((size_t)n, sizeof(size_t[10]));
+    size_t (*scan_end)[MAX_SCANS] = (size_t(*)[MAX_SCANS])calloc((size_t)n, sizeof(size_t[MAX_SCANS]));
 #ifdef _OPENMP
     if (nthreads > 0) omp_set_num_threads(nthreads);
 #endif

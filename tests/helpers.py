@@ -66,6 +66,27 @@ def mask_truth(truth: np.ndarray, W: int, H: int, k: int) -> np.ndarray:
     return out
 
 
+def mask_truth_script(truth: np.ndarray, W: int, H: int, script, k: int) -> np.ndarray:
+    """What a decoder holds after scans 1..k of an arbitrary script, written from the meaning of
+    the script alone: a coefficient is known to the precision Al of the last scan <= k that
+    covers its component and zigzag position (DC: floor shift, AC: magnitude shift toward zero),
+    and is zero if no such scan exists.  script: [(components, Ss, Se, Ah, Al)]."""
+    comp = comp_of_block(W, H)
+    out = np.zeros_like(truth)
+    for comps, Ss, Se, _Ah, Al in script[:k]:
+        for c in comps:
+            sel = comp == c
+            sub = truth[sel][:, Ss:Se + 1].astype(np.int32)
+            if Ss == 0:
+                v = ((sub >> Al) << Al).astype(np.int16)
+            else:
+                v = _trunc(sub, Al)
+            blk = out[sel]
+            blk[:, Ss:Se + 1] = v
+            out[sel] = blk
+    return out
+
+
 def zigzag_natural():
     """zigzag position -> natural index, from the definition (sort by anti-diagonal, alternating)."""
     order = sorted(range(64), key=lambda i: (i // 8 + i % 8, (i // 8) if (i // 8 + i % 8) % 2 else (i % 8)))

@@ -1,0 +1,87 @@
+"""Other scan scripts than the ten-scan default (the paper, Section 4.2: scans that are not used
+can be left out; a record is one scan per group whatever the script).  The oracle is pinned on
+them against the generator's ground truth and the script's own meaning; the CUDA path is then
+compared with the oracle at every fidelity."""
+import numpy as np
+import pytest
+
+import pcr_synth
+from oracle import pcr_oracle as O
+
+from helpers import mask_truth, mask_truth_script
+
+SCRIPTS = {"spectral4": pcr_synth.SCRIPT_SPECTRAL_4, "mixed6": pcr_synth.SCRIPT_MIXED_6, "deep14": pcr_synth.SCRIPT_DEEP_14}
+TEN = [((0, 1, 2), 0, 0, 0, 1), ((0,), 1, 5, 0, 2), ((2,), 1, 63, 0, 1), ((1,), 1, 63, 0, 1), ((0,), 6, 63, 0, 2),
+       ((0,), 1, 63, 2, 1), ((0, 1, 2), 0, 0, 1, 0), ((2,), 1, 63, 1, 0), ((1,), 1, 63, 1, 0), ((0,), 1, 63, 1, 0)]
+
+
+def _record(name, config=2, n=3, **kw):
+    with pcr_synth.scan_script(SCRIPTS[name]):
+        return pcr_synth.make_record(config, n_images=n, **kw)
+
+
+def test_general_mask_agrees_with_the_ten_scan_closed_form(rec2_small):
+    W, H = rec2_small.dims[0]
+    t = rec2_small.truth(0)
+    for k in range(1, 11):
+        assert np.array_equal(mask_truth_script(t, W, H, TEN, k), mask_truth(t, W, H, k))
+
+
+@pytest.mark.parametrize("name", sorted(SCRIPTS))
+def test_oracle_on_other_scripts_every_k(name):
+    rec = _record(name)
+    n, G = O.record_info(rec.bytes)
+    assert G == len(SCRIPTS[name])
+    for i in range(n):
+        W, H = rec.dims[i]
+        for k in range(1, G + 1):
+            got = O.decode_image(rec.bytes, i, k, False)
+            got = got[0] if isinstance(got, tuple) else got
+            assert np.array_equal(got, mask_truth_script(rec.truth(i), W, H, SCRIPTS[name], k)), (name, i, k)
+
+
+@pytest.mark.parametrize("name", sorted(SCRIPTS))
+def test_oracle_other_scripts_without_restart_markers(name):
+    rec = _record(name, config=0, n=4, restart_rows=False)
+    _, G = O.record_info(rec.bytes)
+    for i in range(4):
+        got = O.decode_image(rec.bytes, i, G, False)
+        got = got[0] if isinstance(got, tuple) else got
+        assert np.array_equal(got, rec.truth(i))
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("name", sorted(SCRIPTS))
+@pytest.mark.parametrize("restart_rows", [True, False])
+def test_gpu_other_scripts_every_k(name, restart_rows):
+    import torch
+    from paper_1911_00472_b200 import Decoder, pcr_image_blocks
+    rec = _record(name, config=2, n=5, restart_rows=restart_rows)
+    dec = Decoder(rec.bytes)
+    try:
+        G = dec.n_groups
+        assert G == len(SCRIPTS[name])
+        for k in range(1, G + 1):
+            out = dec.decode(k)
+            torch.cuda.synchronize()
+            assert dec.status() == (-1, 0), (name, k)
+            coef = dec.coeffs().cpu().numpy()
+            out_h = out.cpu().numpy()
+            for i in range(rec.n_images):
+                want_c, want_rgb = O.decode_image(rec.bytes, i, k)
+                a, b = pcr_image_blocks(dec.handle, i)
+                assert np.array_equal(coef[a:a + b], want_c), (name, i, k)
+                inf = dec.info[i]
+                got = out_h[inf.out_offset:inf.out_offset + inf.out_bytes].reshape(inf.height, inf.width, 3)
+                assert np.array_equal(got, want_rgb), (name, i, k)
+        # raising the fidelity step by step ends at the same pixels
+        dec.decode(1)
+        for k in range(2, G + 1):
+            out = dec.decode_more(k)
+        torch.cuda.synchronize()
+        full = dec.decode(G, dec.alloc_out())
+        torch.cuda.synchronize()
+        for i in range(rec.n_images):
+            assert torch.equal(dec.image(out, i), dec.image(full, i)), (name, i)
+    finally:
+        dec.close()
