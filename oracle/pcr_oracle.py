@@ -237,3 +237,86 @@ def training_tensor(rgb: np.ndarray, crop, size: int, mean, std, dtype=np.float1
     m = np.asarray(mean, dtype=np.float64).reshape(3, 1, 1)
     s = np.asarray(std, dtype=np.float64).reshape(3, 1, 1)
     return ((out / 255.0 - m) / s).astype(dtype)
+
+
+# --------------------------------------------------------------------------------------
+# Multi-scale structural similarity (the paper's Section 4.3 and appendix figure "reconstruction
+# quality": MSSIM between the image decoded from scans 1..k and the full-fidelity image, used as
+# a diagnostic for choosing k).  The measure is Wang, Simoncelli and Bovik's (2003); the paper
+# does not say which implementation it ran.  Reading taken here, the common one:
+#   * luminance Y = 0.299 R + 0.587 G + 0.114 B of the decoded 8-bit pixels, dynamic range L = 255;
+#   * at every scale, local statistics under an 11x11 Gaussian window (sigma 1.5, normalised),
+#     evaluated only where the window lies inside the image;
+#   * cs = (2 s_xy + C2) / (s_x^2 + s_y^2 + C2), l = (2 m_x m_y + C1) / (m_x^2 + m_y^2 + C1),
+#     C1 = (0.01 L)^2, C2 = (0.03 L)^2, averaged over the positions of the scale;
+#   * next scale: 2x2 block averages (an odd last row or column is dropped);
+#   * result = prod_j max(mean cs_j, 0)^w_j * max(mean l_M, 0)^w_M over the M scales with the
+#     published weights (0.0448, 0.2856, 0.3001, 0.2363, 0.1333); images too small for five
+#     scales (a side below 11 * 2^(M-1)) use the first M weights, rescaled to sum to one (the
+#     five published weights are used as printed; they sum to 1.0001).
+# Plain float64, windows written out by the definition.
+# --------------------------------------------------------------------------------------
+MSSSIM_WEIGHTS = (0.0448, 0.2856, 0.3001, 0.2363, 0.1333)
+
+
+def gaussian_window(size: int = 11, sigma: float = 1.5) -> np.ndarray:
+    x = np.arange(size, dtype=np.float64) - (size - 1) / 2.0
+    g = np.exp(-(x * x) / (2.0 * sigma * sigma))
+    return g / g.sum()
+
+
+def luminance(rgb: np.ndarray) -> np.ndarray:
+    r = rgb.astype(np.float64)
+    return 0.299 * r[..., 0] + 0.587 * r[..., 1] + 0.114 * r[..., 2]
+
+
+def _valid_filter(a: np.ndarray, g: np.ndarray) -> np.ndarray:
+    """sum_{i,j} g[i] g[j] a[y+i, x+j] for every position where the window fits."""
+    n = g.size
+    H, W = a.shape
+    rows = np.zeros((H, W - n + 1), dtype=np.float64)
+    for j in range(n):
+        rows += g[j] * a[:, j:j + W - n + 1]
+    out = np.zeros((H - n + 1, W - n + 1), dtype=np.float64)
+    for i in range(n):
+        out += g[i] * rows[i:i + H - n + 1, :]
+    return out
+
+
+def msssim_scales(W: int, H: int, window: int = 11) -> int:
+    m = 0
+    while m < len(MSSSIM_WEIGHTS) and (min(W, H) >> m) >= window:
+        m += 1
+    return m
+
+
+def msssim(rgb_a: np.ndarray, rgb_b: np.ndarray) -> float:
+    """Multi-scale SSIM of two (H, W, 3) uint8 images of the same size (nan if a side is below 11)."""
+    if rgb_a.shape != rgb_b.shape:
+        raise ValueError("images differ in size")
+    x, y = luminance(rgb_a), luminance(rgb_b)
+    H, W = x.shape
+    M = msssim_scales(W, H)
+    if M == 0:
+        return float("nan")
+    w = np.array(MSSSIM_WEIGHTS[:M], dtype=np.float64)
+    if M < len(MSSSIM_WEIGHTS):
+        w = w / w.sum()
+    g = gaussian_window()
+    C1, C2 = (0.01 * 255.0) ** 2, (0.03 * 255.0) ** 2
+    result = 1.0
+    for j in range(M):
+        mx, my = _valid_filter(x, g), _valid_filter(y, g)
+        sxx = _valid_filter(x * x, g) - mx * mx
+        syy = _valid_filter(y * y, g) - my * my
+        sxy = _valid_filter(x * y, g) - mx * my
+        cs = ((2.0 * sxy + C2) / (sxx + syy + C2)).mean()
+        if j == M - 1:
+            lum = ((2.0 * mx * my + C1) / (mx * mx + my * my + C1)).mean()
+            result *= max(lum, 0.0) ** w[j]
+        result *= max(cs, 0.0) ** w[j]
+        if j < M - 1:
+            h2, w2 = x.shape[0] // 2, x.shape[1] // 2
+            x = x[:2 * h2, :2 * w2].reshape(h2, 2, w2, 2).mean(axis=(1, 3))
+            y = y[:2 * h2, :2 * w2].reshape(h2, 2, w2, 2).mean(axis=(1, 3))
+    return float(result)
