@@ -147,6 +147,26 @@ typedef struct {
 int pcr_decode_tensor(pcr_record* rec, int k, const pcr_crop* crops, int size, const float* mean, const float* std,
                       int dtype, void* rgb, void* tensor, void* stream);
 
+/* Multi-scale structural similarity between two decodes of the record, image by image (Section
+ * 4.3 and the appendix figure on reconstruction quality: the MSSIM of the image decoded from scan
+ * groups 1..k against the full-fidelity image is the paper's diagnostic for choosing k; scan
+ * groups of 5 and more reach 95 % there).  The measure is Wang, Simoncelli and Bovik's (2003) in
+ * its common form: luminance 0.299 R + 0.587 G + 0.114 B of the 8-bit pixels; per scale an 11x11
+ * Gaussian window (sigma 1.5) at the positions where it fits; cs = (2 s_xy + C2) / (s_x^2 + s_y^2
+ * + C2) and l = (2 m_x m_y + C1) / (m_x^2 + m_y^2 + C1) with C1 = 2.55^2, C2 = 7.65^2, averaged
+ * over the scale; the next scale is the 2x2 block average (an odd last row or column dropped);
+ * score = prod_j max(mean cs_j, 0)^w_j * max(mean l_M, 0)^w_M with the weights 0.0448, 0.2856,
+ * 0.3001, 0.2363, 0.1333; an image with a side below 176 has fewer scales (M = the number of j
+ * with min(W, H) >> j >= 11) and uses the first M weights rescaled to sum to one; M = 0: NaN.
+ *   rgb_a, rgb_b : DEVICE, two outputs of pcr_decode / pcr_decode_more of THIS record.
+ *   scratch      : DEVICE, pcr_msssim_scratch_bytes(rec) bytes, 16-byte aligned, caller-owned
+ *                  (two luminance pyramids per image and the per-scale sums).
+ *   dev_scores   : DEVICE, pcr_num_images floats, score of image i at index i.
+ * Enqueues on `stream` and returns.  The first call on a record uploads a small per-image table
+ * (one allocation).  Errors: PCR_E_ARG, PCR_E_NOMEM, PCR_E_CUDA. */
+size_t pcr_msssim_scratch_bytes(pcr_record* rec);
+int pcr_msssim(pcr_record* rec, const void* rgb_a, const void* rgb_b, void* scratch, float* dev_scores, void* stream);
+
 /* Forget which record bytes are resident on the device: the next pcr_decode copies its whole
  * prefix again (what a loader that streams each record once from host memory pays). */
 int pcr_evict(pcr_record* rec);

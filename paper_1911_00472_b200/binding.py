@@ -17,7 +17,7 @@ PCR_E_ARG, PCR_E_FORMAT, PCR_E_CORRUPT, PCR_E_TIMEOUT, PCR_E_CUDA, PCR_E_NOMEM =
 EXPORTS = ("pcr_open", "pcr_num_images", "pcr_num_groups", "pcr_get_image", "pcr_out_bytes", "pcr_prefix_bytes",
            "pcr_decode", "pcr_evict", "pcr_status", "pcr_coeffs", "pcr_image_blocks", "pcr_launch_count",
            "pcr_strerror", "pcr_close", "pcr_get_scan", "pcr_set_profiling", "pcr_get_profile",
-           "pcr_pixels_noalloc", "pcr_decode_more", "pcr_release_cached_memory", "pcr_decode_tensor")
+           "pcr_pixels_noalloc", "pcr_decode_more", "pcr_release_cached_memory", "pcr_decode_tensor", "pcr_msssim", "pcr_msssim_scratch_bytes")
 
 
 class ImageInfo(C.Structure):
@@ -62,6 +62,9 @@ def lib():
         L.pcr_decode.argtypes = [vp, C.c_int, vp, vp]
         L.pcr_decode_more.argtypes = [vp, C.c_int, vp, vp]
         L.pcr_decode_tensor.argtypes = [vp, C.c_int, vp, C.c_int, vp, vp, C.c_int, vp, vp, vp]
+        L.pcr_msssim_scratch_bytes.restype = C.c_size_t
+        L.pcr_msssim_scratch_bytes.argtypes = [vp]
+        L.pcr_msssim.argtypes = [vp, vp, vp, vp, vp, vp]
         L.pcr_evict.argtypes = [vp]
         L.pcr_status.argtypes = [vp, C.POINTER(C.c_int), C.POINTER(C.c_int)]
         L.pcr_coeffs.argtypes = [vp, C.POINTER(vp), C.POINTER(C.c_size_t)]
@@ -137,7 +140,16 @@ PCR_F16, PCR_F32 = 0, 1
 def pcr_decode_tensor(handle: int, k: int, crops_host_ptr: int, size: int, mean_host_ptr: int, std_host_ptr: int,
                       dtype: int, rgb_dev_ptr: int, tensor_dev_ptr: int, stream: int = 0) -> None:
     _chk(lib().pcr_decode_tensor(handle, k, crops_host_ptr, size, mean_host_ptr, std_host_ptr, dtype,
-                                 rgb_dev_ptr, tensor_dev_ptr, stream), "pcr_decode_tensor")
+                                 rgb_dev_ptr, tensor_dev_ptr, stream), "pcr_decode_tensor", "pcr_msssim", "pcr_msssim_scratch_bytes")
+
+
+def pcr_msssim_scratch_bytes(handle: int) -> int:
+    return lib().pcr_msssim_scratch_bytes(handle)
+
+
+def pcr_msssim(handle: int, rgb_a_dev_ptr: int, rgb_b_dev_ptr: int, scratch_dev_ptr: int, scores_dev_ptr: int,
+               stream: int = 0) -> None:
+    _chk(lib().pcr_msssim(handle, rgb_a_dev_ptr, rgb_b_dev_ptr, scratch_dev_ptr, scores_dev_ptr, stream), "pcr_msssim")
 
 
 def pcr_evict(handle: int) -> None:

@@ -22,6 +22,7 @@
 
 #include "../../include/pcr.h"
 #include "pcr_entropy.cuh"
+#include "pcr_msssim.cuh"
 #include "pcr_pixels.cuh"
 #include "pcr_types.h"
 
@@ -176,6 +177,9 @@ struct pcr_record {
     Unit* d_units = nullptr;
     uint16_t* d_qtab = nullptr;
     uint32_t* d_order = nullptr;  // processing order of the images (slices are runs of it)
+    MsDesc* d_ms = nullptr;       // per-image table of pcr_msssim (built on first use)
+    size_t ms_scratch = 0;        // bytes of scratch pcr_msssim needs
+    uint64_t ms_floats = 0;       // floats of all pyramids (the sums follow them)
     CropRect* d_crops = nullptr;  // crop rectangles of the last pcr_decode_tensor (allocated on first use)
     int* d_status = nullptr;
     std::vector<int> h_status;
@@ -986,6 +990,68 @@ int pcr_decode_tensor(pcr_record* rec, int k, const pcr_crop* crops, int size, c
     const int rc = decode_range(rec, 0, k, rgb, stream, &T);
     rec->decoded_k = 0;          // rows outside the crops were not decoded: nothing to raise the fidelity of
     return rc;
+}
+
+static void msssim_layout(pcr_record* rec, std::vector<MsDesc>* table) {
+    uint64_t floats = 0;
+    if (table) table->resize(rec->N);
+    for (int i = 0; i < rec->N; ++i) {
+        const uint32_t W = rec->info[i].width, H = rec->info[i].height;
+        uint32_t M = 0;
+        while (M < (uint32_t)kMsMaxScales && (std::min(W, H) >> M) >= (uint32_t)kMsWin) ++M;
+        uint64_t len = 0;
+        for (uint32_t j = 0; j < M; ++j) len += (uint64_t)(W >> j) * (H >> j);
+        if (table) {
+            MsDesc& d = (*table)[i];
+            d.W = W; d.H = H; d.M = M; d.rsvd = 0;
+            d.rgb_off = rec->info[i].out_offset; d.plane_off = floats; d.plane_len = len;
+        }
+        floats += 2 * len;
+    }
+    floats = (floats + 1) & ~1ull;                      // the double-precision sums start 8-byte aligned
+    rec->ms_floats = floats;
+    rec->ms_scratch = (size_t)(floats * 4 + (uint64_t)rec->N * kMsMaxScales * 2 * 8);
+}
+
+size_t pcr_msssim_scratch_bytes(pcr_record* rec) {
+    if (!rec) return 0;
+    if (!rec->ms_scratch) msssim_layout(rec, nullptr);
+    return rec->ms_scratch;
+}
+
+int pcr_msssim(pcr_record* rec, const void* rgb_a, const void* rgb_b, void* scratch, float* dev_scores, void* stream) {
+    if (!rec || !rgb_a || !rgb_b || !scratch || !dev_scores) return PCR_E_ARG;
+    if ((reinterpret_cast<uintptr_t>(scratch) & 15u) || (reinterpret_cast<uintptr_t>(dev_scores) & 3u)) return PCR_E_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!rec->d_ms) {
+        std::vector<MsDesc> table;
+        msssim_layout(rec, &table);
+        if (int rc = upload(rec, &rec->d_ms, table)) return rc;
+    }
+    float* planes = static_cast<float*>(scratch);
+    double* sums = reinterpret_cast<double*>(planes + rec->ms_floats);
+    if (cudaMemsetAsync(sums, 0, (size_t)rec->N * kMsMaxScales * 2 * 8, st) != cudaSuccess) return PCR_E_CUDA;
+    MsWindow win;
+    {
+        double g[kMsWin], tot = 0.0;
+        for (int k = 0; k < kMsWin; ++k) { const double x = k - (kMsWin - 1) / 2.0; g[k] = exp(-(x * x) / (2.0 * 1.5 * 1.5)); tot += g[k]; }
+        for (int k = 0; k < kMsWin; ++k) win.g[k] = (float)(g[k] / tot);
+    }
+    const unsigned N = (unsigned)rec->N;
+    ms_luma_kernel<<<dim3(64, N), 256, 0, st>>>(rec->d_ms, static_cast<const uint8_t*>(rgb_a), static_cast<const uint8_t*>(rgb_b), planes);
+    ++g_launches;
+    for (int j = 0; j < kMsMaxScales; ++j) {
+        ms_scale_kernel<<<dim3(j == 0 ? 32 : (j == 1 ? 8 : 2), N), kMsTile * kMsTile, 0, st>>>(rec->d_ms, planes, sums, j, win);
+        ++g_launches;
+        if (j + 1 < kMsMaxScales) {
+            ms_pool_kernel<<<dim3(j == 0 ? 32 : 8, N), 256, 0, st>>>(rec->d_ms, planes, j);
+            ++g_launches;
+        }
+    }
+    ms_final_kernel<<<(N + 255) / 256, 256, 0, st>>>(rec->d_ms, sums, dev_scores, (int)N);
+    ++g_launches;
+    if (cudaGetLastError() != cudaSuccess) return PCR_E_CUDA;
+    return PCR_OK;
 }
 
 int pcr_status(pcr_record* rec, int* first_bad_image, int* code) {

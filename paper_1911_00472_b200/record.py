@@ -82,6 +82,19 @@ class Decoder:
                                 s.cuda_stream)
         return tensor
 
+    def msssim(self, rgb_a: torch.Tensor, rgb_b: torch.Tensor, stream: torch.cuda.Stream | None = None) -> torch.Tensor:
+        """Multi-scale SSIM of every image between two decodes of this record: (N,) float32 on the
+        device.  Marshalling only (scratch and result tensors); the work is pcr_msssim's."""
+        need = B.pcr_msssim_scratch_bytes(self.handle)
+        if getattr(self, "_ms_scratch", None) is None or self._ms_scratch.numel() < need:
+            self._ms_scratch = torch.empty(max(need, 16), dtype=torch.uint8, device=self.device)
+        scores = torch.empty(self.n_images, dtype=torch.float32, device=self.device)
+        s = stream if stream is not None else torch.cuda.current_stream(self.device)
+        with torch.cuda.device(self.device):
+            B.pcr_msssim(self.handle, rgb_a.data_ptr(), rgb_b.data_ptr(), self._ms_scratch.data_ptr(), scores.data_ptr(),
+                         s.cuda_stream)
+        return scores
+
     def evict(self) -> None:
         B.pcr_evict(self.handle)
 
