@@ -140,7 +140,7 @@ PCR_F16, PCR_F32 = 0, 1
 def pcr_decode_tensor(handle: int, k: int, crops_host_ptr: int, size: int, mean_host_ptr: int, std_host_ptr: int,
                       dtype: int, rgb_dev_ptr: int, tensor_dev_ptr: int, stream: int = 0) -> None:
     _chk(lib().pcr_decode_tensor(handle, k, crops_host_ptr, size, mean_host_ptr, std_host_ptr, dtype,
-                                 rgb_dev_ptr, tensor_dev_ptr, stream), "pcr_decode_tensor", "pcr_msssim", "pcr_msssim_scratch_bytes")
+                                 rgb_dev_ptr, tensor_dev_ptr, stream), "pcr_decode_tensor")
 
 
 def pcr_msssim_scratch_bytes(handle: int) -> int:

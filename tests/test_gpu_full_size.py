@@ -85,3 +85,29 @@ def test_imagenet_shaped_full_record_training_tensor():
                 assert np.abs(got[i] - want).max() <= 2.0 ** -9, (k, i)
     finally:
         dec.close()
+
+
+def test_imagenet_shaped_full_record_msssim():
+    """pcr_msssim at full record size: sampled images against the oracle, every score in (0, 1],
+    more scan groups never score lower on average."""
+    import torch
+    from paper_1911_00472_b200 import Decoder
+    rec = pcr_synth.make_record(1, 0)
+    dec = Decoder(rec.bytes)
+    try:
+        full = dec.decode(10, dec.alloc_out())
+        means = []
+        for k in (1, 5):
+            part = dec.decode(k, dec.alloc_out())
+            s = dec.msssim(part, full)
+            torch.cuda.synchronize()
+            v = s.cpu().numpy()
+            assert np.all(v > 0) and np.all(v <= 1.0 + 1e-6)
+            means.append(v.mean())
+            for i in (3, 700):
+                _, lo = O.decode_image(rec.bytes, i, k)
+                _, hi = O.decode_image(rec.bytes, i, 10)
+                assert abs(float(v[i]) - O.msssim(lo, hi)) <= 2e-4, (k, i)
+        assert means[1] > means[0]
+    finally:
+        dec.close()
