@@ -335,6 +335,8 @@ def main():
     ap.add_argument("--k", type=int, default=10, help="scan group (fidelity) of the headline number")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--headline-only", action="store_true",
+                    help="only the timed steps, the end-to-end loop and the stage profile (no per-k, tensor, fidelity extras)")
     ap.add_argument("--images", type=int, default=0, help="images per record (default: the workload's 1024)")
     ap.add_argument("--sweep", action="store_true", help="run the streamed multi-record sweep over k = 1..10 instead")
     ap.add_argument("--records", type=int, default=16, help="records of the sweep")
@@ -463,75 +465,77 @@ def main():
     e2e["with_open_close"] = {"value": total_images * n_open / open_s, "unit": UNIT, "ms_per_step": 1000.0 * open_s / n_open,
                               "note": "pcr_open + pcr_decode from pinned host bytes + synchronise + pcr_status + pcr_close per step"}
 
-    # per-k numbers and the stage profile (this rank's GPU)
-    per_k = {}
-    for kk in pcr_synth.WORKLOADS[WORKLOAD].ks:
-        for _ in range(2):
+    per_k, raise_ms, training_tensor, fidelity = {}, {}, None, None
+    if not args.headline_only:
+        # per-k numbers and the stage profile (this rank's GPU)
+        per_k = {}
+        for kk in pcr_synth.WORKLOADS[WORKLOAD].ks:
+            for _ in range(2):
+                dec.decode(kk, out)
+            torch.cuda.synchronize(dev)
+            st = 5
+            per_k[str(kk)] = n_img * st / (timed_steps(kk, st) / 1000.0)
+        # decode straight to a fixed-size training batch (random-resized crops, flip, 224 x 224, fp16)
+        crops = pcr_synth.random_resized_crops(infos, 1000 + rank)
+        t_size = 224
+        t_mean, t_std = (0.485, 0.456, 0.406), (0.229, 0.224, 0.225)
+        tensor = torch.empty((n_img, 3, t_size, t_size), dtype=torch.float16, device=dev)
+        tensor_by_k = {}
+        for kk in pcr_synth.WORKLOADS[WORKLOAD].ks:
+            for _ in range(2):
+                dec.decode_tensor(kk, crops, t_size, t_mean, t_std, rgb=out, tensor=tensor)
+            torch.cuda.synchronize(dev)
+            st, acc = 5, 0.0
+            for _ in range(st):
+                flush.fill_(1)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                dec.decode_tensor(kk, crops, t_size, t_mean, t_std, rgb=out, tensor=tensor)
+                b.record(stream)
+                torch.cuda.synchronize(dev)
+                acc += a.elapsed_time(b)
+            tensor_by_k[str(kk)] = n_img * st / (acc / 1000.0)
+        crop_frac = float(sum(int(c[2]) * int(c[3]) for c in crops)) / float(sum(w * h for w, h in infos))
+        training_tensor = {"size": t_size, "dtype": "f16", "images_per_s_by_k": tensor_by_k,
+                           "crop_area_fraction": crop_frac,
+                           "note": "pcr_decode_tensor: random-resized crops (area 8-100 %, aspect 3/4-4/3), flip, bilinear, normalise; "
+                                   "only the MCUs a crop touches are transformed"}
+        # the paper's fidelity diagnostic: multi-scale SSIM of scan group k against full fidelity
+        full = dec.alloc_out()
+        dec.decode(dec.n_groups, full)
+        ms_by_k = {}
+        for kk in range(1, dec.n_groups):
             dec.decode(kk, out)
-        torch.cuda.synchronize(dev)
-        st = 5
-        per_k[str(kk)] = n_img * st / (timed_steps(kk, st) / 1000.0)
-    # decode straight to a fixed-size training batch (random-resized crops, flip, 224 x 224, fp16)
-    crops = pcr_synth.random_resized_crops(infos, 1000 + rank)
-    t_size = 224
-    t_mean, t_std = (0.485, 0.456, 0.406), (0.229, 0.224, 0.225)
-    tensor = torch.empty((n_img, 3, t_size, t_size), dtype=torch.float16, device=dev)
-    tensor_by_k = {}
-    for kk in pcr_synth.WORKLOADS[WORKLOAD].ks:
-        for _ in range(2):
-            dec.decode_tensor(kk, crops, t_size, t_mean, t_std, rgb=out, tensor=tensor)
-        torch.cuda.synchronize(dev)
-        st, acc = 5, 0.0
-        for _ in range(st):
-            flush.fill_(1)
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            dec.decode_tensor(kk, crops, t_size, t_mean, t_std, rgb=out, tensor=tensor)
-            b.record(stream)
+            sc = dec.msssim(out, full)
             torch.cuda.synchronize(dev)
-            acc += a.elapsed_time(b)
-        tensor_by_k[str(kk)] = n_img * st / (acc / 1000.0)
-    crop_frac = float(sum(int(c[2]) * int(c[3]) for c in crops)) / float(sum(w * h for w, h in infos))
-    training_tensor = {"size": t_size, "dtype": "f16", "images_per_s_by_k": tensor_by_k,
-                       "crop_area_fraction": crop_frac,
-                       "note": "pcr_decode_tensor: random-resized crops (area 8-100 %, aspect 3/4-4/3), flip, bilinear, normalise; "
-                               "only the MCUs a crop touches are transformed"}
-    # the paper's fidelity diagnostic: multi-scale SSIM of scan group k against full fidelity
-    full = dec.alloc_out()
-    dec.decode(dec.n_groups, full)
-    ms_by_k = {}
-    for kk in range(1, dec.n_groups):
-        dec.decode(kk, out)
-        sc = dec.msssim(out, full)
+            v = sc.float().cpu().numpy()
+            ms_by_k[str(kk)] = {"mean": float(np.nanmean(v)), "q25": float(np.nanpercentile(v, 25)), "q75": float(np.nanpercentile(v, 75))}
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(5):
+            dec.msssim(out, full)
+        b.record(stream)
         torch.cuda.synchronize(dev)
-        v = sc.float().cpu().numpy()
-        ms_by_k[str(kk)] = {"mean": float(np.nanmean(v)), "q25": float(np.nanpercentile(v, 25)), "q75": float(np.nanpercentile(v, 75))}
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record(stream)
-    for _ in range(5):
-        dec.msssim(out, full)
-    b.record(stream)
-    torch.cuda.synchronize(dev)
-    fidelity = {"msssim_vs_full_by_k": ms_by_k, "msssim_images_per_s": n_img * 5 / (a.elapsed_time(b) / 1000.0),
-                "note": "pcr_msssim on the decoded pixels of this record; the paper reports 95 %+ from scan group 5 on for its datasets"}
-    del full
-    # raising the fidelity of a resident decode: only the new scan groups are decoded
-    raise_ms = {}
-    for k_from, k_to in ((1, 10), (5, 10), (2, 5)):
-        if k_to > dec.n_groups:
-            continue
-        acc = 0.0
-        reps = 5
-        for _ in range(reps):
-            dec.decode(k_from, out)
-            flush.fill_(1)
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            dec.decode_more(k_to, out)
-            b.record(stream)
-            torch.cuda.synchronize(dev)
-            acc += a.elapsed_time(b) / reps
-        raise_ms[f"{k_from}->{k_to}"] = acc
+        fidelity = {"msssim_vs_full_by_k": ms_by_k, "msssim_images_per_s": n_img * 5 / (a.elapsed_time(b) / 1000.0),
+                    "note": "pcr_msssim on the decoded pixels of this record; the paper reports 95 %+ from scan group 5 on for its datasets"}
+        del full
+        # raising the fidelity of a resident decode: only the new scan groups are decoded
+        raise_ms = {}
+        for k_from, k_to in ((1, 10), (5, 10), (2, 5)):
+            if k_to > dec.n_groups:
+                continue
+            acc = 0.0
+            reps = 5
+            for _ in range(reps):
+                dec.decode(k_from, out)
+                flush.fill_(1)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                dec.decode_more(k_to, out)
+                b.record(stream)
+                torch.cuda.synchronize(dev)
+                acc += a.elapsed_time(b) / reps
+            raise_ms[f"{k_from}->{k_to}"] = acc
     binding.pcr_set_profiling(dec.handle, True)
     stage_ms, stage_n = {}, {}
     reps = 5
