@@ -134,6 +134,7 @@ struct pcr_record {
     std::vector<pcr_image_info> info;
     std::vector<uint64_t> blk_base, nblk;
     uint64_t total_blocks = 0, total_segs = 0;
+    bool widths_mult16 = true;    // every image is a multiple of 16 pixels wide (the DC-only pixel kernel's condition)
     size_t out_bytes = 0;
     // scan script analysis
     std::vector<ScanScript> script;
@@ -476,6 +477,7 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
         pcr_image_info& inf = r->info[i];
         inf.out_offset = out_off;
         out_off += (inf.out_bytes + 127) & ~127ull;
+        if (imgs[i].W & 15u) r->widths_mult16 = false;
         r->blk_base[i] = blocks; r->nblk[i] = 6ull * imgs[i].mx * imgs[i].my;
         imgs[i].blk_base = blocks; imgs[i].out_off = inf.out_offset;
         blocks += r->nblk[i];
@@ -828,13 +830,15 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
             const unsigned grid = nu;
             uint8_t* o8 = static_cast<uint8_t*>(out);
             if (!targs) {
-                if (dc_only) pixel_kernel<false, 2><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+                if (dc_only && rec->widths_mult16) dc_pixel_kernel<false><<<grid, 128, 0, q>>>(Q, o8);
+                else if (dc_only) pixel_kernel<false, 2><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
                 else if (head_only && any_refine) pixel_kernel<true, 3><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
                 else if (head_only) pixel_kernel<false, 3><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
                 else if (any_refine) pixel_kernel<true, 1><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
                 else pixel_kernel<false, 1><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
             } else {
-                if (dc_only) pixel_kernel<false, 2, true><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+                if (dc_only && rec->widths_mult16) dc_pixel_kernel<true><<<grid, 128, 0, q>>>(Q, o8);
+                else if (dc_only) pixel_kernel<false, 2, true><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
                 else if (head_only && any_refine) pixel_kernel<true, 3, true><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
                 else if (head_only) pixel_kernel<false, 3, true><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
                 else if (any_refine) pixel_kernel<true, 1, true><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);

@@ -296,6 +296,63 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
     }
 }
 
+// Pixel stage when nothing but DC coefficients has been decoded and every image is a multiple of
+// 16 pixels wide: each 8x8 luminance block is one constant sample, each MCU one chroma pair, so
+// an MCU row of the output is runs of eight equal pixels.  A CTA takes one work unit (8 MCUs of
+// one MCU row): 32 threads turn the unit's 32 luminance blocks into RGB triples (the same
+// arithmetic as the general kernel: the transform collapses to its k = 0 term, samples clamp to
+// 0..255), then every thread writes 16-byte vectors whose bytes are picked from the two triples
+// of the vector's MCU half-row.  48 bytes per MCU row = 3 vectors, so a vector never leaves its MCU.
+template <bool kRoi>
+__global__ void __launch_bounds__(128) dc_pixel_kernel(Params P, uint8_t* __restrict__ out) {
+    __shared__ uint32_t s_tri[2][2 * kPixMcus];        // [block row of the MCU row][block column]: R | G << 8 | B << 16
+    const int tid = threadIdx.x;
+    const Unit un = P.units[blockIdx.x];
+    const ImgDesc im = P.imgs[un.img];
+    const int nm = min((int)kPixMcus, (int)im.mx - (int)un.mcol0);
+    if (kRoi) {
+        const CropRect r = P.roi[un.img];
+        const uint32_t ux0 = 16u * un.mcol0, uy0 = 16u * un.mrow;
+        if (ux0 >= r.x0 + r.w || ux0 + 16u * (uint32_t)nm <= r.x0 || uy0 >= r.y0 + r.h || uy0 + 16u <= r.y0) return;
+    }
+    if (tid < 4 * nm) {
+        constexpr uint32_t K4 = 5793;
+        const int brow = tid / (2 * nm), bcol = tid % (2 * nm);
+        const uint16_t* q = P.qtab + (size_t)un.img * 192;
+        auto sample = [&](uint64_t blk, int comp) {
+            const int F = (int)P.head[blk * 8] * (int)q[64 * comp];
+            const int T = (int)(K4 * (uint32_t)F + (1u << 11)) >> 12;
+            const int smp = (int)(K4 * (uint32_t)T + (1u << 15) + (128u << 16)) >> 16;
+            return min(max(smp, 0), 255);
+        };
+        const uint64_t mcus = (uint64_t)im.mx * im.my;
+        const uint64_t yb = im.blk_base + (uint64_t)(2 * un.mrow + brow) * (2 * im.mx) + 2 * un.mcol0 + bcol;
+        const uint64_t cbk = im.blk_base + 4 * mcus + (uint64_t)un.mrow * im.mx + un.mcol0 + (bcol >> 1);
+        const int Y = sample(yb, 0), cb = sample(cbk, 1) - 128, cr = sample(cbk + mcus, 2) - 128;
+        const int R = Y + ((91881 * cr + 32768) >> 16);
+        const int G = Y + ((-22553 * cb - 46802 * cr + 32768) >> 16);
+        const int B = Y + ((116130 * cb + 32768) >> 16);
+        s_tri[brow][bcol] = (uint32_t)min(max(R, 0), 255) | ((uint32_t)min(max(G, 0), 255) << 8) | ((uint32_t)min(max(B, 0), 255) << 16);
+    }
+    __syncthreads();
+    const int nrows = min(16, (int)im.H - 16 * (int)un.mrow);
+    const size_t gpitch = (size_t)im.W * 3;
+    uint8_t* gbase = out + im.out_off + ((uint64_t)(16 * un.mrow) * im.W + 16 * (uint64_t)un.mcol0) * 3;
+    const int vec = 3 * nm;                                 // 16-byte vectors per output row of this unit
+    for (int i = tid; i < nrows * vec; i += 128) {
+        const int row = i / vec, v = i - row * vec, mcu = v / 3, kk = v - 3 * mcu;
+        const uint32_t A = s_tri[row >> 3][2 * mcu], Bt = s_tri[row >> 3][2 * mcu + 1];
+        // four-byte words of a run of equal pixels repeat with period three: RGBR GBRG BRGB
+        const uint32_t aw0 = __byte_perm(A, 0, 0x0210), aw1 = __byte_perm(A, 0, 0x1021), aw2 = __byte_perm(A, 0, 0x2102);
+        const uint32_t bw0 = __byte_perm(Bt, 0, 0x0210), bw1 = __byte_perm(Bt, 0, 0x1021), bw2 = __byte_perm(Bt, 0, 0x2102);
+        uint4 o;
+        if (kk == 0) o = make_uint4(aw0, aw1, aw2, aw0);           // bytes 0..15: left pixels
+        else if (kk == 1) o = make_uint4(aw1, aw2, bw0, bw1);      // bytes 16..23 left, 24..31 right
+        else o = make_uint4(bw2, bw0, bw1, bw2);                   // bytes 32..47: right pixels
+        *reinterpret_cast<uint4*>(gbase + row * gpitch + 16 * v) = o;
+    }
+}
+
 // Training-tensor epilogue: crop, optional mirror, bilinear resize to size x size with half-pixel
 // centres (the crop's edge pixels repeated, no low-pass filter), (v / 255 - mean) / std, planar
 // output [image][channel][row][column].  Images pos0 .. pos0 + gridDim.y - 1 of the processing order.

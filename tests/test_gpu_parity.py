@@ -194,3 +194,20 @@ def test_corrupt_entropy_data_sets_status_not_a_fault(rec0):
         inf = dec.info[i]
         assert torch.equal(out[inf.out_offset:inf.out_offset + inf.out_bytes], good[inf.out_offset:inf.out_offset + inf.out_bytes])
     dec.close(); ref.close()
+
+
+def test_widths_multiple_of_16_odd_heights_dc_only_path():
+    """Images 16-pixel aligned in width (the DC-only pixel kernel's condition) with heights that
+    end inside an MCU row, random coefficient fields: every k, k = 1 included."""
+    rng = np.random.default_rng(7)
+    dims = [(48, 37), (16, 1), (64, 100), (32, 8), (496, 23)]
+    coeffs = []
+    for w, h in dims:
+        c = np.zeros((pcr_synth.num_blocks(w, h), 64), dtype=np.int16)
+        c[:, 0] = rng.integers(-300, 300, c.shape[0])
+        hit = rng.random(c.shape) < 0.08
+        hit[:, 0] = False
+        c[hit] = rng.integers(-12, 13, int(hit.sum()))
+        coeffs.append(c)
+    rec = pcr_synth.record_from_coeffs(dims, coeffs)
+    _compare(rec, (1, 2, 7, 10))
