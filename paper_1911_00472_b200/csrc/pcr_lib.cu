@@ -185,6 +185,9 @@ struct pcr_record {
     int* d_status = nullptr;
     std::vector<int> h_status;
     std::vector<std::pair<void*, size_t>> bufs;   // every device buffer of the record with its size
+    cudaStream_t up_stream = nullptr;             // pcr_open's uploads and memsets (never the default stream:
+                                                  // that one would wait for every other record's decode)
+    cudaEvent_t ev_ready = nullptr;               // the record's device state is set up
     cudaEvent_t ev_done = nullptr;                // end of the last decode enqueued
     bool decode_enqueued = false;
     // optional stage timing
@@ -329,8 +332,13 @@ int parse_chunk(const uint8_t* rec, uint64_t off, uint32_t len, bool first, Imag
 }
 
 void free_device(pcr_record* r) {
-    // nothing is handed on before the record's last decode has finished
+    // nothing is handed on before the record's set-up and its last decode have finished
+    if (r->up_stream) cudaStreamSynchronize(r->up_stream);
     if (r->ev_done && r->decode_enqueued) cudaEventSynchronize(r->ev_done);
+    if (r->ev_ready) pool_event_put(r->ev_ready, r->device);
+    r->ev_ready = nullptr;
+    if (r->up_stream) pool_stream_put(r->up_stream, r->device);
+    r->up_stream = nullptr;
     r->decode_enqueued = false;
     for (cudaStream_t q : r->streams) pool_stream_put(q, r->device);
     r->streams.clear();
@@ -374,7 +382,8 @@ template <class T>
 int upload(pcr_record* r, T** dst, const std::vector<T>& v) {
     size_t n = std::max<size_t>(v.size(), 1) * sizeof(T);
     if (int rc = take(r, dst, n)) return rc;
-    if (!v.empty() && cudaMemcpy(*dst, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice) != cudaSuccess) return PCR_E_CUDA;
+    // pageable source: the call returns once the bytes sit in the driver's staging memory
+    if (!v.empty() && cudaMemcpyAsync(*dst, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice, r->up_stream) != cudaSuccess) return PCR_E_CUDA;
     return PCR_OK;
 }
 
@@ -604,17 +613,19 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
 
     // device state
     if (cudaGetDevice(&r->device) != cudaSuccess) return PCR_E_CUDA;
+    if (!(r->up_stream = pool_stream_get(r->device))) return PCR_E_CUDA;
     if (int rc = take(r, &r->d_aux, (size_t)(std::max<uint64_t>(aux_words, 2) * 8))) return rc;
-    if (cudaMemset(r->d_aux, 0, std::max<uint64_t>(aux_words, 2) * 8) != cudaSuccess) return PCR_E_CUDA;
+    if (cudaMemsetAsync(r->d_aux, 0, std::max<uint64_t>(aux_words, 2) * 8, r->up_stream) != cudaSuccess) return PCR_E_CUDA;
     if (int rc = take(r, &r->d_rec, (size_t)(len + 64))) return rc;
     if (int rc = take(r, &r->d_ubuf, (size_t)(len + 256))) return rc;
-    if (cudaMemset(r->d_ubuf, 0, len + 256) != cudaSuccess) return PCR_E_CUDA;
+    if (cudaMemsetAsync(r->d_ubuf, 0, len + 256, r->up_stream) != cudaSuccess) return PCR_E_CUDA;
     if (int rc = take(r, &r->d_planes, (size_t)(std::max<uint64_t>(blocks, 1) * 128))) return rc;
     if (int rc = take(r, &r->d_head, (size_t)(std::max<uint64_t>(blocks, 1) * 16))) return rc;
-    if (cudaMemset(r->d_head, 0, std::max<uint64_t>(blocks, 1) * 16) != cudaSuccess) return PCR_E_CUDA;
+    if (cudaMemsetAsync(r->d_head, 0, std::max<uint64_t>(blocks, 1) * 16, r->up_stream) != cudaSuccess) return PCR_E_CUDA;
     if (int rc = take(r, &r->d_seg, (size_t)((segs + 1) * 4))) return rc;
     if (int rc = take(r, &r->d_status, (size_t)((size_t)N * 4))) return rc;
-    if (cudaMemset(r->d_seg, 0, (segs + 1) * 4) != cudaSuccess || cudaMemset(r->d_status, 0, (size_t)N * 4) != cudaSuccess) return PCR_E_CUDA;
+    if (cudaMemsetAsync(r->d_seg, 0, (segs + 1) * 4, r->up_stream) != cudaSuccess ||
+        cudaMemsetAsync(r->d_status, 0, (size_t)N * 4, r->up_stream) != cudaSuccess) return PCR_E_CUDA;
     int rc;
     if ((rc = upload(r, &r->d_script, r->script))) return rc;
     if ((rc = upload(r, &r->d_saux, r->saux))) return rc;
@@ -627,8 +638,9 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     r->h_status.assign(N, 0);
     r->resident = 0;
     if (!(r->ev_done = pool_event_get(r->device))) return PCR_E_CUDA;
-    // the zeroing above ran on the default stream; decodes may run on streams that do not wait for it
-    if (cudaStreamSynchronize(cudaStreamLegacy) != cudaSuccess) return PCR_E_CUDA;
+    // the set-up above runs on the record's own stream; every decode waits for this event first
+    if (!(r->ev_ready = pool_event_get(r->device))) return PCR_E_CUDA;
+    if (cudaEventRecord(r->ev_ready, r->up_stream) != cudaSuccess) return PCR_E_CUDA;
     if (r->n_slices > 1) {
         if (!(r->ev_fork = pool_event_get(r->device))) return PCR_E_CUDA;
         if (!(r->copy_stream = pool_stream_get(r->device))) return PCR_E_CUDA;
@@ -718,6 +730,7 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
         rec->stages.push_back(t);
         cudaEventRecord(rec->events[rec->stages.size()], st);
     };
+    if (cudaStreamWaitEvent(st, rec->ev_ready, 0) != cudaSuccess) return PCR_E_CUDA;      // pcr_open's uploads
     if (prof) cudaEventRecord(rec->events[0], st);
     const bool pipelined = rec->n_slices > 1 && !prof;
     if (!pipelined && rec->resident < need) {
@@ -1031,7 +1044,9 @@ int pcr_msssim(pcr_record* rec, const void* rgb_a, const void* rgb_b, void* scra
         std::vector<MsDesc> table;
         msssim_layout(rec, &table);
         if (int rc = upload(rec, &rec->d_ms, table)) return rc;
+        if (cudaEventRecord(rec->ev_ready, rec->up_stream) != cudaSuccess) return PCR_E_CUDA;
     }
+    if (cudaStreamWaitEvent(st, rec->ev_ready, 0) != cudaSuccess) return PCR_E_CUDA;
     float* planes = static_cast<float*>(scratch);
     double* sums = reinterpret_cast<double*>(planes + rec->ms_floats);
     if (cudaMemsetAsync(sums, 0, (size_t)rec->N * kMsMaxScales * 2 * 8, st) != cudaSuccess) return PCR_E_CUDA;
