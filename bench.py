@@ -461,14 +461,20 @@ def main():
     # the same with the record opened and closed inside every step (what a loader pays that sees
     # every record once: host-side parse, table uploads, copy, decode)
     n_open = max(5, min(args.steps, 30))
-    sync_all()
-    to = time.perf_counter()
-    for _ in range(n_open):
+
+    def open_decode_close():
         h = binding.pcr_open(dec.host.data_ptr(), dec.host.numel())
         binding.pcr_decode(h, k, out.data_ptr(), stream.cuda_stream)
         torch.cuda.synchronize(dev)
         binding.pcr_status(h)
         binding.pcr_close(h)
+
+    for _ in range(2):                 # the first opens allocate the second record's device buffers
+        open_decode_close()
+    sync_all()
+    to = time.perf_counter()
+    for _ in range(n_open):
+        open_decode_close()
     open_s = reduce_max(time.perf_counter() - to, world)
     e2e["with_open_close"] = {"value": total_images * n_open / open_s, "unit": UNIT, "ms_per_step": 1000.0 * open_s / n_open,
                               "note": "pcr_open + pcr_decode from pinned host bytes + synchronise + pcr_status + pcr_close per step"}

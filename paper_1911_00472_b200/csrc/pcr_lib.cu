@@ -176,6 +176,7 @@ struct pcr_record {
     uint32_t* d_seg = nullptr;
     Item* d_items = nullptr;
     Unit* d_units = nullptr;
+    uint32_t* d_unit_prefix = nullptr;
     uint16_t* d_qtab = nullptr;
     uint32_t* d_order = nullptr;  // processing order of the images (slices are runs of it)
     MsDesc* d_ms = nullptr;       // per-image table of pcr_msssim (built on first use)
@@ -200,6 +201,19 @@ static const int kMaxStages = 16;
 
 static inline uint32_t rd32(const uint8_t* p) { return (uint32_t)p[0] | ((uint32_t)p[1] << 8) | ((uint32_t)p[2] << 16) | ((uint32_t)p[3] << 24); }
 static inline uint64_t rd64(const uint8_t* p) { return (uint64_t)rd32(p) | ((uint64_t)rd32(p + 4) << 32); }
+
+// Writes the list of pixel work units at set-up: block = position of the processing order.
+__global__ void __launch_bounds__(128) units_kernel(const ImgDesc* __restrict__ imgs, const uint32_t* __restrict__ order,
+                                                    const uint32_t* __restrict__ prefix, Unit* __restrict__ units) {
+    const uint32_t img = order[blockIdx.x];
+    const uint32_t per_row = (imgs[img].mx + kPixMcus - 1) / kPixMcus, n = per_row * imgs[img].my;
+    Unit* dst = units + prefix[blockIdx.x];
+    for (uint32_t j = threadIdx.x; j < n; j += 128) {
+        Unit un;
+        un.img = img; un.mrow = (uint16_t)(j / per_row); un.mcol0 = (uint16_t)((j % per_row) * kPixMcus);
+        dst[j] = un;
+    }
+}
 
 namespace {
 
@@ -513,7 +527,9 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     for (uint32_t s = 0; s < G; ++s) r->wave_scans[r->wave_of_scan[s]].push_back((int)s);
     // slices: enough images each to fill the machine, few enough to keep launches cheap
     {
-        int want = (int)std::min<uint32_t>(8, std::max<uint32_t>(1, N / 128));
+        // four at most: one record decodes as fast with four slices as with eight, and two records
+        // in flight then stay close to the eight hardware queues that streams are mapped onto
+        int want = (int)std::min<uint32_t>(4, std::max<uint32_t>(1, N / 128));
         if (const char* e = getenv("PCR_SLICES")) want = std::max(1, std::min(64, atoi(e)));
         r->n_slices = (int)std::min<uint32_t>((uint32_t)want, N);
         r->slice_img.resize(r->n_slices + 1);
@@ -559,20 +575,19 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
                 if (!items.empty() && items.back().next == kItemOpen) items.back().next = 0;
                 r->item_count[(size_t)g * G + s] = (uint32_t)items.size() - r->item_begin[(size_t)g * G + s];
             }
-    std::vector<Unit> units;
-    units.reserve((size_t)(blocks / 24 + N));
-    r->slice_unit.assign(r->n_slices + 1, 0);
-    for (int g = 0; g < r->n_slices; ++g) {
-        r->slice_unit[g] = (uint32_t)units.size();
-        for (uint32_t pos = r->slice_img[g]; pos < r->slice_img[g + 1]; ++pos)
-            for (uint32_t i = order[pos], row = 0; row < imgs[i].my; ++row)
-                for (uint32_t col = 0; col < imgs[i].mx; col += kPixMcus) {
-                    if (imgs[i].my > 65535 || imgs[i].mx > 65535) return PCR_E_FORMAT;
-                    units.push_back(Unit{i, (uint16_t)row, (uint16_t)col});
-                }
+    // pixel work units (8 MCUs of one MCU row), image by image in processing order, inside an image
+    // MCU row by MCU row.  The host only counts them; a small kernel writes the list at set-up.
+    std::vector<uint32_t> unit_prefix(N + 1, 0);
+    for (uint32_t pos = 0; pos < N; ++pos) {
+        const ImgDesc& im = imgs[order[pos]];
+        if (im.my > 65535 || im.mx > 65535) return PCR_E_FORMAT;
+        const uint64_t nu = (uint64_t)((im.mx + kPixMcus - 1) / kPixMcus) * im.my;
+        if (unit_prefix[pos] + nu >= (1ull << 32)) return PCR_E_FORMAT;
+        unit_prefix[pos + 1] = unit_prefix[pos] + (uint32_t)nu;
     }
-    r->slice_unit[r->n_slices] = (uint32_t)units.size();
-    r->n_units = (uint32_t)units.size();
+    r->slice_unit.assign(r->n_slices + 1, 0);
+    for (int g = 0; g <= r->n_slices; ++g) r->slice_unit[g] = unit_prefix[r->slice_img[g]];
+    r->n_units = unit_prefix[N];
 
     // side data of the AC scans: one word per block for a first pass, four for a refinement
     const uint64_t total_mcus = blocks / 6;
@@ -615,26 +630,34 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     if (cudaGetDevice(&r->device) != cudaSuccess) return PCR_E_CUDA;
     if (!(r->up_stream = pool_stream_get(r->device))) return PCR_E_CUDA;
     if (int rc = take(r, &r->d_aux, (size_t)(std::max<uint64_t>(aux_words, 2) * 8))) return rc;
-    if (cudaMemsetAsync(r->d_aux, 0, std::max<uint64_t>(aux_words, 2) * 8, r->up_stream) != cudaSuccess) return PCR_E_CUDA;
+    // zeroing is enqueued after the table uploads: a copy from pageable memory first waits for
+    // everything already in its stream
+    std::vector<std::pair<void*, size_t>> zero;
+    zero.push_back({r->d_aux, (size_t)(std::max<uint64_t>(aux_words, 2) * 8)});
     if (int rc = take(r, &r->d_rec, (size_t)(len + 64))) return rc;
     if (int rc = take(r, &r->d_ubuf, (size_t)(len + 256))) return rc;
-    if (cudaMemsetAsync(r->d_ubuf, 0, len + 256, r->up_stream) != cudaSuccess) return PCR_E_CUDA;
+    zero.push_back({r->d_ubuf, len + 256});
     if (int rc = take(r, &r->d_planes, (size_t)(std::max<uint64_t>(blocks, 1) * 128))) return rc;
     if (int rc = take(r, &r->d_head, (size_t)(std::max<uint64_t>(blocks, 1) * 16))) return rc;
-    if (cudaMemsetAsync(r->d_head, 0, std::max<uint64_t>(blocks, 1) * 16, r->up_stream) != cudaSuccess) return PCR_E_CUDA;
+    zero.push_back({r->d_head, (size_t)(std::max<uint64_t>(blocks, 1) * 16)});
     if (int rc = take(r, &r->d_seg, (size_t)((segs + 1) * 4))) return rc;
     if (int rc = take(r, &r->d_status, (size_t)((size_t)N * 4))) return rc;
-    if (cudaMemsetAsync(r->d_seg, 0, (segs + 1) * 4, r->up_stream) != cudaSuccess ||
-        cudaMemsetAsync(r->d_status, 0, (size_t)N * 4, r->up_stream) != cudaSuccess) return PCR_E_CUDA;
+    zero.push_back({r->d_seg, (size_t)((segs + 1) * 4)});
+    zero.push_back({r->d_status, (size_t)N * 4});
     int rc;
     if ((rc = upload(r, &r->d_script, r->script))) return rc;
     if ((rc = upload(r, &r->d_saux, r->saux))) return rc;
     if ((rc = upload(r, &r->d_scans, scans))) return rc;
     if ((rc = upload(r, &r->d_imgs, imgs))) return rc;
     if ((rc = upload(r, &r->d_items, items))) return rc;
-    if ((rc = upload(r, &r->d_units, units))) return rc;
     if ((rc = upload(r, &r->d_qtab, qtab))) return rc;
+    if ((rc = upload(r, &r->d_unit_prefix, unit_prefix))) return rc;
+    if ((rc = take(r, &r->d_units, (size_t)std::max<uint32_t>(r->n_units, 1) * sizeof(Unit)))) return rc;
     if ((rc = upload(r, &r->d_order, order))) return rc;
+    units_kernel<<<N, 128, 0, r->up_stream>>>(r->d_imgs, r->d_order, r->d_unit_prefix, r->d_units);
+    ++g_launches;
+    for (auto& z : zero)
+        if (cudaMemsetAsync(z.first, 0, z.second, r->up_stream) != cudaSuccess) return PCR_E_CUDA;
     r->h_status.assign(N, 0);
     r->resident = 0;
     if (!(r->ev_done = pool_event_get(r->device))) return PCR_E_CUDA;
