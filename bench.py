@@ -342,6 +342,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--k", type=int, default=10, help="scan group (fidelity) of the headline number")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=WORKLOAD, choices=[1, 2, 3],
+                    help="1 ImageNet-shaped (the headline), 2 CelebA-shaped, 3 HAM10000-shaped (no restart markers)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--headline-only", action="store_true",
                     help="only the timed steps, the end-to-end loop and the stage profile (no per-k, tensor, fidelity extras)")
@@ -368,7 +370,11 @@ def main():
     import pcr_synth
 
     # input record of this rank; the oracle's process pool starts before the first GPU call
-    rec = pcr_synth.make_record(WORKLOAD, rank_record_index(rank), n_images=args.images or None)
+    wl = args.workload
+    wl_desc = WORKLOAD_DESC if wl == WORKLOAD else {
+        2: "celeba_shaped: 1 record x 1024 images per GPU, 178x218, q95, 4:2:0, 10-scan script, restart per MCU row",
+        3: "ham10000_shaped: 1 record x 1024 images per GPU, 600x450, q90, 4:2:0, 10-scan script, no restart markers"}[wl]
+    rec = pcr_synth.make_record(wl, rank_record_index(rank), n_images=args.images or None)
     pool = None
     tmpdir = None
     cores = len(os.sched_getaffinity(0))
@@ -483,7 +489,7 @@ def main():
     if not args.headline_only:
         # per-k numbers and the stage profile (this rank's GPU)
         per_k = {}
-        for kk in pcr_synth.WORKLOADS[WORKLOAD].ks:
+        for kk in pcr_synth.WORKLOADS[wl].ks:
             for _ in range(2):
                 dec.decode(kk, out)
             torch.cuda.synchronize(dev)
@@ -495,7 +501,7 @@ def main():
         t_mean, t_std = (0.485, 0.456, 0.406), (0.229, 0.224, 0.225)
         tensor = torch.empty((n_img, 3, t_size, t_size), dtype=torch.float16, device=dev)
         tensor_by_k = {}
-        for kk in pcr_synth.WORKLOADS[WORKLOAD].ks:
+        for kk in pcr_synth.WORKLOADS[wl].ks:
             for _ in range(2):
                 dec.decode_tensor(kk, crops, t_size, t_mean, t_std, rgb=out, tensor=tensor)
             torch.cuda.synchronize(dev)
@@ -606,7 +612,7 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_max / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "int16/u8", "data": "synthetic",
-            "config": {"workload": WORKLOAD_DESC, "k": k, "images_per_step_per_gpu": n_img,
+            "config": {"workload": wl_desc, "k": k, "images_per_step_per_gpu": n_img,
                        "l2": "flushed by a 256 MiB write before every timed step",
                        "record_bytes": int(rec.bytes.size), "prefix_bytes_at_k": int(prefix),
                        "mean_compressed_bytes_per_image_by_scan": [c / n_img for c in comp]},
