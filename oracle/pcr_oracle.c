@@ -124,6 +124,7 @@ typedef struct {
     htab dc[4], ac[4];
     int ri;
     int have_frame;
+    int sequential;          /* frame header was SOF0: one interleaved scan carries whole blocks */
     int16_t* coef;          /* canonical layout: comp, block row, block col, zigzag */
 } jdec;
 
@@ -226,7 +227,27 @@ static int decode_scan(jdec* J, const scan_hdr* S, const uint8_t* data, size_t n
                 for (int bx = 0; bx < nh; ++bx) {
                     size_t brow = (size_t)mrow * nv + by, bcol = (size_t)mcol * nh + bx;
                     int16_t* blk = J->coef + (J->coff[c] + brow * J->bw[c] + bcol) * 64;
-                    if (S->Ss == 0) {
+                    if (S->Ss == 0 && S->Se == 63) {
+                        /* sequential DCT scan (F.2.2): the block's DC difference, then its AC
+                         * coefficients as (run, size) symbols up to an end-of-block symbol */
+                        int s0 = decode_sym(&b, &J->dc[S->td[si]], &err);
+                        if (s0 > 15) err = 1;
+                        pred[c] += extend(receive(&b, s0), s0);
+                        blk[0] = (int16_t)pred[c];
+                        int k = 1;
+                        while (k <= 63 && !err) {
+                            int rs = decode_sym(&b, &J->ac[S->ta[si]], &err);
+                            int r = rs >> 4, s = rs & 15;
+                            if (s != 0) {
+                                k += r;
+                                if (k > 63) { err = 1; break; }
+                                blk[k] = (int16_t)extend(receive(&b, s), s);
+                                ++k;
+                            } else if (r == 15) k += 16;
+                            else if (r == 0) break;                    /* end of block */
+                            else { err = 1; break; }                   /* end-of-band runs exist in progressive scans only */
+                        }
+                    } else if (S->Ss == 0) {
                         if (S->Ah == 0) {                              /* DC first (G.2.1) */
                             int s = decode_sym(&b, &J->dc[S->td[si]], &err);
                             if (s > 15) err = 1;
@@ -325,7 +346,8 @@ static int jpeg_decode_coeffs(jdec* J, const uint8_t* d, size_t n, int16_t* coef
                 }
                 J->qdef[tq] = 1;
             }
-        } else if (mk == 0xC2) {                    /* SOF2: progressive, Huffman */
+        } else if (mk == 0xC2 || mk == 0xC0) {      /* SOF2: progressive, Huffman; SOF0: baseline sequential */
+            J->sequential = mk == 0xC0;
             if (sl < 6 || s[0] != 8) return ORC_E_UNSUPPORTED;
             J->H = (s[1] << 8) | s[2]; J->W = (s[3] << 8) | s[4]; J->ncomp = s[5];
             if (J->ncomp != 3 || sl < 6 + 9 || J->W == 0 || J->H == 0) return ORC_E_UNSUPPORTED;
@@ -340,7 +362,7 @@ static int jpeg_decode_coeffs(jdec* J, const uint8_t* d, size_t n, int16_t* coef
             J->coef = coef;
             memset(coef, 0, ncoef * sizeof(int16_t));
             J->have_frame = 1;
-        } else if (mk == 0xC0 || mk == 0xC1 || (mk >= 0xC3 && mk <= 0xCF && mk != 0xC4 && mk != 0xC8 && mk != 0xCC)) {
+        } else if (mk == 0xC1 || (mk >= 0xC3 && mk <= 0xCF && mk != 0xC4 && mk != 0xC8 && mk != 0xCC)) {
             return ORC_E_UNSUPPORTED;               /* other frame types */
         } else if (mk == 0xC4) {                    /* DHT */
             size_t q = 0;
@@ -373,7 +395,11 @@ static int jpeg_decode_coeffs(jdec* J, const uint8_t* d, size_t n, int16_t* coef
             }
             S.Ss = s[1 + 2 * S.ns]; S.Se = s[2 + 2 * S.ns]; S.Ah = s[3 + 2 * S.ns] >> 4; S.Al = s[3 + 2 * S.ns] & 15;
             if (S.Ss > S.Se || S.Se > 63 || S.Al > 13) return ORC_E_CORRUPT;
-            if (S.Ss == 0 && S.Se != 0) return ORC_E_CORRUPT;      /* DC and AC never share a scan */
+            if (J->sequential) {                                   /* one kind of scan: everything of its components */
+                if (S.Ss != 0 || S.Se != 63 || S.Ah != 0 || S.Al != 0 || S.ns != 3) return ORC_E_UNSUPPORTED;
+                for (int i = 0; i < S.ns; ++i)
+                    if (!J->dc[S.td[i]].defined || !J->ac[S.ta[i]].defined) return ORC_E_CORRUPT;
+            } else if (S.Ss == 0 && S.Se != 0) return ORC_E_CORRUPT;  /* DC and AC never share a progressive scan */
             if (S.Ss > 0 && S.ns != 1) return ORC_E_CORRUPT;       /* AC scans hold one component */
             if (S.Ah != 0 && S.Ah != S.Al + 1) return ORC_E_CORRUPT;
             for (int i = 0; i < S.ns; ++i) {
@@ -518,7 +544,7 @@ int oracle_jpeg_dims(const uint8_t* d, size_t n, uint32_t* W, uint32_t* H) {
         int mk = d[p + 1];
         if (mk == 0xFF) { ++p; continue; }
         size_t L = ((size_t)d[p + 2] << 8) | d[p + 3];
-        if (mk == 0xC2) {
+        if (mk == 0xC2 || mk == 0xC0) {
             if (p + 9 > n) return ORC_E_CORRUPT;
             *H = ((uint32_t)d[p + 5] << 8) | d[p + 6]; *W = ((uint32_t)d[p + 7] << 8) | d[p + 8];
             return ORC_OK;

@@ -324,6 +324,10 @@ SCRIPT_DEEP_14 = [((0, 1, 2), 0, 0, 0, 2), ((0,), 1, 9, 0, 3), ((0,), 10, 63, 0,
                   ((1,), 1, 63, 1, 0), ((2,), 1, 63, 1, 0)]
 
 
+# baseline (sequential) JPEG: one interleaved scan with the DC and all AC coefficients of every block
+SCRIPT_BASELINE = [((0, 1, 2), 0, 63, 0, 0)]
+
+
 class scan_script:
     """Context manager: records made inside use `script` (a list of (components, Ss, Se, Ah, Al),
     at most 16 scans) instead of the ten-scan default.  Not thread safe (a process-wide setting)."""

@@ -394,6 +394,22 @@ static void enc_ac_first(scan_enc* e, const int16_t* blk, int Ss, int Se, int Al
     }
 }
 
+/* a whole block of a sequential (baseline) scan: the AC part ends with a plain end-of-block
+ * symbol unless position 63 is non-zero; there are no end-of-band runs */
+static void enc_ac_sequential(scan_enc* e, const int16_t* blk, int slot) {
+    int run = 0;
+    for (int k = 1; k <= 63; ++k) {
+        int v = blk[k], a = v < 0 ? -v : v;
+        if (a == 0) { ++run; continue; }
+        while (run > 15) { tk_sym(&e->tok, slot, 0xF0); run -= 16; }
+        int s = bitlen(a);
+        tk_sym(&e->tok, slot, (run << 4) | s);
+        tk_bits(&e->tok, (uint32_t)(v < 0 ? ~a : a), s);
+        run = 0;
+    }
+    if (run > 0) tk_sym(&e->tok, slot, 0x00);
+}
+
 static void enc_ac_refine(scan_enc* e, const int16_t* blk, int Ss, int Se, int Al, int slot) {
     int mag[64], last_new = -1;
     for (int k = Ss; k <= Se; ++k) {
@@ -490,6 +506,7 @@ static void encode_scan(enc_state* st, const geom_t* g, const int16_t* coef, con
     scan_enc* e = &st->se;
     e->tok.n = 0; e->ncorr = 0; e->eobrun = 0; e->eobslot = 0;
     int inter = sc->ncomp > 1;
+    int sequential = sc->Ss == 0 && sc->Se == 63;      /* DC and AC of every block in one scan: baseline */
     int c0 = sc->comp[0];
     int mcu_w = inter ? g->mx : g->ubw[c0];
     int mcu_h = inter ? g->my : g->ubh[c0];
@@ -514,7 +531,13 @@ static void encode_scan(enc_state* st, const geom_t* g, const int16_t* coef, con
                         size_t brow = (size_t)my * hv + by, bcol = (size_t)mxi * hv + bx;
                         const int16_t* blk = coef + (g->coff[c] + brow * g->bw[c] + bcol) * 64;
                         int slot = c == 0 ? 0 : 1;
-                        if (sc->Ss == 0) {
+                        if (sequential) {
+                            int v = blk[0], d = v - pred[c]; pred[c] = v;
+                            int a = d < 0 ? -d : d, s = bitlen(a);
+                            tk_sym(&e->tok, slot, s);
+                            tk_bits(&e->tok, (uint32_t)(d < 0 ? d - 1 : d), s);
+                            enc_ac_sequential(e, blk, 2 + slot);
+                        } else if (sc->Ss == 0) {
                             if (sc->Ah == 0) {
                                 int v = blk[0] >> sc->Al;      /* arithmetic shift: floor */
                                 int d = v - pred[c]; pred[c] = v;
@@ -533,16 +556,22 @@ static void encode_scan(enc_state* st, const geom_t* g, const int16_t* coef, con
     (void)total;
 
     /* statistics -> tables */
-    long freq[2][256]; memset(freq, 0, sizeof freq);
-    int used[2] = {0, 0};
+    long freq[4][256]; memset(freq, 0, sizeof freq);
+    int used[4] = {0, 0, 0, 0};
     for (size_t i = 0; i < e->tok.n; ++i) {
         uint32_t t = e->tok.t[i];
         if ((t >> 30) == TOK_SYM) { int slot = (t >> 8) & 3; ++freq[slot][t & 255]; used[slot] = 1; }
     }
-    hufftab tab[2];
+    hufftab tab[4];
     int is_dc = sc->Ss == 0;
-    for (int s = 0; s < 2; ++s)
-        if (used[s]) { huff_build(freq[s], &tab[s]); write_dht(out, is_dc ? 0 : 1, s, &tab[s]); }
+    /* progressive scans use slots 0, 1 of one table class; a sequential scan uses DC tables 0, 1
+     * (slots 0, 1) and AC tables 0, 1 (slots 2, 3) */
+    for (int s = 0; s < 4; ++s)
+        if (used[s]) {
+            huff_build(freq[s], &tab[s]);
+            if (sequential) write_dht(out, s >= 2 ? 1 : 0, s & 1, &tab[s]);
+            else write_dht(out, is_dc ? 0 : 1, s, &tab[s]);
+        }
     if (ri != st->cur_ri) {
         bb_put16(out, 0xFFDD); bb_put16(out, 4); bb_put16(out, ri);
         st->cur_ri = ri;
@@ -553,7 +582,7 @@ static void encode_scan(enc_state* st, const geom_t* g, const int16_t* coef, con
     for (int ci = 0; ci < sc->ncomp; ++ci) {
         int c = sc->comp[ci], slot = c == 0 ? 0 : 1;
         bb_put(out, c + 1);
-        bb_put(out, is_dc ? (slot << 4) : slot);
+        bb_put(out, sequential ? ((slot << 4) | slot) : (is_dc ? (slot << 4) : slot));
     }
     bb_put(out, sc->Ss); bb_put(out, sc->Se); bb_put(out, (sc->Ah << 4) | sc->Al);
     bitw w = {out, 0, 0};
@@ -585,7 +614,10 @@ static void encode_image(enc_state* st, const geom_t* g, const int16_t* coef, co
         const uint8_t* q = t ? qc : qy;
         for (int k = 0; k < 64; ++k) bb_put(out, q[ZZ[k]]);
     }
-    bb_put16(out, 0xFFC2); bb_put16(out, 17); bb_put(out, 8);
+    int ns0;
+    const scan_spec* script0 = cur_script(&ns0);
+    int baseline = ns0 == 1 && script0[0].Ss == 0 && script0[0].Se == 63;
+    bb_put16(out, baseline ? 0xFFC0 : 0xFFC2); bb_put16(out, 17); bb_put(out, 8);
     bb_put16(out, g->H); bb_put16(out, g->W); bb_put(out, 3);
     bb_put(out, 1); bb_put(out, 0x22); bb_put(out, 0);
     bb_put(out, 2); bb_put(out, 0x11); bb_put(out, 1);

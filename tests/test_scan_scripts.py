@@ -85,3 +85,43 @@ def test_gpu_other_scripts_every_k(name, restart_rows):
             assert torch.equal(dec.image(out, i), dec.image(full, i)), (name, i)
     finally:
         dec.close()
+
+
+# ---- baseline (sequential) JPEG records: the paper's Table 2 compares progressive decoding with it
+def _baseline(config, n, **kw):
+    with pcr_synth.scan_script(pcr_synth.SCRIPT_BASELINE):
+        return pcr_synth.make_record(config, n_images=n, **kw)
+
+
+@pytest.mark.parametrize("config,restart_rows", [(0, True), (2, True), (2, False), (3, False)])
+def test_oracle_on_baseline_records_matches_ground_truth(config, restart_rows):
+    rec = _baseline(config, 3, restart_rows=restart_rows)
+    n, G = O.record_info(rec.bytes)
+    assert G == 1
+    for i in range(n):
+        got, _ = O.decode_image(rec.bytes, i, 1)
+        assert np.array_equal(got, rec.truth(i))
+
+
+def test_baseline_files_cross_checked_with_pillow():
+    """Pillow decodes this generator's baseline files and the oracle decodes Pillow's: luminance
+    planes within one level both ways (chroma upsampling differs by design, luminance does not)."""
+    PIL = pytest.importorskip("PIL.Image")
+    import io
+    from helpers import pillow_y
+    rec = _baseline(2, 2)
+    for i in range(2):
+        jpg = rec.jpeg(i)
+        assert not PIL.open(io.BytesIO(jpg)).info.get("progressive")
+        W, H = rec.dims[i]
+        _, _, (Y, _, _) = O.jpeg_decode(jpg, want_planes=True)
+        assert np.abs(pillow_y(jpg).astype(int) - Y[:H, :W].astype(int)).max() <= 1
+    rng = np.random.default_rng(3)
+    img = np.clip(np.cumsum(rng.normal(0, 4, (70, 90, 3)), axis=1) + 128, 0, 255).astype(np.uint8)
+    for opt, rst in ((True, 0), (False, 0), (True, 1)):
+        buf = io.BytesIO()
+        kw = {"restart_marker_rows": rst} if rst else {}
+        PIL.fromarray(img).save(buf, "JPEG", quality=90, subsampling=2, progressive=False, optimize=opt, **kw)
+        jpg = buf.getvalue()
+        _, _, (Y, _, _) = O.jpeg_decode(jpg, want_planes=True)
+        assert np.abs(pillow_y(jpg).astype(int) - Y[:70, :90].astype(int)).max() <= 1
