@@ -22,8 +22,10 @@
  *   g = 1 from SOI (tables, frame header), for every g the scan's DHT/DRI/SOS segments and
  *   entropy-coded bytes.  The file's EOI is not stored.  One scan per group.
  *
- * Supported streams: 8-bit, three components, 4:2:0 (2x2, 1x1, 1x1), progressive Huffman
- * (SOF2), any scan script that is the same for all images of a record, any restart interval.
+ * Supported streams: 8-bit, three components, 4:2:0 (2x2, 1x1, 1x1), Huffman coded; progressive
+ * (SOF2) with any scan script that is the same for all images of a record, or baseline
+ * sequential (SOF0, one interleaved scan = one scan group: the conventional JPEG that the paper's
+ * Table 2 compares against); any restart interval.
  *
  * All functions return an int status: PCR_OK (0) or a negative PCR_E_* code.  Nothing here
  * throws, aborts or prints.  Unless said otherwise pointers are HOST pointers.

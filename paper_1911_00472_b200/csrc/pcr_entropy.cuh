@@ -634,4 +634,114 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
     if (bad) atomicMin(&P.status[img], kErrCorrupt);
 }
 
+// ---------------------------------------------------------------------------------------
+// Sequential (baseline) scans: one interleaved scan carries, block after block, the DC difference
+// and then the AC coefficients up to an end-of-block symbol.  Same decomposition as above (one
+// lane per restart interval, one Huffman symbol per step), four tables per warp (DC and AC,
+// luminance and chrominance).  Coefficients go where the progressive first passes put them:
+// zigzag positions 0..7 into the dense head plane, the rest into the block's line.
+// ---------------------------------------------------------------------------------------
+constexpr int kSeqWarps = 2;
+
+template <bool kRoi>
+__global__ void __launch_bounds__(32 * kSeqWarps) sequential_kernel(Params P, uint32_t item_begin, uint32_t item_count) {
+    __shared__ HuffTab tabs[kSeqWarps][4];                    // DC 0, DC 1, AC 0, AC 1
+    __shared__ uint32_t s_ring[kSeqWarps][kRingWords][32];
+    const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t it = blockIdx.x * kSeqWarps + wid;
+    if (it >= item_count) return;                             // whole warp
+    const Item item = P.items[item_begin + it];
+    const ScanDesc sd = P.scans[item.si];
+    const int img = (int)(item.si % (uint32_t)P.N);
+    bool done = (uint32_t)lane >= item.count;
+    uint32_t seg = item.seg0 + lane;
+    if (seg >= sd.nseg) { done = true; seg = 0; }
+    const ImgDesc im = P.imgs[img];
+    const Geometry g = make_geometry(im);
+    const uint32_t mcu_w = g.mx, total = g.mx * g.my;
+    const uint32_t m0 = sd.ri ? seg * sd.ri : 0;
+    const uint32_t m1 = sd.ri ? min(m0 + sd.ri, total) : total;
+    const unsigned full = 0xffffffffu;
+    if (kRoi) {
+        if (!done && m1 > m0) {
+            const CropRect rc = P.roi[img];
+            const uint32_t lo = 16u * (rc.y0 >> 4), hi = 16u * ((rc.y0 + rc.h + 15u) >> 4);
+            const uint32_t r0 = m0 / mcu_w, r1 = (m1 - 1u) / mcu_w;
+            if ((r1 + 1u) * 16u <= lo || r0 * 16u >= hi) done = true;
+        }
+        if (__all_sync(full, done)) return;
+    }
+    build_hufftab(tabs[wid][0], P.rec + sd.tab_off[0], lane);
+    if (sd.tab_off[1]) build_hufftab(tabs[wid][1], P.rec + sd.tab_off[1], lane);
+    build_hufftab(tabs[wid][2], P.rec + sd.tab_ac[0], lane);
+    if (sd.tab_ac[1]) build_hufftab(tabs[wid][3], P.rec + sd.tab_ac[1], lane);
+    const uint32_t* segtab = P.seg_start + sd.seg_base;
+    uint32_t bstart = segtab[seg];
+    uint32_t bend = segtab[seg + 1] - 2;
+    bool bad = false;
+    if (!done && (bstart < sd.data_off || bend > sd.data_end || bend < bstart)) { bad = true; done = true; }
+    if (done) { bstart = sd.data_off; bend = sd.data_off; }
+    BitReader br;
+    br.init(&s_ring[wid][0][lane], P.ubuf, bstart, bend);
+    br.topup(!done);
+    br.prime();
+
+    uint32_t m = m0, mrow = m0 / mcu_w, mcol = m0 % mcu_w;
+    int j = 0;                                            // block inside the MCU: Y00 Y01 Y10 Y11 Cb Cr
+    int k = 0;                                            // 0: the block's DC symbol comes next
+    int pred0 = 0, pred1 = 0, pred2 = 0;
+    if (m >= m1) done = true;
+    for (;;) {
+        br.topup(!done);
+        __syncwarp(full);
+        if (__all_sync(full, done)) break;
+#pragma unroll 1
+        for (int t = 0; t < kDecodeSteps; ++t) {
+            if (done || !br.ready()) continue;
+            br.refill();
+            const uint32_t win = br.top32();
+            const int c = j < 4 ? 0 : j - 3;
+            uint64_t blk;
+            if (c == 0) blk = g.coff[0] + (uint64_t)(2 * mrow + (j >> 1)) * g.bw[0] + 2 * mcol + (j & 1);
+            else blk = (c == 1 ? g.coff[1] : g.coff[2]) + (uint64_t)mrow * g.mx + mcol;
+            const bool is_dc = k == 0;
+            const int ti = is_dc ? (int)((sd.slots >> (2 * c)) & 1u) : 2 + (int)((sd.slots_ac >> (2 * c)) & 1u);
+            const HuffTab& tab = tabs[wid][ti];
+            uint32_t e = tab.lut[win >> (32 - kLutBits)];
+            if (e == 0) e = huff_lookup(tab, win);
+            const int len = (int)(e >> 8), r = is_dc ? 0 : (int)(e >> 4) & 15, sz = is_dc ? (int)(e & 255u) : (int)(e & 15u);
+            const bool is_coef = sz != 0, is_zrl = !is_dc && sz == 0 && r == 15, is_eob = !is_dc && sz == 0 && r == 0;
+            const int kk = k + r;
+            const bool fail = e == 0 || sz > 15 || (!is_dc && !is_coef && !is_zrl && !is_eob) || (is_coef && kk > 63);
+            if (fail) { bad = true; done = true; continue; }
+            const int extra = is_coef ? sz : 0;
+            const int v = extend_bits(top_bits(win << len, extra), extra);
+            br.skip(len + extra);
+            if (is_dc) {
+                const int pv = (c == 0 ? pred0 : (c == 1 ? pred1 : pred2)) + v;
+                if (c == 0) pred0 = pv; else if (c == 1) pred1 = pv; else pred2 = pv;
+                P.head[blk * 8] = (int16_t)pv;
+                k = 1;
+            } else if (is_coef) {
+                if (kk < 8) P.head[blk * 8 + kk] = (int16_t)v;
+                else P.planes[blk * 64 + kk] = (int16_t)v;
+                k = kk + 1;
+            } else if (is_zrl) {
+                k += 16;
+            }
+            if (is_eob || k > 63) {                       // block finished
+                k = 0;
+                if (++j == 6) {
+                    j = 0; ++m;
+                    if (++mcol == mcu_w) { mcol = 0; ++mrow; }
+                }
+            }
+            if (br.overran()) { bad = true; done = true; }
+            if (m >= m1) done = true;
+        }
+        __syncwarp(full);
+    }
+    if (bad) atomicMin(&P.status[img], kErrCorrupt);
+}
+
 }  // namespace pcr

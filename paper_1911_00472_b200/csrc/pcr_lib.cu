@@ -227,11 +227,13 @@ struct ImageParse {
     TableRef dc[4], ac[4];
     uint32_t ri = 0;
     bool have_frame = false;
+    bool sequential = false;      // SOF0: one interleaved scan carries whole blocks
 };
 
 struct ScanParse {
     ScanScript sc;
     uint32_t tab[3];       // table body offset per scan component (0 when the scan uses none)
+    uint32_t tab_ac[3];    // sequential scans: the AC table per component (tab then holds the DC tables)
     uint32_t data_off, data_end, ri;
 };
 
@@ -278,8 +280,9 @@ int parse_chunk(const uint8_t* rec, uint64_t off, uint32_t len, bool first, Imag
                 }
                 im.qdef[tq] = true;
             }
-        } else if (mk == 0xC2) {
+        } else if (mk == 0xC2 || mk == 0xC0) {            // progressive / baseline sequential, Huffman
             if (im.have_frame || sl < 15 || s[0] != 8 || s[5] != 3) return PCR_E_FORMAT;
+            im.sequential = mk == 0xC0;
             im.H = ((uint32_t)s[1] << 8) | s[2];
             im.W = ((uint32_t)s[3] << 8) | s[4];
             for (int c = 0; c < 3; ++c) {
@@ -325,11 +328,17 @@ int parse_chunk(const uint8_t* rec, uint64_t off, uint32_t len, bool first, Imag
             sc.Ss = s[1 + 2 * ns]; sc.Se = s[2 + 2 * ns];
             sc.Ah = s[3 + 2 * ns] >> 4; sc.Al = s[3 + 2 * ns] & 15;
             if (sc.Ss > sc.Se || sc.Se > 63 || sc.Al > 13) return PCR_E_FORMAT;
-            if (sc.Ss == 0 && sc.Se != 0) return PCR_E_FORMAT;
+            if (im.sequential) {
+                if (sc.Ss != 0 || sc.Se != 63 || sc.Ah != 0 || sc.Al != 0 || ns != 3) return PCR_E_FORMAT;
+            } else if (sc.Ss == 0 && sc.Se != 0) return PCR_E_FORMAT;
             if (sc.Ss > 0 && ns != 1) return PCR_E_FORMAT;
             if (ns > 1 && ns != 3) return PCR_E_FORMAT;     // interleaved scans hold all three components
             if (sc.Ah != 0 && sc.Ah != sc.Al + 1) return PCR_E_FORMAT;
-            for (int i = 0; i < 3; ++i) out.tab[i] = 0;
+            for (int i = 0; i < 3; ++i) out.tab[i] = out.tab_ac[i] = 0;
+            for (int i = 0; i < ns && im.sequential; ++i) {
+                out.tab_ac[i] = im.ac[ta[i]].off;
+                if (!out.tab_ac[i]) return PCR_E_FORMAT;
+            }
             for (int i = 0; i < ns; ++i) {
                 if (sc.Ss == 0 && sc.Ah == 0) { out.tab[i] = im.dc[td[i]].off; if (!out.tab[i]) return PCR_E_FORMAT; }
                 if (sc.Ss > 0) { out.tab[i] = im.ac[ta[i]].off; if (!out.tab[i]) return PCR_E_FORMAT; }
@@ -443,6 +452,13 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
             ScanDesc& sd = scans[(size_t)g * N + i];
             sd.data_off = sp.data_off; sd.data_end = sp.data_end; sd.ri = sp.ri;
             // up to two distinct tables per scan
+            sd.tab_ac[0] = sp.tab_ac[0]; sd.tab_ac[1] = 0; sd.slots_ac = 0;
+            for (int ci = 1; ci < sp.sc.ncomp && sp.tab_ac[0]; ++ci) {
+                if (sp.tab_ac[ci] == sd.tab_ac[0]) continue;
+                if (sd.tab_ac[1] == 0) sd.tab_ac[1] = sp.tab_ac[ci];
+                if (sp.tab_ac[ci] != sd.tab_ac[1]) return PCR_E_FORMAT;
+                sd.slots_ac |= 1u << (2 * ci);
+            }
             sd.tab_off[0] = sp.tab[0]; sd.tab_off[1] = 0; sd.slots = 0;
             for (int ci = 1; ci < sp.sc.ncomp; ++ci) {
                 if (sp.tab[ci] == sd.tab_off[0]) continue;
@@ -786,7 +802,7 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
     }
     bool dc_only = true, head_only = true;      // no AC scan at all / no scan beyond zigzag position 7
     for (int s = 0; s < k; ++s) {
-        if (rec->script[s].Ss > 0) dc_only = false;
+        if (rec->script[s].Ss > 0 || rec->script[s].Se > 0) dc_only = false;
         if (rec->script[s].Se > 7) head_only = false;
     }
     rec->dc_merged = false;
@@ -854,6 +870,13 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
                 count += rec->item_count[(size_t)g * G + s];
             }
             if (!count) return true;
+            const ScanScript& first = rec->script[rec->wave_scans[w][0]];
+            if (first.Ss == 0 && first.Se == 63) {        // a baseline record: its one scan is sequential
+                if (targs) sequential_kernel<true><<<(count + kSeqWarps - 1) / kSeqWarps, 32 * kSeqWarps, 0, q>>>(P, begin, count);
+                else sequential_kernel<false><<<(count + kSeqWarps - 1) / kSeqWarps, 32 * kSeqWarps, 0, q>>>(P, begin, count);
+                ++g_launches;
+                return true;
+            }
             if (targs) entropy_kernel<true><<<(count + kEntropyWarps - 1) / kEntropyWarps, 32 * kEntropyWarps, 0, q>>>(P, begin, count);
             else entropy_kernel<false><<<(count + kEntropyWarps - 1) / kEntropyWarps, 32 * kEntropyWarps, 0, q>>>(P, begin, count);
             ++g_launches;

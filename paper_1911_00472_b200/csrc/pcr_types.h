@@ -44,6 +44,8 @@ struct ScanDesc {
     uint32_t ri;          // restart interval in MCUs (0 = none)
     uint32_t tab_off[2];  // offsets of up to two DHT table bodies (16 counts, then values)
     uint32_t slots;       // 2 bits per scan component: which of tab_off it uses
+    uint32_t tab_ac[2];   // sequential scans only: up to two AC table bodies (tab_off then holds the DC tables)
+    uint32_t slots_ac;    // 2 bits per scan component: which of tab_ac it uses
 };
 
 struct ImgDesc {

@@ -125,3 +125,39 @@ def test_baseline_files_cross_checked_with_pillow():
         jpg = buf.getvalue()
         _, _, (Y, _, _) = O.jpeg_decode(jpg, want_planes=True)
         assert np.abs(pillow_y(jpg).astype(int) - Y[:70, :90].astype(int)).max() <= 1
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("config,n,restart_rows", [(0, 32, True), (1, 6, True), (2, 5, True), (2, 5, False), (3, 2, False)])
+def test_gpu_baseline_records(config, n, restart_rows):
+    """A record of baseline JPEGs (one scan group): coefficients and pixels bit-equal to the oracle,
+    and the training-tensor path on top of it."""
+    import torch
+    from paper_1911_00472_b200 import Decoder, pcr_image_blocks
+    rec = _baseline(config, n, restart_rows=restart_rows)
+    dec = Decoder(rec.bytes)
+    try:
+        assert dec.n_groups == 1
+        out = dec.decode(1)
+        torch.cuda.synchronize()
+        assert dec.status() == (-1, 0)
+        coef = dec.coeffs().cpu().numpy()
+        out_h = out.cpu().numpy()
+        for i in range(rec.n_images):
+            want_c, want_rgb = O.decode_image(rec.bytes, i, 1)
+            a, b = pcr_image_blocks(dec.handle, i)
+            assert np.array_equal(coef[a:a + b], want_c), (config, i)
+            inf = dec.info[i]
+            got = out_h[inf.out_offset:inf.out_offset + inf.out_bytes].reshape(inf.height, inf.width, 3)
+            assert np.array_equal(got, want_rgb), (config, i)
+        crops = pcr_synth.random_resized_crops([(int(w), int(h)) for w, h in rec.dims], 31)
+        mean, std = (0.485, 0.456, 0.406), (0.229, 0.224, 0.225)
+        t = dec.decode_tensor(1, crops, 24, mean, std)
+        torch.cuda.synchronize()
+        got_t = t.cpu().numpy().astype(np.float64)
+        for i in range(0, rec.n_images, 3):
+            _, rgb = O.decode_image(rec.bytes, i, 1)
+            want = O.training_tensor(rgb, crops[i], 24, mean, std).astype(np.float64)
+            assert np.abs(got_t[i] - want).max() <= 2.0 ** -9, (config, i)
+    finally:
+        dec.close()
