@@ -125,12 +125,12 @@ int pcr_decode_more(pcr_record* rec, int k, void* out, void* stream);
  *   fx = clamp((u + 0.5) * w / size - 0.5, 0, w - 1), fy likewise with h (half-pixel centres,
  *   the crop's edge pixels repeated, no low-pass filter); v = bilinear interpolation of the four
  *   pixels around (x0 + fx, y0 + fy); tensor[i][c][oy][ox] = (v_c / 255 - mean[c]) / std[c],
- *   evaluated in single precision, stored as dtype (half: round to nearest even).
+ *   evaluated in single precision, stored as dtype (half, bfloat16: round to nearest even).
  *   crops  : HOST array of pcr_num_images entries (read before the call returns); every
  *            rectangle must lie inside its image, w, h >= 1, flip 0 or 1 (else PCR_E_ARG; also
  *            when an image has 2 GiB of pixels or more).
  *            The random draws of an augmentation policy are the caller's.
- *   size   : 1..4096.   mean, std : HOST, three floats each, std > 0.   dtype : PCR_F16 / PCR_F32.
+ *   size   : 1..4096.   mean, std : HOST, three floats each, std > 0.   dtype : PCR_F16 / PCR_F32 / PCR_BF16.
  *   rgb    : DEVICE scratch as pcr_decode's `out` (same size and alignment); afterwards it holds
  *            the decoded pixels of the transformed MCUs, other bytes are left as they were.
  *   tensor : DEVICE, pcr_num_images * 3 * size * size elements of dtype, image i at index i.
@@ -142,6 +142,7 @@ int pcr_decode_more(pcr_record* rec, int k, void* out, void* stream);
  * a small device array for the rectangles. */
 #define PCR_F16 0
 #define PCR_F32 1
+#define PCR_BF16 2
 typedef struct {
     uint32_t x0, y0, w, h; /* crop rectangle in pixels of the decoded image */
     uint32_t flip;         /* 1: mirror the columns                         */

@@ -134,7 +134,7 @@ def pcr_decode_more(handle: int, k: int, out_dev_ptr: int, stream: int = 0) -> N
     _chk(lib().pcr_decode_more(handle, k, out_dev_ptr, stream), "pcr_decode_more")
 
 
-PCR_F16, PCR_F32 = 0, 1
+PCR_F16, PCR_F32, PCR_BF16 = 0, 1, 2
 
 
 def pcr_decode_tensor(handle: int, k: int, crops_host_ptr: int, size: int, mean_host_ptr: int, std_host_ptr: int,

@@ -906,7 +906,8 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
             ++g_launches;
             if (targs && i1 > i0) {
                 const dim3 tg((unsigned)((targs->size + kTensorRows - 1) / kTensorRows), i1 - i0);
-                if (targs->f32) tensor_kernel<float><<<tg, 256, 0, q>>>(P, *targs, static_cast<const uint8_t*>(out), i0);
+                if (targs->f32 == 2) tensor_kernel<__nv_bfloat16><<<tg, 256, 0, q>>>(P, *targs, static_cast<const uint8_t*>(out), i0);
+                else if (targs->f32) tensor_kernel<float><<<tg, 256, 0, q>>>(P, *targs, static_cast<const uint8_t*>(out), i0);
                 else tensor_kernel<__half><<<tg, 256, 0, q>>>(P, *targs, static_cast<const uint8_t*>(out), i0);
                 ++g_launches;
             }
@@ -1030,7 +1031,7 @@ int pcr_decode_more(pcr_record* rec, int k, void* out, void* stream) {
 int pcr_decode_tensor(pcr_record* rec, int k, const pcr_crop* crops, int size, const float* mean, const float* std_,
                       int dtype, void* rgb, void* tensor, void* stream) {
     if (!rec || !crops || !mean || !std_ || !rgb || !tensor || k < 1 || k > rec->G) return PCR_E_ARG;
-    if (size < 1 || size > 4096 || (dtype != PCR_F16 && dtype != PCR_F32)) return PCR_E_ARG;
+    if (size < 1 || size > 4096 || (dtype != PCR_F16 && dtype != PCR_F32 && dtype != PCR_BF16)) return PCR_E_ARG;
     if (reinterpret_cast<uintptr_t>(rgb) & 15u) return PCR_E_ARG;
     if (reinterpret_cast<uintptr_t>(tensor) & (dtype == PCR_F32 ? 3u : 1u)) return PCR_E_ARG;
     static_assert(sizeof(pcr_crop) == sizeof(CropRect), "pcr_crop and CropRect have the same layout");
@@ -1048,7 +1049,7 @@ int pcr_decode_tensor(pcr_record* rec, int k, const pcr_crop* crops, int size, c
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (cudaMemcpyAsync(rec->d_crops, crops, (size_t)rec->N * sizeof(CropRect), cudaMemcpyHostToDevice, st) != cudaSuccess) return PCR_E_CUDA;
     TensorArgs T;
-    T.crops = rec->d_crops; T.out = tensor; T.size = size; T.f32 = dtype == PCR_F32 ? 1 : 0;
+    T.crops = rec->d_crops; T.out = tensor; T.size = size; T.f32 = dtype == PCR_F32 ? 1 : (dtype == PCR_BF16 ? 2 : 0);
     for (int c = 0; c < 3; ++c) { T.mean[c] = mean[c]; T.inv_std[c] = 1.0f / std_[c]; }
     const int rc = decode_range(rec, 0, k, rgb, stream, &T);
     rec->decoded_k = 0;          // rows outside the crops were not decoded: nothing to raise the fidelity of

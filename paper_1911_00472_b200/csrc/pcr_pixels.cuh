@@ -12,6 +12,7 @@
 //   R = clamp(Y + ((91881 cr + 32768) >> 16)), G = clamp(Y + ((-22553 cb - 46802 cr + 32768) >> 16)),
 //   B = clamp(Y + ((116130 cb + 32768) >> 16)) with cb, cr = sample - 128 of chroma (x>>1, y>>1).
 #pragma once
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -360,12 +361,13 @@ struct TensorArgs {
     const CropRect* crops;     // [N], by image index
     void* out;                 // [N][3][size][size]
     int32_t size;
-    int32_t f32;               // 0: half precision output, 1: single precision
+    int32_t f32;               // output type: 0 half precision, 1 single precision, 2 bfloat16
     float mean[3], inv_std[3];
 };
 
 __device__ __forceinline__ void tensor_store(float* p, float v) { *p = v; }
 __device__ __forceinline__ void tensor_store(__half* p, float v) { *p = __float2half_rn(v); }
+__device__ __forceinline__ void tensor_store(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
 
 // the three bytes at byte offset `off` of a 4-byte-aligned shared buffer, as floats: two aligned
 // words, a funnel shift, and per byte a permute into the mantissa of 2^23 (exact for 0..255)

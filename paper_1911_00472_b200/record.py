@@ -65,8 +65,9 @@ class Decoder:
         crops = np.ascontiguousarray(crops, dtype=np.uint32)
         if crops.shape != (self.n_images, 5):
             raise ValueError("crops must have shape (n_images, 5)")
-        if dtype not in (torch.float16, torch.float32):
-            raise ValueError("dtype must be torch.float16 or torch.float32")
+        codes = {torch.float16: B.PCR_F16, torch.float32: B.PCR_F32, torch.bfloat16: B.PCR_BF16}
+        if dtype not in codes:
+            raise ValueError("dtype must be torch.float16, torch.bfloat16 or torch.float32")
         m = np.ascontiguousarray(mean, dtype=np.float32)
         sd = np.ascontiguousarray(std, dtype=np.float32)
         if rgb is None:
@@ -78,7 +79,7 @@ class Decoder:
         s = stream if stream is not None else torch.cuda.current_stream(self.device)
         with torch.cuda.device(self.device):
             B.pcr_decode_tensor(self.handle, k, crops.ctypes.data, size, m.ctypes.data, sd.ctypes.data,
-                                B.PCR_F16 if dtype == torch.float16 else B.PCR_F32, rgb.data_ptr(), tensor.data_ptr(),
+                                codes[dtype], rgb.data_ptr(), tensor.data_ptr(),
                                 s.cuda_stream)
         return tensor
 

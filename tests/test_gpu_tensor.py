@@ -17,6 +17,7 @@ pytestmark = pytest.mark.gpu
 MEAN = (0.485, 0.456, 0.406)
 STD = (0.229, 0.224, 0.225)
 HALF_ULP_TOL = 2.0 ** -9
+BF16_ULP_TOL = 2.0 ** -6          # one unit in the last place of bfloat16 (8 significant bits) in [2, 4)
 SINGLE_TOL = 1e-5
 
 
@@ -30,11 +31,13 @@ def _check(rec, k, crops, size, images, dtype_name="float16"):
         torch.cuda.synchronize()
         assert dec.status() == (-1, 0)
         assert tuple(t.shape) == (rec.n_images, 3, size, size) and t.dtype == dtype
-        got = t.cpu().numpy().astype(np.float64)
-        tol = HALF_ULP_TOL if dtype_name == "float16" else SINGLE_TOL
+        got = t.float().cpu().numpy().astype(np.float64)       # exact widening of every output type
+        tol = {"float16": HALF_ULP_TOL, "bfloat16": BF16_ULP_TOL, "float32": SINGLE_TOL}[dtype_name]
         for i in images:
             _, rgb = O.decode_image(rec.bytes, i, k)
             want = O.training_tensor(rgb, crops[i], size, MEAN, STD, dtype=np.float16 if dtype_name == "float16" else np.float32)
+            if dtype_name == "bfloat16":       # numpy has no bfloat16: round the oracle's float32 result with torch on the CPU
+                want = torch.from_numpy(want).to(torch.bfloat16).float().numpy()
             err = np.abs(got[i] - want.astype(np.float64)).max()
             assert err <= tol, (i, k, crops[i], err)
     finally:
@@ -56,6 +59,7 @@ def test_full_image_identity_size(rec0):
     crops = np.array([[0, 0, w, h, i & 1] for i, (w, h) in enumerate(_dims(rec0))], dtype=np.uint32)
     _check(rec0, 10, crops, 32, range(rec0.n_images), "float32")
     _check(rec0, 10, crops, 32, range(rec0.n_images), "float16")
+    _check(rec0, 10, crops, 32, range(rec0.n_images), "bfloat16")
 
 
 def test_imagenet_shaped_224_and_160(rec1_small):
