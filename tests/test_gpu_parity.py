@@ -211,3 +211,13 @@ def test_widths_multiple_of_16_odd_heights_dc_only_path():
         coeffs.append(c)
     rec = pcr_synth.record_from_coeffs(dims, coeffs)
     _compare(rec, (1, 2, 7, 10))
+
+
+@pytest.mark.parametrize("slices", ["2", "3"])
+def test_sliced_pipelines_on_small_records(monkeypatch, slices, rec1_small, rec2_small):
+    """The multi-slice path (image slices on their own streams in width-sorted order, index of the
+    later waves on the side stream) on records small enough to compare every image: the slice
+    count is read when a record is opened."""
+    monkeypatch.setenv("PCR_SLICES", slices)
+    _compare(rec1_small, (1, 2, 5, 6, 7, 9, 10))
+    _compare(rec2_small, range(1, G + 1))
