@@ -69,6 +69,11 @@ typedef struct {
  *           BORROWED: it must stay valid and unchanged until pcr_close.
  *   len   : its length in bytes (< 4 GiB).
  *   rec   : receives the handle; NULL on failure.
+ * The device tables are filled on an internal stream and the call does not wait for them: every
+ * decode of the record waits (on the device) for that set-up first.  Different records may be
+ * opened and used from different host threads at the same time (a loader parses the next record
+ * while the current one decodes); one record belongs to one thread at a time.  Device buffers of
+ * closed records are kept for later opens (pcr_release_cached_memory returns them).
  * Errors: PCR_E_ARG, PCR_E_FORMAT, PCR_E_NOMEM, PCR_E_CUDA. */
 int pcr_open(const void* bytes, size_t len, pcr_record** rec);
 
