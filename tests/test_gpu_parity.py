@@ -221,3 +221,37 @@ def test_sliced_pipelines_on_small_records(monkeypatch, slices, rec1_small, rec2
     monkeypatch.setenv("PCR_SLICES", slices)
     _compare(rec1_small, (1, 2, 5, 6, 7, 9, 10))
     _compare(rec2_small, range(1, G + 1))
+
+
+def test_two_records_in_flight_on_two_streams(monkeypatch, rec1_small, rec2_small):
+    """A loader keeps two records in flight (the paper's double buffering): both decodes are enqueued
+    on their own streams before either is waited for, each opened from its own host thread."""
+    import threading
+    import torch
+    from paper_1911_00472_b200 import Decoder
+    monkeypatch.setenv("PCR_SLICES", "2")
+    decs = [None, None]
+
+    def opener(j, rec):
+        torch.cuda.set_device(0)
+        decs[j] = Decoder(rec.bytes)
+
+    ths = [threading.Thread(target=opener, args=(j, r)) for j, r in enumerate((rec1_small, rec2_small))]
+    for t in ths:
+        t.start()
+    for t in ths:
+        t.join()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    try:
+        for k in (5, 10):
+            outs = [d.decode(k, d.alloc_out(), stream=s) for d, s in zip(decs, streams)]
+            torch.cuda.synchronize()
+            for d, rec, out in zip(decs, (rec1_small, rec2_small), outs):
+                assert d.status() == (-1, 0)
+                for i in range(0, rec.n_images, 2):
+                    _, want = O.decode_image(rec.bytes, i, k)
+                    assert np.array_equal(d.image(out, i).cpu().numpy(), want), (k, i)
+    finally:
+        for d in decs:
+            if d is not None:
+                d.close()
