@@ -486,6 +486,7 @@ def main():
                               "note": "pcr_open + pcr_decode from pinned host bytes + synchronise + pcr_status + pcr_close per step"}
 
     per_k, raise_ms, training_tensor, fidelity, baseline_jpeg = {}, {}, None, None, None
+    hbm_by_k = {}
     if not args.headline_only:
         # per-k numbers and the stage profile (this rank's GPU)
         per_k = {}
@@ -495,6 +496,7 @@ def main():
             torch.cuda.synchronize(dev)
             st = 5
             per_k[str(kk)] = n_img * st / (timed_steps(kk, st) / 1000.0)
+            hbm_by_k[str(kk)] = algorithmic_bytes(scans, infos, kk)["total"] * per_k[str(kk)] / n_img / 1e9
         # decode straight to a fixed-size training batch (random-resized crops, flip, 224 x 224, fp16)
         crops = pcr_synth.random_resized_crops(infos, 1000 + rank)
         t_size = 224
@@ -641,7 +643,12 @@ def main():
                        "record_bytes": int(rec.bytes.size), "prefix_bytes_at_k": int(prefix),
                        "mean_compressed_bytes_per_image_by_scan": [c / n_img for c in comp]},
             "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
-            "cpu_baseline": cpu_baseline, "images_per_s_by_k": per_k, "raise_fidelity_ms_per_record": raise_ms,
+            "cpu_baseline": cpu_baseline, "images_per_s_by_k": per_k, "hbm_gbs_by_k": hbm_by_k,
+            "hbm_frac_of_peak_by_k": {kk: v / peak for kk, v in hbm_by_k.items()},
+            "hbm_by_k_note": "algorithmic bytes of the decode at k (compressed prefix, zeroed and written coefficient planes, "
+                             "planes read by the pixel stage, pixels written) / time; below k = 5 the implementation moves fewer "
+                             "bytes than this model (positions 0..7 of every block live in a dense plane, the 128-byte lines are "
+                             "neither zeroed nor read while no scan reaches position 8)", "raise_fidelity_ms_per_record": raise_ms,
             "training_tensor": training_tensor, "predicted_io_speedup_by_k": io_speedup, "fidelity": fidelity, "baseline_jpeg": baseline_jpeg,
         }))
     dec.close()
