@@ -161,3 +161,33 @@ def test_gpu_baseline_records(config, n, restart_rows):
             assert np.abs(got_t[i] - want).max() <= 2.0 ** -9, (config, i)
     finally:
         dec.close()
+
+
+@pytest.mark.gpu
+def test_gpu_baseline_record_with_damaged_bytes_is_flagged():
+    """Damaged entropy-coded bytes in a baseline record: the decode completes, the image is flagged,
+    its neighbours are untouched."""
+    import torch
+    from paper_1911_00472_b200 import Decoder
+    rec = _baseline(0, 32)
+    ref = Decoder(rec.bytes)
+    good = ref.decode(1).clone()
+    torch.cuda.synchronize()
+    b = rec.bytes.copy()
+    N = rec.n_images
+    index_off = int(np.frombuffer(b[32:40].tobytes(), dtype="<u8")[0])
+    ent = index_off + 8 * 2 + 16 * (0 * N + 5)                 # chunk (group 1, image 5)
+    off = int(np.frombuffer(b[ent:ent + 8].tobytes(), dtype="<u8")[0])
+    ln = int(np.frombuffer(b[ent + 8:ent + 12].tobytes(), dtype="<u4")[0])
+    b[off + ln - 40:off + ln] = 0                              # wipes the last restart marker and the data around it
+    dec = Decoder(b)
+    try:
+        out = dec.decode(1)
+        torch.cuda.synchronize()
+        bad, code = dec.status()
+        assert bad == 5 and code == -3
+        for i in (4, 6):
+            inf = dec.info[i]
+            assert torch.equal(out[inf.out_offset:inf.out_offset + inf.out_bytes], good[inf.out_offset:inf.out_offset + inf.out_bytes])
+    finally:
+        dec.close(); ref.close()
