@@ -320,3 +320,38 @@ def msssim(rgb_a: np.ndarray, rgb_b: np.ndarray) -> float:
             x = x[:2 * h2, :2 * w2].reshape(h2, 2, w2, 2).mean(axis=(1, 3))
             y = y[:2 * h2, :2 * w2].reshape(h2, 2, w2, 2).mean(axis=(1, 3))
     return float(result)
+
+
+# --------------------------------------------------------------------------------------
+# Triangle ("linear") chroma upsampling, the filter stock decoders apply by default to 4:2:0
+# data; the paper's decoders were stock ones (Section 5) and it does not name the filter.
+# Reading taken: every pixel mixes its own chroma sample with the horizontally nearer, the
+# vertically nearer and the diagonal neighbour with weights 9, 3, 3, 1 (sum 16, +8 and a shift:
+# round half up); neighbours come from the decoded MCU-padded chroma planes, beyond their border
+# the edge sample repeats.  Then the same colour conversion as with replication.
+# --------------------------------------------------------------------------------------
+def rgb_from_planes(Y: np.ndarray, Cb: np.ndarray, Cr: np.ndarray, W: int, H: int, triangle: bool) -> np.ndarray:
+    """Padded sample planes (Y: 16my x 16mx, Cb/Cr: 8my x 8mx, uint8) -> (H, W, 3) uint8."""
+    ch, cw = Cb.shape
+    ys, xs = np.arange(H), np.arange(W)
+    cy, cx = ys >> 1, xs >> 1
+    if not triangle:
+        cb, cr = Cb[cy][:, cx], Cr[cy][:, cx]
+    else:
+        ny = np.clip(cy + np.where(ys & 1, 1, -1), 0, ch - 1)
+        nx = np.clip(cx + np.where(xs & 1, 1, -1), 0, cw - 1)
+
+        def mix(P):
+            P = P.astype(np.int64)
+            return (9 * P[cy][:, cx] + 3 * P[cy][:, nx] + 3 * P[ny][:, cx] + P[ny][:, nx] + 8) >> 4
+        cb, cr = mix(Cb), mix(Cr)
+    ycc = np.stack([Y[:H, :W].astype(np.uint8), cb.astype(np.uint8), cr.astype(np.uint8)], axis=-1)
+    return ycc_to_rgb_array(ycc.reshape(-1, 3)).reshape(H, W, 3)
+
+
+def decode_image_upsampled(rec, i, k, triangle: bool):
+    """Image i of a record at fidelity k with the chosen chroma upsampling: (coefficients, RGB)."""
+    jpg = reassemble(rec, i, k)
+    coef, _, (Y, Cb, Cr) = jpeg_decode(jpg, want_planes=True)
+    W, H = image_info(rec, i)[:2]
+    return coef, rgb_from_planes(Y, Cb, Cr, W, H, triangle)
