@@ -175,6 +175,20 @@ int pcr_decode_tensor(pcr_record* rec, int k, const pcr_crop* crops, int size, c
 size_t pcr_msssim_scratch_bytes(pcr_record* rec);
 int pcr_msssim(pcr_record* rec, const void* rgb_a, const void* rgb_b, void* scratch, float* dev_scores, void* stream);
 
+/* Chroma upsampling of the decodes that follow (pcr_decode, pcr_decode_more).  The paper hands
+ * its reassembled files to stock decoders (Section 5) and does not name the filter.
+ *   PCR_UPSAMPLE_REPLICATE (default): pixel (x, y) takes chroma sample (x >> 1, y >> 1).
+ *   PCR_UPSAMPLE_TRIANGLE: the filter stock decoders apply by default: every pixel mixes its own
+ *     sample with the horizontally nearer, the vertically nearer and the diagonal neighbour,
+ *     (9 a + 3 b + 3 c + d + 8) >> 4; neighbours come from the decoded MCU-padded chroma planes,
+ *     beyond their border the edge sample repeats.  Costs a second pass over the chroma blocks
+ *     (their samples go through device memory: the first call allocates 128 bytes per MCU).
+ * pcr_decode_tensor works with replication only (PCR_E_ARG otherwise).
+ * Errors: PCR_E_ARG, PCR_E_NOMEM. */
+#define PCR_UPSAMPLE_REPLICATE 0
+#define PCR_UPSAMPLE_TRIANGLE 1
+int pcr_set_upsampling(pcr_record* rec, int mode);
+
 /* Forget which record bytes are resident on the device: the next pcr_decode copies its whole
  * prefix again (what a loader that streams each record once from host memory pays). */
 int pcr_evict(pcr_record* rec);

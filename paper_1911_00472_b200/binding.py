@@ -17,7 +17,7 @@ PCR_E_ARG, PCR_E_FORMAT, PCR_E_CORRUPT, PCR_E_TIMEOUT, PCR_E_CUDA, PCR_E_NOMEM =
 EXPORTS = ("pcr_open", "pcr_num_images", "pcr_num_groups", "pcr_get_image", "pcr_out_bytes", "pcr_prefix_bytes",
            "pcr_decode", "pcr_evict", "pcr_status", "pcr_coeffs", "pcr_image_blocks", "pcr_launch_count",
            "pcr_strerror", "pcr_close", "pcr_get_scan", "pcr_set_profiling", "pcr_get_profile",
-           "pcr_pixels_noalloc", "pcr_decode_more", "pcr_release_cached_memory", "pcr_decode_tensor", "pcr_msssim", "pcr_msssim_scratch_bytes")
+           "pcr_pixels_noalloc", "pcr_decode_more", "pcr_release_cached_memory", "pcr_decode_tensor", "pcr_msssim", "pcr_msssim_scratch_bytes", "pcr_set_upsampling")
 
 
 class ImageInfo(C.Structure):
@@ -65,6 +65,7 @@ def lib():
         L.pcr_msssim_scratch_bytes.restype = C.c_size_t
         L.pcr_msssim_scratch_bytes.argtypes = [vp]
         L.pcr_msssim.argtypes = [vp, vp, vp, vp, vp, vp]
+        L.pcr_set_upsampling.argtypes = [vp, C.c_int]
         L.pcr_evict.argtypes = [vp]
         L.pcr_status.argtypes = [vp, C.POINTER(C.c_int), C.POINTER(C.c_int)]
         L.pcr_coeffs.argtypes = [vp, C.POINTER(vp), C.POINTER(C.c_size_t)]
@@ -150,6 +151,13 @@ def pcr_msssim_scratch_bytes(handle: int) -> int:
 def pcr_msssim(handle: int, rgb_a_dev_ptr: int, rgb_b_dev_ptr: int, scratch_dev_ptr: int, scores_dev_ptr: int,
                stream: int = 0) -> None:
     _chk(lib().pcr_msssim(handle, rgb_a_dev_ptr, rgb_b_dev_ptr, scratch_dev_ptr, scores_dev_ptr, stream), "pcr_msssim")
+
+
+PCR_UPSAMPLE_REPLICATE, PCR_UPSAMPLE_TRIANGLE = 0, 1
+
+
+def pcr_set_upsampling(handle: int, mode: int) -> None:
+    _chk(lib().pcr_set_upsampling(handle, mode), "pcr_set_upsampling")
 
 
 def pcr_evict(handle: int) -> None:

@@ -182,6 +182,8 @@ struct pcr_record {
     MsDesc* d_ms = nullptr;       // per-image table of pcr_msssim (built on first use)
     size_t ms_scratch = 0;        // bytes of scratch pcr_msssim needs
     uint64_t ms_floats = 0;       // floats of all pyramids (the sums follow them)
+    int upsampling = PCR_UPSAMPLE_REPLICATE;
+    uint8_t* d_chroma = nullptr;  // chroma sample planes between the two passes of triangle upsampling
     CropRect* d_crops = nullptr;  // crop rectangles of the last pcr_decode_tensor (allocated on first use)
     int* d_status = nullptr;
     std::vector<int> h_status;
@@ -785,6 +787,7 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
     P.imgs = rec->d_imgs; P.seg_start = rec->d_seg; P.items = rec->d_items; P.units = rec->d_units;
     P.qtab = rec->d_qtab; P.order = rec->d_order; P.status = rec->d_status; P.N = rec->N;
     P.roi = targs ? targs->crops : nullptr;
+    P.chroma = rec->d_chroma;
     FinalizeList fl;
     memset(&fl, 0, sizeof fl);
     bool any_refine = false;
@@ -888,7 +891,23 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
         if (nu) {
             const unsigned grid = nu;
             uint8_t* o8 = static_cast<uint8_t*>(out);
-            if (!targs) {
+            if (!targs && rec->upsampling == PCR_UPSAMPLE_TRIANGLE) {
+                // chroma pass (samples of every chroma block into the sample planes), then the pixel pass
+                if (head_only && any_refine) {
+                    pixel_kernel<true, 3, false, 1><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+                    pixel_kernel<true, 3, false, 2><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+                } else if (head_only) {
+                    pixel_kernel<false, 3, false, 1><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+                    pixel_kernel<false, 3, false, 2><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+                } else if (any_refine) {
+                    pixel_kernel<true, 1, false, 1><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+                    pixel_kernel<true, 1, false, 2><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+                } else {
+                    pixel_kernel<false, 1, false, 1><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+                    pixel_kernel<false, 1, false, 2><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+                }
+                ++g_launches;
+            } else if (!targs) {
                 if (dc_only && rec->widths_mult16) dc_pixel_kernel<false><<<grid, 128, 0, q>>>(Q, o8);
                 else if (dc_only) pixel_kernel<false, 2><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
                 else if (head_only && any_refine) pixel_kernel<true, 3><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
@@ -1031,6 +1050,7 @@ int pcr_decode_more(pcr_record* rec, int k, void* out, void* stream) {
 int pcr_decode_tensor(pcr_record* rec, int k, const pcr_crop* crops, int size, const float* mean, const float* std_,
                       int dtype, void* rgb, void* tensor, void* stream) {
     if (!rec || !crops || !mean || !std_ || !rgb || !tensor || k < 1 || k > rec->G) return PCR_E_ARG;
+    if (rec->upsampling != PCR_UPSAMPLE_REPLICATE) return PCR_E_ARG;      // the tensor path resamples replicated chroma only
     if (size < 1 || size > 4096 || (dtype != PCR_F16 && dtype != PCR_F32 && dtype != PCR_BF16)) return PCR_E_ARG;
     if (reinterpret_cast<uintptr_t>(rgb) & 15u) return PCR_E_ARG;
     if (reinterpret_cast<uintptr_t>(tensor) & (dtype == PCR_F32 ? 3u : 1u)) return PCR_E_ARG;
@@ -1117,6 +1137,15 @@ int pcr_msssim(pcr_record* rec, const void* rgb_a, const void* rgb_b, void* scra
     ms_final_kernel<<<(N + 255) / 256, 256, 0, st>>>(rec->d_ms, sums, dev_scores, (int)N);
     ++g_launches;
     if (cudaGetLastError() != cudaSuccess) return PCR_E_CUDA;
+    return PCR_OK;
+}
+
+int pcr_set_upsampling(pcr_record* rec, int mode) {
+    if (!rec || (mode != PCR_UPSAMPLE_REPLICATE && mode != PCR_UPSAMPLE_TRIANGLE)) return PCR_E_ARG;
+    if (mode == PCR_UPSAMPLE_TRIANGLE && !rec->d_chroma) {
+        if (int rc = take(rec, &rec->d_chroma, (size_t)(std::max<uint64_t>(rec->total_blocks / 6, 1) * 128))) return rc;
+    }
+    rec->upsampling = mode;
     return PCR_OK;
 }
 

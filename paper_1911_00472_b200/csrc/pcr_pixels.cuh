@@ -80,13 +80,21 @@ __device__ __forceinline__ uint32_t pack4_sat(int v0, int v1, int v2, int v3) {
 // coefficient (no AC scan decoded): only the head plane is read and the transform collapses to
 // one value; 3 = no decoded scan reaches beyond position 7: the lines are not read at all.
 // kRoi: only work units that touch their image's crop rectangle (P.roi) are processed.
-template <bool kRefine, int kDcMode, bool kRoi = false>
+//
+// kStage serves triangle chroma upsampling, which needs chroma samples of neighbouring work
+// units: 0 = everything in one launch (2x2 replication); 1 = chroma pass: the chroma blocks are
+// folded, written back, transformed and their samples stored in P.chroma, nothing else; 2 = pixel
+// pass: luminance blocks as in 0, chroma samples with a one-sample border read back from
+// P.chroma, every pixel's chroma = (9 own + 3 horizontally nearer + 3 vertically nearer +
+// 1 diagonal + 8) >> 4, neighbours clamped to the MCU-padded planes.
+template <bool kRefine, int kDcMode, bool kRoi = false, int kStage = 0>
 __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeList fl, uint8_t* __restrict__ out) {
     __shared__ __align__(16) uint32_t s_line[kRefine ? 32 * kPixThreads : 1];
     __shared__ __align__(16) uint8_t s_y[16][16 * kPixMcus];
     __shared__ __align__(16) uint8_t s_c[2][8][8 * kPixMcus];
     __shared__ __align__(16) uint8_t s_stage[16 * kStagePitch];
     __shared__ __align__(16) uint16_t s_q[3][64];
+    __shared__ uint8_t s_ct[kStage == 2 ? 2 : 1][kStage == 2 ? 10 : 1][kStage == 2 ? 8 * kPixMcus + 2 : 1];   // chroma tile + border
 
     const int tid = threadIdx.x;
     const Unit un = P.units[blockIdx.x];
@@ -121,6 +129,12 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
             blk = im.blk_base + (comp == 1 ? 4ull : 5ull) * im.mx * im.my + local;
             local += im.blk_base / 6;
         }
+        if (kStage == 1 && comp == 0) valid = false;          // chroma pass
+        if (kStage == 2 && comp != 0) valid = false;          // pixel pass: chroma comes from the sample planes
+        uint8_t* cplane = nullptr;                            // chroma pass: where this block's samples go
+        if (kStage == 1 && comp != 0)
+            cplane = P.chroma + (im.blk_base / 6) * 128 + (comp == 2 ? 64ull * im.mx * im.my : 0ull) +
+                     (size_t)(8 * un.mrow) * (8 * im.mx) + 8 * (un.mcol0 + ((j - 32) & 7));
         if (valid && kDcMode == 2) {
             // all AC zero: both passes keep only the k = 0 term, every sample of the block is equal
             constexpr uint32_t K4 = 5793;
@@ -218,7 +232,8 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
             // pass 2: rows; the +128 level shift rides in the rounding constant
             uint8_t* dst;
             int pitch;
-            if (j < 32) { dst = &s_y[(j >> 4) * 8][(j & 15) * 8]; pitch = 16 * kPixMcus; }
+            if (kStage == 1) { dst = cplane; pitch = 8 * (int)im.mx; }
+            else if (j < 32) { dst = &s_y[(j >> 4) * 8][(j & 15) * 8]; pitch = 16 * kPixMcus; }
             else { dst = &s_c[(j - 32) >> 3][0][((j - 32) & 7) * 8]; pitch = 8 * kPixMcus; }
 #pragma unroll
             for (int y = 0; y < 8; ++y) {
@@ -230,6 +245,17 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
             }
         }
     }
+    if (kStage == 1) return;                                // chroma pass: no pixels
+    if (kStage == 2) {
+        // chroma tile of the unit with a one-sample border, clamped to the padded planes
+        const int cw = 8 * (int)im.mx, chh = 8 * (int)im.my, tw = 8 * nm + 2;
+        const uint8_t* cbase = P.chroma + (im.blk_base / 6) * 128;
+        for (int i = tid; i < 2 * 10 * tw; i += kPixThreads) {
+            const int c = i / (10 * tw), rem2 = i - c * 10 * tw, r = rem2 / tw, x = rem2 - r * tw;
+            const int gy = min(max(8 * (int)un.mrow + r - 1, 0), chh - 1), gx2 = min(max(8 * (int)un.mcol0 + x - 1, 0), cw - 1);
+            s_ct[c][r][x] = cbase[(size_t)c * cw * chh + (size_t)gy * cw + gx2];
+        }
+    }
     __syncthreads();
 
     // ---- colour: 4 pixels per step, staged as the output's byte layout
@@ -237,9 +263,22 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
         const int row = gi / (4 * kPixMcus), gx = gi % (4 * kPixMcus);
         if (gx >= 4 * nm) continue;
         const uint32_t yw = *reinterpret_cast<const uint32_t*>(&s_y[row][4 * gx]);
+        int px[12];
+        if (kStage == 2) {
+            const int ry = 1 + (row >> 1), rn = ry + ((row & 1) ? 1 : -1);       // own / vertically nearer tile row
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int x = 4 * gx + e, cx = 1 + (x >> 1), cn = cx + ((x & 1) ? 1 : -1);
+                const int cb = ((9 * s_ct[0][ry][cx] + 3 * s_ct[0][ry][cn] + 3 * s_ct[0][rn][cx] + s_ct[0][rn][cn] + 8) >> 4) - 128;
+                const int cr = ((9 * s_ct[1][ry][cx] + 3 * s_ct[1][ry][cn] + 3 * s_ct[1][rn][cx] + s_ct[1][rn][cn] + 8) >> 4) - 128;
+                const int Y = (int)((yw >> (8 * e)) & 255u);
+                px[e * 3 + 0] = Y + ((91881 * cr + 32768) >> 16);
+                px[e * 3 + 1] = Y + ((-22553 * cb - 46802 * cr + 32768) >> 16);
+                px[e * 3 + 2] = Y + ((116130 * cb + 32768) >> 16);
+            }
+        } else {
         const uint32_t cbw = *reinterpret_cast<const uint16_t*>(&s_c[0][row >> 1][2 * gx]);
         const uint32_t crw = *reinterpret_cast<const uint16_t*>(&s_c[1][row >> 1][2 * gx]);
-        int px[12];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const int cb = (int)((cbw >> (8 * h)) & 255u) - 128, cr = (int)((crw >> (8 * h)) & 255u) - 128;
@@ -253,6 +292,7 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
                 px[(2 * h + e) * 3 + 1] = Y + dg;
                 px[(2 * h + e) * 3 + 2] = Y + db;
             }
+        }
         }
         uint32_t* d = reinterpret_cast<uint32_t*>(s_stage + row * kStagePitch + 12 * gx);
         d[0] = pack4_sat(px[0], px[1], px[2], px[3]);

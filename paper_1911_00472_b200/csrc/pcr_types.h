@@ -100,6 +100,8 @@ struct Params {
     const Item* items;
     const Unit* units;
     const uint16_t* qtab;       // [N][3][64] quantisers, zigzag order
+    uint8_t* chroma;            // chroma sample planes (triangle upsampling only): per image, at 128 bytes
+                                // per MCU in front of it, a Cb plane then a Cr plane of 8*my rows x 8*mx bytes
     const uint32_t* order;      // [N] processing order of the images
     const CropRect* roi;        // [N] or null: only work units that touch the image's rectangle are transformed
     int* status;                // [N]

@@ -96,6 +96,10 @@ class Decoder:
                          s.cuda_stream)
         return scores
 
+    def set_upsampling(self, triangle: bool) -> None:
+        """Chroma upsampling of later decodes: 2x2 replication (default) or the triangle filter."""
+        B.pcr_set_upsampling(self.handle, B.PCR_UPSAMPLE_TRIANGLE if triangle else B.PCR_UPSAMPLE_REPLICATE)
+
     def evict(self) -> None:
         B.pcr_evict(self.handle)
 
