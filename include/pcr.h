@@ -85,7 +85,8 @@ int pcr_num_groups(const pcr_record* rec);
 int pcr_get_image(const pcr_record* rec, int i, pcr_image_info* info);
 
 /* Size the output buffer of pcr_decode must have.  Images are packed RGB, row-major,
- * 3*width bytes per row, image i at out_offset (a multiple of 128). */
+ * 3*width bytes per row, image i at out_offset (a multiple of 128).  The size includes 16 spare
+ * bytes behind the last image (never written; pcr_decode_tensor reads pixels as aligned words). */
 size_t pcr_out_bytes(const pcr_record* rec);
 
 /* Bytes [0, pcr_prefix_bytes(rec, k)) are what fidelity k reads (Section 3: "from the

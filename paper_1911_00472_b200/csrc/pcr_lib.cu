@@ -523,7 +523,9 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
         imgs[i].blk_base = blocks; imgs[i].out_off = inf.out_offset;
         blocks += r->nblk[i];
     }
-    r->total_blocks = blocks; r->out_bytes = out_off; r->total_segs = segs;
+    // 16 spare bytes behind the last image: the tensor epilogue reads pixels as aligned words and may
+    // touch up to 8 bytes past a pixel pair
+    r->total_blocks = blocks; r->out_bytes = out_off + 16; r->total_segs = segs;
 
     // dependency waves of the script: a scan waits for every earlier scan that touches an
     // overlapping coefficient band of one of its components

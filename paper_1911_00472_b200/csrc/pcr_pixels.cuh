@@ -409,6 +409,24 @@ __device__ __forceinline__ void tensor_store(float* p, float v) { *p = v; }
 __device__ __forceinline__ void tensor_store(__half* p, float v) { *p = __float2half_rn(v); }
 __device__ __forceinline__ void tensor_store(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
 
+// Two horizontally adjacent RGB pixels (six bytes at any alignment) as floats, read as aligned
+// words: the word holding the first byte, the next one, and a third only when the six bytes reach
+// into it.  `same`: the right neighbour is the pixel itself (clamped at the crop's edge).
+__device__ __forceinline__ void load_rgb_pair(const uint8_t* p, bool same, float& r0, float& g0, float& b0,
+                                              float& r1, float& g1, float& b1) {
+    const uint32_t a = (uint32_t)(reinterpret_cast<uintptr_t>(p) & 3u);
+    const uint32_t* w = reinterpret_cast<const uint32_t*>(p - a);
+    const uint32_t w0 = __ldg(w), w1 = __ldg(w + 1);
+    const uint32_t w2 = (a == 3u && !same) ? __ldg(w + 2) : 0u;
+    const uint32_t lo = __funnelshift_r(w0, w1, 8 * a), hi = __funnelshift_r(w1, w2, 8 * a);   // bytes 0..3, 4..7
+    r0 = __uint_as_float(__byte_perm(lo, 0x4B000000u, 0x7540)) - 8388608.f;      // byte into the mantissa of 2^23
+    g0 = __uint_as_float(__byte_perm(lo, 0x4B000000u, 0x7541)) - 8388608.f;
+    b0 = __uint_as_float(__byte_perm(lo, 0x4B000000u, 0x7542)) - 8388608.f;
+    r1 = same ? r0 : __uint_as_float(__byte_perm(lo, 0x4B000000u, 0x7543)) - 8388608.f;
+    g1 = same ? g0 : __uint_as_float(__byte_perm(hi, 0x4B000000u, 0x7540)) - 8388608.f;
+    b1 = same ? b0 : __uint_as_float(__byte_perm(hi, 0x4B000000u, 0x7541)) - 8388608.f;
+}
+
 #ifndef PCR_TENSOR_ROWS
 #define PCR_TENSOR_ROWS 16
 #endif
@@ -451,17 +469,16 @@ __global__ void __launch_bounds__(256) tensor_kernel(Params P, TensorArgs T, con
         const int ix = (int)floorf(fx);
         const float ax = fx - (float)ix, bx = 1.f - ax;
         const uint8_t* p0 = crop0 + 3 * ix;
-        const uint8_t* p1 = crop0 + 3 * min(ix + 1, (int)r.w - 1);
+        const bool same = ix + 1 > (int)r.w - 1;            // the right tap is clamped onto the left one
         OutT* o = obase + ox;
         for (int dy = 0; dy < nrows; ++dy, o += S) {
             const int q0 = s_off0[dy], q1 = s_off1[dy];
             const float ay = s_ay[dy], by = 1.f - ay;
-            const float tr = bx * (float)__ldg(p0 + q0) + ax * (float)__ldg(p1 + q0);
-            const float tg = bx * (float)__ldg(p0 + q0 + 1) + ax * (float)__ldg(p1 + q0 + 1);
-            const float tb = bx * (float)__ldg(p0 + q0 + 2) + ax * (float)__ldg(p1 + q0 + 2);
-            const float hr = bx * (float)__ldg(p0 + q1) + ax * (float)__ldg(p1 + q1);
-            const float hg = bx * (float)__ldg(p0 + q1 + 1) + ax * (float)__ldg(p1 + q1 + 1);
-            const float hb = bx * (float)__ldg(p0 + q1 + 2) + ax * (float)__ldg(p1 + q1 + 2);
+            float r00, g00, b00, r01, g01, b01, r10, g10, b10, r11, g11, b11;
+            load_rgb_pair(p0 + q0, same, r00, g00, b00, r01, g01, b01);
+            load_rgb_pair(p0 + q1, same, r10, g10, b10, r11, g11, b11);
+            const float tr = bx * r00 + ax * r01, tg = bx * g00 + ax * g01, tb = bx * b00 + ax * b01;
+            const float hr = bx * r10 + ax * r11, hg = bx * g10 + ax * g11, hb = bx * b10 + ax * b11;
             tensor_store(o, ((by * tr + ay * hr) * k255 - m0) * i0);
             tensor_store(o + plane, ((by * tg + ay * hg) * k255 - m1) * i1);
             tensor_store(o + 2 * plane, ((by * tb + ay * hb) * k255 - m2) * i2);
