@@ -120,17 +120,37 @@ def source_hash() -> str:
     return h.hexdigest()[:16]
 
 
-def measured_traffic(stage: str, k: int, n_images: int):
-    """dram__bytes_read + dram__bytes_write per launch of a stage's kernel from the committed ncu
-    capture (whole record, k = 10), or None when the kernels changed since or the case differs."""
+def _traffic_table():
+    """The committed ncu DRAM counters (profiles/traffic_imagenet_shaped.json), or None when the
+    CUDA sources have changed since they were taken."""
     try:
-        with open(os.path.join(ROOT, "profiles", "traffic_imagenet_shaped_k10.json")) as f:
+        with open(os.path.join(ROOT, "profiles", "traffic_imagenet_shaped.json")) as f:
             t = json.load(f)
-        if t["source_sha256_16"] != source_hash() or k != 10 or n_images != 1024:
-            return None
-        return t["bytes_per_launch"].get(stage)
+        return t if t["source_sha256_16"] == source_hash() else None
     except Exception:
         return None
+
+
+def measured_traffic(stage: str, k: int, n_images: int):
+    """dram__bytes_read + dram__bytes_write per launch of a stage's kernel (whole record in one
+    launch) from the committed ncu capture at fidelity k, or None when the kernels changed since
+    or the case was not captured."""
+    t = _traffic_table()
+    if t is None or n_images != 1024:
+        return None
+    return t["by_k"].get(str(k), {}).get("bytes_per_launch", {}).get(stage)
+
+
+def measured_bytes_per_decode(k: int, n_images: int):
+    """All DRAM bytes one decode at fidelity k moves (kernels' ncu counters plus the sizes of the
+    memsets), from the committed capture, or None."""
+    t = _traffic_table()
+    if t is None or n_images != 1024:
+        return None
+    e = t["by_k"].get(str(k))
+    if not e:
+        return None
+    return float(sum(e["bytes_per_launch"].values()) + e.get("memset_bytes", 0.0))
 
 
 class ClockSampler:
@@ -208,6 +228,37 @@ def _oracle_worker(args):
     return hi - lo
 
 
+def _oracle_crc_worker(args):
+    """CRC-32 of the oracle's RGB bytes of images lo..hi-1 at fidelity k (the parity gate)."""
+    path, k, lo, hi = args
+    import zlib
+    import numpy as np
+    from oracle import pcr_oracle as O
+    rec = np.load(path)
+    return [(i, zlib.crc32(O.decode_image(rec, i, k, True)[1].tobytes())) for i in range(lo, hi)]
+
+
+def oracle_crcs(pool, cores: int, rec_path: str, k: int, images) -> dict:
+    """{image: CRC-32 of its oracle pixels at fidelity k} for a list of consecutive image indices."""
+    lo0, hi0 = images[0], images[-1] + 1
+    per = max(1, (hi0 - lo0 + cores * 2 - 1) // (cores * 2))
+    shards = [(rec_path, k, lo, min(lo + per, hi0)) for lo in range(lo0, hi0, per)]
+    out = {}
+    for part in pool.map(_oracle_crc_worker, shards):
+        out.update(part)
+    return out
+
+
+def device_crcs(dec, out, images) -> dict:
+    """CRC-32 of the decoded pixels of the listed images (read back from the device)."""
+    import zlib
+    res = {}
+    for i in images:
+        inf = dec.info[i]
+        res[i] = zlib.crc32(out[inf.out_offset:inf.out_offset + inf.out_bytes].cpu().numpy().tobytes())
+    return res
+
+
 def time_oracle(pool, cores: int, rec_path: str, k: int, n_images: int, passes: int = 1) -> float:
     """Images/s of the oracle decoding images [0, n_images) on `cores` processes."""
     per = max(1, (n_images + cores * 4 - 1) // (cores * 4))
@@ -254,47 +305,75 @@ def run_reference(args, rank: int):
     }))
 
 
-def run_sweep(args):
+def streamed_sweep(dev, recs, ks, peak, pool=None, cores=0, tmpdir=None):
     """Throughput sweep (the fifth workload): R ImageNet-shaped records of 1024 images, streamed
     from pinned host memory on two CUDA streams (two records in flight: the copy of one overlaps
-    the decode of the other), every record decoded once per k, k = 1..10."""
+    the decode of the other), every record opened, copied, decoded and closed once per k.
+
+    Parity: before the timed passes of a k every record goes through the same streamed path once
+    and the CRC-32 of every image's pixels is compared with the oracle's (when the oracle pool of
+    the CPU baseline is available); after the timed pass the outputs of the last two records are
+    compared on the device with a resident decode of the same records."""
+    import zlib
+    from concurrent.futures import ThreadPoolExecutor
     import numpy as np
     import torch
-    import pcr_synth
     from paper_1911_00472_b200 import Decoder, binding
-    from paper_1911_00472_b200 import build as libbuild
-    libbuild.build()
-    dev = torch.device("cuda", 0)
-    torch.cuda.set_device(dev)
-    R = args.records
-    recs = [pcr_synth.make_record(4, r, n_images=args.images or None) for r in range(R)]
+    R = len(recs)
     decs = [Decoder(r.bytes, device=dev) for r in recs]
     n_img = sum(d.n_images for d in decs)
     streams = [torch.cuda.Stream(dev), torch.cuda.Stream(dev)]
-    outs = [torch.empty(max(d.out_bytes for d in decs), dtype=torch.uint8, device=dev) for _ in range(2)]
-    peak = FALLBACK_HBM_GBS
-    try:
-        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
-            peak = float(json.load(f)["hbm_gbs"])
-    except Exception:
-        pass
+    size = max(d.out_bytes for d in decs)
+    outs = [torch.zeros(size, dtype=torch.uint8, device=dev) for _ in range(2)]
+    check = torch.zeros(size, dtype=torch.uint8, device=dev)
     scans0 = []
     for s in range(decs[0].n_groups):
         si = binding.pcr_get_scan(decs[0].handle, s)
         scans0.append((si.ncomp, si.comp[0], si.Ss, si.Se, si.Ah, si.wave))
     per_k = {}
-    from concurrent.futures import ThreadPoolExecutor
     OPEN_AHEAD = 3
     opener = ThreadPoolExecutor(max_workers=OPEN_AHEAD, initializer=lambda: torch.cuda.set_device(dev))
-    for k in range(1, decs[0].n_groups + 1):
+    hasher = ThreadPoolExecutor(max_workers=8)
+    rec_paths = []
+    if pool is not None:
+        for r, rec in enumerate(recs):
+            path = os.path.join(tmpdir, f"sweep_rec{r}.npy")
+            np.save(path, rec.bytes)
+            rec_paths.append(path)
+
+    def image_crcs(d, host):
+        def one(i):
+            inf = d.info[i]
+            return zlib.crc32(host[inf.out_offset:inf.out_offset + inf.out_bytes])
+        return list(hasher.map(one, range(d.n_images)))
+
+    for k in ks:
+        # ---- parity of the streamed path against the oracle, every image of every record
+        checked = 0
+        if pool is not None:
+            for i, d in enumerate(decs):
+                want = oracle_crcs(pool, cores, rec_paths[i], k, list(range(d.n_images)))
+                h = binding.pcr_open(d.host.data_ptr(), d.host.numel())
+                binding.pcr_decode(h, k, outs[i & 1].data_ptr(), streams[i & 1].cuda_stream)
+                streams[i & 1].synchronize()
+                bad, code = binding.pcr_status(h)
+                binding.pcr_close(h)
+                if code != 0:
+                    raise RuntimeError(f"sweep: decode error {code} on image {bad} of record {i}")
+                got = image_crcs(d, memoryview(outs[i & 1].cpu().numpy()))
+                for j in range(d.n_images):
+                    if got[j] != want[j]:
+                        raise RuntimeError(f"sweep parity: record {i} image {j} differs from the oracle at k={k}")
+                checked += d.n_images
         for rep in range(2):                     # first pass warms up, second is timed
             torch.cuda.synchronize(dev)
             t0 = time.perf_counter()
             live = []                            # handles of the records in flight, at most two
             # every record is opened, copied and decoded once, as a loader streaming a data set does.
             # Loader threads parse the next records (pcr_open: host-side marker walk and table
-            # uploads, about a millisecond each) while this thread enqueues decodes.
+            # uploads) while this thread enqueues decodes.
             ahead = [opener.submit(binding.pcr_open, d.host.data_ptr(), d.host.numel()) for d in decs[:OPEN_AHEAD]]
+            last = []
             for i, d in enumerate(decs):
                 h = ahead.pop(0).result()
                 if i + OPEN_AHEAD < len(decs):
@@ -305,33 +384,79 @@ def run_sweep(args):
                 if len(live) > 2:
                     old = live.pop(0)
                     binding.pcr_close(old)       # waits for that record's decode only
-            for h in live:
-                binding.pcr_close(h)
             torch.cuda.synchronize(dev)
             dt = time.perf_counter() - t0
-        # parity gate on the resident decoders (same records, same kernels)
-        for d in decs[:2]:
-            d.decode(k, outs[0])
-        torch.cuda.synchronize(dev)
-        for d in decs[:2]:
+            for h in live:
+                bad, code = binding.pcr_status(h)
+                if code != 0:
+                    raise RuntimeError(f"sweep: decode error {code} on image {bad}")
+                binding.pcr_close(h)
+        # the outputs the timed pass left behind (last two records) against a resident decode
+        for i in range(max(0, R - 2), R):
+            d = decs[i]
+            d.decode(k, check)
+            torch.cuda.synchronize(dev)
             bad, code = d.status()
             if code != 0:
                 raise RuntimeError(f"decode error {code} on image {bad}")
+            for inf in d.info:
+                a, b = inf.out_offset, inf.out_offset + inf.out_bytes
+                if not torch.equal(outs[i & 1][a:b], check[a:b]):
+                    raise RuntimeError(f"sweep: streamed output of record {i} differs from the resident decode at k={k}")
         model = 0.0
         h2d = 0
         for d in decs:
             scans = [sc + (binding.pcr_get_scan(d.handle, s).bytes,) for s, sc in enumerate(scans0)]
             model += algorithmic_bytes(scans, [(i.width, i.height) for i in d.info], k)["total"]
             h2d += d.prefix_bytes(k)
-        per_k[str(k)] = {"images_per_s": n_img / dt, "ms_per_record": 1000.0 * dt / R, "hbm_gbs": model / dt / 1e9,
-                         "frac_of_peak": model / dt / 1e9 / peak, "h2d_bytes_per_record": h2d // R}
-    print(json.dumps({"metric": METRIC, "unit": UNIT, "n_gpus": 1, "data": "synthetic", "dtype": "int16/u8",
-                      "config": {"workload": f"sweep: {R} ImageNet-shaped records x {decs[0].n_images} images, streamed from pinned host "
-                                             "memory on two CUDA streams, each record opened (host parse, three loader threads ahead), copied, decoded and closed once per k, two in flight",
-                                 "timing": "wall clock around enqueue + synchronise, second of two passes"},
-                      "sweep": per_k}))
+        per_k[str(k)] = {"images_per_s": n_img / dt, "ms_per_record": 1000.0 * dt / R, "hbm_gbs_model": model / dt / 1e9,
+                         "model_frac_of_peak": model / dt / 1e9 / peak, "h2d_bytes_per_record": h2d // R,
+                         "parity_images_vs_oracle": checked}
+    n_per = decs[0].n_images
     for d in decs:
         d.close()
+    opener.shutdown()
+    hasher.shutdown()
+    return {"workload": f"sweep: {R} ImageNet-shaped records x {n_per} images, streamed from pinned host memory on two CUDA "
+                        "streams, each record opened (host parse, three loader threads ahead), copied, decoded and closed once per k, two in flight",
+            "timing": "wall clock around enqueue + synchronise, second of two passes",
+            "parity": "every image of every record against the oracle's CRC-32 (streamed path, before timing) when the oracle pool runs; "
+                      "the last two streamed outputs against a resident decode on the device",
+            "by_k": per_k}
+
+
+def hbm_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def run_sweep(args):
+    """The full sweep on its own: --records records, k = 1..10."""
+    import multiprocessing as mp
+    import tempfile
+    import pcr_synth
+    pool, cores, tmp = None, len(os.sched_getaffinity(0)), tempfile.TemporaryDirectory()
+    if not args.no_cpu_baseline:
+        from oracle import pcr_oracle as O
+        O.build()
+        pool = mp.get_context("spawn").Pool(cores)
+        pool.map(abs, range(cores))              # start the workers before the first GPU call
+    import torch
+    from paper_1911_00472_b200 import build as libbuild
+    libbuild.build()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    recs = [pcr_synth.make_record(4, r, n_images=args.images or None) for r in range(args.records)]
+    res = streamed_sweep(dev, recs, list(range(1, 11)), hbm_peak()[0], pool, cores, tmp.name)
+    print(json.dumps({"metric": METRIC, "unit": UNIT, "n_gpus": 1, "data": "synthetic", "dtype": "int16/u8",
+                      "config": {"workload": res["workload"], "timing": res["timing"], "parity": res["parity"]},
+                      "sweep": res["by_k"]}))
+    if pool is not None:
+        pool.close(); pool.join()
+    tmp.cleanup()
 
 
 # ----------------------------------------------------------------------------------------
@@ -387,6 +512,13 @@ def main():
         np.save(rec_path, rec.bytes)
         pool = mp.get_context("spawn").Pool(cores)
         time_oracle(pool, cores, rec_path, 1, min(64, rec.n_images))   # start the workers
+        # parity gate: the oracle's pixels of a sample of the timed record at the timed fidelity
+        # (CRC-32 per image), compared with the device output before anything is timed
+        parity_images = list(range(min(rec.n_images, 128)))
+        parity_want = oracle_crcs(pool, cores, rec_path, args.k, parity_images)
+    sweep_recs = []
+    if do_cpu and wl == WORKLOAD and not args.headline_only and not args.images:
+        sweep_recs = [pcr_synth.make_record(4, r) for r in range(4)]
 
     import torch
     import torch.distributed as dist
@@ -431,6 +563,14 @@ def main():
     bad, code = dec.status()
     if code != 0:
         raise RuntimeError(f"decode reported error {code} on image {bad}")
+    parity_checked = None
+    if do_cpu:
+        got = device_crcs(dec, out, parity_images)
+        diff = [i for i in parity_images if got[i] != parity_want[i]]
+        if diff:
+            raise RuntimeError(f"parity: images {diff[:8]} differ from the oracle at k={k}")
+        parity_checked = {"images": len(parity_images), "k": k, "how": "CRC-32 of every sampled image's RGB bytes, device output "
+                          "against the CPU oracle, before the timed steps"}
 
     sampler = ClockSampler(local_rank)
     for _ in range(args.warmup):
@@ -486,8 +626,9 @@ def main():
                               "note": "pcr_open + pcr_decode from pinned host bytes + synchronise + pcr_status + pcr_close per step"}
 
     per_k, raise_ms, training_tensor, fidelity, baseline_jpeg = {}, {}, None, None, None
-    hbm_by_k = {}
+    hbm_by_k, hbm_meas_by_k = {}, {}
     triangle = None
+    sweep = None
     if not args.headline_only:
         # per-k numbers and the stage profile (this rank's GPU)
         per_k = {}
@@ -498,6 +639,8 @@ def main():
             st = 5
             per_k[str(kk)] = n_img * st / (timed_steps(kk, st) / 1000.0)
             hbm_by_k[str(kk)] = algorithmic_bytes(scans, infos, kk)["total"] * per_k[str(kk)] / n_img / 1e9
+            mb = measured_bytes_per_decode(kk, n_img) if wl == WORKLOAD else None
+            hbm_meas_by_k[str(kk)] = mb * per_k[str(kk)] / n_img / 1e9 if mb is not None else None
         # decode straight to a fixed-size training batch (random-resized crops, flip, 224 x 224, fp16)
         crops = pcr_synth.random_resized_crops(infos, 1000 + rank)
         t_size = 224
@@ -590,6 +733,10 @@ def main():
                 torch.cuda.synchronize(dev)
                 acc += a.elapsed_time(b) / reps
             raise_ms[f"{k_from}->{k_to}"] = acc
+    if sweep_recs:
+        # the streamed multi-record workload, short form: 4 records, k = 1, 5, 10
+        sweep = streamed_sweep(dev, sweep_recs, [1, 5, 10], hbm_peak()[0], pool, cores, tmpdir.name)
+        del sweep_recs
     binding.pcr_set_profiling(dec.handle, True)
     stage_ms, stage_n = {}, {}
     reps = 5
@@ -604,13 +751,7 @@ def main():
     model = algorithmic_bytes(scans, infos, k)
     kernels = {n: t for n, t in stage_ms.items() if stage_n.get(n, 0) > 0}
     dom = max(kernels, key=kernels.get)
-    peak, peak_src = FALLBACK_HBM_GBS, "fallback"
-    try:
-        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
-            peak = float(json.load(f)["hbm_gbs"])
-            peak_src = "measured"
-    except Exception:
-        pass
+    peak, peak_src = hbm_peak()
     achieved = model[dom] / (kernels[dom] * 1e-3) / 1e9
     traffic = measured_traffic(dom, k, n_img)
     whole = model["total"] / (ms_max / args.steps * 1e-3) / 1e9
@@ -618,6 +759,9 @@ def main():
                 "traffic": traffic, "peak_source": peak_src, "kernel_ms": kernels[dom],
                 "algorithmic_bytes_per_launch": model[dom],
                 "whole_path": {"algorithmic_bytes_per_step": model["total"], "achieved": whole, "frac": whole / peak},
+                "step_ms": {"pipelined": ms_max / args.steps, "stages_one_after_the_other": sum(stage_ms.values()),
+                            "note": "value is timed in the pipelined layout (image slices on their own streams); the stage "
+                                    "times below come from the profiling layout, one stage after the other"},
                 "stages_ms": stage_ms,
                 "stage_frac_of_peak": {n: (model.get(n, 0.0) / (t * 1e-3) / 1e9 / peak if t > 0 else None)
                                        for n, t in stage_ms.items()}}
@@ -651,12 +795,18 @@ def main():
                        "record_bytes": int(rec.bytes.size), "prefix_bytes_at_k": int(prefix),
                        "mean_compressed_bytes_per_image_by_scan": [c / n_img for c in comp]},
             "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
-            "cpu_baseline": cpu_baseline, "images_per_s_by_k": per_k, "hbm_gbs_by_k": hbm_by_k,
-            "hbm_frac_of_peak_by_k": {kk: v / peak for kk, v in hbm_by_k.items()},
-            "hbm_by_k_note": "algorithmic bytes of the decode at k (compressed prefix, zeroed and written coefficient planes, "
-                             "planes read by the pixel stage, pixels written) / time; below k = 5 the implementation moves fewer "
-                             "bytes than this model (positions 0..7 of every block live in a dense plane, the 128-byte lines are "
-                             "neither zeroed nor read while no scan reaches position 8)", "raise_fidelity_ms_per_record": raise_ms,
+            "cpu_baseline": cpu_baseline, "parity_checked": parity_checked, "sweep": sweep,
+            "images_per_s_by_k": per_k, "hbm_gbs_model_by_k": hbm_by_k,
+            "hbm_model_frac_of_peak_by_k": {kk: v / peak for kk, v in hbm_by_k.items()},
+            "hbm_gbs_measured_by_k": hbm_meas_by_k,
+            "hbm_measured_frac_of_peak_by_k": {kk: (v / peak if v is not None else None) for kk, v in hbm_meas_by_k.items()},
+            "hbm_by_k_note": "model: algorithmic bytes of the decode at k (compressed prefix, zeroed and written coefficient planes, "
+                             "planes read by the pixel stage, pixels written) / time: a rate of useful work, NOT an achieved "
+                             "bandwidth (below k = 5 the implementation moves far fewer bytes than the model: positions 0..7 of "
+                             "every block live in a dense plane, the 128-byte lines are neither zeroed nor read while no scan "
+                             "reaches position 8).  measured: DRAM bytes the kernels and memsets of one decode really move "
+                             "(ncu dram__bytes of every kernel, committed under profiles/) / the same time; null when the "
+                             "kernels changed since the capture", "raise_fidelity_ms_per_record": raise_ms,
             "training_tensor": training_tensor, "predicted_io_speedup_by_k": io_speedup, "fidelity": fidelity, "baseline_jpeg": baseline_jpeg, "triangle_upsampling": triangle,
         }))
     dec.close()

@@ -172,7 +172,8 @@ int pcr_decode_tensor(pcr_record* rec, int k, const pcr_crop* crops, int size, c
  *                  (two luminance pyramids per image and the per-scale sums).
  *   dev_scores   : DEVICE, pcr_num_images floats, score of image i at index i.
  * Enqueues on `stream` and returns.  The first call on a record uploads a small per-image table
- * (one allocation).  Errors: PCR_E_ARG, PCR_E_NOMEM, PCR_E_CUDA. */
+ * (one allocation).  Records of more than 65535 images are refused (PCR_E_ARG).
+ * Errors: PCR_E_ARG, PCR_E_NOMEM, PCR_E_CUDA. */
 size_t pcr_msssim_scratch_bytes(pcr_record* rec);
 int pcr_msssim(pcr_record* rec, const void* rgb_a, const void* rgb_b, void* scratch, float* dev_scores, void* stream);
 
@@ -253,8 +254,9 @@ int pcr_get_profile(pcr_record* rec, pcr_stage_time* out, int cap, int* n);
  * It turns the int16 coefficient planes of ONE image into packed RGB exactly as pcr_decode's
  * last stage does (dequantise, inverse DCT, 2x2 chroma replication, colour conversion, crop).
  *   dev_coeffs : DEVICE, caller-owned: 6*ceil(W/16)*ceil(H/16) blocks of 64 int16 in the
- *                layout of pcr_coeffs (Y, Cb, Cr; block rows, block columns; zigzag), 4-byte
- *                aligned.  Not modified.
+ *                layout of pcr_coeffs (Y, Cb, Cr; block rows, block columns; zigzag), 16-byte
+ *                aligned (the kernel reads whole 16-byte vectors; any other alignment is
+ *                refused with PCR_E_ARG before anything is launched).  Not modified.
  *   width, height : at most 4096 each; larger images are refused with PCR_E_ARG.
  *   host_qtab  : HOST, 3 x 64 uint16 quantisers (Y, Cb, Cr) in zigzag order; copied by value.
  *   dev_rgb    : DEVICE, caller-owned, 3*W*H bytes, 4-byte aligned start recommended.

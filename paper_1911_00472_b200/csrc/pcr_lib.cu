@@ -925,11 +925,12 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
                 else pixel_kernel<false, 1, true><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
             }
             ++g_launches;
-            if (targs && i1 > i0) {
-                const dim3 tg((unsigned)((targs->size + kTensorRows - 1) / kTensorRows), i1 - i0);
-                if (targs->f32 == 2) tensor_kernel<__nv_bfloat16><<<tg, 256, 0, q>>>(P, *targs, static_cast<const uint8_t*>(out), i0);
-                else if (targs->f32) tensor_kernel<float><<<tg, 256, 0, q>>>(P, *targs, static_cast<const uint8_t*>(out), i0);
-                else tensor_kernel<__half><<<tg, 256, 0, q>>>(P, *targs, static_cast<const uint8_t*>(out), i0);
+            // the grid's second dimension (one image each) holds at most 65535 entries
+            for (uint32_t p0 = i0; targs && p0 < i1; p0 += 65535u) {
+                const dim3 tg((unsigned)((targs->size + kTensorRows - 1) / kTensorRows), std::min(i1 - p0, 65535u));
+                if (targs->f32 == 2) tensor_kernel<__nv_bfloat16><<<tg, 256, 0, q>>>(P, *targs, static_cast<const uint8_t*>(out), p0);
+                else if (targs->f32) tensor_kernel<float><<<tg, 256, 0, q>>>(P, *targs, static_cast<const uint8_t*>(out), p0);
+                else tensor_kernel<__half><<<tg, 256, 0, q>>>(P, *targs, static_cast<const uint8_t*>(out), p0);
                 ++g_launches;
             }
         }
@@ -1108,6 +1109,7 @@ size_t pcr_msssim_scratch_bytes(pcr_record* rec) {
 int pcr_msssim(pcr_record* rec, const void* rgb_a, const void* rgb_b, void* scratch, float* dev_scores, void* stream) {
     if (!rec || !rgb_a || !rgb_b || !scratch || !dev_scores) return PCR_E_ARG;
     if ((reinterpret_cast<uintptr_t>(scratch) & 15u) || (reinterpret_cast<uintptr_t>(dev_scores) & 3u)) return PCR_E_ARG;
+    if (rec->N > 65535) return PCR_E_ARG;       // one grid row per image
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (!rec->d_ms) {
         std::vector<MsDesc> table;
@@ -1138,6 +1140,9 @@ int pcr_msssim(pcr_record* rec, const void* rgb_a, const void* rgb_b, void* scra
     }
     ms_final_kernel<<<(N + 255) / 256, 256, 0, st>>>(rec->d_ms, sums, dev_scores, (int)N);
     ++g_launches;
+    // pcr_close waits for this event before it hands the record's buffers (the table above among them) on
+    if (cudaEventRecord(rec->ev_done, st) != cudaSuccess) return PCR_E_CUDA;
+    rec->decode_enqueued = true;
     if (cudaGetLastError() != cudaSuccess) return PCR_E_CUDA;
     return PCR_OK;
 }
@@ -1286,7 +1291,8 @@ int pcr_pixels_noalloc(const int16_t* dev_coeffs, uint32_t width, uint32_t heigh
                        uint8_t* dev_rgb, void* stream) {
     if (!dev_coeffs || !host_qtab || !dev_rgb || width == 0 || height == 0) return PCR_E_ARG;
     if (width > kNoAllocMaxDim || height > kNoAllocMaxDim) return PCR_E_ARG;   // beyond the fixed scratch
-    if (reinterpret_cast<uintptr_t>(dev_coeffs) & 3u) return PCR_E_ARG;
+    // the pixel kernel reads every block as eight 16-byte vectors
+    if (reinterpret_cast<uintptr_t>(dev_coeffs) & 15u) return PCR_E_ARG;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return PCR_E_CUDA;
     if (dev < 0 || dev >= kMaxDevices) return PCR_E_ARG;

@@ -145,3 +145,34 @@ def pillow_y(jpeg_bytes: bytes) -> np.ndarray:
     im.load()
     assert im.mode == "YCbCr"
     return np.asarray(im)[:, :, 0]
+
+
+def oracle_rgb_shard(args):
+    """Process-pool worker (module level so that spawned children can import it): decodes images
+    lo..hi-1 of the record saved at rec_path with the CPU oracle at fidelity k and writes each
+    image's pixels at its offset into the uint8 file out_path (the GPU output buffer's layout)."""
+    rec_path, out_path, out_bytes, offsets, k, lo, hi = args
+    from oracle import pcr_oracle as O
+    rec = np.load(rec_path)
+    out = np.memmap(out_path, dtype=np.uint8, mode="r+", shape=(out_bytes,))
+    for i in range(lo, hi):
+        _, rgb = O.decode_image(rec, i, k)
+        out[offsets[i]:offsets[i] + rgb.size] = rgb.reshape(-1)
+    out.flush()
+    return hi - lo
+
+
+def oracle_record_pixels(pool, workers, rec_bytes, tmpdir, offsets, out_bytes, k):
+    """All images of a record at fidelity k through the oracle on a process pool: a uint8 array
+    laid out like the output buffer of the decode (bytes between images zero)."""
+    import os
+    rec_path = os.path.join(tmpdir, "rec.npy")
+    if not os.path.exists(rec_path):
+        np.save(rec_path, rec_bytes)
+    out_path = os.path.join(tmpdir, f"oracle_k{k}.u8")
+    np.memmap(out_path, dtype=np.uint8, mode="w+", shape=(out_bytes,)).flush()
+    n = len(offsets)
+    per = max(1, (n + 4 * workers - 1) // (4 * workers))
+    shards = [(rec_path, out_path, out_bytes, offsets, k, lo, min(lo + per, n)) for lo in range(0, n, per)]
+    assert sum(pool.map(oracle_rgb_shard, shards)) == n
+    return np.array(np.memmap(out_path, dtype=np.uint8, mode="r", shape=(out_bytes,)))

@@ -28,6 +28,21 @@ def test_decode_more_equals_decode_from_scratch(fix, request):
     want = {}
     for k in range(1, 11):
         want[k] = _snapshot(ref, ref.decode(k))
+    # what the chains are compared with is itself the oracle's result, for every image and k
+    from paper_1911_00472_b200 import pcr_image_blocks
+    oracle = {k: [O.decode_image(rec.bytes, i, k) for i in range(rec.n_images)] for k in range(1, 11)}
+
+    def assert_oracle(snap, k, what):
+        out_h, coef_h = snap[0].cpu().numpy(), snap[1].cpu().numpy()
+        for i in range(rec.n_images):
+            inf = ref.info[i]
+            a, b = pcr_image_blocks(ref.handle, i)
+            want_c, want_rgb = oracle[k][i]
+            assert np.array_equal(coef_h[a:a + b], want_c), (fix, what, k, i)
+            assert np.array_equal(out_h[inf.out_offset:inf.out_offset + inf.out_bytes].reshape(inf.height, inf.width, 3), want_rgb), (fix, what, k, i)
+
+    for k in range(1, 11):
+        assert_oracle(want[k], k, "from scratch")
     # one scan group at a time, and a few jumps (from DC only, across the refinement waves)
     chains = [list(range(1, 11)), [1, 10], [2, 6, 7], [5, 8, 10], [4, 9]]
     for chain in chains:
@@ -39,6 +54,7 @@ def test_decode_more_equals_decode_from_scratch(fix, request):
             got = _snapshot(inc, out)
             assert torch.equal(got[0], want[k][0]), (fix, chain, k)
             assert torch.equal(got[1], want[k][1]), (fix, chain, k)
+        assert_oracle(got, chain[-1], chain)             # the end of every chain against the oracle directly
     # the end of the longest chain against the oracle directly
     coef, rgb = O.decode_image(rec.bytes, 0, 10)
     inf = inc.info[0]

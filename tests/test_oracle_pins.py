@@ -178,6 +178,28 @@ def test_scan_script_and_one_bit_dc_refinement(rec1_small):
     assert abs((s[6] - s[5]) * 1024 - blocks / 8) < 0.1 * 1024 + 64
 
 
+def test_size_ratio_shape_of_the_paper_tables(rec1_small):
+    """Table 1 of the paper: the ratio full size / size of the prefix up to scan group k falls with
+    k and is 1 at k = 10 for every data set.  The synthetic record has the same shape (its values
+    are reported by the benchmark, not asserted: the content recipe is not the paper's data)."""
+    rows = {}
+    with open(os.path.join(os.path.dirname(__file__), "golden", "paper_tables.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            t = line.split()
+            rows[t[0]] = [float(v) for v in t[1:5]]
+    assert set(rows) == {"imagenet", "ham10000", "cars", "celebahq"}
+    for name, r in rows.items():
+        assert r[0] > r[1] > r[2] > r[3] == 1.0, name
+    rec = rec1_small.bytes
+    data0 = O.prefix_bytes(rec, 1) - sum(len(O.reassemble(rec, i, 1)) - 2 for i in range(rec1_small.n_images))
+    full = O.prefix_bytes(rec, 10) - data0          # scan-group bytes without header and index
+    ratios = [full / (O.prefix_bytes(rec, k) - data0) for k in (1, 2, 5, 10)]
+    assert ratios[0] > ratios[1] > ratios[2] > ratios[3] == 1.0
+    assert ratios[0] > 4.0                          # the first scan group is a small fraction of the image
+
+
 def test_quant_tables_match_a_stock_encoder():
     """The typed-in base tables and the quality scaling agree with a stock encoder's tables."""
     from PIL import Image

@@ -5,7 +5,8 @@ another framework's memory pool, or after the training job has taken the whole d
 `pcr_pixels_noalloc` serves them: it keeps its small tables in a fixed array inside the
 library instead of cudaMalloc'd buffers.  Here it must reproduce, byte for byte, the pixels
 that `pcr_decode` writes for the same coefficients, on two calls in a row (the second call
-reuses the array the first one filled, with a different image size).
+reuses the array the first one filled, with a different image size), and both must equal what
+the CPU oracle makes of the same coefficients.
 
 This file sorts last on purpose, so a run that stops at the first failure has already run
 every other test.
@@ -14,6 +15,7 @@ import numpy as np
 import pytest
 
 import pcr_synth
+from oracle import pcr_oracle as O
 
 pytestmark = pytest.mark.gpu
 
@@ -50,8 +52,23 @@ def test_noalloc_pixels_match_decode_on_two_calls_in_a_row():
         inf = dec.info[i]
         want = out[inf.out_offset:inf.out_offset + inf.out_bytes]
         assert torch.equal(rgb, want), f"image {i}"
+        # ... and the oracle's pixels from the same coefficients (which are the ground truth at k = 10)
+        coef_h = dec.coeffs(i).cpu().numpy()
+        assert np.array_equal(coef_h, rec.truth(i)), f"image {i}"
+        want_o = O.pixels_from_coeffs(coef_h, inf.width, inf.height, q[:64], q[64:128])
+        assert np.array_equal(rgb.cpu().numpy().reshape(inf.height, inf.width, 3), want_o), f"image {i}"
     # sizes beyond the fixed array are refused with a clear error, nothing is launched
     with pytest.raises(binding.PcrError) as e:
         binding.pcr_pixels_noalloc(results[0][1].data_ptr(), 4112, 16, q.ctypes.data, results[0][1].data_ptr(), 0)
     assert e.value.code == binding.PCR_E_ARG
+    # the kernel reads the coefficients as 16-byte vectors: a pointer that is only 4-byte aligned
+    # is refused before anything is launched
+    coef = dec.coeffs(0).contiguous()
+    inf = dec.info[0]
+    for shift in (4, 8, 12):
+        with pytest.raises(binding.PcrError) as e:
+            binding.pcr_pixels_noalloc(coef.data_ptr() + shift, inf.width, inf.height, q.ctypes.data,
+                                       results[0][1].data_ptr(), stream.cuda_stream)
+        assert e.value.code == binding.PCR_E_ARG
+    torch.cuda.synchronize()
     dec.close()
