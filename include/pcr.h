@@ -47,7 +47,10 @@ extern "C" {
                                images disagree on the scan script, unsupported JPEG features     */
 #define PCR_E_CORRUPT (-3)  /* found while decoding on the device: undefined Huffman code,
                                segment overrun, wrong number of restart markers                   */
-#define PCR_E_TIMEOUT (-4)  /* a bounded device-side wait gave up                                */
+#define PCR_E_TIMEOUT (-4)  /* a bounded device-side wait gave up: in records without restart
+                               markers a refinement scan follows, block by block, the earlier
+                               refinement of the same component that another warp of its CTA
+                               decodes; its polls for that warp's progress are counted          */
 #define PCR_E_CUDA (-5)     /* a CUDA runtime call failed                                        */
 #define PCR_E_NOMEM (-6)    /* host or device allocation failed                                  */
 
@@ -272,6 +275,13 @@ int pcr_get_profile(pcr_record* rec, pcr_stage_time* out, int cap, int* n);
  * beyond 63), PCR_E_CUDA. */
 int pcr_pixels_noalloc(const int16_t* dev_coeffs, uint32_t width, uint32_t height, const uint16_t* host_qtab,
                        uint8_t* dev_rgb, void* stream);
+
+/* Test hook for the bounded device-side wait behind PCR_E_TIMEOUT (the paper has no counterpart):
+ * launches one warp that waits, with the decoder's own wait routine and a limit of 2000 polls,
+ * for a flag that nothing sets.  *gave_up = 1 if the wait ended by its limit (the kernel returns
+ * normally and the context stays usable), 0 if it claims to have seen the flag.
+ * Errors: PCR_E_ARG, PCR_E_NOMEM, PCR_E_CUDA. */
+int pcr_selftest_bounded_wait(int* gave_up);
 
 /* Counts kernel launches issued by this library since it was loaded (all records). */
 uint64_t pcr_launch_count(void);

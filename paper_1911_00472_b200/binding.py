@@ -17,7 +17,8 @@ PCR_E_ARG, PCR_E_FORMAT, PCR_E_CORRUPT, PCR_E_TIMEOUT, PCR_E_CUDA, PCR_E_NOMEM =
 EXPORTS = ("pcr_open", "pcr_num_images", "pcr_num_groups", "pcr_get_image", "pcr_out_bytes", "pcr_prefix_bytes",
            "pcr_decode", "pcr_evict", "pcr_status", "pcr_coeffs", "pcr_image_blocks", "pcr_launch_count",
            "pcr_strerror", "pcr_close", "pcr_get_scan", "pcr_set_profiling", "pcr_get_profile",
-           "pcr_pixels_noalloc", "pcr_decode_more", "pcr_release_cached_memory", "pcr_decode_tensor", "pcr_msssim", "pcr_msssim_scratch_bytes", "pcr_set_upsampling")
+           "pcr_pixels_noalloc", "pcr_decode_more", "pcr_release_cached_memory", "pcr_decode_tensor", "pcr_msssim", "pcr_msssim_scratch_bytes", "pcr_set_upsampling",
+           "pcr_selftest_bounded_wait")
 
 
 class ImageInfo(C.Structure):
@@ -74,6 +75,7 @@ def lib():
         L.pcr_set_profiling.argtypes = [vp, C.c_int]
         L.pcr_get_profile.argtypes = [vp, C.POINTER(StageTime), C.c_int, C.POINTER(C.c_int)]
         L.pcr_pixels_noalloc.argtypes = [vp, C.c_uint32, C.c_uint32, vp, vp, vp]
+        L.pcr_selftest_bounded_wait.argtypes = [C.POINTER(C.c_int)]
         L.pcr_launch_count.restype = C.c_uint64
         L.pcr_launch_count.argtypes = []
         L.pcr_strerror.restype = C.c_char_p
@@ -210,6 +212,13 @@ def pcr_pixels_noalloc(dev_coeffs_ptr: int, width: int, height: int, host_qtab_p
     device coefficients + host quantisers -> device RGB, enqueued on `stream`."""
     _chk(lib().pcr_pixels_noalloc(dev_coeffs_ptr, width, height, host_qtab_ptr, dev_rgb_ptr, stream),
          "pcr_pixels_noalloc")
+
+
+def pcr_selftest_bounded_wait() -> bool:
+    """True if the decoder's bounded device-side wait, pointed at a flag nothing sets, gave up at its limit."""
+    v = C.c_int(-1)
+    _chk(lib().pcr_selftest_bounded_wait(C.byref(v)), "pcr_selftest_bounded_wait")
+    return v.value == 1
 
 
 def pcr_release_cached_memory() -> None:

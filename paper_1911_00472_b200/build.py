@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libpcr_b200.so")
 SOURCES = ["pcr_lib.cu"]
-HEADERS = ["pcr_types.h", "pcr_entropy.cuh", "pcr_pixels.cuh", "pcr_msssim.cuh"]
+HEADERS = ["pcr_types.h", "pcr_entropy.cuh", "pcr_long.cuh", "pcr_pixels.cuh", "pcr_msssim.cuh"]
 
 
 def _nvcc() -> str:

@@ -147,7 +147,7 @@ __device__ __forceinline__ uint32_t huff_lookup(const HuffTab& t, uint32_t win) 
     const uint32_t w16 = win >> 16;
     for (int l = kLutBits + 1; l <= 16; ++l) {
         uint32_t d = (w16 >> (16 - l)) - t.first[l];
-        if (d < t.cnt[l]) return ((uint32_t)l << 8) | t.vals[t.idx[l] + d];
+        if (d < t.cnt[l]) return ((uint32_t)l << 8) | t.vals[(t.idx[l] + d) & 255u];   // (index masked: damaged tables stay in bounds)
     }
     return 0;
 }
@@ -330,8 +330,7 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
     const ScanDesc sd0 = P.scans[item.si];
     const int s = item.si / P.N;
     const ScanScript sc = P.script[s];
-    const bool dc = sc.Ss == 0;
-    const bool huff = !(dc && sc.Ah != 0);
+    const bool dc = sc.Ss == 0;              // a DC first pass (DC refinement scans go to dc_refine_kernel)
     // tables: a DC scan may use two tables of one image; an AC item may span two images
     const bool two_images = item.next != 0;
     const uint32_t si1 = two_images ? item.next - 1u : item.si;
@@ -364,11 +363,9 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
         }
         if (__all_sync(full, done)) return;                               // nothing of this item is wanted
     }
-    if (huff) {
-        build_hufftab(tabs[wid][0], P.rec + sd0.tab_off[0], lane);
-        if (two_images) build_hufftab(tabs[wid][1], P.rec + P.scans[si1].tab_off[0], lane);
-        else if (sd0.tab_off[1]) build_hufftab(tabs[wid][1], P.rec + sd0.tab_off[1], lane);
-    }
+    build_hufftab(tabs[wid][0], P.rec + sd0.tab_off[0], lane);
+    if (two_images) build_hufftab(tabs[wid][1], P.rec + P.scans[si1].tab_off[0], lane);
+    else if (sd0.tab_off[1]) build_hufftab(tabs[wid][1], P.rec + sd0.tab_off[1], lane);
     const uint32_t* segtab = P.seg_start + sd.seg_base;
     uint32_t bstart = segtab[seg];
     uint32_t bend = segtab[seg + 1] - 2;
@@ -384,7 +381,7 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
     const int Al = sc.Al, p1 = 1 << sc.Al;
 
     if (dc) {
-        // ---- DC scans: one block per step
+        // ---- DC first pass: one block per step
         const int bpm = inter ? 6 : 1;                     // blocks per MCU
         uint32_t m = m0, mrow = m0 / mcu_w, mcol = m0 % mcu_w;
         int j = 0;                                         // block inside the MCU: Y00 Y01 Y10 Y11 Cb Cr
@@ -405,7 +402,7 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
                 if (inter && c == 0) blk = g.coff[0] + (uint64_t)(2 * mrow + (j >> 1)) * g.bw[0] + 2 * mcol + (j & 1);
                 else blk = g.coff[c] + (uint64_t)mrow * g.bw[c] + mcol;
                 int16_t* dcv = P.head + blk * 8;
-                if (sc.Ah == 0) {
+                {
                     const HuffTab& tab = tabs[wid][(sd.slots >> (2 * ci)) & 1u];
                     const uint32_t e = huff_lookup(tab, win);
                     const int len = (int)(e >> 8), sz = (int)(e & 255u);
@@ -415,11 +412,6 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
                     const int pv = (c == 0 ? pred0 : (c == 1 ? pred1 : pred2)) + d;
                     if (c == 0) pred0 = pv; else if (c == 1) pred1 = pv; else pred2 = pv;
                     *dcv = (int16_t)(pv << Al);
-                } else {
-                    // coefficient 0 is the low half of the block's first head word; position 1 in the
-                    // upper half may be written by an AC scan of the same wave, hence the atomic
-                    if (win >> 31) atomicOr(reinterpret_cast<unsigned int*>(dcv), (unsigned int)p1);
-                    br.skip(1);
                 }
                 if (++j == bpm) {
                     j = 0; ++m;

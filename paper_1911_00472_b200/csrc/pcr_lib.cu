@@ -22,6 +22,7 @@
 
 #include "../../include/pcr.h"
 #include "pcr_entropy.cuh"
+#include "pcr_long.cuh"
 #include "pcr_msssim.cuh"
 #include "pcr_pixels.cuh"
 #include "pcr_types.h"
@@ -134,6 +135,7 @@ struct pcr_record {
     std::vector<pcr_image_info> info;
     std::vector<uint64_t> blk_base, nblk;
     uint64_t total_blocks = 0, total_segs = 0;
+    unsigned dc_refine_chunks = 1;  // 256-MCU chunks of the largest image, at most 8 (dc_refine_kernel's grid)
     bool widths_mult16 = true;    // every image is a multiple of 16 pixels wide (the DC-only pixel kernel's condition)
     size_t out_bytes = 0;
     // scan script analysis
@@ -146,6 +148,13 @@ struct pcr_record {
     std::vector<uint32_t> slice_img;                            // [n_slices + 1] first image of each slice
     std::vector<uint32_t> slice_unit;                           // [n_slices + 1] first pixel unit of each slice
     std::vector<uint32_t> item_begin, item_count;               // [n_slices][G]
+    // Scans that are one long restart interval take kernels of their own (pcr_long.cuh): first passes
+    // as (scan, image) pairs sorted by (slice, wave, scan); AC refinements as (component, image)
+    // groups sorted by slice (all refinement scans of the component that a call decodes, in one CTA)
+    std::vector<uint32_t> long_begin, long_count;               // [n_slices][G]
+    uint32_t* d_long = nullptr;
+    std::vector<uint32_t> group_begin, group_count;             // [n_slices]
+    uint32_t* d_group = nullptr;
     std::vector<cudaStream_t> streams;                          // one per slice
     std::vector<cudaEvent_t> ev_index;                          // [n_waves] index of wave w done (side stream)
     cudaEvent_t ev_start = nullptr;                             // index of the first wave done
@@ -447,6 +456,7 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
             uint32_t clen = rd32(c + 8);
             uint64_t padded = ((uint64_t)clen + 15) & ~15ull;
             if ((off & 15) || off < r->group_end[g] || off + padded > r->group_end[g + 1]) return PCR_E_FORMAT;
+            if (clen >= (1u << 28)) return PCR_E_FORMAT;        // bit positions inside a scan are 32-bit
             ScanParse sp;
             int rc = parse_chunk(rec, off, clen, g == 0, im, sp);
             if (rc) return rc;
@@ -519,6 +529,7 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
         inf.out_offset = out_off;
         out_off += (inf.out_bytes + 127) & ~127ull;
         if (imgs[i].W & 15u) r->widths_mult16 = false;
+        r->dc_refine_chunks = std::max(r->dc_refine_chunks, std::min(8u, (imgs[i].mx * imgs[i].my + 255u) / 256u));
         r->blk_base[i] = blocks; r->nblk[i] = 6ull * imgs[i].mx * imgs[i].my;
         imgs[i].blk_base = blocks; imgs[i].out_off = inf.out_offset;
         blocks += r->nblk[i];
@@ -569,13 +580,64 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     std::vector<Item> items;
     items.reserve((size_t)(segs / 24 + (uint64_t)N * G));
     r->item_begin.assign((size_t)r->n_slices * G, 0); r->item_count.assign((size_t)r->n_slices * G, 0);
+    // A scan that is one restart interval of at least this many bytes goes to the kernels for long
+    // intervals; DC refinement scans have a kernel of their own and no items at all.
+    uint32_t long_min = 1024;
+    if (const char* e = getenv("PCR_LONG_MIN_BYTES")) long_min = (uint32_t)std::max(0, atoi(e));
+    auto is_long = [&](int s, uint32_t i) {
+        const ScanScript& sc = r->script[s];
+        const ScanDesc& sd = scans[(size_t)s * N + i];
+        if (sc.Ss == 0 && sc.Se == 63) return false;           // a baseline record's sequential scan
+        return sd.nseg == 1 && sd.data_end - sd.data_off >= long_min;
+    };
+    // the AC refinements of one component of one image go together: all of them one interval each,
+    // at least one of them long
+    std::vector<uint8_t> grouped((size_t)N * 3, 0);
+    for (uint32_t i = 0; i < N; ++i)
+        for (int c = 0; c < 3; ++c) {
+            bool any = false, one_interval = true, big = false;
+            for (uint32_t s = 0; s < G; ++s) {
+                const ScanScript& sc = r->script[s];
+                if (sc.Ss == 0 || sc.Ah == 0 || sc.comp[0] != c) continue;
+                any = true;
+                one_interval = one_interval && scans[(size_t)s * N + i].nseg == 1;
+                big = big || is_long((int)s, i);
+            }
+            grouped[(size_t)i * 3 + c] = any && one_interval && big;
+        }
+    auto takes_long_kernel = [&](int s, uint32_t i) {
+        const ScanScript& sc = r->script[s];
+        if (sc.Ss > 0 && sc.Ah != 0) return grouped[(size_t)i * 3 + sc.comp[0]] != 0;
+        return is_long(s, i);
+    };
+    std::vector<uint32_t> longs, groups;
+    r->long_begin.assign((size_t)r->n_slices * G, 0); r->long_count.assign((size_t)r->n_slices * G, 0);
+    r->group_begin.assign(r->n_slices, 0); r->group_count.assign(r->n_slices, 0);
+    for (int g = 0; g < r->n_slices; ++g) {
+        for (int w = 0; w < r->n_waves; ++w)
+            for (int s : r->wave_scans[w]) {
+                const ScanScript& sc = r->script[s];
+                if (sc.Ah != 0) continue;                      // first passes only
+                r->long_begin[(size_t)g * G + s] = (uint32_t)longs.size();
+                for (uint32_t pos = r->slice_img[g]; pos < r->slice_img[g + 1]; ++pos)
+                    if (is_long(s, order[pos])) longs.push_back((uint32_t)(s * N + order[pos]));
+                r->long_count[(size_t)g * G + s] = (uint32_t)longs.size() - r->long_begin[(size_t)g * G + s];
+            }
+        r->group_begin[g] = (uint32_t)groups.size();
+        for (uint32_t pos = r->slice_img[g]; pos < r->slice_img[g + 1]; ++pos)
+            for (int c = 0; c < 3; ++c)
+                if (grouped[(size_t)order[pos] * 3 + c]) groups.push_back(((uint32_t)c << 28) | order[pos]);
+        r->group_count[g] = (uint32_t)groups.size() - r->group_begin[g];
+    }
     for (int g = 0; g < r->n_slices; ++g)
         for (int w = 0; w < r->n_waves; ++w)
             for (int s : r->wave_scans[w]) {
                 r->item_begin[(size_t)g * G + s] = (uint32_t)items.size();
                 const bool ac = r->script[s].Ss > 0;
-                for (uint32_t pos = r->slice_img[g]; pos < r->slice_img[g + 1]; ++pos) {
+                const bool dc_refine = r->script[s].Ss == 0 && r->script[s].Ah != 0;
+                for (uint32_t pos = r->slice_img[g]; pos < r->slice_img[g + 1] && !dc_refine; ++pos) {
                     const uint32_t i = order[pos];
+                    if (takes_long_kernel((int)s, i)) continue;
                     const ScanDesc& sd = scans[(size_t)s * N + i];
                     // full warps of 32 restart intervals; in AC scans the last warp of an image
                     // runs on into the first intervals of the next image (two tables per warp)
@@ -670,6 +732,8 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     if ((rc = upload(r, &r->d_scans, scans))) return rc;
     if ((rc = upload(r, &r->d_imgs, imgs))) return rc;
     if ((rc = upload(r, &r->d_items, items))) return rc;
+    if ((rc = upload(r, &r->d_long, longs))) return rc;
+    if ((rc = upload(r, &r->d_group, groups))) return rc;
     if ((rc = upload(r, &r->d_qtab, qtab))) return rc;
     if ((rc = upload(r, &r->d_unit_prefix, unit_prefix))) return rc;
     if ((rc = take(r, &r->d_units, (size_t)std::max<uint32_t>(r->n_units, 1) * sizeof(Unit)))) return rc;
@@ -805,6 +869,10 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
             any_refine = true;
         }
     }
+    int first_refine_wave = -1;                 // wave of the first AC refinement this call decodes
+    for (int s = k0; s < k; ++s)
+        if (rec->script[s].Ss > 0 && rec->script[s].Ah > 0 && (first_refine_wave < 0 || rec->wave_of_scan[s] < first_refine_wave))
+            first_refine_wave = rec->wave_of_scan[s];
     bool dc_only = true, head_only = true;      // no AC scan at all / no scan beyond zigzag position 7
     for (int s = 0; s < k; ++s) {
         if (rec->script[s].Ss > 0 || rec->script[s].Se > 0) dc_only = false;
@@ -874,17 +942,52 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
                 if (!any) { begin = rec->item_begin[(size_t)g * G + s]; any = true; }
                 count += rec->item_count[(size_t)g * G + s];
             }
-            if (!count) return true;
             const ScanScript& first = rec->script[rec->wave_scans[w][0]];
-            if (first.Ss == 0 && first.Se == 63) {        // a baseline record: its one scan is sequential
+            if (count && first.Ss == 0 && first.Se == 63) {        // a baseline record: its one scan is sequential
                 if (targs) sequential_kernel<true><<<(count + kSeqWarps - 1) / kSeqWarps, 32 * kSeqWarps, 0, q>>>(P, begin, count);
                 else sequential_kernel<false><<<(count + kSeqWarps - 1) / kSeqWarps, 32 * kSeqWarps, 0, q>>>(P, begin, count);
                 ++g_launches;
                 return true;
             }
-            if (targs) entropy_kernel<true><<<(count + kEntropyWarps - 1) / kEntropyWarps, 32 * kEntropyWarps, 0, q>>>(P, begin, count);
-            else entropy_kernel<false><<<(count + kEntropyWarps - 1) / kEntropyWarps, 32 * kEntropyWarps, 0, q>>>(P, begin, count);
-            ++g_launches;
+            if (count) {
+                if (targs) entropy_kernel<true><<<(count + kEntropyWarps - 1) / kEntropyWarps, 32 * kEntropyWarps, 0, q>>>(P, begin, count);
+                else entropy_kernel<false><<<(count + kEntropyWarps - 1) / kEntropyWarps, 32 * kEntropyWarps, 0, q>>>(P, begin, count);
+                ++g_launches;
+            }
+            // scans that are one long restart interval: the first passes of the wave (a contiguous run
+            // of the list) ...
+            {
+                uint32_t lb = 0, lc = 0;
+                bool lany = false;
+                for (int s : rec->wave_scans[w]) {
+                    if (s >= k) break;
+                    if (s < k0 || rec->script[s].Ah != 0) continue;
+                    if (!lany) { lb = rec->long_begin[(size_t)g * G + s]; lany = true; }
+                    lc += rec->long_count[(size_t)g * G + s];
+                }
+                if (lc) {
+                    first_pass_long_kernel<<<(lc + kLongWarps - 1) / kLongWarps, 32 * kLongWarps, 0, q>>>(P, rec->d_long + lb, lc);
+                    ++g_launches;
+                }
+            }
+            // ... all their AC refinements of this call in the wave of the first one (a refinement
+            // depends on first passes, which every wave-0 launch above has finished, and on earlier
+            // refinements of its component, which run in the same CTA) ...
+            if (w == first_refine_wave && rec->group_count[g]) {
+                int warps = std::max(fl.n[0], std::max(fl.n[1], fl.n[2]));
+                ac_refine_group_kernel<<<rec->group_count[g], 32 * warps, 0, q>>>(P, fl, rec->d_group + rec->group_begin[g]);
+                ++g_launches;
+            }
+            // ... and the DC refinement scans of every record
+            for (int s : rec->wave_scans[w]) {
+                if (s >= k) break;
+                const ScanScript& sc = rec->script[s];
+                if (s < k0 || sc.Ss != 0 || sc.Ah == 0) continue;
+                for (uint32_t p0 = i0; p0 < i1; p0 += 65535u) {
+                    dc_refine_kernel<<<dim3(rec->dc_refine_chunks, std::min(i1 - p0, 65535u)), 256, 0, q>>>(P, s, p0);
+                    ++g_launches;
+                }
+            }
             return true;
         }
         Params Q = P;
@@ -1231,6 +1334,23 @@ int pcr_get_profile(pcr_record* rec, pcr_stage_time* out, int cap, int* n) {
 }
 
 uint64_t pcr_launch_count(void) { return g_launches.load(); }
+
+int pcr_selftest_bounded_wait(int* gave_up) {
+    if (!gave_up) return PCR_E_ARG;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return PCR_E_CUDA;
+    int* d = static_cast<int*>(dev_alloc(sizeof(int), dev));
+    if (!d) return PCR_E_NOMEM;
+    int rc = PCR_OK;
+    if (cudaMemset(d, 0xFF, sizeof(int)) != cudaSuccess) rc = PCR_E_CUDA;
+    if (rc == PCR_OK) {
+        bounded_wait_probe_kernel<<<1, 32>>>(2000u, d);      // 2000 polls of about 64 ns: the wait ends by itself
+        ++g_launches;
+        if (cudaMemcpy(gave_up, d, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) rc = PCR_E_CUDA;
+    }
+    dev_release(d, sizeof(int), dev);
+    return rc;
+}
 
 const char* pcr_strerror(int code) {
     switch (code) {

@@ -1,0 +1,616 @@
+// Entropy stage for scans that are ONE long restart interval (records written without restart
+// markers: one entropy-coded segment per image and scan), and the DC refinement scans of any record.
+//
+// A Huffman stream is a serial chain, so a whole scan on one lane takes tens of thousands of
+// dependent steps.  Three kernels shorten or remove that chain:
+//
+//  * dc_refine_kernel: a DC refinement scan carries exactly one raw bit per block, so after
+//    unstuffing bit j of a restart interval is block j of the interval in scan order: one thread
+//    per MCU, no chain at all.  Used for every record.
+//  * first_pass_long_kernel: DC and AC first passes.  One warp per (scan, image); the segment is cut
+//    into 32 subsequences of equal bit length and every lane decodes its own.  A lane that starts
+//    in the middle of the stream does not know where a code begins nor which coefficient (or which
+//    block of the MCU) it is at; it starts anyway, and because Huffman streams re-synchronise, its
+//    state at the end of its subsequence is usually right.  The lanes then hand their end states on:
+//    a lane whose predecessor ended in a state other than the one it started from decodes again
+//    from there; the rounds stop when nothing changes (at the latest after 32: lane 0 starts at
+//    the true beginning, so after round r lanes 0..r are exact).  A prefix sum of the blocks each
+//    lane finished (and of the DC differences per component) gives every lane its first block and
+//    its predictors, and a last pass decodes once more and writes.
+//  * ac_refine_chain_kernel: an AC refinement cannot be entered in the middle (how many correction
+//    bits follow a symbol depends on which coefficients of the block are already non-zero, i.e. on
+//    the block number).  One warp per (scan, image): lane 0 walks the chain with ordinary branches
+//    (no other lane shares its instruction stream), the other lanes fetch the bitstream into a
+//    shared-memory ring, gather the masks of the next 32 blocks and write the side data out.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "pcr_entropy.cuh"
+#include "pcr_types.h"
+
+namespace pcr {
+
+// ---------------------------------------------------------------------------------------
+// DC refinement: thread per MCU of the scan.  grid = (chunks of MCUs, images of the run).
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) dc_refine_kernel(Params P, int s, uint32_t pos0) {
+    const int img = (int)P.order[pos0 + blockIdx.y];
+    const ScanDesc sd = P.scans[(size_t)s * P.N + img];
+    const ScanScript sc = P.script[s];
+    const ImgDesc im = P.imgs[img];
+    const Geometry g = make_geometry(im);
+    const bool inter = sc.ncomp > 1;
+    const int c0 = sc.comp[0];
+    const uint32_t mcu_w = inter ? g.mx : g.ubw[c0];
+    const uint32_t mcu_h = inter ? g.my : g.ubh[c0];
+    const uint32_t total = mcu_w * mcu_h;
+    const uint32_t bpm = inter ? 6u : 1u;                      // blocks (= bits) per MCU
+    const uint32_t* segtab = P.seg_start + sd.seg_base;
+    const uint32_t* words = reinterpret_cast<const uint32_t*>(P.ubuf);
+    const int p1 = 1 << sc.Al;
+    bool bad = false;
+    for (uint32_t m = blockIdx.x * 256u + threadIdx.x; m < total; m += gridDim.x * 256u) {
+        const uint32_t seg = sd.ri ? m / sd.ri : 0u;
+        if (seg >= sd.nseg) { bad = true; continue; }
+        const uint32_t m0 = seg * sd.ri;                       // 0 without restart markers
+        const uint32_t bstart = segtab[seg], bend = segtab[seg + 1] - 2u;
+        if (bstart < sd.data_off || bend > sd.data_end || bend < bstart) { bad = true; continue; }   // a missing marker left a hole
+        const uint32_t bit = bpm * (m - m0);
+        if (bit + bpm > 8u * (bend - bstart)) { bad = true; continue; }                             // the interval is too short
+        const uint32_t p = 8u * (bstart & 3u) + bit;           // from the first bit of word bstart >> 2
+        const uint32_t wi = (bstart >> 2) + (p >> 5);
+        const uint32_t w0 = __ldg(words + wi), w1 = __ldg(words + wi + 1);   // the copy has spare bytes behind its end
+        const uint32_t v = __funnelshift_l(w1, w0, p & 31u) >> (32u - bpm);  // the MCU's bits, first block in the top bit
+        const uint32_t mrow = m / mcu_w, mcol = m - mrow * mcu_w;
+#pragma unroll
+        for (uint32_t j = 0; j < 6; ++j) {
+            if (j >= bpm) break;
+            if (!((v >> (bpm - 1u - j)) & 1u)) continue;
+            uint64_t blk;
+            if (!inter) blk = g.coff[c0] + (uint64_t)mrow * g.bw[c0] + mcol;
+            else if (j < 4) blk = g.coff[0] + (uint64_t)(2 * mrow + (j >> 1)) * g.bw[0] + 2 * mcol + (j & 1);
+            else blk = g.coff[j - 3] + (uint64_t)mrow * g.bw[j - 3] + mcol;
+            // coefficient 0 is the first int16 of the block's head entry; no other scan of the wave writes it
+            int16_t* dcv = P.head + blk * 8;
+            *dcv = (int16_t)(*dcv | p1);
+        }
+    }
+    if (bad) atomicMin(&P.status[img], kErrCorrupt);
+}
+
+// ---------------------------------------------------------------------------------------
+// Bit reader of one lane over the unstuffed big-endian words: a 64-bit window, the next word
+// already requested while the current bits are consumed.  Positions are bits counted from the
+// first bit of a base word.
+// ---------------------------------------------------------------------------------------
+struct WordReader {
+    const uint32_t* w;     // base word
+    uint32_t rd;           // index of the word held in `ahead`
+    uint64_t buf;          // left-aligned window
+    int nbits;
+    uint32_t ahead;
+    __device__ __forceinline__ void init(const uint32_t* base, uint32_t pos) {
+        w = base;
+        rd = pos >> 5;
+        const uint32_t first = __ldg(w + rd) << (pos & 31u);
+        buf = (uint64_t)first << 32;
+        nbits = 32 - (int)(pos & 31u);
+        ++rd;
+        ahead = __ldg(w + rd);
+    }
+    __device__ __forceinline__ void refill() {                 // afterwards at least 33 bits are held
+        if (nbits <= 32) {
+            buf |= (uint64_t)ahead << (32 - nbits);
+            nbits += 32;
+            ++rd;
+            ahead = __ldg(w + rd);
+        }
+    }
+    __device__ __forceinline__ uint32_t top32() const { return (uint32_t)(buf >> 32); }
+    __device__ __forceinline__ void skip(int n) { buf <<= n; nbits -= n; }
+    __device__ __forceinline__ uint32_t pos() const { return rd * 32u - (uint32_t)nbits; }
+};
+
+constexpr int kLongWarps = 3;
+
+// What one lane needs to write the coefficients of an AC first pass.
+struct AcWrite {
+    int16_t* plane;        // the component's lines
+    int16_t* headp;        // the component's head entries
+    unsigned long long* maskp;   // the scan's non-zero masks, by block number inside the component
+    uint32_t mcu_w, bw;    // blocks per row of the scan's (unpadded) grid / of the padded grid
+    uint32_t m, m1;        // next block of the scan, one past its last
+    int p1;
+};
+
+// Decodes the symbols of an AC first pass that START in [pos, pos_end), from zigzag position k of the
+// current block.  Every step consumes at least one bit, so the loop ends.  Without kWrite (search
+// for the true entry state) an undefined code is skipped by one bit and a coefficient beyond the
+// band ends the block: the lane is then reading from a wrong entry point and only has to arrive
+// somewhere.  With kWrite the entry state is the true one, such events mean a corrupt stream.
+template <bool kWrite>
+__device__ __forceinline__ void ac_first_span(const HuffTab& tab, const uint32_t* base, uint32_t pos, int k, uint32_t pos_end,
+                                              int Ss, int Se, uint32_t& pos_out, int& k_out, uint32_t& nblk, AcWrite& W, bool& bad) {
+    WordReader br;
+    br.init(base, pos);
+    uint32_t nb = 0;
+    unsigned long long M = 0;
+    uint32_t bcol = 0, bi = 0;
+    if (kWrite) { bcol = W.m % W.mcu_w; bi = (W.m / W.mcu_w) * W.bw + bcol; }
+    bool stop = kWrite && W.m >= W.m1;
+    while (!stop && br.pos() < pos_end) {
+        br.refill();
+        const uint32_t win = br.top32();
+        uint32_t e = tab.lut[win >> (32 - kLutBits)];
+        if (e == 0) e = huff_lookup(tab, win);
+        if (e == 0) {
+            if (kWrite) { bad = true; break; }
+            br.skip(1);
+            continue;
+        }
+        const int len = (int)(e >> 8), r = (int)(e >> 4) & 15, sz = (int)(e & 15u);
+        const bool is_coef = sz != 0, is_eob = sz == 0 && r < 15;
+        const int kk = k + r;
+        const bool over = is_coef && kk > Se;
+        if (kWrite && over) { bad = true; break; }
+        const int extra = is_coef ? sz : (is_eob ? r : 0);
+        const uint32_t xb = top_bits(win << len, extra);
+        br.skip(len + extra);
+        if (kWrite && is_coef) {
+            const int16_t val = (int16_t)(extend_bits(xb, sz) * W.p1);
+            if (kk < 8) W.headp[(uint64_t)bi * 8 + kk] = val;
+            else W.plane[(uint64_t)bi * 64 + kk] = val;
+            M |= 1ull << kk;
+        }
+        k = is_coef ? kk + 1 : (is_eob ? k : k + 16);
+        if (is_eob || over || k > Se) {                        // the block ends, an end-of-band run skips more
+            const uint32_t adv = 1u + (is_eob ? (1u << r) + xb - 1u : 0u);
+            nb += adv;
+            k = Ss;
+            if (kWrite) {
+                if (M) atomicOr(W.maskp + bi, M);              // a block may be shared with the neighbouring lane
+                M = 0;
+                W.m += adv;
+                if (W.m >= W.m1) stop = true;
+                else if (adv == 1u) { if (++bcol == W.mcu_w) { bcol = 0; bi += W.bw - W.mcu_w + 1u; } else ++bi; }
+                else { bcol = W.m % W.mcu_w; bi = (W.m / W.mcu_w) * W.bw + bcol; }
+            }
+        }
+    }
+    if (kWrite && M) atomicOr(W.maskp + bi, M);                // the part of a block that ends in the next lane's span
+    pos_out = br.pos();
+    k_out = k;
+    nblk = nb;
+}
+
+// The same for a DC first pass: one symbol (size category, then that many difference bits) per block;
+// j = the block's place in its MCU (Y00 Y01 Y10 Y11 Cb Cr, or always 0 in a one-component scan).
+struct DcWrite {
+    int16_t* head;
+    uint64_t coff[3];
+    uint32_t bw[3];
+    uint32_t mcu_w;
+    uint32_t n, n1;        // next block of the scan in scan order, one past its last
+    int pred[3];
+    int Al;
+};
+
+template <bool kWrite>
+__device__ __forceinline__ void dc_first_span(const HuffTab* tabs2, uint32_t slots, bool inter, int c0, const uint32_t* base,
+                                              uint32_t pos, int j, uint32_t pos_end, uint32_t& pos_out, int& j_out, uint32_t& nblk,
+                                              int& sum0, int& sum1, int& sum2, DcWrite& W, bool& bad) {
+    WordReader br;
+    br.init(base, pos);
+    const int bpm = inter ? 6 : 1;
+    uint32_t nb = 0;
+    int s0 = 0, s1 = 0, s2 = 0;
+    uint32_t mrow = 0, mcol = 0;
+    if (kWrite) { const uint32_t m = W.n / (uint32_t)bpm; mrow = m / W.mcu_w; mcol = m - mrow * W.mcu_w; }
+    bool stop = kWrite && W.n >= W.n1;
+    while (!stop && br.pos() < pos_end) {
+        br.refill();
+        const uint32_t win = br.top32();
+        const int ci = inter ? (j < 4 ? 0 : j - 3) : 0;
+        const int c = inter ? ci : c0;
+        const HuffTab& tab = tabs2[(slots >> (2 * ci)) & 1u];
+        const uint32_t e = huff_lookup(tab, win);
+        const int len = (int)(e >> 8), sz = (int)(e & 255u);
+        if (e == 0 || sz > 15) {
+            if (kWrite) { bad = true; break; }
+            br.skip(1);
+            continue;
+        }
+        const int d = extend_bits(top_bits(win << len, sz), sz);
+        br.skip(len + sz);
+        if (c == 0) s0 += d; else if (c == 1) s1 += d; else s2 += d;
+        if (kWrite) {
+            const int pv = (c == 0 ? W.pred[0] : (c == 1 ? W.pred[1] : W.pred[2])) + d;
+            if (c == 0) W.pred[0] = pv; else if (c == 1) W.pred[1] = pv; else W.pred[2] = pv;
+            uint64_t blk;
+            if (inter && c == 0) blk = W.coff[0] + (uint64_t)(2 * mrow + (uint32_t)(j >> 1)) * W.bw[0] + 2 * mcol + (uint32_t)(j & 1);
+            else blk = W.coff[c] + (uint64_t)mrow * W.bw[c] + mcol;
+            W.head[blk * 8] = (int16_t)(pv << W.Al);
+            if (++W.n >= W.n1) stop = true;
+        }
+        ++nb;
+        if (++j == bpm) {
+            j = 0;
+            if (kWrite) { if (++mcol == W.mcu_w) { mcol = 0; ++mrow; } }
+        }
+    }
+    pos_out = br.pos();
+    j_out = j;
+    nblk = nb;
+    sum0 = s0; sum1 = s1; sum2 = s2;
+}
+
+// One warp per listed (scan, image) whose scan is one restart interval; first passes only.
+__global__ void __launch_bounds__(32 * kLongWarps) first_pass_long_kernel(Params P, const uint32_t* __restrict__ list, uint32_t count) {
+    __shared__ HuffTab tabs[kLongWarps][2];
+    const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t it = blockIdx.x * kLongWarps + wid;
+    if (it >= count) return;                                   // whole warp
+    const uint32_t si = list[it];
+    const int s = (int)(si / (uint32_t)P.N), img = (int)(si % (uint32_t)P.N);
+    const ScanDesc sd = P.scans[si];
+    const ScanScript sc = P.script[s];
+    const ImgDesc im = P.imgs[img];
+    const Geometry g = make_geometry(im);
+    const bool dc = sc.Ss == 0, inter = sc.ncomp > 1;
+    const int c0 = sc.comp[0];
+    const uint32_t mcu_w = inter ? g.mx : g.ubw[c0];
+    const uint32_t mcu_h = inter ? g.my : g.ubh[c0];
+    const uint32_t total = mcu_w * mcu_h;                      // MCUs of the scan (one interval)
+    const unsigned full = 0xffffffffu;
+    build_hufftab(tabs[wid][0], P.rec + sd.tab_off[0], lane);
+    if (sd.tab_off[1]) build_hufftab(tabs[wid][1], P.rec + sd.tab_off[1], lane);
+    const uint32_t* segtab = P.seg_start + sd.seg_base;
+    const uint32_t bstart = segtab[0], bend = segtab[1] - 2u;
+    if (bstart < sd.data_off || bend > sd.data_end || bend < bstart) {
+        if (lane == 0) atomicMin(&P.status[img], kErrCorrupt);
+        return;
+    }
+    const uint32_t* base = reinterpret_cast<const uint32_t*>(P.ubuf) + (bstart >> 2);
+    const uint32_t lead = 8u * (bstart & 3u), endbit = lead + 8u * (bend - bstart);
+    // 32 subsequences of S bits (whole words, at least 8 of them)
+    const uint32_t nwords = (endbit + 31u) >> 5;
+    const uint32_t S = 32u * max(8u, (nwords + 31u) / 32u);
+    const uint32_t my_begin = min(max((uint32_t)lane * S, lead), endbit), my_end = min(((uint32_t)lane + 1u) * S, endbit);
+    bool bad = false;
+    if (dc) {
+        DcWrite W;
+        W.head = P.head; W.mcu_w = mcu_w; W.Al = sc.Al;
+#pragma unroll
+        for (int c = 0; c < 3; ++c) { W.coff[c] = g.coff[c]; W.bw[c] = g.bw[c]; W.pred[c] = 0; }
+        W.n = 0; W.n1 = total * (inter ? 6u : 1u);
+        uint32_t pos = my_begin, pos_x, nb;
+        int j = 0, j_x, a0, a1, a2;
+        bool again = true;
+        for (int round = 0; round < 33; ++round) {
+            if (again) dc_first_span<false>(tabs[wid], sd.slots, inter, c0, base, pos, j, my_end, pos_x, j_x, nb, a0, a1, a2, W, bad);
+            const uint32_t ppos = min(__shfl_up_sync(full, pos_x, 1), endbit);
+            const int pj = __shfl_up_sync(full, j_x, 1);
+            again = lane > 0 && (ppos != pos || pj != j);
+            if (again) { pos = ppos; j = pj; }
+            if (!__any_sync(full, again)) break;
+        }
+        // first block and predictors of every lane: exclusive prefix sums
+        uint32_t nin = nb;
+        int b0 = a0, b1 = a1, b2 = a2;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t on = __shfl_up_sync(full, nin, d);
+            const int o0 = __shfl_up_sync(full, b0, d), o1 = __shfl_up_sync(full, b1, d), o2 = __shfl_up_sync(full, b2, d);
+            if (lane >= d) { nin += on; b0 += o0; b1 += o1; b2 += o2; }
+        }
+        const uint32_t all = __shfl_sync(full, nin, 31);
+        W.n = min(nin - nb, W.n1); W.pred[0] = b0 - a0; W.pred[1] = b1 - a1; W.pred[2] = b2 - a2;
+        // the place inside the MCU follows from the block number (equal to the handed-on state unless
+        // the stream is damaged; taking it from the block number keeps every store inside the image)
+        if (nb && (uint32_t)j != W.n % (inter ? 6u : 1u)) bad = true;
+        j = (int)(W.n % (inter ? 6u : 1u));
+        dc_first_span<true>(tabs[wid], sd.slots, inter, c0, base, pos, j, my_end, pos_x, j_x, nb, a0, a1, a2, W, bad);
+        if (all < total * (inter ? 6u : 1u)) bad = true;                     // the stream ends before the last block
+    } else {
+        const int c = c0, Ss = sc.Ss, Se = sc.Se;
+        const ScanAux ax = P.saux[s];
+        AcWrite W;
+        W.plane = P.planes + g.coff[c] * 64; W.headp = P.head + g.coff[c] * 8;
+        W.maskp = reinterpret_cast<unsigned long long*>(P.aux + ax.base + g.loff[c]);
+        W.mcu_w = mcu_w; W.bw = g.bw[c]; W.m = 0; W.m1 = total; W.p1 = 1 << sc.Al;
+        const HuffTab& tab = tabs[wid][0];
+        uint32_t pos = my_begin, pos_x, nb;
+        int k = Ss, k_x;
+        bool again = true;
+        for (int round = 0; round < 33; ++round) {
+            if (again) ac_first_span<false>(tab, base, pos, k, my_end, Ss, Se, pos_x, k_x, nb, W, bad);
+            const uint32_t ppos = min(__shfl_up_sync(full, pos_x, 1), endbit);
+            const int pk = __shfl_up_sync(full, k_x, 1);
+            again = lane > 0 && (ppos != pos || pk != k);
+            if (again) { pos = ppos; k = pk; }
+            if (!__any_sync(full, again)) break;
+        }
+        uint32_t nin = nb;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t on = __shfl_up_sync(full, nin, d);
+            if (lane >= d) nin += on;
+        }
+        const uint32_t all = __shfl_sync(full, nin, 31);
+        W.m = min(nin - nb, total);
+        ac_first_span<true>(tab, base, pos, k, my_end, Ss, Se, pos_x, k_x, nb, W, bad);
+        if (all < total) bad = true;                                         // the stream ends before the last block
+    }
+    if (__any_sync(full, bad) && lane == 0) atomicMin(&P.status[img], kErrCorrupt);
+}
+
+// ---------------------------------------------------------------------------------------
+// AC refinements of scans that are one restart interval.  One CTA per listed (image,
+// component), one warp per refinement scan of that component that the call decodes (at most
+// four, in scan order).  Side data written per block is that of entropy_kernel's refinement
+// branch: {non-zero mask of the band after the scan, correction bits in reading order from bit
+// 63 down, newly non-zero positions, the positive ones among them}.
+//
+// The time of a scan is the number of instructions lane 0 executes per symbol (a warp or two
+// per scheduler: every instruction waits for the one before), so lane 0 only follows the chain:
+// Huffman symbol -> run r -> position of the (r+1)-th still-zero coefficient -> number of
+// correction bits passed -> next symbol.  For every symbol it leaves a record {bit position
+// behind the sign, new position, number of correction bits}; afterwards all lanes turn the
+// records of 32 blocks into the side data in parallel (one lane per block, reading sign and
+// correction bits back from the ring).
+//
+// A later refinement of the same component needs the masks the earlier one leaves, block by
+// block.  Both walk the same block grid in the same order, so the later warp runs behind the
+// earlier one instead of after it: every warp publishes the number of blocks whose side data it
+// has written (shared memory, after a fence), and a warp that depends on it waits, with a bounded
+// number of polls, until the blocks it is about to read are there.  Producer and consumer share
+// a CTA, so both are resident while either waits.
+// ---------------------------------------------------------------------------------------
+constexpr int kGroupWarps = 4;           // refinement scans of one component in one call (pcr_open admits four)
+constexpr int kChainRing = 128;          // words of bitstream per warp in shared memory
+constexpr int kChainRecs = 320;          // symbol records per batch of blocks
+constexpr uint32_t kChainBlockWords = 44;   // a block never needs more: 63 symbols of at most 17 bits, 3 sixteen-zero runs, one run length, 63 correction bits
+constexpr uint32_t kSpinLimit = 1u << 22;   // polls (of at least 64 ns) before a wait gives up
+constexpr int kErrTimeout = -4;
+
+struct ChainBits {
+    const uint32_t* ring;
+    uint32_t w0, w1, w2;   // the word the next bit lies in and the two after it
+    uint32_t o;            // bits of w0 already consumed (0..31)
+    uint32_t rd;           // ring word that follows w2 (absolute word index)
+    uint32_t base;         // first word of the interval
+    __device__ __forceinline__ void init(const uint32_t* r, uint32_t first, uint32_t lead) {
+        ring = r;
+        base = first;
+        w0 = r[first & (kChainRing - 1)]; w1 = r[(first + 1) & (kChainRing - 1)]; w2 = r[(first + 2) & (kChainRing - 1)];
+        rd = first + 3;
+        o = lead;
+    }
+    __device__ __forceinline__ uint32_t win() const { return __funnelshift_l(w1, w0, o); }   // the next 32 bits
+    __device__ __forceinline__ void skip(uint32_t n) {        // n <= 32
+        o += n;
+        if (o >= 32u) { o -= 32u; w0 = w1; w1 = w2; w2 = ring[rd & (kChainRing - 1)]; ++rd; }
+    }
+    __device__ __forceinline__ uint32_t pos() const { return (rd - 3u - base) * 32u + o; }   // bits from the first bit of the interval's first word
+};
+
+// the n bits (1..32) at bit position p (counted from the first bit of word `base`) of the ring
+__device__ __forceinline__ uint32_t ring_bits(const uint32_t* ring, uint32_t base, uint32_t p, uint32_t n) {
+    const uint32_t a = ring[(base + (p >> 5)) & (kChainRing - 1)], b = ring[(base + (p >> 5) + 1u) & (kChainRing - 1)];
+    return __funnelshift_l(b, a, p & 31u) >> (32u - n);
+}
+
+// Polls *flag until it reaches `need`; false after `limit` polls.
+__device__ __forceinline__ bool wait_at_least(const volatile uint32_t* flag, uint32_t need, uint32_t limit) {
+    for (uint32_t i = 0; i < limit; ++i) {
+        if (*flag >= need) return true;
+        __nanosleep(64);
+    }
+    return false;
+}
+
+struct ChainShared {
+    HuffTab tab;
+    uint32_t ring[kChainRing];
+    uint64_t h[32];
+    uint2 rec[kChainRecs];             // {bit position behind the sign bit, corrections | position << 7 | new << 13}
+    uint32_t first[33];                // first record of each block of the batch
+};
+
+__global__ void __launch_bounds__(32 * kGroupWarps) ac_refine_group_kernel(Params P, FinalizeList fl, const uint32_t* __restrict__ list) {
+    __shared__ ChainShared s_sh[kGroupWarps];
+    __shared__ uint32_t s_progress[kGroupWarps];              // blocks whose side data each warp has written
+    const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t entry = list[blockIdx.x];
+    const int c = (int)(entry >> 28), img = (int)(entry & 0x0FFFFFFFu);
+    if (threadIdx.x < kGroupWarps) s_progress[threadIdx.x] = 0;
+    __syncthreads();
+    if (wid >= fl.n[c]) return;                                // whole warp: fewer scans than warps
+    const int s = fl.scan[c][wid];
+    const uint32_t si = (uint32_t)s * (uint32_t)P.N + (uint32_t)img;
+    const ScanDesc sd = P.scans[si];
+    const ScanScript sc = P.script[s];
+    const ImgDesc im = P.imgs[img];
+    const Geometry g = make_geometry(im);
+    const uint32_t Ss = (uint32_t)sc.Ss, Se = (uint32_t)sc.Se;
+    const uint32_t mcu_w = g.ubw[c], total = g.ubw[c] * g.ubh[c], bw = g.bw[c];
+    const unsigned full = 0xffffffffu;
+    ChainShared& sh = s_sh[wid];
+    volatile uint32_t* my_progress = &s_progress[wid];
+    build_hufftab(sh.tab, P.rec + sd.tab_off[0], lane);
+    const uint32_t* segtab = P.seg_start + sd.seg_base;
+    const uint32_t bstart = segtab[0], bend = segtab[1] - 2u;
+    if (bstart < sd.data_off || bend > sd.data_end || bend < bstart) {
+        if (lane == 0) { atomicMin(&P.status[img], kErrCorrupt); *my_progress = 0xFFFFFFFFu; }   // nobody waits for this scan
+        return;
+    }
+    const uint32_t* words = reinterpret_cast<const uint32_t*>(P.ubuf);
+    const uint32_t rd0 = bstart >> 2, lead = 8u * (bstart & 3u);
+    const uint32_t limit = lead + 8u * (bend - bstart);        // first bit behind the interval, counted from word rd0
+    const uint32_t wlim = ((bend + 3u) >> 2) + 2u;             // words beyond are not read (zeros instead)
+    // masks of the positions that are already non-zero: the union of up to four earlier scans; a
+    // source that this CTA decodes itself is waited for (prod* = its progress word)
+    const ScanAux ax = P.saux[s];
+    const uint64_t band = low_mask((int)Se + 1) & ~low_mask((int)Ss);
+    const uint64_t* src0 = nullptr; const uint64_t* src1 = nullptr; const uint64_t* src2 = nullptr; const uint64_t* src3 = nullptr;
+    uint32_t st0 = 0, st1 = 0, st2 = 0, st3 = 0;
+    const volatile uint32_t* prod0 = nullptr; const volatile uint32_t* prod1 = nullptr;
+    {
+        auto producer = [&](int scan) -> const volatile uint32_t* {
+            for (int w = 0; w < wid; ++w) if (fl.scan[c][w] == scan) return &s_progress[w];
+            return nullptr;
+        };
+        auto note = [&](const volatile uint32_t* p) { if (p) { if (!prod0) prod0 = p; else prod1 = p; } };
+        const ScanAux x0 = P.saux[ax.src[0]];
+        src0 = P.aux + x0.base + g.loff[c] * x0.stride; st0 = x0.stride; note(producer(ax.src[0]));
+        if (ax.nsrc > 1) { const ScanAux x = P.saux[ax.src[1]]; src1 = P.aux + x.base + g.loff[c] * x.stride; st1 = x.stride; note(producer(ax.src[1])); }
+        if (ax.nsrc > 2) { const ScanAux x = P.saux[ax.src[2]]; src2 = P.aux + x.base + g.loff[c] * x.stride; st2 = x.stride; note(producer(ax.src[2])); }
+        if (ax.nsrc > 3) { const ScanAux x = P.saux[ax.src[3]]; src3 = P.aux + x.base + g.loff[c] * x.stride; st3 = x.stride; note(producer(ax.src[3])); }
+    }
+    uint64_t* outp = P.aux + ax.base + g.loff[c] * 4ull;
+    uint32_t* ring = sh.ring;
+    const uint16_t* lut = sh.tab.lut;
+    uint32_t wr = rd0;                                         // next word to fetch
+    ChainBits B;
+    B.ring = ring; B.w0 = B.w1 = B.w2 = 0; B.o = 0; B.rd = rd0; B.base = rd0;
+    uint32_t eobrun = 0, m = 0;
+    int err = 0;
+    bool primed = false;
+    while (m < total && !err) {
+        // ---- all lanes: the masks of the next 32 blocks (once their producers have written them), the ring topped up
+        const uint32_t nblk = min(32u, total - m);
+        if (prod0 && !wait_at_least(prod0, m + nblk, kSpinLimit)) { err = kErrTimeout; break; }
+        if (prod1 && !wait_at_least(prod1, m + nblk, kSpinLimit)) { err = kErrTimeout; break; }
+        __threadfence();
+        uint32_t bi = 0;
+        if ((uint32_t)lane < nblk) {
+            const uint32_t x = m + lane, row = x / mcu_w;
+            bi = row * bw + (x - row * mcu_w);
+            uint64_t v = __ldcg(src0 + (uint64_t)bi * st0);    // not through L1: a line may hold blocks written later
+            if (src1) v |= __ldcg(src1 + (uint64_t)bi * st1);
+            if (src2) v |= __ldcg(src2 + (uint64_t)bi * st2);
+            if (src3) v |= __ldcg(src3 + (uint64_t)bi * st3);
+            sh.h[lane] = v & band;
+        }
+        const uint32_t rd_now = __shfl_sync(full, B.rd - (primed ? 3u : 0u), 0);   // lane 0's reader: w0 is the oldest word still in use
+        while (wr - rd_now + 32u <= (uint32_t)kChainRing) {
+            ring[(wr + lane) & (kChainRing - 1)] = wr + lane < wlim ? __ldg(words + wr + lane) : 0u;
+            wr += 32u;
+        }
+        __syncwarp(full);
+        // ---- lane 0: the chain
+        uint32_t nd = 0;
+        if (lane == 0) {
+            if (!primed) { B.init(ring, rd0, lead); primed = true; }
+            uint32_t nrec = 0;
+            for (; nd < nblk; ++nd) {
+                if (wr - B.rd < kChainBlockWords || nrec > (uint32_t)kChainRecs - 64u) break;   // fetch more / flush first
+                sh.first[nd] = nrec;
+                uint64_t Hs = sh.h[nd] >> Ss;                  // non-zero positions; bit 0 = the position that comes next
+                uint32_t k = Ss, rem = Se - Ss + 1u;
+                if (eobrun == 0) {
+                    while (rem) {
+                        const uint32_t win = B.win();
+                        uint32_t e = lut[win >> (32 - kLutBits)];
+                        if (e == 0) { e = huff_lookup(sh.tab, win); if (e == 0) { err = kErrCorrupt; break; } }
+                        const uint32_t len = e >> 8, rs = e & 255u;
+                        if (rs & 14u) { err = kErrCorrupt; break; }   // a refinement symbol has size 0 or 1
+                        const uint32_t newc = rs & 1u, r = rs >> 4;
+                        if (rs < 0xF0u && !newc) {             // end of band for this block and eobrun - 1 more
+                            eobrun = 1u << r;
+                            if (r) eobrun += (win << len) >> (32u - r);
+                            B.skip(len + r);
+                            break;
+                        }
+                        B.skip(len + newc);                    // the sign comes before the correction bits
+                        // distance d of the (r+1)-th position that is still zero: d = r + (non-zero positions up to d),
+                        // iterated from d = r; the count reached is the number of correction bits that follow
+                        uint32_t d = r, cnt = 0;
+                        {
+                            const uint32_t lo = (uint32_t)Hs;
+                            bool settled = false;
+                            while (d < 32u) {
+                                cnt = (uint32_t)__popc(lo & ((2u << d) - 1u));
+                                if (r + cnt == d) { settled = true; break; }
+                                d = r + cnt;
+                            }
+                            while (!settled) {                 // beyond the low word (d <= 78)
+                                cnt = (uint32_t)__popcll(Hs & low_mask((int)d + 1));
+                                if (r + cnt == d) break;
+                                d = r + cnt;
+                            }
+                        }
+                        uint32_t flag = newc;
+                        if (d >= rem) { d = rem; cnt = (uint32_t)__popcll(Hs); flag = 0; }   // past the band: nothing new
+                        sh.rec[nrec++] = make_uint2(B.pos(), cnt | ((k + d) << 7) | (flag << 13));
+                        if (cnt > 32u) { B.skip(32u); B.skip(cnt - 32u); } else B.skip(cnt);
+                        const uint32_t adv = min(d + 1u, rem);
+                        k += adv;
+                        rem -= adv;
+                        Hs >>= adv;                            // adv <= 63
+                    }
+                }
+                if (err) break;
+                if (rem) {                                     // inside an end-of-band run: corrections for the rest of the band
+                    const uint32_t cnt = (uint32_t)__popcll(Hs);
+                    sh.rec[nrec++] = make_uint2(B.pos(), cnt);
+                    if (cnt > 32u) { B.skip(32u); B.skip(cnt - 32u); } else B.skip(cnt);
+                    --eobrun;
+                }
+                if (B.pos() > limit) { err = kErrCorrupt; break; }   // read past the end of the interval
+            }
+            sh.first[nd] = nrec;
+        }
+        __syncwarp(full);
+        nd = __shfl_sync(full, nd, 0);
+        err = __shfl_sync(full, err, 0);
+        // ---- all lanes: one block each, records -> side data
+        bool over = false;
+        if ((uint32_t)lane < nd) {
+            uint64_t cstr = 0, Nw = 0, NS = 0;
+            uint32_t cn = 0;
+            for (uint32_t i = sh.first[lane]; i < sh.first[lane + 1]; ++i) {
+                const uint2 rc = sh.rec[i];
+                uint32_t n = rc.y & 127u;
+                if (rc.y >> 13) {
+                    const uint64_t bit = 1ull << ((rc.y >> 7) & 63u);
+                    Nw |= bit;
+                    if (ring_bits(ring, rd0, rc.x - 1u, 1u)) NS |= bit;
+                }
+                if (cn + n > 64u) { over = true; break; }
+                cn += n;
+                uint32_t p = rc.x;
+                while (n) {
+                    const uint32_t q = min(n, 32u);
+                    cstr = (cstr << q) | (uint64_t)ring_bits(ring, rd0, p, q);
+                    p += q; n -= q;
+                }
+            }
+            if (cn) cstr <<= 64u - cn;                         // first correction bit at bit 63
+            ulonglong2* o = reinterpret_cast<ulonglong2*>(outp + (uint64_t)bi * 4);
+            o[0] = make_ulonglong2((sh.h[lane] | Nw), cstr);
+            o[1] = make_ulonglong2(Nw, NS);
+        }
+        if (__any_sync(full, over)) err = kErrCorrupt;
+        m += nd;
+        __threadfence();                                       // the side data before the count
+        __syncwarp(full);
+        if (lane == 0) *my_progress = m;
+    }
+    if (lane == 0) {
+        *my_progress = 0xFFFFFFFFu;                            // a scan that failed must not keep a later one waiting
+        if (err) atomicMin(&P.status[img], err);
+    }
+}
+
+// Test hook: the bounded wait on a flag that nothing sets; *result = 1 if it gave up as it should.
+__global__ void bounded_wait_probe_kernel(uint32_t limit, int* result) {
+    __shared__ uint32_t s_flag;
+    if (threadIdx.x == 0) s_flag = 0;
+    __syncthreads();
+    const bool ok = wait_at_least(&s_flag, 1u, limit);
+    if (threadIdx.x == 0) *result = ok ? 0 : 1;
+}
+
+}  // namespace pcr
