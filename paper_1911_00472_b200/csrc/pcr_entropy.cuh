@@ -34,17 +34,20 @@ constexpr int kErrCorrupt = -3;
 constexpr int kLutBits = PCR_LUT_BITS;
 constexpr int kEntropyWarps = PCR_ENTROPY_WARPS;
 
-// Decoder tables of one Huffman table: a direct lookup on the next kLutBits bits for short
+// Decoder tables of one Huffman table: a direct lookup on the next kBits bits for short
 // codes, and the canonical first-code / count / index triple per length for the rest.
-struct HuffTab {
-    uint16_t lut[1 << kLutBits];  // (length << 8) | symbol, 0 = longer than kLutBits (or undefined)
+template <int kBits>
+struct HuffTabT {
+    uint16_t lut[1 << kBits];  // (length << 8) | symbol, 0 = longer than kBits (or undefined)
     uint32_t first[17];
     uint16_t cnt[17];
     uint16_t idx[17];
     uint8_t vals[256];
 };
+using HuffTab = HuffTabT<kLutBits>;
 
-__device__ __forceinline__ void build_hufftab(HuffTab& t, const uint8_t* __restrict__ dht, int lane) {
+template <int kBits>
+__device__ __forceinline__ void build_hufftab(HuffTabT<kBits>& t, const uint8_t* __restrict__ dht, int lane) {
     // dht: 16 length counts, then the symbol values in code order
     uint32_t code = 0, p = 0;
     for (int l = 1; l <= 16; ++l) {
@@ -56,16 +59,16 @@ __device__ __forceinline__ void build_hufftab(HuffTab& t, const uint8_t* __restr
     const uint32_t nvals = min(p, 256u);
     for (uint32_t j = lane; j < nvals; j += 32) t.vals[j] = dht[16 + j];
     uint32_t* lw = reinterpret_cast<uint32_t*>(t.lut);
-    for (int e = lane; e < (1 << kLutBits) / 2; e += 32) lw[e] = 0;
+    for (int e = lane; e < (1 << kBits) / 2; e += 32) lw[e] = 0;
     __syncwarp();
-    // every symbol with a short code fills its 2^(kLutBits - length) entries, all lanes together
+    // every symbol with a short code fills its 2^(kBits - length) entries, all lanes together
     uint32_t j = 0;
-    for (int l = 1; l <= kLutBits; ++l) {
-        const uint32_t c = t.cnt[l], f = t.first[l], span = 1u << (kLutBits - l);
+    for (int l = 1; l <= kBits; ++l) {
+        const uint32_t c = t.cnt[l], f = t.first[l], span = 1u << (kBits - l);
         for (uint32_t i = 0; i < c && j < nvals; ++i, ++j) {
-            const uint32_t base = (f + i) << (kLutBits - l);
+            const uint32_t base = (f + i) << (kBits - l);
             const uint16_t entry = (uint16_t)(((uint32_t)l << 8) | t.vals[j]);
-            if (base + span <= (1u << kLutBits))
+            if (base + span <= (1u << kBits))
                 for (uint32_t e = lane; e < span; e += 32) t.lut[base + e] = entry;
         }
     }
@@ -141,11 +144,12 @@ struct BitReader {
 };
 
 // Huffman symbol at the top of the 32-bit window; returns (length << 8) | symbol, 0 if undefined
-__device__ __forceinline__ uint32_t huff_lookup(const HuffTab& t, uint32_t win) {
-    uint32_t e = t.lut[win >> (32 - kLutBits)];
+template <int kBits>
+__device__ __forceinline__ uint32_t huff_lookup(const HuffTabT<kBits>& t, uint32_t win) {
+    uint32_t e = t.lut[win >> (32 - kBits)];
     if (e) return e;
     const uint32_t w16 = win >> 16;
-    for (int l = kLutBits + 1; l <= 16; ++l) {
+    for (int l = kBits + 1; l <= 16; ++l) {
         uint32_t d = (w16 >> (16 - l)) - t.first[l];
         if (d < t.cnt[l]) return ((uint32_t)l << 8) | t.vals[(t.idx[l] + d) & 255u];   // (index masked: damaged tables stay in bounds)
     }

@@ -624,8 +624,8 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
                 r->long_count[(size_t)g * G + s] = (uint32_t)longs.size() - r->long_begin[(size_t)g * G + s];
             }
         r->group_begin[g] = (uint32_t)groups.size();
-        for (uint32_t pos = r->slice_img[g]; pos < r->slice_img[g + 1]; ++pos)
-            for (int c = 0; c < 3; ++c)
+        for (int c = 0; c < 3; ++c)                            // luminance first: its chains are the longest
+            for (uint32_t pos = r->slice_img[g]; pos < r->slice_img[g + 1]; ++pos)
                 if (grouped[(size_t)order[pos] * 3 + c]) groups.push_back(((uint32_t)c << 28) | order[pos]);
         r->group_count[g] = (uint32_t)groups.size() - r->group_begin[g];
     }
@@ -904,6 +904,13 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
         ++g_launches;
         return 1;
     };
+    // the restart-interval index (and unstuffed copy) of waves w0.. is complete before what follows on q
+    auto wait_index_from = [&](int w0, cudaStream_t q) -> bool {
+        if (!pipelined) return true;                 // indexed up front on the same stream
+        for (int w = std::max(w0, 1); w < rec->n_waves; ++w)
+            if (indexed[w] && cudaStreamWaitEvent(q, rec->ev_index[w], 0) != cudaSuccess) return false;
+        return true;
+    };
     auto run_stage = [&](int stage, int g, cudaStream_t q) -> bool {
         const uint32_t i0 = rec->slice_img[g], i1 = rec->slice_img[g + 1];
         const uint32_t u0 = rec->slice_unit[g], nu = rec->slice_unit[g + 1] - u0;
@@ -934,24 +941,26 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
                     if (cudaStreamWaitEvent(q, rec->ev_index[w], 0) != cudaSuccess) return false;
                 }
             }
+            const ScanScript& first = rec->script[rec->wave_scans[w][0]];
+            const bool sequential = first.Ss == 0 && first.Se == 63;   // a baseline record: its one scan is sequential
+            // the items of the wave's scans lie one after the other
             uint32_t begin = 0, count = 0;
-            bool any = false;
             for (int s : rec->wave_scans[w]) {
                 if (s >= k) break;   // scans of a wave are stored in ascending order
                 if (s < k0) continue;
-                if (!any) { begin = rec->item_begin[(size_t)g * G + s]; any = true; }
+                if (!count) begin = rec->item_begin[(size_t)g * G + s];
                 count += rec->item_count[(size_t)g * G + s];
             }
-            const ScanScript& first = rec->script[rec->wave_scans[w][0]];
-            if (count && first.Ss == 0 && first.Se == 63) {        // a baseline record: its one scan is sequential
+            if (count && sequential) {
                 if (targs) sequential_kernel<true><<<(count + kSeqWarps - 1) / kSeqWarps, 32 * kSeqWarps, 0, q>>>(P, begin, count);
                 else sequential_kernel<false><<<(count + kSeqWarps - 1) / kSeqWarps, 32 * kSeqWarps, 0, q>>>(P, begin, count);
                 ++g_launches;
                 return true;
             }
             if (count) {
-                if (targs) entropy_kernel<true><<<(count + kEntropyWarps - 1) / kEntropyWarps, 32 * kEntropyWarps, 0, q>>>(P, begin, count);
-                else entropy_kernel<false><<<(count + kEntropyWarps - 1) / kEntropyWarps, 32 * kEntropyWarps, 0, q>>>(P, begin, count);
+                const unsigned nb = (count + kEntropyWarps - 1) / kEntropyWarps;
+                if (targs) entropy_kernel<true><<<nb, 32 * kEntropyWarps, 0, q>>>(P, begin, count);
+                else entropy_kernel<false><<<nb, 32 * kEntropyWarps, 0, q>>>(P, begin, count);
                 ++g_launches;
             }
             // scans that are one long restart interval: the first passes of the wave (a contiguous run
@@ -974,8 +983,9 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
             // depends on first passes, which every wave-0 launch above has finished, and on earlier
             // refinements of its component, which run in the same CTA) ...
             if (w == first_refine_wave && rec->group_count[g]) {
+                if (!wait_index_from(w + 1, q)) return false;    // the launch reads scans of later waves too
                 int warps = std::max(fl.n[0], std::max(fl.n[1], fl.n[2]));
-                ac_refine_group_kernel<<<rec->group_count[g], 32 * warps, 0, q>>>(P, fl, rec->d_group + rec->group_begin[g]);
+                ac_refine_group_kernel<<<rec->group_count[g], 32 * warps, (size_t)warps * sizeof(ChainShared), q>>>(P, fl, rec->d_group + rec->group_begin[g]);
                 ++g_launches;
             }
             // ... and the DC refinement scans of every record

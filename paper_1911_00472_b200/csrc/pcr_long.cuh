@@ -369,7 +369,8 @@ __global__ void __launch_bounds__(32 * kLongWarps) first_pass_long_kernel(Params
 // ---------------------------------------------------------------------------------------
 constexpr int kGroupWarps = 4;           // refinement scans of one component in one call (pcr_open admits four)
 constexpr int kChainRing = 128;          // words of bitstream per warp in shared memory
-constexpr int kChainRecs = 320;          // symbol records per batch of blocks
+constexpr int kChainRecs = 192;          // symbol records per batch of blocks
+constexpr int kChainLutBits = 9;         // refinement alphabets are small (runs 0..15 with size 0 or 1): short codes
 constexpr uint32_t kChainBlockWords = 44;   // a block never needs more: 63 symbols of at most 17 bits, 3 sixteen-zero runs, one run length, 63 correction bits
 constexpr uint32_t kSpinLimit = 1u << 22;   // polls (of at least 64 ns) before a wait gives up
 constexpr int kErrTimeout = -4;
@@ -411,7 +412,7 @@ __device__ __forceinline__ bool wait_at_least(const volatile uint32_t* flag, uin
 }
 
 struct ChainShared {
-    HuffTab tab;
+    HuffTabT<kChainLutBits> tab;
     uint32_t ring[kChainRing];
     uint64_t h[32];
     uint2 rec[kChainRecs];             // {bit position behind the sign bit, corrections | position << 7 | new << 13}
@@ -419,7 +420,8 @@ struct ChainShared {
 };
 
 __global__ void __launch_bounds__(32 * kGroupWarps) ac_refine_group_kernel(Params P, FinalizeList fl, const uint32_t* __restrict__ list) {
-    __shared__ ChainShared s_sh[kGroupWarps];
+    extern __shared__ __align__(16) unsigned char s_dyn[];     // one ChainShared per warp of the launch
+    ChainShared* s_sh = reinterpret_cast<ChainShared*>(s_dyn);
     __shared__ uint32_t s_progress[kGroupWarps];              // blocks whose side data each warp has written
     const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t entry = list[blockIdx.x];
@@ -512,7 +514,7 @@ __global__ void __launch_bounds__(32 * kGroupWarps) ac_refine_group_kernel(Param
                 if (eobrun == 0) {
                     while (rem) {
                         const uint32_t win = B.win();
-                        uint32_t e = lut[win >> (32 - kLutBits)];
+                        uint32_t e = lut[win >> (32 - kChainLutBits)];
                         if (e == 0) { e = huff_lookup(sh.tab, win); if (e == 0) { err = kErrCorrupt; break; } }
                         const uint32_t len = e >> 8, rs = e & 255u;
                         if (rs & 14u) { err = kErrCorrupt; break; }   // a refinement symbol has size 0 or 1
