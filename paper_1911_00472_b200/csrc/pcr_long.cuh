@@ -17,11 +17,12 @@
 //    the true beginning, so after round r lanes 0..r are exact).  A prefix sum of the blocks each
 //    lane finished (and of the DC differences per component) gives every lane its first block and
 //    its predictors, and a last pass decodes once more and writes.
-//  * ac_refine_chain_kernel: an AC refinement cannot be entered in the middle (how many correction
+//  * ac_refine_group_kernel: an AC refinement cannot be entered in the middle (how many correction
 //    bits follow a symbol depends on which coefficients of the block are already non-zero, i.e. on
-//    the block number).  One warp per (scan, image): lane 0 walks the chain with ordinary branches
-//    (no other lane shares its instruction stream), the other lanes fetch the bitstream into a
-//    shared-memory ring, gather the masks of the next 32 blocks and write the side data out.
+//    the block number).  One warp per scan: lane 0 walks the chain with ordinary branches (no other
+//    lane shares its instruction stream), the other lanes fetch the bitstream into a shared-memory
+//    ring, gather the masks of the next 32 blocks and turn lane 0's symbol records into side data.
+//    The refinements of one component share a CTA and run behind one another, block by block.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
