@@ -306,12 +306,20 @@ static int decode_scan(jdec* J, const scan_hdr* S, const uint8_t* data, size_t n
     return ORC_OK;
 }
 
+/* T.81 A.1.1 / A.2: component c has ceil(W * Hc / Hmax) x ceil(H * Vc / Vmax) samples; an
+ * interleaved MCU holds Hc x Vc blocks of it, so the MCU-padded grid is (mx * Hc) x (my * Vc) blocks
+ * with mx = ceil(W / (8 Hmax)).  A frame with one component is never interleaved: its grid is the
+ * unpadded one and its sampling factors play no role (taken as 1 x 1). */
 static void set_geometry(jdec* J) {
-    J->mx = (J->W + 15) / 16; J->my = (J->H + 15) / 16;
+    int hmax = 1, vmax = 1;
+    if (J->ncomp == 1) { J->hs[0] = 1; J->vs[0] = 1; }
+    for (int c = 0; c < J->ncomp; ++c) { if (J->hs[c] > hmax) hmax = J->hs[c]; if (J->vs[c] > vmax) vmax = J->vs[c]; }
+    J->mx = (J->W + 8 * hmax - 1) / (8 * hmax); J->my = (J->H + 8 * vmax - 1) / (8 * vmax);
     size_t off = 0;
     for (int c = 0; c < 3; ++c) {
+        if (c >= J->ncomp) { J->bw[c] = J->bh[c] = J->ubw[c] = J->ubh[c] = 0; J->coff[c] = off; continue; }
         J->bw[c] = J->mx * J->hs[c]; J->bh[c] = J->my * J->vs[c];
-        int wc = (J->W * J->hs[c] + 1) / 2, hc = (J->H * J->vs[c] + 1) / 2;
+        int wc = (J->W * J->hs[c] + hmax - 1) / hmax, hc = (J->H * J->vs[c] + vmax - 1) / vmax;
         J->ubw[c] = (wc + 7) / 8; J->ubh[c] = (hc + 7) / 8;
         J->coff[c] = off; off += (size_t)J->bw[c] * J->bh[c];
     }
@@ -350,13 +358,14 @@ static int jpeg_decode_coeffs(jdec* J, const uint8_t* d, size_t n, int16_t* coef
             J->sequential = mk == 0xC0;
             if (sl < 6 || s[0] != 8) return ORC_E_UNSUPPORTED;
             J->H = (s[1] << 8) | s[2]; J->W = (s[3] << 8) | s[4]; J->ncomp = s[5];
-            if (J->ncomp != 3 || sl < 6 + 9 || J->W == 0 || J->H == 0) return ORC_E_UNSUPPORTED;
-            for (int c = 0; c < 3; ++c) {
+            if ((J->ncomp != 3 && J->ncomp != 1) || sl < (size_t)(6 + 3 * J->ncomp) || J->W == 0 || J->H == 0) return ORC_E_UNSUPPORTED;
+            for (int c = 0; c < J->ncomp; ++c) {
                 J->cid[c] = s[6 + 3 * c]; J->hs[c] = s[7 + 3 * c] >> 4; J->vs[c] = s[7 + 3 * c] & 15; J->tq[c] = s[8 + 3 * c];
                 if (J->tq[c] > 3) return ORC_E_CORRUPT;
+                if (J->hs[c] < 1 || J->hs[c] > 2 || J->vs[c] < 1 || J->vs[c] > 2) return ORC_E_UNSUPPORTED;
             }
-            if (J->hs[0] != 2 || J->vs[0] != 2 || J->hs[1] != 1 || J->vs[1] != 1 || J->hs[2] != 1 || J->vs[2] != 1)
-                return ORC_E_UNSUPPORTED;               /* 4:2:0 only */
+            /* luminance 1 or 2 blocks per MCU in each direction, chroma one block: 4:4:4, 4:2:2, 4:4:0, 4:2:0, grey */
+            if (J->ncomp == 3 && (J->hs[1] != 1 || J->vs[1] != 1 || J->hs[2] != 1 || J->vs[2] != 1)) return ORC_E_UNSUPPORTED;
             set_geometry(J);
             if (J->nblocks * 64 != ncoef) return ORC_E_ARG;
             J->coef = coef;
@@ -388,7 +397,7 @@ static int jpeg_decode_coeffs(jdec* J, const uint8_t* d, size_t n, int16_t* coef
             if (S.ns < 1 || S.ns > 3 || sl != (size_t)(4 + 2 * S.ns)) return ORC_E_CORRUPT;
             for (int i = 0; i < S.ns; ++i) {
                 int id = s[1 + 2 * i], found = -1;
-                for (int c = 0; c < 3; ++c) if (J->cid[c] == id) found = c;
+                for (int c = 0; c < J->ncomp; ++c) if (J->cid[c] == id) found = c;
                 if (found < 0) return ORC_E_CORRUPT;
                 S.ci[i] = found; S.td[i] = s[2 + 2 * i] >> 4; S.ta[i] = s[2 + 2 * i] & 15;
                 if (S.td[i] > 3 || S.ta[i] > 3) return ORC_E_CORRUPT;
@@ -396,7 +405,7 @@ static int jpeg_decode_coeffs(jdec* J, const uint8_t* d, size_t n, int16_t* coef
             S.Ss = s[1 + 2 * S.ns]; S.Se = s[2 + 2 * S.ns]; S.Ah = s[3 + 2 * S.ns] >> 4; S.Al = s[3 + 2 * S.ns] & 15;
             if (S.Ss > S.Se || S.Se > 63 || S.Al > 13) return ORC_E_CORRUPT;
             if (J->sequential) {                                   /* one kind of scan: everything of its components */
-                if (S.Ss != 0 || S.Se != 63 || S.Ah != 0 || S.Al != 0 || S.ns != 3) return ORC_E_UNSUPPORTED;
+                if (S.Ss != 0 || S.Se != 63 || S.Ah != 0 || S.Al != 0 || S.ns != J->ncomp) return ORC_E_UNSUPPORTED;
                 for (int i = 0; i < S.ns; ++i)
                     if (!J->dc[S.td[i]].defined || !J->ac[S.ta[i]].defined) return ORC_E_CORRUPT;
             } else if (S.Ss == 0 && S.Se != 0) return ORC_E_CORRUPT;  /* DC and AC never share a progressive scan */
@@ -479,20 +488,25 @@ void oracle_ycc_to_rgb_array(const uint8_t* ycc, size_t n, uint8_t* rgb) {
 }
 
 /* coefficients (canonical layout) + per-component zigzag quantisers -> packed RGB (H*W*3).
- * planes, if not NULL, receives the three sample planes over the padded grids
- * (Y: 16mx x 16my, then Cb and Cr: 8mx x 8my each). */
-int oracle_pixels_from_coeffs(const int16_t* coef, uint32_t W, uint32_t H, const uint16_t* qy, const uint16_t* qcb,
-                              const uint16_t* qcr, uint8_t* rgb, uint8_t* planes) {
+ * hs x vs: luminance blocks per MCU (chroma has one), ncomp 3 or 1.  Pixel (x, y) takes the
+ * chroma sample (x / hs, y / vs) (replication); a greyscale image has no chroma: every pixel is
+ * (Y, Y, Y), which is what the colour formula gives for Cb = Cr = 128.
+ * planes, if not NULL, receives the sample planes over the padded grids
+ * (Y: 8 hs mx x 8 vs my, then Cb and Cr: 8mx x 8my each). */
+int oracle_pixels_from_coeffs_s(const int16_t* coef, uint32_t W, uint32_t H, int hs, int vs, int ncomp, const uint16_t* qy,
+                                const uint16_t* qcb, const uint16_t* qcr, uint8_t* rgb, uint8_t* planes) {
     init_consts();
-    if (!coef || W == 0 || H == 0) return ORC_E_ARG;
-    int mx = (int)((W + 15) / 16), my = (int)((H + 15) / 16);
-    int bw[3] = {2 * mx, mx, mx}, bh[3] = {2 * my, my, my};
-    size_t psz[3] = {(size_t)256 * mx * my, (size_t)64 * mx * my, (size_t)64 * mx * my};
+    if (!coef || W == 0 || H == 0 || (ncomp != 1 && ncomp != 3) || hs < 1 || hs > 2 || vs < 1 || vs > 2) return ORC_E_ARG;
+    if (ncomp == 1) { hs = 1; vs = 1; }
+    int mx = (int)((W + 8 * hs - 1) / (8 * hs)), my = (int)((H + 8 * vs - 1) / (8 * vs));
+    int bw[3] = {hs * mx, mx, mx}, bh[3] = {vs * my, my, my};
+    size_t psz[3] = {(size_t)64 * bw[0] * bh[0], (size_t)64 * mx * my, (size_t)64 * mx * my};
+    if (ncomp == 1) psz[1] = psz[2] = 0;
     uint8_t* own = planes ? NULL : (uint8_t*)malloc(psz[0] + psz[1] + psz[2]);
     uint8_t* pl[3]; pl[0] = planes ? planes : own; pl[1] = pl[0] + psz[0]; pl[2] = pl[1] + psz[1];
     const uint16_t* q[3] = {qy, qcb, qcr};
     size_t boff = 0;
-    for (int c = 0; c < 3; ++c) {
+    for (int c = 0; c < ncomp; ++c) {
         int pw = bw[c] * 8;
         for (int by = 0; by < bh[c]; ++by)
             for (int bx = 0; bx < bw[c]; ++bx) {
@@ -504,17 +518,25 @@ int oracle_pixels_from_coeffs(const int16_t* coef, uint32_t W, uint32_t H, const
         boff += (size_t)bw[c] * bh[c];
     }
     if (rgb) {
-        int yw = 16 * mx, cw = 8 * mx;
+        int yw = 8 * bw[0], cw = 8 * mx;
         for (uint32_t y = 0; y < H; ++y)
             for (uint32_t x = 0; x < W; ++x) {
                 int Yv = pl[0][(size_t)y * yw + x];
-                int cb = pl[1][(size_t)(y >> 1) * cw + (x >> 1)];   /* 2x2 replication */
-                int cr = pl[2][(size_t)(y >> 1) * cw + (x >> 1)];
+                int cb = 128, cr = 128;
+                if (ncomp == 3) {
+                    cb = pl[1][(size_t)(y / (uint32_t)vs) * cw + (x / (uint32_t)hs)];   /* replication */
+                    cr = pl[2][(size_t)(y / (uint32_t)vs) * cw + (x / (uint32_t)hs)];
+                }
                 ycc_to_rgb(Yv, cb, cr, rgb + ((size_t)y * W + x) * 3);
             }
     }
     free(own);
     return ORC_OK;
+}
+
+int oracle_pixels_from_coeffs(const int16_t* coef, uint32_t W, uint32_t H, const uint16_t* qy, const uint16_t* qcb,
+                              const uint16_t* qcr, uint8_t* rgb, uint8_t* planes) {
+    return oracle_pixels_from_coeffs_s(coef, W, H, 2, 2, 3, qy, qcb, qcr, rgb, planes);
 }
 
 /* A progressive JPEG byte string -> coefficients (+ optional RGB and planes).
@@ -527,12 +549,41 @@ int oracle_jpeg_decode(const uint8_t* jpg, size_t n, int16_t* coef, size_t ncoef
     if (rc == ORC_OK) {
         if (W) *W = (uint32_t)J->W;
         if (H) *H = (uint32_t)J->H;
-        for (int c = 0; c < 3; ++c) if (!J->qdef[J->tq[c]]) rc = ORC_E_CORRUPT;
+        for (int c = 0; c < J->ncomp; ++c) if (!J->qdef[J->tq[c]]) rc = ORC_E_CORRUPT;
         if (rc == ORC_OK && (rgb || planes))
-            rc = oracle_pixels_from_coeffs(coef, (uint32_t)J->W, (uint32_t)J->H, J->q[J->tq[0]], J->q[J->tq[1]], J->q[J->tq[2]], rgb, planes);
+            rc = oracle_pixels_from_coeffs_s(coef, (uint32_t)J->W, (uint32_t)J->H, J->hs[0], J->vs[0], J->ncomp, J->q[J->tq[0]],
+                                             J->q[J->tq[J->ncomp == 3 ? 1 : 0]], J->q[J->tq[J->ncomp == 3 ? 2 : 0]], rgb, planes);
     }
     free(J);
     return rc;
+}
+
+/* frame size, luminance sampling and component count of a JPEG byte string (reads up to the frame header) */
+int oracle_jpeg_info(const uint8_t* d, size_t n, uint32_t* W, uint32_t* H, int* hs, int* vs, int* ncomp) {
+    size_t p = 2;
+    if (n < 4 || d[0] != 0xFF || d[1] != 0xD8) return ORC_E_FORMAT;
+    while (p + 4 <= n) {
+        if (d[p] != 0xFF) return ORC_E_CORRUPT;
+        int mk = d[p + 1];
+        if (mk == 0xFF) { ++p; continue; }
+        size_t L = ((size_t)d[p + 2] << 8) | d[p + 3];
+        if (mk == 0xC2 || mk == 0xC0) {
+            if (p + 12 > n) return ORC_E_CORRUPT;
+            *H = ((uint32_t)d[p + 5] << 8) | d[p + 6]; *W = ((uint32_t)d[p + 7] << 8) | d[p + 8];
+            *ncomp = d[p + 9];
+            *hs = *ncomp == 1 ? 1 : d[p + 11] >> 4; *vs = *ncomp == 1 ? 1 : d[p + 11] & 15;
+            return ORC_OK;
+        }
+        if (mk == 0xDA || mk == 0xD9) break;
+        p += 2 + L;
+    }
+    return ORC_E_FORMAT;
+}
+
+size_t oracle_num_blocks_s(uint32_t W, uint32_t H, int hs, int vs, int ncomp) {
+    if (ncomp == 1) { hs = 1; vs = 1; }
+    size_t mx = (W + 8 * (uint32_t)hs - 1) / (8 * (uint32_t)hs), my = (H + 8 * (uint32_t)vs - 1) / (8 * (uint32_t)vs);
+    return ((size_t)hs * vs + (ncomp == 3 ? 2 : 0)) * mx * my;
 }
 
 /* frame size of a JPEG byte string without decoding it (reads up to the SOF2 segment) */

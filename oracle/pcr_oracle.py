@@ -47,6 +47,10 @@ def _load():
             lib.oracle_jpeg_decode.argtypes = [vp, sz, vp, sz, vp, vp, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]
             lib.oracle_jpeg_dims.argtypes = [vp, sz, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]
             lib.oracle_pixels_from_coeffs.argtypes = [vp, C.c_uint32, C.c_uint32, vp, vp, vp, vp, vp]
+            lib.oracle_jpeg_info.argtypes = [vp, sz, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32), C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int)]
+            lib.oracle_pixels_from_coeffs_s.argtypes = [vp, C.c_uint32, C.c_uint32, C.c_int, C.c_int, C.c_int, vp, vp, vp, vp, vp]
+            lib.oracle_num_blocks_s.restype = sz
+            lib.oracle_num_blocks_s.argtypes = [C.c_uint32, C.c_uint32, C.c_int, C.c_int, C.c_int]
             lib.oracle_num_blocks.restype = sz
             lib.oracle_num_blocks.argtypes = [C.c_uint32, C.c_uint32]
             lib.oracle_block_idct.argtypes = [vp, vp, vp]
@@ -104,59 +108,78 @@ def reassemble(rec, i, k) -> bytes:
     return out.tobytes()
 
 
-def num_blocks(W, H) -> int:
-    return int(_load().oracle_num_blocks(W, H))
+def num_blocks(W, H, sampling=(2, 2, 3)) -> int:
+    """Blocks of the MCU-padded grids of all components; sampling = (hs, vs, components)."""
+    return int(_load().oracle_num_blocks_s(W, H, *sampling))
+
+
+def jpeg_info(jpg):
+    """(W, H, (hs, vs, components)) from the frame header of a JPEG byte string."""
+    a = _u8(jpg)
+    W, H = C.c_uint32(), C.c_uint32()
+    hs, vs, nc = C.c_int(), C.c_int(), C.c_int()
+    _chk(_load().oracle_jpeg_info(a.ctypes.data, a.size, C.byref(W), C.byref(H), C.byref(hs), C.byref(vs), C.byref(nc)))
+    return W.value, H.value, (hs.value, vs.value, nc.value)
+
+
+def image_sampling(rec, i):
+    """(hs, vs, components) of image i: read from the frame header at the head of its first chunk."""
+    return jpeg_info(reassemble(rec, i, 1))[2]
 
 
 def decode_image(rec, i, k, want_rgb=True):
     """Image i at fidelity k -> (coefficients (blocks, 64) int16 zigzag, RGB (H, W, 3) uint8 or None)."""
     rec = _u8(rec)
     W, H, _ = image_info(rec, i)
-    coef = np.empty((num_blocks(W, H), 64), dtype=np.int16)
+    coef = np.empty((num_blocks(W, H, image_sampling(rec, i)), 64), dtype=np.int16)
     rgb = np.empty((H, W, 3), dtype=np.uint8) if want_rgb else None
     _chk(_load().oracle_decode_image(rec.ctypes.data, rec.size, i, k, coef.ctypes.data, coef.size,
                                      rgb.ctypes.data if want_rgb else None))
     return coef, rgb
 
 
+def _split_planes(planes, W, H, sampling):
+    hs, vs, nc = sampling
+    mx, my = (W + 8 * hs - 1) // (8 * hs), (H + 8 * vs - 1) // (8 * vs)
+    ny = 64 * hs * vs * mx * my
+    Y = planes[:ny].reshape(8 * vs * my, 8 * hs * mx)
+    if nc == 1:
+        return (Y,)
+    Cb = planes[ny:ny + 64 * mx * my].reshape(8 * my, 8 * mx)
+    Cr = planes[ny + 64 * mx * my:].reshape(8 * my, 8 * mx)
+    return Y, Cb, Cr
+
+
 def jpeg_decode(jpg: bytes, want_planes=False):
     """A progressive JPEG byte string -> (coefficients, RGB[, (Y, Cb, Cr) padded planes])."""
     lib = _load()
     a = _u8(jpg)
-    W, H = C.c_uint32(), C.c_uint32()
-    _chk(lib.oracle_jpeg_dims(a.ctypes.data, a.size, C.byref(W), C.byref(H)))
-    W, H = W.value, H.value
-    coef = np.empty((num_blocks(W, H), 64), dtype=np.int16)
+    W, H, samp = jpeg_info(a)
+    nb = num_blocks(W, H, samp)
+    coef = np.empty((nb, 64), dtype=np.int16)
     rgb = np.empty((H, W, 3), dtype=np.uint8)
-    mx, my = (W + 15) // 16, (H + 15) // 16
-    planes = np.empty(384 * mx * my, dtype=np.uint8) if want_planes else None
+    planes = np.empty(64 * nb, dtype=np.uint8) if want_planes else None
     _chk(lib.oracle_jpeg_decode(a.ctypes.data, a.size, coef.ctypes.data, coef.size, rgb.ctypes.data,
                                 planes.ctypes.data if want_planes else None, None, None))
     if not want_planes:
         return coef, rgb
-    ny = 256 * mx * my
-    Y = planes[:ny].reshape(16 * my, 16 * mx)
-    Cb = planes[ny:ny + 64 * mx * my].reshape(8 * my, 8 * mx)
-    Cr = planes[ny + 64 * mx * my:].reshape(8 * my, 8 * mx)
-    return coef, rgb, (Y, Cb, Cr)
+    return coef, rgb, _split_planes(planes, W, H, samp)
 
 
-def pixels_from_coeffs(coef, W, H, qy_zz, qc_zz, want_planes=False):
+def pixels_from_coeffs(coef, W, H, qy_zz, qc_zz, want_planes=False, sampling=(2, 2, 3)):
     """Sequential-style decode of given coefficients: canonical (blocks, 64) int16 + zigzag-order
     quantisers -> RGB (H, W, 3)."""
     coef = np.ascontiguousarray(coef, dtype=np.int16)
     qy = np.ascontiguousarray(qy_zz, dtype=np.uint16)
     qc = np.ascontiguousarray(qc_zz, dtype=np.uint16)
     rgb = np.empty((H, W, 3), dtype=np.uint8)
-    mx, my = (W + 15) // 16, (H + 15) // 16
-    planes = np.empty(384 * mx * my, dtype=np.uint8) if want_planes else None
-    _chk(_load().oracle_pixels_from_coeffs(coef.ctypes.data, W, H, qy.ctypes.data, qc.ctypes.data, qc.ctypes.data,
-                                           rgb.ctypes.data, planes.ctypes.data if want_planes else None))
+    planes = np.empty(64 * num_blocks(W, H, sampling), dtype=np.uint8) if want_planes else None
+    _chk(_load().oracle_pixels_from_coeffs_s(coef.ctypes.data, W, H, sampling[0], sampling[1], sampling[2],
+                                             qy.ctypes.data, qc.ctypes.data, qc.ctypes.data,
+                                             rgb.ctypes.data, planes.ctypes.data if want_planes else None))
     if not want_planes:
         return rgb
-    ny = 256 * mx * my
-    return rgb, (planes[:ny].reshape(16 * my, 16 * mx), planes[ny:ny + 64 * mx * my].reshape(8 * my, 8 * mx),
-                 planes[ny + 64 * mx * my:].reshape(8 * my, 8 * mx))
+    return rgb, _split_planes(planes, W, H, sampling)
 
 
 def block_idct(coef_zz, q_zz) -> np.ndarray:

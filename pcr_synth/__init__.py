@@ -70,6 +70,7 @@ def _load():
             lib.synth_num_blocks.argtypes = [C.c_uint32, C.c_uint32]
             lib.synth_zigzag.argtypes = [C.c_void_p]
             lib.synth_set_script.argtypes = [C.c_void_p, C.c_int]
+            lib.synth_set_sampling.argtypes = [C.c_int, C.c_int, C.c_int]
             lib.synth_rgb_to_coeffs.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
             _lib = lib
     return _lib
@@ -153,6 +154,7 @@ class Record:
     def __init__(self, handle):
         self._lib = _load()
         self._h = C.c_void_p(handle)
+        self.sampling = _sampling          # (hs, vs, components) the record was made with
         n = C.c_size_t()
         p = self._lib.synth_record_bytes(self._h, C.byref(n))
         self.n_images = self._lib.synth_record_num_images(self._h)
@@ -268,13 +270,14 @@ def zigzag() -> np.ndarray:
     return out
 
 
-def block_grids(W: int, H: int):
-    """(padded, unpadded) block grids per component as [(bw, bh)] * 3, and block offsets."""
-    mx, my = (W + 15) // 16, (H + 15) // 16
-    padded = [(2 * mx, 2 * my), (mx, my), (mx, my)]
-    cw, ch = (W + 1) // 2, (H + 1) // 2
-    unp = [((W + 7) // 8, (H + 7) // 8), ((cw + 7) // 8, (ch + 7) // 8), ((cw + 7) // 8, (ch + 7) // 8)]
-    off = [0, padded[0][0] * padded[0][1], padded[0][0] * padded[0][1] + mx * my]
+def block_grids(W: int, H: int, sampling=(2, 2, 3)):
+    """(padded, unpadded) block grids per component as [(bw, bh)] * components, and block offsets."""
+    hs, vs, nc = sampling
+    mx, my = (W + 8 * hs - 1) // (8 * hs), (H + 8 * vs - 1) // (8 * vs)
+    padded = [(hs * mx, vs * my)] + [(mx, my)] * (nc - 1)
+    cw, ch = (W + hs - 1) // hs, (H + vs - 1) // vs
+    unp = [((W + 7) // 8, (H + 7) // 8)] + [((cw + 7) // 8, (ch + 7) // 8)] * (nc - 1)
+    off = [0, padded[0][0] * padded[0][1], padded[0][0] * padded[0][1] + mx * my][:nc]
     return padded, unp, off
 
 
@@ -326,6 +329,32 @@ SCRIPT_DEEP_14 = [((0, 1, 2), 0, 0, 0, 2), ((0,), 1, 9, 0, 3), ((0,), 10, 63, 0,
 
 # baseline (sequential) JPEG: one interleaved scan with the DC and all AC coefficients of every block
 SCRIPT_BASELINE = [((0, 1, 2), 0, 63, 0, 0)]
+
+
+_sampling = (2, 2, 3)
+
+
+class sampling:
+    """Context manager: records made inside have luminance sampling hs x vs (1 or 2 each; 2 x 2 =
+    4:2:0, 2 x 1 = 4:2:2, 1 x 1 = 4:4:4) and `components` components (1 = greyscale: the scans of
+    the chroma components drop out of the script).  Not thread safe (a process-wide setting)."""
+
+    def __init__(self, hs: int, vs: int, components: int = 3):
+        self.new = (1, 1, 1) if components == 1 else (hs, vs, components)
+
+    def __enter__(self):
+        global _sampling
+        self.old = _sampling
+        if _load().synth_set_sampling(*self.new) != 0:
+            raise ValueError("unsupported sampling")
+        _sampling = self.new
+        return self
+
+    def __exit__(self, *exc):
+        global _sampling
+        _load().synth_set_sampling(*self.old)
+        _sampling = self.old
+        return False
 
 
 class scan_script:

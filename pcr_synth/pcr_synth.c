@@ -63,8 +63,19 @@ typedef struct {
     uint64_t seed;
 } synth_image_spec;
 
+/* Chroma sampling of the images made from here on (process-wide, like the scan script): the
+ * luminance component has hs x vs blocks per MCU, the chroma components one each; ncomp = 1 makes
+ * greyscale images (one component, no MCU padding: a lone component is never interleaved). */
+static int g_hs = 2, g_vs = 2, g_nc = 3;
+int synth_set_sampling(int hs, int vs, int ncomp) {
+    if ((hs != 1 && hs != 2) || (vs != 1 && vs != 2) || (ncomp != 1 && ncomp != 3)) return -1;
+    g_hs = ncomp == 1 ? 1 : hs; g_vs = ncomp == 1 ? 1 : vs; g_nc = ncomp;
+    return 0;
+}
+
 typedef struct {
     int W, H, mx, my;
+    int hs, vs, nc;       /* luminance blocks per MCU (horizontal, vertical), components */
     int bw[3], bh[3];     /* padded block grid per component                    */
     int ubw[3], ubh[3];   /* unpadded block grid per component                  */
     size_t coff[3];       /* first block of each component in the image array   */
@@ -73,12 +84,13 @@ typedef struct {
 
 static void geom_init(geom_t* g, int W, int H) {
     g->W = W; g->H = H;
-    g->mx = (W + 15) / 16; g->my = (H + 15) / 16;
-    g->bw[0] = 2 * g->mx; g->bh[0] = 2 * g->my;
-    g->bw[1] = g->bw[2] = g->mx; g->bh[1] = g->bh[2] = g->my;
+    g->hs = g_hs; g->vs = g_vs; g->nc = g_nc;
+    g->mx = (W + 8 * g->hs - 1) / (8 * g->hs); g->my = (H + 8 * g->vs - 1) / (8 * g->vs);
+    g->bw[0] = g->hs * g->mx; g->bh[0] = g->vs * g->my;
+    g->bw[1] = g->bw[2] = g->nc == 3 ? g->mx : 0; g->bh[1] = g->bh[2] = g->nc == 3 ? g->my : 0;
     g->ubw[0] = (W + 7) / 8; g->ubh[0] = (H + 7) / 8;
-    int cw = (W + 1) / 2, ch = (H + 1) / 2;
-    g->ubw[1] = g->ubw[2] = (cw + 7) / 8; g->ubh[1] = g->ubh[2] = (ch + 7) / 8;
+    int cw = (W + g->hs - 1) / g->hs, ch = (H + g->vs - 1) / g->vs;
+    g->ubw[1] = g->ubw[2] = g->nc == 3 ? (cw + 7) / 8 : 0; g->ubh[1] = g->ubh[2] = g->nc == 3 ? (ch + 7) / 8 : 0;
     g->coff[0] = 0;
     g->coff[1] = (size_t)g->bw[0] * g->bh[0];
     g->coff[2] = g->coff[1] + (size_t)g->bw[1] * g->bh[1];
@@ -247,7 +259,7 @@ static void fdct_quant_plane(const double* plane, int pw, int bw, int bh, const 
 void synth_rgb_to_coeffs(const uint8_t* rgb, int W, int H, const uint8_t qy[64], const uint8_t qc[64], int16_t* coef) {
     init_tables();
     geom_t g; geom_init(&g, W, H);
-    int PW = 16 * g.mx, PH = 16 * g.my;
+    int PW = 8 * g.hs * g.mx, PH = 8 * g.vs * g.my;
     double* Y = (double*)malloc(sizeof(double) * (size_t)PW * PH);
     double* Cb = (double*)malloc(sizeof(double) * (size_t)PW * PH);
     double* Cr = (double*)malloc(sizeof(double) * (size_t)PW * PH);
@@ -262,18 +274,26 @@ void synth_rgb_to_coeffs(const uint8_t* rgb, int W, int H, const uint8_t qy[64],
             Cr[(size_t)y * PW + x] = 128.0 + 0.5 * R - 0.418688 * G - 0.081312 * B;
         }
     }
-    int CW = PW / 2, CH = PH / 2;
+    int CW = PW / g.hs, CH = PH / g.vs;
     double* cb2 = (double*)malloc(sizeof(double) * (size_t)CW * CH);
     double* cr2 = (double*)malloc(sizeof(double) * (size_t)CW * CH);
+    const double inv = 1.0 / (g.hs * g.vs);                    /* box average over the hs x vs pixels of a chroma sample */
     for (int y = 0; y < CH; ++y)
         for (int x = 0; x < CW; ++x) {
-            size_t a = (size_t)(2 * y) * PW + 2 * x;
-            cb2[(size_t)y * CW + x] = 0.25 * (Cb[a] + Cb[a + 1] + Cb[a + PW] + Cb[a + PW + 1]);
-            cr2[(size_t)y * CW + x] = 0.25 * (Cr[a] + Cr[a + 1] + Cr[a + PW] + Cr[a + PW + 1]);
+            double sb = 0.0, sr = 0.0;
+            for (int dy = 0; dy < g.vs; ++dy)
+                for (int dx = 0; dx < g.hs; ++dx) {
+                    size_t a = (size_t)(g.vs * y + dy) * PW + g.hs * x + dx;
+                    sb += Cb[a]; sr += Cr[a];
+                }
+            cb2[(size_t)y * CW + x] = inv * sb;
+            cr2[(size_t)y * CW + x] = inv * sr;
         }
     fdct_quant_plane(Y, PW, g.bw[0], g.bh[0], qy, coef + g.coff[0] * 64);
-    fdct_quant_plane(cb2, CW, g.bw[1], g.bh[1], qc, coef + g.coff[1] * 64);
-    fdct_quant_plane(cr2, CW, g.bw[2], g.bh[2], qc, coef + g.coff[2] * 64);
+    if (g.nc == 3) {
+        fdct_quant_plane(cb2, CW, g.bw[1], g.bh[1], qc, coef + g.coff[1] * 64);
+        fdct_quant_plane(cr2, CW, g.bw[2], g.bh[2], qc, coef + g.coff[2] * 64);
+    }
     free(Y); free(Cb); free(Cr); free(cb2); free(cr2);
 }
 
@@ -328,6 +348,24 @@ static int g_nscans = 0;
 static const scan_spec* cur_script(int* n) {
     if (g_nscans > 0) { *n = g_nscans; return g_script; }
     *n = 10; return SCRIPT10;
+}
+/* What a record really holds: for greyscale images the scans of the chroma components fall away
+ * and an interleaved scan becomes a luminance scan. */
+static int eff_script(scan_spec* out) {
+    int n;
+    const scan_spec* sc = cur_script(&n);
+    int m = 0;
+    for (int s = 0; s < n; ++s) {
+        scan_spec t = sc[s];
+        if (g_nc == 1) {
+            int has_y = 0;
+            for (int c = 0; c < t.ncomp; ++c) if (t.comp[c] == 0) has_y = 1;
+            if (!has_y) continue;
+            t.ncomp = 1; t.comp[0] = 0;
+        }
+        out[m++] = t;
+    }
+    return m;
 }
 int synth_set_script(const int* flat, int n) {
     if (n < 0 || n > MAX_SCANS) return -1;
@@ -525,10 +563,10 @@ static void encode_scan(enc_state* st, const geom_t* g, const int16_t* coef, con
             }
             for (int ci = 0; ci < sc->ncomp; ++ci) {
                 int c = sc->comp[ci];
-                int hv = inter ? (c == 0 ? 2 : 1) : 1;
+                int hh = inter && c == 0 ? g->hs : 1, hv = inter && c == 0 ? g->vs : 1;
                 for (int by = 0; by < hv; ++by)
-                    for (int bx = 0; bx < hv; ++bx) {
-                        size_t brow = (size_t)my * hv + by, bcol = (size_t)mxi * hv + bx;
+                    for (int bx = 0; bx < hh; ++bx) {
+                        size_t brow = (size_t)my * hv + by, bcol = (size_t)mxi * hh + bx;
                         const int16_t* blk = coef + (g->coff[c] + brow * g->bw[c] + bcol) * 64;
                         int slot = c == 0 ? 0 : 1;
                         if (sequential) {
@@ -614,16 +652,16 @@ static void encode_image(enc_state* st, const geom_t* g, const int16_t* coef, co
         const uint8_t* q = t ? qc : qy;
         for (int k = 0; k < 64; ++k) bb_put(out, q[ZZ[k]]);
     }
-    int ns0;
-    const scan_spec* script0 = cur_script(&ns0);
-    int baseline = ns0 == 1 && script0[0].Ss == 0 && script0[0].Se == 63;
-    bb_put16(out, baseline ? 0xFFC0 : 0xFFC2); bb_put16(out, 17); bb_put(out, 8);
-    bb_put16(out, g->H); bb_put16(out, g->W); bb_put(out, 3);
-    bb_put(out, 1); bb_put(out, 0x22); bb_put(out, 0);
-    bb_put(out, 2); bb_put(out, 0x11); bb_put(out, 1);
-    bb_put(out, 3); bb_put(out, 0x11); bb_put(out, 1);
-    int ns;
-    const scan_spec* script = cur_script(&ns);
+    scan_spec script[MAX_SCANS];
+    int ns = eff_script(script);
+    int baseline = ns == 1 && script[0].Ss == 0 && script[0].Se == 63;
+    bb_put16(out, baseline ? 0xFFC0 : 0xFFC2); bb_put16(out, 8 + 3 * g->nc); bb_put(out, 8);
+    bb_put16(out, g->H); bb_put16(out, g->W); bb_put(out, g->nc);
+    bb_put(out, 1); bb_put(out, (g->hs << 4) | g->vs); bb_put(out, 0);
+    if (g->nc == 3) {
+        bb_put(out, 2); bb_put(out, 0x11); bb_put(out, 1);
+        bb_put(out, 3); bb_put(out, 0x11); bb_put(out, 1);
+    }
     for (int s = 0; s < ns; ++s) {
         encode_scan(st, g, coef, &script[s], restart_rows, restart_fixed, out);
         scan_end[s] = out->n;
@@ -646,8 +684,8 @@ static void put32(uint8_t* p, uint32_t v) { p[0] = v; p[1] = v >> 8; p[2] = v >>
 static void put64(uint8_t* p, uint64_t v) { put32(p, (uint32_t)v); put32(p + 4, (uint32_t)(v >> 32)); }
 
 static void assemble_record(synth_record* r, const int32_t* labels, size_t (*scan_end)[MAX_SCANS]) {
-    int N = r->n, G;
-    (void)cur_script(&G);                 /* one scan per group */
+    scan_spec eff[MAX_SCANS];
+    int N = r->n, G = eff_script(eff);    /* one scan per group */
     size_t meta_off = 64;
     size_t index_off = meta_off + 16 * (size_t)N;
     size_t data_off = index_off + 8 * (size_t)(G + 1) + 16 * (size_t)G * N;

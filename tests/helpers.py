@@ -7,17 +7,24 @@ import struct
 import numpy as np
 
 
-def block_grids(W, H):
-    mx, my = (W + 15) // 16, (H + 15) // 16
-    padded = [(2 * mx, 2 * my), (mx, my), (mx, my)]
-    off = [0, 4 * mx * my, 5 * mx * my]
+def block_grids(W, H, sampling=(2, 2, 3)):
+    """MCU grid, padded block grid per component and block offsets; sampling = (hs, vs, components):
+    hs x vs luminance blocks per MCU, one block per chroma component; one component = no MCU padding."""
+    hs, vs, nc = sampling
+    mx, my = (W + 8 * hs - 1) // (8 * hs), (H + 8 * vs - 1) // (8 * vs)
+    padded = [(hs * mx, vs * my)] + [(mx, my)] * (nc - 1)
+    off = [0, hs * vs * mx * my, (hs * vs + 1) * mx * my][:nc]
     return mx, my, padded, off
 
 
-def comp_of_block(W, H):
+def comp_of_block(W, H, sampling=(2, 2, 3)):
     """Component index (0 Y, 1 Cb, 2 Cr) of every block of the canonical layout."""
-    mx, my, _, _ = block_grids(W, H)
-    return np.concatenate([np.zeros(4 * mx * my, int), np.ones(mx * my, int), 2 * np.ones(mx * my, int)])
+    hs, vs, nc = sampling
+    mx, my, _, _ = block_grids(W, H, sampling)
+    parts = [np.zeros(hs * vs * mx * my, int)]
+    if nc == 3:
+        parts += [np.ones(mx * my, int), 2 * np.ones(mx * my, int)]
+    return np.concatenate(parts)
 
 
 def _trunc(c, bits):
@@ -66,12 +73,12 @@ def mask_truth(truth: np.ndarray, W: int, H: int, k: int) -> np.ndarray:
     return out
 
 
-def mask_truth_script(truth: np.ndarray, W: int, H: int, script, k: int) -> np.ndarray:
+def mask_truth_script(truth: np.ndarray, W: int, H: int, script, k: int, sampling=(2, 2, 3)) -> np.ndarray:
     """What a decoder holds after scans 1..k of an arbitrary script, written from the meaning of
     the script alone: a coefficient is known to the precision Al of the last scan <= k that
     covers its component and zigzag position (DC: floor shift, AC: magnitude shift toward zero),
     and is zero if no such scan exists.  script: [(components, Ss, Se, Ah, Al)]."""
-    comp = comp_of_block(W, H)
+    comp = comp_of_block(W, H, sampling)
     out = np.zeros_like(truth)
     for comps, Ss, Se, _Ah, Al in script[:k]:
         for c in comps:
