@@ -22,7 +22,10 @@
  *   g = 1 from SOI (tables, frame header), for every g the scan's DHT/DRI/SOS segments and
  *   entropy-coded bytes.  The file's EOI is not stored.  One scan per group.
  *
- * Supported streams: 8-bit, three components, 4:2:0 (2x2, 1x1, 1x1), Huffman coded; progressive
+ * Supported streams: 8-bit, Huffman coded; three components with the luminance at 1 or 2 blocks per
+ * MCU in each direction and one block per chroma component (4:2:0, 4:2:2, 4:4:0, 4:4:4: the paper's
+ * per-scan example for HAM10000 is a 4:4:4 file), or one component (greyscale: every output pixel
+ * is (Y, Y, Y)); one sampling per record; progressive
  * (SOF2) with any scan script that is the same for all images of a record, or baseline
  * sequential (SOF0, one interleaved scan = one scan group: the conventional JPEG that the paper's
  * Table 2 compares against); any restart interval.
@@ -188,7 +191,8 @@ int pcr_msssim(pcr_record* rec, const void* rgb_a, const void* rgb_b, void* scra
  *     (9 a + 3 b + 3 c + d + 8) >> 4; neighbours come from the decoded MCU-padded chroma planes,
  *     beyond their border the edge sample repeats.  Costs a second pass over the chroma blocks
  *     (their samples go through device memory: the first call allocates 128 bytes per MCU).
- * pcr_decode_tensor works with replication only (PCR_E_ARG otherwise).
+ * pcr_decode_tensor works with replication only (PCR_E_ARG otherwise).  The triangle filter is
+ * built for 4:2:0 records (PCR_E_ARG for other samplings).
  * Errors: PCR_E_ARG, PCR_E_NOMEM. */
 #define PCR_UPSAMPLE_REPLICATE 0
 #define PCR_UPSAMPLE_TRIANGLE 1
@@ -229,6 +233,13 @@ typedef struct {
     uint64_t bytes;     /* bytes of this scan group in the record                    */
 } pcr_scan_info;
 int pcr_get_scan(const pcr_record* rec, int s, pcr_scan_info* info);   /* s in 0..G-1 */
+
+/* Chroma sampling of the record's images (Section 2: chroma subsampling is part of the JPEG data):
+ * *hs x *vs luminance blocks per MCU (2 x 2 = 4:2:0, 2 x 1 = 4:2:2, 1 x 2 = 4:4:0, 1 x 1 = 4:4:4),
+ * *ncomp = 3, or 1 for greyscale (then 1 x 1).  The block grid of pcr_coeffs follows from it: the
+ * luminance plane has hs*ceil(W/(8 hs)) x vs*ceil(H/(8 vs)) blocks, each chroma plane
+ * ceil(W/(8 hs)) x ceil(H/(8 vs)). */
+int pcr_get_sampling(const pcr_record* rec, int* hs, int* vs, int* ncomp);
 
 /* Stage timing for benchmarks.  With profiling enabled every pcr_decode records CUDA events
  * on its stream around each stage; after the stream has been synchronised pcr_get_profile

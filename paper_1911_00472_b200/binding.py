@@ -18,7 +18,7 @@ EXPORTS = ("pcr_open", "pcr_num_images", "pcr_num_groups", "pcr_get_image", "pcr
            "pcr_decode", "pcr_evict", "pcr_status", "pcr_coeffs", "pcr_image_blocks", "pcr_launch_count",
            "pcr_strerror", "pcr_close", "pcr_get_scan", "pcr_set_profiling", "pcr_get_profile",
            "pcr_pixels_noalloc", "pcr_decode_more", "pcr_release_cached_memory", "pcr_decode_tensor", "pcr_msssim", "pcr_msssim_scratch_bytes", "pcr_set_upsampling",
-           "pcr_selftest_bounded_wait")
+           "pcr_selftest_bounded_wait", "pcr_get_sampling")
 
 
 class ImageInfo(C.Structure):
@@ -76,6 +76,7 @@ def lib():
         L.pcr_get_profile.argtypes = [vp, C.POINTER(StageTime), C.c_int, C.POINTER(C.c_int)]
         L.pcr_pixels_noalloc.argtypes = [vp, C.c_uint32, C.c_uint32, vp, vp, vp]
         L.pcr_selftest_bounded_wait.argtypes = [C.POINTER(C.c_int)]
+        L.pcr_get_sampling.argtypes = [vp, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int)]
         L.pcr_launch_count.restype = C.c_uint64
         L.pcr_launch_count.argtypes = []
         L.pcr_strerror.restype = C.c_char_p
@@ -212,6 +213,13 @@ def pcr_pixels_noalloc(dev_coeffs_ptr: int, width: int, height: int, host_qtab_p
     device coefficients + host quantisers -> device RGB, enqueued on `stream`."""
     _chk(lib().pcr_pixels_noalloc(dev_coeffs_ptr, width, height, host_qtab_ptr, dev_rgb_ptr, stream),
          "pcr_pixels_noalloc")
+
+
+def pcr_get_sampling(handle: int):
+    """(hs, vs, components) of the record's images."""
+    a, b, c = C.c_int(), C.c_int(), C.c_int()
+    _chk(lib().pcr_get_sampling(handle, C.byref(a), C.byref(b), C.byref(c)), "pcr_get_sampling")
+    return a.value, b.value, c.value
 
 
 def pcr_selftest_bounded_wait() -> bool:

@@ -285,19 +285,34 @@ struct Geometry {
     uint64_t loff[3];         // first block of each component counted inside its component
 };
 
-__device__ __forceinline__ Geometry make_geometry(const ImgDesc& im) {
+__device__ __forceinline__ Geometry make_geometry(const ImgDesc& im, const Params& P) {
     Geometry g;
+    const uint32_t hs = (uint32_t)P.hs, vs = (uint32_t)P.vs, ny = hs * vs;      // luminance blocks per MCU
     g.mx = im.mx; g.my = im.my;
-    g.bw[0] = 2 * im.mx; g.bw[1] = g.bw[2] = im.mx;
+    g.bw[0] = hs * im.mx; g.bw[1] = g.bw[2] = im.mx;
     g.ubw[0] = (im.W + 7) / 8; g.ubh[0] = (im.H + 7) / 8;
-    uint32_t cw = (im.W + 1) / 2, ch = (im.H + 1) / 2;
+    uint32_t cw = (im.W + hs - 1) / hs, ch = (im.H + vs - 1) / vs;
     g.ubw[1] = g.ubw[2] = (cw + 7) / 8; g.ubh[1] = g.ubh[2] = (ch + 7) / 8;
     g.coff[0] = im.blk_base;
-    g.coff[1] = im.blk_base + 4ull * im.mx * im.my;
-    g.coff[2] = im.blk_base + 5ull * im.mx * im.my;
-    const uint64_t mcus_before = im.blk_base / 6;      // every image holds 6 blocks per MCU
-    g.loff[0] = 4 * mcus_before; g.loff[1] = g.loff[2] = mcus_before;
+    g.coff[1] = im.blk_base + (uint64_t)ny * im.mx * im.my;
+    g.coff[2] = g.coff[1] + (uint64_t)im.mx * im.my;
+    const uint64_t mcus_before = im.blk_base / (ny + (P.nc == 3 ? 2u : 0u));   // every image holds the same blocks per MCU
+    g.loff[0] = ny * mcus_before; g.loff[1] = g.loff[2] = mcus_before;
     return g;
+}
+
+// Block number (in the planes) of block j of MCU (mrow, mcol) in an interleaved scan: the luminance
+// blocks of the MCU row by row, then Cb, then Cr.  *comp = its component.
+__device__ __forceinline__ uint64_t mcu_block(const Geometry& g, const Params& P, uint32_t mrow, uint32_t mcol, int j, int* comp) {
+    const int ny = P.hs * P.vs;
+    if (j < ny) {
+        const uint32_t r = (uint32_t)j >> (P.hs - 1), c = (uint32_t)j & (uint32_t)(P.hs - 1);
+        *comp = 0;
+        return g.coff[0] + (uint64_t)((uint32_t)P.vs * mrow + r) * g.bw[0] + (uint32_t)P.hs * mcol + c;
+    }
+    const int cc = j - ny + 1;
+    *comp = cc;
+    return g.coff[cc] + (uint64_t)mrow * g.bw[cc] + mcol;
 }
 
 __device__ __forceinline__ uint64_t low_mask(int p) { return p >= 64 ? ~0ull : ((1ull << p) - 1ull); }
@@ -347,7 +362,7 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
     const int img = (int)((which ? si1 : item.si) % (uint32_t)P.N);
     if (seg >= sd.nseg) { done = true; seg = 0; }
     const ImgDesc im = P.imgs[img];
-    const Geometry g = make_geometry(im);
+    const Geometry g = make_geometry(im, P);
 
     const bool inter = sc.ncomp > 1;
     const int c0 = sc.comp[0];
@@ -360,8 +375,9 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
     if (kRoi) {
         if (!done && m1 > m0) {
             const CropRect rc = P.roi[img];
-            const uint32_t ph = (inter || c0 != 0) ? 16u : 8u;             // pixel rows per MCU row of this scan
-            const uint32_t lo = 16u * (rc.y0 >> 4), hi = 16u * ((rc.y0 + rc.h + 15u) >> 4);
+            const uint32_t mh = 8u * (uint32_t)P.vs;                       // pixel rows of an MCU row
+            const uint32_t ph = (inter || c0 != 0) ? mh : 8u;              // pixel rows per MCU row of this scan
+            const uint32_t lo = mh * (rc.y0 / mh), hi = mh * ((rc.y0 + rc.h + mh - 1u) / mh);
             const uint32_t r0 = m0 / mcu_w, r1 = (m1 - 1u) / mcu_w;
             if ((r1 + 1u) * ph <= lo || r0 * ph >= hi) done = true;
         }
@@ -386,9 +402,9 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
 
     if (dc) {
         // ---- DC first pass: one block per step
-        const int bpm = inter ? 6 : 1;                     // blocks per MCU
+        const int bpm = inter ? P.hs * P.vs + 2 : 1;       // blocks per MCU
         uint32_t m = m0, mrow = m0 / mcu_w, mcol = m0 % mcu_w;
-        int j = 0;                                         // block inside the MCU: Y00 Y01 Y10 Y11 Cb Cr
+        int j = 0;                                         // block inside the MCU: the luminance blocks, Cb, Cr
         int pred0 = 0, pred1 = 0, pred2 = 0;
         if (m >= m1) done = true;
         for (;;) {
@@ -400,11 +416,11 @@ __global__ void __launch_bounds__(32 * kEntropyWarps) entropy_kernel(Params P, u
                 if (done || !br.ready()) continue;
                 br.refill();
                 const uint32_t win = br.top32();
-                const int ci = inter ? (j < 4 ? 0 : j - 3) : 0;
-                const int c = inter ? ci : c0;
+                int ci = 0;
                 uint64_t blk;
-                if (inter && c == 0) blk = g.coff[0] + (uint64_t)(2 * mrow + (j >> 1)) * g.bw[0] + 2 * mcol + (j & 1);
-                else blk = g.coff[c] + (uint64_t)mrow * g.bw[c] + mcol;
+                if (inter) blk = mcu_block(g, P, mrow, mcol, j, &ci);
+                else blk = g.coff[c0] + (uint64_t)mrow * g.bw[c0] + mcol;
+                const int c = inter ? ci : c0;
                 int16_t* dcv = P.head + blk * 8;
                 {
                     const HuffTab& tab = tabs[wid][(sd.slots >> (2 * ci)) & 1u];
@@ -653,7 +669,7 @@ __global__ void __launch_bounds__(32 * kSeqWarps) sequential_kernel(Params P, ui
     uint32_t seg = item.seg0 + lane;
     if (seg >= sd.nseg) { done = true; seg = 0; }
     const ImgDesc im = P.imgs[img];
-    const Geometry g = make_geometry(im);
+    const Geometry g = make_geometry(im, P);
     const uint32_t mcu_w = g.mx, total = g.mx * g.my;
     const uint32_t m0 = sd.ri ? seg * sd.ri : 0;
     const uint32_t m1 = sd.ri ? min(m0 + sd.ri, total) : total;
@@ -661,9 +677,10 @@ __global__ void __launch_bounds__(32 * kSeqWarps) sequential_kernel(Params P, ui
     if (kRoi) {
         if (!done && m1 > m0) {
             const CropRect rc = P.roi[img];
-            const uint32_t lo = 16u * (rc.y0 >> 4), hi = 16u * ((rc.y0 + rc.h + 15u) >> 4);
+            const uint32_t mh = 8u * (uint32_t)P.vs;                       // pixel rows of an MCU row
+            const uint32_t lo = mh * (rc.y0 / mh), hi = mh * ((rc.y0 + rc.h + mh - 1u) / mh);
             const uint32_t r0 = m0 / mcu_w, r1 = (m1 - 1u) / mcu_w;
-            if ((r1 + 1u) * 16u <= lo || r0 * 16u >= hi) done = true;
+            if ((r1 + 1u) * mh <= lo || r0 * mh >= hi) done = true;
         }
         if (__all_sync(full, done)) return;
     }
@@ -683,7 +700,8 @@ __global__ void __launch_bounds__(32 * kSeqWarps) sequential_kernel(Params P, ui
     br.prime();
 
     uint32_t m = m0, mrow = m0 / mcu_w, mcol = m0 % mcu_w;
-    int j = 0;                                            // block inside the MCU: Y00 Y01 Y10 Y11 Cb Cr
+    const int bpm = P.nc == 3 ? P.hs * P.vs + 2 : 1;      // blocks per MCU (a lone component: one block, no padding)
+    int j = 0;                                            // block inside the MCU: the luminance blocks, Cb, Cr
     int k = 0;                                            // 0: the block's DC symbol comes next
     int pred0 = 0, pred1 = 0, pred2 = 0;
     if (m >= m1) done = true;
@@ -696,10 +714,8 @@ __global__ void __launch_bounds__(32 * kSeqWarps) sequential_kernel(Params P, ui
             if (done || !br.ready()) continue;
             br.refill();
             const uint32_t win = br.top32();
-            const int c = j < 4 ? 0 : j - 3;
-            uint64_t blk;
-            if (c == 0) blk = g.coff[0] + (uint64_t)(2 * mrow + (j >> 1)) * g.bw[0] + 2 * mcol + (j & 1);
-            else blk = (c == 1 ? g.coff[1] : g.coff[2]) + (uint64_t)mrow * g.mx + mcol;
+            int c = 0;
+            const uint64_t blk = P.nc == 3 ? mcu_block(g, P, mrow, mcol, j, &c) : g.coff[0] + (uint64_t)mrow * g.bw[0] + mcol;
             const bool is_dc = k == 0;
             const int ti = is_dc ? (int)((sd.slots >> (2 * c)) & 1u) : 2 + (int)((sd.slots_ac >> (2 * c)) & 1u);
             const HuffTab& tab = tabs[wid][ti];
@@ -727,7 +743,7 @@ __global__ void __launch_bounds__(32 * kSeqWarps) sequential_kernel(Params P, ui
             }
             if (is_eob || k > 63) {                       // block finished
                 k = 0;
-                if (++j == 6) {
+                if (++j == bpm) {
                     j = 0; ++m;
                     if (++mcol == mcu_w) { mcol = 0; ++mrow; }
                 }

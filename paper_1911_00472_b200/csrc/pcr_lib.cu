@@ -135,6 +135,8 @@ struct pcr_record {
     std::vector<pcr_image_info> info;
     std::vector<uint64_t> blk_base, nblk;
     uint64_t total_blocks = 0, total_segs = 0;
+    int hs = 2, vs = 2, nc = 3;     // chroma sampling, the same for every image of the record
+    uint32_t unit_mcus = kPixMcus;  // MCUs of a pixel work unit
     unsigned dc_refine_chunks = 1;  // 256-MCU chunks of the largest image, at most 8 (dc_refine_kernel's grid)
     bool widths_mult16 = true;    // every image is a multiple of 16 pixels wide (the DC-only pixel kernel's condition)
     size_t out_bytes = 0;
@@ -215,13 +217,13 @@ static inline uint64_t rd64(const uint8_t* p) { return (uint64_t)rd32(p) | ((uin
 
 // Writes the list of pixel work units at set-up: block = position of the processing order.
 __global__ void __launch_bounds__(128) units_kernel(const ImgDesc* __restrict__ imgs, const uint32_t* __restrict__ order,
-                                                    const uint32_t* __restrict__ prefix, Unit* __restrict__ units) {
+                                                    const uint32_t* __restrict__ prefix, Unit* __restrict__ units, uint32_t unit_mcus) {
     const uint32_t img = order[blockIdx.x];
-    const uint32_t per_row = (imgs[img].mx + kPixMcus - 1) / kPixMcus, n = per_row * imgs[img].my;
+    const uint32_t per_row = (imgs[img].mx + unit_mcus - 1) / unit_mcus, n = per_row * imgs[img].my;
     Unit* dst = units + prefix[blockIdx.x];
     for (uint32_t j = threadIdx.x; j < n; j += 128) {
         Unit un;
-        un.img = img; un.mrow = (uint16_t)(j / per_row); un.mcol0 = (uint16_t)((j % per_row) * kPixMcus);
+        un.img = img; un.mrow = (uint16_t)(j / per_row); un.mcol0 = (uint16_t)((j % per_row) * unit_mcus);
         dst[j] = un;
     }
 }
@@ -239,6 +241,7 @@ struct ImageParse {
     uint32_t ri = 0;
     bool have_frame = false;
     bool sequential = false;      // SOF0: one interleaved scan carries whole blocks
+    int hs = 2, vs = 2, nc = 3;   // luminance blocks per MCU, components
 };
 
 struct ScanParse {
@@ -292,17 +295,21 @@ int parse_chunk(const uint8_t* rec, uint64_t off, uint32_t len, bool first, Imag
                 im.qdef[tq] = true;
             }
         } else if (mk == 0xC2 || mk == 0xC0) {            // progressive / baseline sequential, Huffman
-            if (im.have_frame || sl < 15 || s[0] != 8 || s[5] != 3) return PCR_E_FORMAT;
+            if (im.have_frame || sl < 9 || s[0] != 8 || (s[5] != 3 && s[5] != 1) || sl < 6u + 3u * s[5]) return PCR_E_FORMAT;
             im.sequential = mk == 0xC0;
             im.H = ((uint32_t)s[1] << 8) | s[2];
             im.W = ((uint32_t)s[3] << 8) | s[4];
-            for (int c = 0; c < 3; ++c) {
+            im.nc = s[5];
+            for (int c = 0; c < im.nc; ++c) {
                 im.cid[c] = s[6 + 3 * c];
                 int hv = s[7 + 3 * c];
                 im.tq[c] = s[8 + 3 * c];
                 if (im.tq[c] > 3) return PCR_E_FORMAT;
-                if (hv != (c == 0 ? 0x22 : 0x11)) return PCR_E_FORMAT;   // 4:2:0 only
+                // luminance 1 or 2 blocks per MCU in each direction, chroma one: 4:4:4, 4:2:2, 4:4:0, 4:2:0
+                if (c == 0) { im.hs = hv >> 4; im.vs = hv & 15; if (im.hs < 1 || im.hs > 2 || im.vs < 1 || im.vs > 2) return PCR_E_FORMAT; }
+                else if (hv != 0x11) return PCR_E_FORMAT;
             }
+            if (im.nc == 1) im.hs = im.vs = 1;                // a lone component is never interleaved: no MCU padding
             if (im.W == 0 || im.H == 0) return PCR_E_FORMAT;
             im.have_frame = true;
         } else if (mk == 0xC4) {
@@ -328,7 +335,7 @@ int parse_chunk(const uint8_t* rec, uint64_t off, uint32_t len, bool first, Imag
             int td[3] = {0, 0, 0}, ta[3] = {0, 0, 0};
             for (int i = 0; i < ns; ++i) {
                 int id = s[1 + 2 * i], found = -1;
-                for (int c = 0; c < 3; ++c) if (im.cid[c] == id) found = c;
+                for (int c = 0; c < im.nc; ++c) if (im.cid[c] == id) found = c;
                 if (found < 0) return PCR_E_FORMAT;
                 for (int j = 0; j < i; ++j) if (sc.comp[j] >= found) return PCR_E_FORMAT;   // frame order
                 sc.comp[i] = found;
@@ -340,10 +347,10 @@ int parse_chunk(const uint8_t* rec, uint64_t off, uint32_t len, bool first, Imag
             sc.Ah = s[3 + 2 * ns] >> 4; sc.Al = s[3 + 2 * ns] & 15;
             if (sc.Ss > sc.Se || sc.Se > 63 || sc.Al > 13) return PCR_E_FORMAT;
             if (im.sequential) {
-                if (sc.Ss != 0 || sc.Se != 63 || sc.Ah != 0 || sc.Al != 0 || ns != 3) return PCR_E_FORMAT;
+                if (sc.Ss != 0 || sc.Se != 63 || sc.Ah != 0 || sc.Al != 0 || ns != im.nc) return PCR_E_FORMAT;
             } else if (sc.Ss == 0 && sc.Se != 0) return PCR_E_FORMAT;
             if (sc.Ss > 0 && ns != 1) return PCR_E_FORMAT;
-            if (ns > 1 && ns != 3) return PCR_E_FORMAT;     // interleaved scans hold all three components
+            if (ns > 1 && ns != im.nc) return PCR_E_FORMAT; // interleaved scans hold all three components
             if (sc.Ah != 0 && sc.Ah != sc.Al + 1) return PCR_E_FORMAT;
             for (int i = 0; i < 3; ++i) out.tab[i] = out.tab_ac[i] = 0;
             for (int i = 0; i < ns && im.sequential; ++i) {
@@ -447,6 +454,7 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     // every image's chunks are walked independently (a few host threads for large records); the
     // running sums over images follow in one serial pass
     std::vector<ScanScript> scripts((size_t)N * G);
+    std::vector<uint8_t> samplings(N, 0);
     auto parse_image = [&](uint32_t i) -> int {
         ImageParse im;
         const uint8_t* m = rec + meta_off + 16ull * i;
@@ -478,25 +486,27 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
                 if (sp.tab[ci] != sd.tab_off[1]) return PCR_E_FORMAT;
                 sd.slots |= 1u << (2 * ci);
             }
-            uint32_t mx = (im.W + 15) / 16, my = (im.H + 15) / 16;
+            uint32_t mx = (im.W + 8 * im.hs - 1) / (8 * im.hs), my = (im.H + 8 * im.vs - 1) / (8 * im.vs);
             uint64_t total_mcu;
             if (sp.sc.ncomp > 1) total_mcu = (uint64_t)mx * my;
             else {
-                uint32_t wc = sp.sc.comp[0] == 0 ? im.W : (im.W + 1) / 2, hc = sp.sc.comp[0] == 0 ? im.H : (im.H + 1) / 2;
+                uint32_t wc = sp.sc.comp[0] == 0 ? im.W : (im.W + im.hs - 1) / im.hs, hc = sp.sc.comp[0] == 0 ? im.H : (im.H + im.vs - 1) / im.vs;
                 total_mcu = (uint64_t)((wc + 7) / 8) * ((hc + 7) / 8);
             }
             sd.nseg = sd.ri ? (uint32_t)((total_mcu + sd.ri - 1) / sd.ri) : 1u;
         }
         if (!im.have_frame) return PCR_E_FORMAT;
         if (rd32(m + 4) != im.W || rd32(m + 8) != im.H) return PCR_E_FORMAT;   // metadata and frame header agree
-        for (int c = 0; c < 3; ++c) {
+        for (int c = 0; c < im.nc; ++c) {
             if (!im.qdef[im.tq[c]]) return PCR_E_FORMAT;
             memcpy(&qtab[(size_t)i * 192 + 64 * c], im.q[im.tq[c]], 128);
         }
+        samplings[i] = (uint8_t)(im.hs | (im.vs << 2) | (im.nc << 4));
         pcr_image_info& inf = r->info[i];
         inf.width = im.W; inf.height = im.H; inf.label = (int32_t)rd32(m); inf.rsvd = 0;
         inf.out_bytes = 3ull * im.W * im.H;
-        imgs[i].W = im.W; imgs[i].H = im.H; imgs[i].mx = (im.W + 15) / 16; imgs[i].my = (im.H + 15) / 16;
+        imgs[i].W = im.W; imgs[i].H = im.H;
+        imgs[i].mx = (im.W + 8 * im.hs - 1) / (8 * im.hs); imgs[i].my = (im.H + 8 * im.vs - 1) / (8 * im.vs);
         return PCR_OK;
     };
     {
@@ -516,6 +526,9 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
         for (int rc : rcs) if (rc != PCR_OK) return rc;
     }
     uint64_t blocks = 0, out_off = 0, segs = 0;
+    r->hs = samplings[0] & 3; r->vs = (samplings[0] >> 2) & 3; r->nc = samplings[0] >> 4;
+    const uint32_t bpm = (uint32_t)(r->hs * r->vs + (r->nc == 3 ? 2 : 0));      // blocks per MCU
+    r->unit_mcus = r->nc == 3 && r->hs == 2 ? 8u : 16u;                         // a work unit is 128 pixels wide
     for (uint32_t g = 0; g < G; ++g) r->script[g] = scripts[g];
     for (uint32_t i = 0; i < N; ++i) {
         if (i && memcmp(&scripts[(size_t)i * G], &scripts[0], sizeof(ScanScript) * G) != 0) return PCR_E_FORMAT;   // one script per record
@@ -530,7 +543,8 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
         out_off += (inf.out_bytes + 127) & ~127ull;
         if (imgs[i].W & 15u) r->widths_mult16 = false;
         r->dc_refine_chunks = std::max(r->dc_refine_chunks, std::min(8u, (imgs[i].mx * imgs[i].my + 255u) / 256u));
-        r->blk_base[i] = blocks; r->nblk[i] = 6ull * imgs[i].mx * imgs[i].my;
+        if (samplings[i] != samplings[0]) return PCR_E_FORMAT;                                  // one sampling per record
+        r->blk_base[i] = blocks; r->nblk[i] = (uint64_t)bpm * imgs[i].mx * imgs[i].my;
         imgs[i].blk_base = blocks; imgs[i].out_off = inf.out_offset;
         blocks += r->nblk[i];
     }
@@ -663,7 +677,7 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     for (uint32_t pos = 0; pos < N; ++pos) {
         const ImgDesc& im = imgs[order[pos]];
         if (im.my > 65535 || im.mx > 65535) return PCR_E_FORMAT;
-        const uint64_t nu = (uint64_t)((im.mx + kPixMcus - 1) / kPixMcus) * im.my;
+        const uint64_t nu = (uint64_t)((im.mx + r->unit_mcus - 1) / r->unit_mcus) * im.my;
         if (unit_prefix[pos] + nu >= (1ull << 32)) return PCR_E_FORMAT;
         unit_prefix[pos + 1] = unit_prefix[pos] + (uint32_t)nu;
     }
@@ -672,7 +686,7 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     r->n_units = unit_prefix[N];
 
     // side data of the AC scans: one word per block for a first pass, four for a refinement
-    const uint64_t total_mcus = blocks / 6;
+    const uint64_t total_mcus = blocks / bpm;
     uint64_t aux_words = 0;
     r->saux.assign(G, ScanAux{});
     int n_refine[3] = {0, 0, 0};
@@ -684,7 +698,7 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
         if (sc.Ss == 0) continue;
         ax.stride = sc.Ah ? 4u : 1u;
         ax.base = aux_words;
-        aux_words += (sc.comp[0] == 0 ? 4ull : 1ull) * total_mcus * ax.stride;
+        aux_words += (sc.comp[0] == 0 ? (uint64_t)(r->hs * r->vs) : 1ull) * total_mcus * ax.stride;
         aux_words = (aux_words + 1) & ~1ull;      // 16-byte alignment of every scan's area
         if (sc.Ah) {
             // positions already non-zero = union of the masks of earlier scans on this band; an
@@ -738,7 +752,7 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     if ((rc = upload(r, &r->d_unit_prefix, unit_prefix))) return rc;
     if ((rc = take(r, &r->d_units, (size_t)std::max<uint32_t>(r->n_units, 1) * sizeof(Unit)))) return rc;
     if ((rc = upload(r, &r->d_order, order))) return rc;
-    units_kernel<<<N, 128, 0, r->up_stream>>>(r->d_imgs, r->d_order, r->d_unit_prefix, r->d_units);
+    units_kernel<<<N, 128, 0, r->up_stream>>>(r->d_imgs, r->d_order, r->d_unit_prefix, r->d_units, r->unit_mcus);
     ++g_launches;
     for (auto& z : zero)
         if (cudaMemsetAsync(z.first, 0, z.second, r->up_stream) != cudaSuccess) return PCR_E_CUDA;
@@ -821,6 +835,12 @@ int pcr_evict(pcr_record* rec) {
 
 }  // extern "C"
 
+template <int kSamp>
+static void launch_pixels_sampled(bool refine, unsigned grid, cudaStream_t q, const Params& Q, const FinalizeList& fl, uint8_t* o8) {
+    if (refine) pixel_kernel<true, 1, false, 0, kSamp><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+    else pixel_kernel<false, 1, false, 0, kSamp><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+}
+
 // Decode scans k0 .. k-1 on top of the state scans 0 .. k0-1 left behind (k0 = 0: from scratch),
 // then produce the pixels of fidelity k.
 static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream, const TensorArgs* targs = nullptr) {
@@ -852,7 +872,8 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
     P.saux = rec->d_saux; P.aux = rec->d_aux;
     P.imgs = rec->d_imgs; P.seg_start = rec->d_seg; P.items = rec->d_items; P.units = rec->d_units;
     P.qtab = rec->d_qtab; P.order = rec->d_order; P.status = rec->d_status; P.N = rec->N;
-    P.roi = targs ? targs->crops : nullptr;
+    P.hs = rec->hs; P.vs = rec->vs; P.nc = rec->nc;
+    P.roi = targs ? targs->crops : nullptr;          // (only read by the crop-restricted kernels)
     P.chroma = rec->d_chroma;
     FinalizeList fl;
     memset(&fl, 0, sizeof fl);
@@ -878,6 +899,10 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
         if (rec->script[s].Ss > 0 || rec->script[s].Se > 0) dc_only = false;
         if (rec->script[s].Se > 7) head_only = false;
     }
+    // the specialised pixel kernels (DC only, head plane only, crop-restricted) exist for 4:2:0
+    const bool s420 = rec->hs == 2 && rec->vs == 2 && rec->nc == 3;
+    if (!s420) { dc_only = false; head_only = false; }
+    const bool roi = targs && s420;                 // decode only the MCU rows the crops touch
     rec->dc_merged = false;
     // the planes must be zero before the first AC scan writes into them
     const bool clear_planes = !head_only && (k0 == 0 || !rec->planes_cleared);
@@ -952,14 +977,14 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
                 count += rec->item_count[(size_t)g * G + s];
             }
             if (count && sequential) {
-                if (targs) sequential_kernel<true><<<(count + kSeqWarps - 1) / kSeqWarps, 32 * kSeqWarps, 0, q>>>(P, begin, count);
+                if (roi) sequential_kernel<true><<<(count + kSeqWarps - 1) / kSeqWarps, 32 * kSeqWarps, 0, q>>>(P, begin, count);
                 else sequential_kernel<false><<<(count + kSeqWarps - 1) / kSeqWarps, 32 * kSeqWarps, 0, q>>>(P, begin, count);
                 ++g_launches;
                 return true;
             }
             if (count) {
                 const unsigned nb = (count + kEntropyWarps - 1) / kEntropyWarps;
-                if (targs) entropy_kernel<true><<<nb, 32 * kEntropyWarps, 0, q>>>(P, begin, count);
+                if (roi) entropy_kernel<true><<<nb, 32 * kEntropyWarps, 0, q>>>(P, begin, count);
                 else entropy_kernel<false><<<nb, 32 * kEntropyWarps, 0, q>>>(P, begin, count);
                 ++g_launches;
             }
@@ -1006,7 +1031,15 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
         if (nu) {
             const unsigned grid = nu;
             uint8_t* o8 = static_cast<uint8_t*>(out);
-            if (!targs && rec->upsampling == PCR_UPSAMPLE_TRIANGLE) {
+            if (!s420) {
+                // other samplings: one general kernel per sampling (positions 0..7 from the head plane, the
+                // rest from the lines, which are always cleared for these records)
+                const int code = rec->nc == 1 ? kSampGrey : (rec->hs == 2 ? kSamp422 : (rec->vs == 2 ? kSamp440 : kSamp444));
+                if (code == kSamp422) launch_pixels_sampled<kSamp422>(any_refine, grid, q, Q, fl, o8);
+                else if (code == kSamp440) launch_pixels_sampled<kSamp440>(any_refine, grid, q, Q, fl, o8);
+                else if (code == kSamp444) launch_pixels_sampled<kSamp444>(any_refine, grid, q, Q, fl, o8);
+                else launch_pixels_sampled<kSampGrey>(any_refine, grid, q, Q, fl, o8);
+            } else if (!targs && rec->upsampling == PCR_UPSAMPLE_TRIANGLE) {
                 // chroma pass (samples of every chroma block into the sample planes), then the pixel pass
                 if (head_only && any_refine) {
                     pixel_kernel<true, 3, false, 1><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
@@ -1262,8 +1295,9 @@ int pcr_msssim(pcr_record* rec, const void* rgb_a, const void* rgb_b, void* scra
 
 int pcr_set_upsampling(pcr_record* rec, int mode) {
     if (!rec || (mode != PCR_UPSAMPLE_REPLICATE && mode != PCR_UPSAMPLE_TRIANGLE)) return PCR_E_ARG;
+    if (mode == PCR_UPSAMPLE_TRIANGLE && !(rec->hs == 2 && rec->vs == 2 && rec->nc == 3)) return PCR_E_ARG;   // built for 4:2:0
     if (mode == PCR_UPSAMPLE_TRIANGLE && !rec->d_chroma) {
-        if (int rc = take(rec, &rec->d_chroma, (size_t)(std::max<uint64_t>(rec->total_blocks / 6, 1) * 128))) return rc;
+        if (int rc = take(rec, &rec->d_chroma, (size_t)(std::max<uint64_t>(rec->total_blocks / 6, 1) * 128)   /* 4:2:0: six blocks per MCU */)) return rc;
     }
     rec->upsampling = mode;
     return PCR_OK;
@@ -1316,6 +1350,12 @@ int pcr_get_scan(const pcr_record* rec, int s, pcr_scan_info* info) {
     info->wave = rec->wave_of_scan[s];
     info->rsvd = 0;
     info->bytes = rec->group_end[s + 1] - rec->group_end[s];
+    return PCR_OK;
+}
+
+int pcr_get_sampling(const pcr_record* rec, int* hs, int* vs, int* ncomp) {
+    if (!rec || !hs || !vs || !ncomp) return PCR_E_ARG;
+    *hs = rec->hs; *vs = rec->vs; *ncomp = rec->nc;
     return PCR_OK;
 }
 

@@ -40,13 +40,13 @@ __global__ void __launch_bounds__(256) dc_refine_kernel(Params P, int s, uint32_
     const ScanDesc sd = P.scans[(size_t)s * P.N + img];
     const ScanScript sc = P.script[s];
     const ImgDesc im = P.imgs[img];
-    const Geometry g = make_geometry(im);
+    const Geometry g = make_geometry(im, P);
     const bool inter = sc.ncomp > 1;
     const int c0 = sc.comp[0];
     const uint32_t mcu_w = inter ? g.mx : g.ubw[c0];
     const uint32_t mcu_h = inter ? g.my : g.ubh[c0];
     const uint32_t total = mcu_w * mcu_h;
-    const uint32_t bpm = inter ? 6u : 1u;                      // blocks (= bits) per MCU
+    const uint32_t bpm = inter ? (uint32_t)(P.hs * P.vs + 2) : 1u;   // blocks (= bits) per MCU
     const uint32_t* segtab = P.seg_start + sd.seg_base;
     const uint32_t* words = reinterpret_cast<const uint32_t*>(P.ubuf);
     const int p1 = 1 << sc.Al;
@@ -69,9 +69,9 @@ __global__ void __launch_bounds__(256) dc_refine_kernel(Params P, int s, uint32_
             if (j >= bpm) break;
             if (!((v >> (bpm - 1u - j)) & 1u)) continue;
             uint64_t blk;
+            int comp;
             if (!inter) blk = g.coff[c0] + (uint64_t)mrow * g.bw[c0] + mcol;
-            else if (j < 4) blk = g.coff[0] + (uint64_t)(2 * mrow + (j >> 1)) * g.bw[0] + 2 * mcol + (j & 1);
-            else blk = g.coff[j - 3] + (uint64_t)mrow * g.bw[j - 3] + mcol;
+            else blk = mcu_block(g, P, mrow, mcol, (int)j, &comp);
             // coefficient 0 is the first int16 of the block's head entry; no other scan of the wave writes it
             int16_t* dcv = P.head + blk * 8;
             *dcv = (int16_t)(*dcv | p1);
@@ -192,6 +192,7 @@ struct DcWrite {
     uint64_t coff[3];
     uint32_t bw[3];
     uint32_t mcu_w;
+    uint32_t hs, vs;       // luminance blocks per MCU
     uint32_t n, n1;        // next block of the scan in scan order, one past its last
     int pred[3];
     int Al;
@@ -203,7 +204,7 @@ __device__ __forceinline__ void dc_first_span(const HuffTab* tabs2, uint32_t slo
                                               int& sum0, int& sum1, int& sum2, DcWrite& W, bool& bad) {
     WordReader br;
     br.init(base, pos);
-    const int bpm = inter ? 6 : 1;
+    const int ny = (int)(W.hs * W.vs), bpm = inter ? ny + 2 : 1;
     uint32_t nb = 0;
     int s0 = 0, s1 = 0, s2 = 0;
     uint32_t mrow = 0, mcol = 0;
@@ -212,7 +213,7 @@ __device__ __forceinline__ void dc_first_span(const HuffTab* tabs2, uint32_t slo
     while (!stop && br.pos() < pos_end) {
         br.refill();
         const uint32_t win = br.top32();
-        const int ci = inter ? (j < 4 ? 0 : j - 3) : 0;
+        const int ci = inter ? (j < ny ? 0 : j - ny + 1) : 0;
         const int c = inter ? ci : c0;
         const HuffTab& tab = tabs2[(slots >> (2 * ci)) & 1u];
         const uint32_t e = huff_lookup(tab, win);
@@ -229,7 +230,7 @@ __device__ __forceinline__ void dc_first_span(const HuffTab* tabs2, uint32_t slo
             const int pv = (c == 0 ? W.pred[0] : (c == 1 ? W.pred[1] : W.pred[2])) + d;
             if (c == 0) W.pred[0] = pv; else if (c == 1) W.pred[1] = pv; else W.pred[2] = pv;
             uint64_t blk;
-            if (inter && c == 0) blk = W.coff[0] + (uint64_t)(2 * mrow + (uint32_t)(j >> 1)) * W.bw[0] + 2 * mcol + (uint32_t)(j & 1);
+            if (inter && c == 0) blk = W.coff[0] + (uint64_t)(W.vs * mrow + ((uint32_t)j >> (W.hs - 1u))) * W.bw[0] + W.hs * mcol + ((uint32_t)j & (W.hs - 1u));
             else blk = W.coff[c] + (uint64_t)mrow * W.bw[c] + mcol;
             W.head[blk * 8] = (int16_t)(pv << W.Al);
             if (++W.n >= W.n1) stop = true;
@@ -257,7 +258,7 @@ __global__ void __launch_bounds__(32 * kLongWarps) first_pass_long_kernel(Params
     const ScanDesc sd = P.scans[si];
     const ScanScript sc = P.script[s];
     const ImgDesc im = P.imgs[img];
-    const Geometry g = make_geometry(im);
+    const Geometry g = make_geometry(im, P);
     const bool dc = sc.Ss == 0, inter = sc.ncomp > 1;
     const int c0 = sc.comp[0];
     const uint32_t mcu_w = inter ? g.mx : g.ubw[c0];
@@ -281,10 +282,11 @@ __global__ void __launch_bounds__(32 * kLongWarps) first_pass_long_kernel(Params
     bool bad = false;
     if (dc) {
         DcWrite W;
-        W.head = P.head; W.mcu_w = mcu_w; W.Al = sc.Al;
+        W.head = P.head; W.mcu_w = mcu_w; W.Al = sc.Al; W.hs = (uint32_t)P.hs; W.vs = (uint32_t)P.vs;
+        const uint32_t bpm = inter ? (uint32_t)(P.hs * P.vs + 2) : 1u;
 #pragma unroll
         for (int c = 0; c < 3; ++c) { W.coff[c] = g.coff[c]; W.bw[c] = g.bw[c]; W.pred[c] = 0; }
-        W.n = 0; W.n1 = total * (inter ? 6u : 1u);
+        W.n = 0; W.n1 = total * bpm;
         uint32_t pos = my_begin, pos_x, nb;
         int j = 0, j_x, a0, a1, a2;
         bool again = true;
@@ -309,10 +311,10 @@ __global__ void __launch_bounds__(32 * kLongWarps) first_pass_long_kernel(Params
         W.n = min(nin - nb, W.n1); W.pred[0] = b0 - a0; W.pred[1] = b1 - a1; W.pred[2] = b2 - a2;
         // the place inside the MCU follows from the block number (equal to the handed-on state unless
         // the stream is damaged; taking it from the block number keeps every store inside the image)
-        if (nb && (uint32_t)j != W.n % (inter ? 6u : 1u)) bad = true;
-        j = (int)(W.n % (inter ? 6u : 1u));
+        if (nb && (uint32_t)j != W.n % bpm) bad = true;
+        j = (int)(W.n % bpm);
         dc_first_span<true>(tabs[wid], sd.slots, inter, c0, base, pos, j, my_end, pos_x, j_x, nb, a0, a1, a2, W, bad);
-        if (all < total * (inter ? 6u : 1u)) bad = true;                     // the stream ends before the last block
+        if (all < total * bpm) bad = true;                     // the stream ends before the last block
     } else {
         const int c = c0, Ss = sc.Ss, Se = sc.Se;
         const ScanAux ax = P.saux[s];
@@ -435,7 +437,7 @@ __global__ void __launch_bounds__(32 * kGroupWarps) ac_refine_group_kernel(Param
     const ScanDesc sd = P.scans[si];
     const ScanScript sc = P.script[s];
     const ImgDesc im = P.imgs[img];
-    const Geometry g = make_geometry(im);
+    const Geometry g = make_geometry(im, P);
     const uint32_t Ss = (uint32_t)sc.Ss, Se = (uint32_t)sc.Se;
     const uint32_t mcu_w = g.ubw[c], total = g.ubw[c] * g.ubh[c], bw = g.bw[c];
     const unsigned full = 0xffffffffu;

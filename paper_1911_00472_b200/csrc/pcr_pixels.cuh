@@ -21,10 +21,21 @@
 
 namespace pcr {
 
-constexpr int kPixMcus = 8;                   // MCUs per CTA
-constexpr int kPixBlocks = 6 * kPixMcus;      // 32 Y + 8 Cb + 8 Cr
-constexpr int kPixThreads = 64;               // one thread per block for the transform (48 used)
-constexpr int kStagePitch = 3 * 16 * kPixMcus + 16;   // bytes per staged RGB row (+ spare, keeps rows 16-byte aligned)
+constexpr int kPixMcus = 8;                   // MCUs per CTA (4:2:0)
+constexpr int kPixThreads = 64;               // one thread per block for the transform
+constexpr int kStagePitch = 3 * 128 + 16;     // bytes per staged RGB row (+ spare, keeps rows 16-byte aligned)
+
+// Chroma sampling of a record as a template code: luminance blocks per MCU (horizontal, vertical),
+// components, and the MCUs of one work unit, chosen so that a unit is 128 pixels wide and has at
+// most 64 blocks: 4:2:0 -> 8 MCUs (32 Y + 8 Cb + 8 Cr), 4:2:2 -> 8 (16 + 8 + 8), 4:4:0 -> 16
+// (32 + 16 + 16), 4:4:4 -> 16 (16 + 16 + 16), greyscale -> 16 (16 Y).
+enum { kSamp420 = 0, kSamp422 = 1, kSamp440 = 2, kSamp444 = 3, kSampGrey = 4 };
+template <int kSamp> struct Sampling;
+template <> struct Sampling<kSamp420> { static constexpr int HS = 2, VS = 2, NC = 3, U = 8; };
+template <> struct Sampling<kSamp422> { static constexpr int HS = 2, VS = 1, NC = 3, U = 8; };
+template <> struct Sampling<kSamp440> { static constexpr int HS = 1, VS = 2, NC = 3, U = 16; };
+template <> struct Sampling<kSamp444> { static constexpr int HS = 1, VS = 1, NC = 3, U = 16; };
+template <> struct Sampling<kSampGrey> { static constexpr int HS = 1, VS = 1, NC = 1, U = 16; };
 
 // zigzag position -> natural index, by walking the anti-diagonals
 struct ZigzagTable {
@@ -87,54 +98,66 @@ __device__ __forceinline__ uint32_t pack4_sat(int v0, int v1, int v2, int v3) {
 // pass: luminance blocks as in 0, chroma samples with a one-sample border read back from
 // P.chroma, every pixel's chroma = (9 own + 3 horizontally nearer + 3 vertically nearer +
 // 1 diagonal + 8) >> 4, neighbours clamped to the MCU-padded planes.
-template <bool kRefine, int kDcMode, bool kRoi = false, int kStage = 0>
+// kSamp: the record's chroma sampling (see Sampling); the triangle filter (kStage 1, 2) exists for
+// 4:2:0 only.  A greyscale record has no chroma: every pixel is (Y, Y, Y).
+template <bool kRefine, int kDcMode, bool kRoi = false, int kStage = 0, int kSamp = kSamp420>
 __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeList fl, uint8_t* __restrict__ out) {
+    using S = Sampling<kSamp>;
+    constexpr int HS = S::HS, VS = S::VS, NC = S::NC, U = S::U;
+    constexpr int kYCols = HS * U;                            // luminance blocks per block row of a unit
+    constexpr int kYBlocks = VS * kYCols;                      // luminance blocks of a unit
+    constexpr int kBlocks = kYBlocks + (NC == 3 ? 2 * U : 0);
+    constexpr int kBpm = HS * VS + (NC == 3 ? 2 : 0);          // blocks per MCU
+    constexpr int kPxW = 8 * HS, kPxH = 8 * VS;                // pixels per MCU
+    static_assert(kBlocks <= kPixThreads && kPxW * U == 128, "a unit is 128 pixels wide and has at most 64 blocks");
+    static_assert(kStage == 0 || kSamp == kSamp420, "triangle upsampling is built for 4:2:0");
     __shared__ __align__(16) uint32_t s_line[kRefine ? 32 * kPixThreads : 1];
-    __shared__ __align__(16) uint8_t s_y[16][16 * kPixMcus];
-    __shared__ __align__(16) uint8_t s_c[2][8][8 * kPixMcus];
-    __shared__ __align__(16) uint8_t s_stage[16 * kStagePitch];
+    __shared__ __align__(16) uint8_t s_y[kPxH][128];
+    __shared__ __align__(16) uint8_t s_c[2][8][8 * U];
+    __shared__ __align__(16) uint8_t s_stage[kPxH * kStagePitch];
     __shared__ __align__(16) uint16_t s_q[3][64];
     __shared__ uint8_t s_ct[kStage == 2 ? 2 : 1][kStage == 2 ? 10 : 1][kStage == 2 ? 8 * kPixMcus + 2 : 1];   // chroma tile + border
 
     const int tid = threadIdx.x;
     const Unit un = P.units[blockIdx.x];
     const ImgDesc im = P.imgs[un.img];
-    const int nm = min((int)kPixMcus, (int)im.mx - (int)un.mcol0);   // MCUs in this unit
+    const int nm = min(U, (int)im.mx - (int)un.mcol0);                // MCUs in this unit
     if (kRoi) {                                                       // whole CTA: nothing of this unit is wanted
         const CropRect r = P.roi[un.img];
-        const uint32_t ux0 = 16u * un.mcol0, uy0 = 16u * un.mrow;
-        if (ux0 >= r.x0 + r.w || ux0 + 16u * (uint32_t)nm <= r.x0 || uy0 >= r.y0 + r.h || uy0 + 16u <= r.y0) return;
+        const uint32_t ux0 = (uint32_t)kPxW * un.mcol0, uy0 = (uint32_t)kPxH * un.mrow;
+        if (ux0 >= r.x0 + r.w || ux0 + (uint32_t)(kPxW * nm) <= r.x0 || uy0 >= r.y0 + r.h || uy0 + (uint32_t)kPxH <= r.y0) return;
     }
     for (int i = tid; i < 96; i += kPixThreads)
         reinterpret_cast<uint32_t*>(&s_q[0][0])[i] = __ldg(reinterpret_cast<const uint32_t*>(P.qtab + (size_t)un.img * 192) + i);
     __syncthreads();
 
-    // ---- transform: thread j owns block j; block order Y row 0 (16), Y row 1 (16), Cb (8), Cr (8)
+    // ---- transform: thread j owns block j; block order: the unit's luminance block rows, then Cb, then Cr
     {
         const int j = tid;
         int comp = 0;
         bool valid = false;
         uint64_t blk = 0, local = 0;      // block number in the planes / inside its component
-        if (j < 32) {
-            const int r = j >> 4, c = j & 15;
-            valid = c < 2 * nm;
-            local = (uint64_t)(2 * un.mrow + r) * (2 * im.mx) + 2 * un.mcol0 + c;
+        int yr = 0, yc = 0;               // block row / column inside the unit
+        if (j < kYBlocks) {
+            yr = j / kYCols; yc = j % kYCols;
+            valid = yc < HS * nm;
+            local = (uint64_t)(VS * un.mrow + yr) * (HS * im.mx) + HS * un.mcol0 + yc;
             blk = im.blk_base + local;
-            local += 4 * (im.blk_base / 6);
-        } else if (j < kPixBlocks) {
-            const int c = (j - 32) & 7;
-            comp = 1 + ((j - 32) >> 3);
-            valid = c < nm;
-            local = (uint64_t)un.mrow * im.mx + un.mcol0 + c;
-            blk = im.blk_base + (comp == 1 ? 4ull : 5ull) * im.mx * im.my + local;
-            local += im.blk_base / 6;
+            local += (uint64_t)(HS * VS) * (im.blk_base / kBpm);
+        } else if (j < kBlocks) {
+            yc = (j - kYBlocks) % U;
+            comp = 1 + (j - kYBlocks) / U;
+            valid = yc < nm;
+            local = (uint64_t)un.mrow * im.mx + un.mcol0 + yc;
+            blk = im.blk_base + (uint64_t)(HS * VS + comp - 1) * im.mx * im.my + local;
+            local += im.blk_base / kBpm;
         }
         if (kStage == 1 && comp == 0) valid = false;          // chroma pass
         if (kStage == 2 && comp != 0) valid = false;          // pixel pass: chroma comes from the sample planes
         uint8_t* cplane = nullptr;                            // chroma pass: where this block's samples go
         if (kStage == 1 && comp != 0)
             cplane = P.chroma + (im.blk_base / 6) * 128 + (comp == 2 ? 64ull * im.mx * im.my : 0ull) +
-                     (size_t)(8 * un.mrow) * (8 * im.mx) + 8 * (un.mcol0 + ((j - 32) & 7));
+                     (size_t)(8 * un.mrow) * (8 * im.mx) + 8 * (un.mcol0 + yc);
         if (valid && kDcMode == 2) {
             // all AC zero: both passes keep only the k = 0 term, every sample of the block is equal
             constexpr uint32_t K4 = 5793;
@@ -144,8 +167,8 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
             const uint32_t w = pack4_sat(smp, smp, smp, smp);
             uint8_t* dst;
             int pitch;
-            if (j < 32) { dst = &s_y[(j >> 4) * 8][(j & 15) * 8]; pitch = 16 * kPixMcus; }
-            else { dst = &s_c[(j - 32) >> 3][0][((j - 32) & 7) * 8]; pitch = 8 * kPixMcus; }
+            if (comp == 0) { dst = &s_y[yr * 8][yc * 8]; pitch = 128; }
+            else { dst = &s_c[comp - 1][0][yc * 8]; pitch = 8 * U; }
 #pragma unroll
             for (int y = 0; y < 8; ++y) *reinterpret_cast<uint2*>(dst + y * pitch) = make_uint2(w, w);
         } else if (valid) {
@@ -233,8 +256,8 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
             uint8_t* dst;
             int pitch;
             if (kStage == 1) { dst = cplane; pitch = 8 * (int)im.mx; }
-            else if (j < 32) { dst = &s_y[(j >> 4) * 8][(j & 15) * 8]; pitch = 16 * kPixMcus; }
-            else { dst = &s_c[(j - 32) >> 3][0][((j - 32) & 7) * 8]; pitch = 8 * kPixMcus; }
+            else if (comp == 0) { dst = &s_y[yr * 8][yc * 8]; pitch = 128; }
+            else { dst = &s_c[comp - 1][0][yc * 8]; pitch = 8 * U; }
 #pragma unroll
             for (int y = 0; y < 8; ++y) {
                 idct8(v[8 * y], v[8 * y + 1], v[8 * y + 2], v[8 * y + 3], v[8 * y + 4], v[8 * y + 5], v[8 * y + 6], v[8 * y + 7],
@@ -259,9 +282,9 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
     __syncthreads();
 
     // ---- colour: 4 pixels per step, staged as the output's byte layout
-    for (int gi = tid; gi < 16 * 4 * kPixMcus; gi += kPixThreads) {
-        const int row = gi / (4 * kPixMcus), gx = gi % (4 * kPixMcus);
-        if (gx >= 4 * nm) continue;
+    for (int gi = tid; gi < kPxH * 32; gi += kPixThreads) {
+        const int row = gi / 32, gx = gi % 32;                  // 32 groups of four pixels per row
+        if (4 * gx >= kPxW * nm) continue;
         const uint32_t yw = *reinterpret_cast<const uint32_t*>(&s_y[row][4 * gx]);
         int px[12];
         if (kStage == 2) {
@@ -276,9 +299,24 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
                 px[e * 3 + 1] = Y + ((-22553 * cb - 46802 * cr + 32768) >> 16);
                 px[e * 3 + 2] = Y + ((116130 * cb + 32768) >> 16);
             }
+        } else if (NC == 1) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) px[3 * e] = px[3 * e + 1] = px[3 * e + 2] = (int)((yw >> (8 * e)) & 255u);
+        } else if (HS == 1) {
+            // every pixel its own chroma sample of row (row / VS)
+            const uint32_t cbw = *reinterpret_cast<const uint32_t*>(&s_c[0][row / VS][4 * gx]);
+            const uint32_t crw = *reinterpret_cast<const uint32_t*>(&s_c[1][row / VS][4 * gx]);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int cb = (int)((cbw >> (8 * e)) & 255u) - 128, cr = (int)((crw >> (8 * e)) & 255u) - 128;
+                const int Y = (int)((yw >> (8 * e)) & 255u);
+                px[e * 3 + 0] = Y + ((91881 * cr + 32768) >> 16);
+                px[e * 3 + 1] = Y + ((-22553 * cb - 46802 * cr + 32768) >> 16);
+                px[e * 3 + 2] = Y + ((116130 * cb + 32768) >> 16);
+            }
         } else {
-        const uint32_t cbw = *reinterpret_cast<const uint16_t*>(&s_c[0][row >> 1][2 * gx]);
-        const uint32_t crw = *reinterpret_cast<const uint16_t*>(&s_c[1][row >> 1][2 * gx]);
+        const uint32_t cbw = *reinterpret_cast<const uint16_t*>(&s_c[0][row / VS][2 * gx]);
+        const uint32_t crw = *reinterpret_cast<const uint16_t*>(&s_c[1][row / VS][2 * gx]);
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const int cb = (int)((cbw >> (8 * h)) & 255u) - 128, cr = (int)((crw >> (8 * h)) & 255u) - 128;
@@ -302,11 +340,11 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
     __syncthreads();
 
     // ---- store: each staged row is a contiguous byte run of the output
-    const int x0 = 16 * (int)un.mcol0;
-    const int npx = min(16 * nm, (int)im.W - x0);
-    const int nrows = min(16, (int)im.H - 16 * (int)un.mrow);
+    const int x0 = kPxW * (int)un.mcol0;
+    const int npx = min(kPxW * nm, (int)im.W - x0);
+    const int nrows = min(kPxH, (int)im.H - kPxH * (int)un.mrow);
     const int nbytes = 3 * npx;
-    uint8_t* gbase = out + im.out_off + ((uint64_t)(16 * un.mrow) * im.W + x0) * 3;
+    uint8_t* gbase = out + im.out_off + ((uint64_t)(kPxH * un.mrow) * im.W + x0) * 3;
     const size_t gpitch = (size_t)im.W * 3;
     if (((reinterpret_cast<uintptr_t>(gbase) | gpitch | (uintptr_t)nbytes) & 15u) == 0) {
         // rows start and end on 16-byte boundaries: whole 16-byte vectors

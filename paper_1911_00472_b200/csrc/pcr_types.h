@@ -106,6 +106,10 @@ struct Params {
     const CropRect* roi;        // [N] or null: only work units that touch the image's rectangle are transformed
     int* status;                // [N]
     int32_t N;
+    // chroma sampling of the record's images: the luminance component has hs x vs blocks per MCU
+    // (1 or 2 each), every chroma component one; nc = 3, or 1 for greyscale (then hs = vs = 1 and
+    // the block grid has no MCU padding)
+    int32_t hs, vs, nc;
 };
 
 }  // namespace pcr
