@@ -365,7 +365,12 @@ def streamed_sweep(dev, recs, ks, peak, pool=None, cores=0, tmpdir=None):
                     if got[j] != want[j]:
                         raise RuntimeError(f"sweep parity: record {i} image {j} differs from the oracle at k={k}")
                 checked += d.n_images
-        for rep in range(2):                     # first pass warms up, second is timed
+        rates = {}
+        for rep in range(4):
+            # passes 0, 1: every open parses the record (pass 0 warms up, pass 1 is timed); passes 2, 3: with
+            # the cache of closed records on, as in the second and later epochs of a loader (pass 2 fills it)
+            if rep == 2:
+                binding.pcr_set_record_cache(64 << 30)
             torch.cuda.synchronize(dev)
             t0 = time.perf_counter()
             live = []                            # handles of the records in flight, at most two
@@ -391,6 +396,9 @@ def streamed_sweep(dev, recs, ks, peak, pool=None, cores=0, tmpdir=None):
                 if code != 0:
                     raise RuntimeError(f"sweep: decode error {code} on image {bad}")
                 binding.pcr_close(h)
+            rates[rep] = dt
+        binding.pcr_set_record_cache(0)
+        dt = rates[1]
         # the outputs the timed pass left behind (last two records) against a resident decode
         for i in range(max(0, R - 2), R):
             d = decs[i]
@@ -411,6 +419,7 @@ def streamed_sweep(dev, recs, ks, peak, pool=None, cores=0, tmpdir=None):
             h2d += d.prefix_bytes(k)
         per_k[str(k)] = {"images_per_s": n_img / dt, "ms_per_record": 1000.0 * dt / R, "hbm_gbs_model": model / dt / 1e9,
                          "model_frac_of_peak": model / dt / 1e9 / peak, "h2d_bytes_per_record": h2d // R,
+                         "images_per_s_records_seen_before": n_img / rates[3],
                          "parity_images_vs_oracle": checked}
     n_per = decs[0].n_images
     for d in decs:
@@ -419,7 +428,8 @@ def streamed_sweep(dev, recs, ks, peak, pool=None, cores=0, tmpdir=None):
     hasher.shutdown()
     return {"workload": f"sweep: {R} ImageNet-shaped records x {n_per} images, streamed from pinned host memory on two CUDA "
                         "streams, each record opened (host parse, three loader threads ahead), copied, decoded and closed once per k, two in flight",
-            "timing": "wall clock around enqueue + synchronise, second of two passes",
+            "timing": "wall clock around enqueue + synchronise, second of two passes; images_per_s_records_seen_before: the same "
+                      "with pcr_set_record_cache on, every record having been opened and closed once before (a later epoch)",
             "parity": "every image of every record against the oracle's CRC-32 (streamed path, before timing) when the oracle pool runs; "
                       "the last two streamed outputs against a resident decode on the device",
             "by_k": per_k}
@@ -624,6 +634,18 @@ def main():
     open_s = reduce_max(time.perf_counter() - to, world)
     e2e["with_open_close"] = {"value": total_images * n_open / open_s, "unit": UNIT, "ms_per_step": 1000.0 * open_s / n_open,
                               "note": "pcr_open + pcr_decode from pinned host bytes + synchronise + pcr_status + pcr_close per step"}
+    binding.pcr_set_record_cache(8 << 30)
+    for _ in range(2):
+        open_decode_close()
+    sync_all()
+    to = time.perf_counter()
+    for _ in range(n_open):
+        open_decode_close()
+    open_s = reduce_max(time.perf_counter() - to, world)
+    binding.pcr_set_record_cache(0)
+    e2e["with_open_close_record_seen_before"] = {
+        "value": total_images * n_open / open_s, "unit": UNIT, "ms_per_step": 1000.0 * open_s / n_open,
+        "note": "the same with pcr_set_record_cache on: the record was opened and closed before, as in a loader's later epochs"}
 
     per_k, raise_ms, training_tensor, fidelity, baseline_jpeg = {}, {}, None, None, None
     hbm_by_k, hbm_meas_by_k = {}, {}

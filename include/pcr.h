@@ -307,7 +307,24 @@ const char* pcr_strerror(int code);
  * cudaMalloc/cudaFree each time. */
 void pcr_close(pcr_record* rec);
 
-/* Returns the cached device buffers of closed records to the driver. */
+/* Cache of closed records (Section 5: a loader reads the same records epoch after epoch).  With a
+ * limit above zero pcr_close parks the whole record (parse results, device tables and buffers:
+ * about 1.5 GB for a 1024-image ImageNet-shaped record) instead of freeing it, and a later pcr_open
+ * of the same record takes it back, which saves the host-side walk over every image's marker
+ * segments and the table uploads (about 0.7 ms per 1024 images).  The handle it returns is fresh:
+ * nothing resident, nothing decoded, default settings.  A record is recognised by the address and
+ * length of its bytes, the PCR_SLICES / PCR_LONG_MIN_BYTES settings, the current device, and a
+ * hash of its header, sample metadata, index (position and length of every chunk) and the first
+ * 256 bytes of every image's first chunk (frame header, quantisation and Huffman tables).  Bytes
+ * that changed elsewhere under the same address are the caller's responsibility, exactly as for
+ * an open handle.
+ *   max_device_bytes : device memory the parked records may hold together; the least recently
+ *                      closed ones are freed beyond it; 0 (the default) switches the cache off
+ *                      and frees what it holds.
+ * Errors: none (always PCR_OK). */
+int pcr_set_record_cache(size_t max_device_bytes);
+
+/* Returns the cached device buffers of closed records (and parked records) to the driver. */
 void pcr_release_cached_memory(void);
 
 #ifdef __cplusplus

@@ -18,7 +18,7 @@ EXPORTS = ("pcr_open", "pcr_num_images", "pcr_num_groups", "pcr_get_image", "pcr
            "pcr_decode", "pcr_evict", "pcr_status", "pcr_coeffs", "pcr_image_blocks", "pcr_launch_count",
            "pcr_strerror", "pcr_close", "pcr_get_scan", "pcr_set_profiling", "pcr_get_profile",
            "pcr_pixels_noalloc", "pcr_decode_more", "pcr_release_cached_memory", "pcr_decode_tensor", "pcr_msssim", "pcr_msssim_scratch_bytes", "pcr_set_upsampling",
-           "pcr_selftest_bounded_wait", "pcr_get_sampling")
+           "pcr_selftest_bounded_wait", "pcr_get_sampling", "pcr_set_record_cache")
 
 
 class ImageInfo(C.Structure):
@@ -76,6 +76,7 @@ def lib():
         L.pcr_get_profile.argtypes = [vp, C.POINTER(StageTime), C.c_int, C.POINTER(C.c_int)]
         L.pcr_pixels_noalloc.argtypes = [vp, C.c_uint32, C.c_uint32, vp, vp, vp]
         L.pcr_selftest_bounded_wait.argtypes = [C.POINTER(C.c_int)]
+        L.pcr_set_record_cache.argtypes = [C.c_size_t]
         L.pcr_get_sampling.argtypes = [vp, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int)]
         L.pcr_launch_count.restype = C.c_uint64
         L.pcr_launch_count.argtypes = []
@@ -227,6 +228,11 @@ def pcr_selftest_bounded_wait() -> bool:
     v = C.c_int(-1)
     _chk(lib().pcr_selftest_bounded_wait(C.byref(v)), "pcr_selftest_bounded_wait")
     return v.value == 1
+
+
+def pcr_set_record_cache(max_device_bytes: int) -> None:
+    """Park closed records (up to this much device memory) for later opens of the same bytes; 0 = off."""
+    _chk(lib().pcr_set_record_cache(max_device_bytes), "pcr_set_record_cache")
 
 
 def pcr_release_cached_memory() -> None:

@@ -204,6 +204,11 @@ struct pcr_record {
     cudaEvent_t ev_ready = nullptr;               // the record's device state is set up
     cudaEvent_t ev_done = nullptr;                // end of the last decode enqueued
     bool decode_enqueued = false;
+    // identity of the record for the cache of closed records (pcr_set_record_cache): valid when key_len != 0
+    uint64_t key_hash = 0;
+    size_t key_len = 0;
+    uint32_t key_env = 0;                         // the tuning variables read when it was opened
+    size_t device_bytes = 0;                      // what its device buffers add up to
     // optional stage timing
     bool profiling = false;
     std::vector<cudaEvent_t> events;
@@ -789,11 +794,99 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
 
 }  // namespace
 
+// ---------------------------------------------------------------------------------------
+// Cache of closed records.  A loader reads the same records epoch after epoch; with the cache
+// on, pcr_close parks the whole record (parse results, device tables and buffers) and a later
+// pcr_open of the same bytes takes it back instead of walking every image's marker segments and
+// uploading the tables again.  A record is recognised by its address, its length, the tuning
+// variables in force and a hash of its header, sample metadata, index (position and length of every
+// chunk) and the head of every image's first chunk (frame header and tables).
+// ---------------------------------------------------------------------------------------
+namespace {
+struct RecordCache {
+    std::mutex mu;
+    std::vector<pcr_record*> lru;     // most recently closed last
+    size_t bytes = 0, limit = 0;
+} g_rcache;
+
+inline uint64_t mix64(uint64_t h, uint64_t v) {
+    h ^= v + 0x9E3779B97F4A7C15ull + (h << 6) + (h >> 2);
+    h *= 0xFF51AFD7ED558CCDull;
+    return h ^ (h >> 29);
+}
+uint64_t hash_bytes(uint64_t h, const uint8_t* p, size_t n) {
+    size_t i = 0;
+    for (; i + 8 <= n; i += 8) { uint64_t v; memcpy(&v, p + i, 8); h = mix64(h, v); }
+    uint64_t tail = 0;
+    if (i < n) { memcpy(&tail, p + i, n - i); h = mix64(h, tail ^ ((uint64_t)(n - i) << 56)); }
+    return h;
+}
+uint32_t env_key() {
+    const char* a = getenv("PCR_SLICES"); const char* b = getenv("PCR_LONG_MIN_BYTES");
+    return (uint32_t)((a ? atoi(a) + 1 : 0) * 1000003 + (b ? atoi(b) + 1 : 0));
+}
+// 0 when the bytes do not even look like a record (pcr_open then reports the error)
+uint64_t record_identity(const uint8_t* rec, size_t len) {
+    if (len < 64 || len >= (1ull << 32) || memcmp(rec, "PCR1", 4) != 0) return 0;
+    const uint32_t N = rd32(rec + 8), G = rd32(rec + 12);
+    const uint64_t index_off = rd64(rec + 32), data_off = rd64(rec + 40);
+    if (N == 0 || G == 0 || G > 64 || N > (1u << 24) || data_off > len) return 0;
+    if (index_off < 64 || index_off + 8ull * (G + 1) + 16ull * G * N > data_off) return 0;
+    uint64_t h = hash_bytes(len, rec, (size_t)data_off);        // header, sample metadata, index
+    const uint8_t* chunk = rec + index_off + 8ull * (G + 1);
+    for (uint64_t j = 0; j < (uint64_t)N; ++j) {              // the chunks of scan group 1: frame header and tables of every image
+        const uint64_t off = rd64(chunk + 16 * j);
+        const uint32_t clen = rd32(chunk + 16 * j + 8);
+        if (off > len || clen > len - off) return 0;
+        h = hash_bytes(h, rec + off, std::min<size_t>(clen, 256));
+    }
+    return h ? h : 1;
+}
+void evict_records_locked(std::vector<pcr_record*>* out) {
+    while (g_rcache.bytes > g_rcache.limit && !g_rcache.lru.empty()) {
+        pcr_record* r = g_rcache.lru.front();
+        g_rcache.lru.erase(g_rcache.lru.begin());
+        g_rcache.bytes -= r->device_bytes;
+        out->push_back(r);
+    }
+}
+}  // namespace
+
 extern "C" {
+
+int pcr_set_record_cache(size_t max_device_bytes) {
+    std::vector<pcr_record*> gone;
+    {
+        std::lock_guard<std::mutex> lk(g_rcache.mu);
+        g_rcache.limit = max_device_bytes;
+        evict_records_locked(&gone);
+    }
+    for (pcr_record* r : gone) { free_device(r); delete r; }
+    return PCR_OK;
+}
 
 int pcr_open(const void* bytes, size_t len, pcr_record** rec) {
     if (rec) *rec = nullptr;
     if (!bytes || !rec) return PCR_E_ARG;
+    uint64_t key = 0;
+    const uint32_t ekey = env_key();
+    if (g_rcache.limit) {
+        key = record_identity(static_cast<const uint8_t*>(bytes), len);
+        int dev = -1;
+        cudaGetDevice(&dev);
+        std::lock_guard<std::mutex> lk(g_rcache.mu);
+        for (size_t i = g_rcache.lru.size(); key && i-- > 0;) {
+            pcr_record* c = g_rcache.lru[i];
+            if (c->host != bytes || c->key_len != len || c->key_hash != key || c->key_env != ekey || c->device != dev) continue;
+            g_rcache.lru.erase(g_rcache.lru.begin() + (long)i);
+            g_rcache.bytes -= c->device_bytes;
+            // a fresh handle: nothing resident, nothing decoded, default settings
+            c->resident = 0; c->decoded_k = 0; c->upsampling = PCR_UPSAMPLE_REPLICATE; c->profiling = false;
+            c->decode_enqueued = false;
+            *rec = c;
+            return PCR_OK;
+        }
+    }
     pcr_record* r = new (std::nothrow) pcr_record();
     if (!r) return PCR_E_NOMEM;
     int rc;
@@ -807,6 +900,8 @@ int pcr_open(const void* bytes, size_t len, pcr_record** rec) {
         delete r;
         return rc;
     }
+    r->key_hash = key; r->key_len = key ? len : 0; r->key_env = ekey;
+    for (auto& b : r->bufs) r->device_bytes += size_class(b.second);
     *rec = r;
     return PCR_OK;
 }
@@ -1177,6 +1272,15 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
 extern "C" {
 
 void pcr_release_cached_memory(void) {
+    {
+        std::vector<pcr_record*> gone;
+        {
+            std::lock_guard<std::mutex> lk(g_rcache.mu);
+            gone.swap(g_rcache.lru);
+            g_rcache.bytes = 0;
+        }
+        for (pcr_record* r : gone) { free_device(r); delete r; }
+    }
     std::lock_guard<std::mutex> lk(g_cache.mu);
     for (auto& kv : g_cache.free_) cudaFree(kv.second);
     g_cache.free_.clear();
@@ -1496,6 +1600,25 @@ int pcr_pixels_noalloc(const int16_t* dev_coeffs, uint32_t width, uint32_t heigh
 
 void pcr_close(pcr_record* rec) {
     if (!rec) return;
+    if (g_rcache.limit && rec->key_len) {
+        // park it: its set-up and its last decode have to be complete before another handle may use it
+        if (rec->up_stream) cudaStreamSynchronize(rec->up_stream);
+        if (rec->ev_done && rec->decode_enqueued) cudaEventSynchronize(rec->ev_done);
+        rec->device_bytes = 0;
+        for (auto& b : rec->bufs) rec->device_bytes += size_class(b.second);
+        std::vector<pcr_record*> gone;
+        {
+            std::lock_guard<std::mutex> lk(g_rcache.mu);
+            if (rec->device_bytes <= g_rcache.limit) {
+                g_rcache.lru.push_back(rec);
+                g_rcache.bytes += rec->device_bytes;
+                rec = nullptr;
+                evict_records_locked(&gone);
+            }
+        }
+        for (pcr_record* r : gone) { free_device(r); delete r; }
+        if (!rec) return;
+    }
     free_device(rec);
     delete rec;
 }

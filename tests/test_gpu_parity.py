@@ -257,3 +257,43 @@ def test_two_records_in_flight_on_two_streams(monkeypatch, rec1_small, rec2_smal
         for d in decs:
             if d is not None:
                 d.close()
+
+
+def test_record_cache_reopens_the_same_record_and_only_that(rec0, rec1_small):
+    """With the cache of closed records on, reopening the same bytes gives a fresh handle that
+    decodes to the same result; other bytes, or the same bytes changed in what pcr_open reads, are
+    parsed anew."""
+    import torch
+    from paper_1911_00472_b200 import Decoder, binding
+    binding.pcr_set_record_cache(1 << 30)
+    try:
+        dec = Decoder(rec0.bytes)
+        host = dec.host                                   # keep the pinned bytes: the identity includes their address
+        want = dec.decode(7).clone()
+        torch.cuda.synchronize()
+        dec.close()
+        n0 = binding.pcr_launch_count()
+        h = binding.pcr_open(host.data_ptr(), host.numel())      # a hit: no set-up kernel is launched
+        assert binding.pcr_launch_count() == n0
+        out = torch.zeros_like(want)
+        with pytest.raises(binding.PcrError):             # a fresh handle: nothing decoded yet
+            binding.pcr_decode_more(h, 9, out.data_ptr(), 0)
+        binding.pcr_decode(h, 7, out.data_ptr(), 0)
+        torch.cuda.synchronize()
+        assert binding.pcr_status(h) == (-1, 0)
+        assert torch.equal(out, want)
+        binding.pcr_close(h)
+        # a label changes (sample metadata is part of what pcr_open reads): parsed anew, new label seen
+        host[64] ^= 0x5A
+        n1 = binding.pcr_launch_count()
+        h = binding.pcr_open(host.data_ptr(), host.numel())
+        assert binding.pcr_launch_count() == n1 + 1        # the set-up kernel of a real open
+        assert binding.pcr_get_image(h, 0).label == (dec.info[0].label ^ 0x5A)
+        binding.pcr_close(h)
+        host[64] ^= 0x5A
+        # another record is not confused with it
+        other = Decoder(rec1_small.bytes)
+        assert other.n_images == rec1_small.n_images
+        other.close()
+    finally:
+        binding.pcr_set_record_cache(0)
