@@ -21,6 +21,9 @@
 
 namespace pcr {
 
+#ifndef PCR_PIX_MIN_CTAS
+#define PCR_PIX_MIN_CTAS 1                    // CTAs per SM the compiler must leave registers for
+#endif
 constexpr int kPixMcus = 8;                   // MCUs per CTA (4:2:0)
 constexpr int kPixThreads = 64;               // one thread per block for the transform
 constexpr int kStagePitch = 3 * 128 + 16;     // bytes per staged RGB row (+ spare, keeps rows 16-byte aligned)
@@ -101,7 +104,7 @@ __device__ __forceinline__ uint32_t pack4_sat(int v0, int v1, int v2, int v3) {
 // kSamp: the record's chroma sampling (see Sampling); the triangle filter (kStage 1, 2) exists for
 // 4:2:0 only.  A greyscale record has no chroma: every pixel is (Y, Y, Y).
 template <bool kRefine, int kDcMode, bool kRoi = false, int kStage = 0, int kSamp = kSamp420>
-__global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeList fl, uint8_t* __restrict__ out) {
+__global__ void __launch_bounds__(kPixThreads, PCR_PIX_MIN_CTAS) pixel_kernel(Params P, FinalizeList fl, uint8_t* __restrict__ out) {
     using S = Sampling<kSamp>;
     constexpr int HS = S::HS, VS = S::VS, NC = S::NC, U = S::U;
     constexpr int kYCols = HS * U;                            // luminance blocks per block row of a unit
@@ -176,6 +179,19 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
             uint4 raw[8];
             const uint4* headv = reinterpret_cast<const uint4*>(P.head + blk * 8);
             if (kRefine && fl.n[comp] > 0) {
+                // the side data of the first two refinement scans is requested before the lines: all of the
+                // block's loads are then in flight together
+                const int nref = fl.n[comp];
+                const ulonglong2 zero2 = make_ulonglong2(0ull, 0ull);
+                ulonglong2 a0 = zero2, b0 = zero2, a1 = zero2, b1 = zero2;
+                {
+                    const ulonglong2* o = reinterpret_cast<const ulonglong2*>(P.aux + fl.base[comp][0] + local * 4);
+                    a0 = __ldg(o); b0 = __ldg(o + 1);                        // {mask, corrections}, {new, signs}
+                    if (nref > 1) {
+                        const ulonglong2* o1 = reinterpret_cast<const ulonglong2*>(P.aux + fl.base[comp][1] + local * 4);
+                        a1 = __ldg(o1); b1 = __ldg(o1 + 1);
+                    }
+                }
                 if (kDcMode == 3) {
 #pragma unroll
                     for (int q = 1; q < 8; ++q) raw[q] = make_uint4(0, 0, 0, 0);
@@ -190,34 +206,52 @@ __global__ void __launch_bounds__(kPixThreads) pixel_kernel(Params P, FinalizeLi
                     col[(4 * q) * kPixThreads] = raw[q].x; col[(4 * q + 1) * kPixThreads] = raw[q].y;
                     col[(4 * q + 2) * kPixThreads] = raw[q].z; col[(4 * q + 3) * kPixThreads] = raw[q].w;
                 }
-                bool dirty = false;
-                for (int i = 0; i < fl.n[comp]; ++i) {
+                uint32_t dirty = 0;                                         // 16-byte chunks of the line that changed
+                for (int i = 0; i < nref; ++i) {
                     const int p1 = fl.p1[comp][i];
-                    const ulonglong2* o = reinterpret_cast<const ulonglong2*>(P.aux + fl.base[comp][i] + local * 4);
-                    const ulonglong2 a = __ldg(o), b = __ldg(o + 1);       // {mask, corrections}, {new, signs}
-                    uint64_t h = a.x & ~b.x, cc = a.y;
-                    while (cc) {
-                        const int pos = __ffsll((long long)h) - 1;
-                        if (pos < 0) break;
-                        h &= h - 1;
-                        if (cc >> 63) {
-                            int16_t* e = reinterpret_cast<int16_t*>(col + (pos >> 1) * kPixThreads) + (pos & 1);
-                            const int v = *e;
-                            if ((v & p1) == 0) { *e = (int16_t)(v >= 0 ? v + p1 : v - p1); dirty = true; }
-                        }
-                        cc <<= 1;
+                    ulonglong2 a = i == 0 ? a0 : a1, b = i == 0 ? b0 : b1;
+                    if (i > 1) {
+                        const ulonglong2* o = reinterpret_cast<const ulonglong2*>(P.aux + fl.base[comp][i] + local * 4);
+                        a = __ldg(o); b = __ldg(o + 1);
                     }
-                    uint64_t nw = b.x;
-                    while (nw) {
-                        const int pos = __ffsll((long long)nw) - 1;
-                        nw &= nw - 1;
-                        *(reinterpret_cast<int16_t*>(col + (pos >> 1) * kPixThreads) + (pos & 1)) = (int16_t)(((b.y >> pos) & 1ull) ? p1 : -p1);
-                        dirty = true;
+                    // corrections: the coefficients that were non-zero before the scan, in zigzag order, take the
+                    // correction bits in reading order (from bit 63 down); the walk ends with the last set bit.
+                    // Positions 0..31 and 32..63 are walked as 32-bit masks.
+                    const uint64_t hist = a.x & ~b.x;
+                    uint64_t cc = a.y;
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        uint32_t h32 = half ? (uint32_t)(hist >> 32) : (uint32_t)hist;
+                        uint32_t* hb = col + half * 16 * kPixThreads;
+                        while (h32 && cc) {
+                            const int pos = __ffs((int)h32) - 1;
+                            h32 &= h32 - 1u;
+                            if ((long long)cc < 0) {
+                                int16_t* e = reinterpret_cast<int16_t*>(hb + (pos >> 1) * kPixThreads) + (pos & 1);
+                                const int v = *e;
+                                if ((v & p1) == 0) { *e = (int16_t)(v >= 0 ? v + p1 : v - p1); dirty |= 1u << ((pos >> 3) + 4 * half); }
+                            }
+                            cc <<= 1;
+                        }
+                    }
+                    // new coefficients: +-2^Al at positions that were zero
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        uint32_t nw = half ? (uint32_t)(b.x >> 32) : (uint32_t)b.x;
+                        const uint32_t sg = half ? (uint32_t)(b.y >> 32) : (uint32_t)b.y;
+                        uint32_t* hb = col + half * 16 * kPixThreads;
+                        while (nw) {
+                            const int pos = __ffs((int)nw) - 1;
+                            nw &= nw - 1u;
+                            *(reinterpret_cast<int16_t*>(hb + (pos >> 1) * kPixThreads) + (pos & 1)) = (int16_t)(((sg >> pos) & 1u) ? p1 : -p1);
+                            dirty |= 1u << ((pos >> 3) + 4 * half);
+                        }
                     }
                 }
-                if (dirty) {
+                // only the chunks that changed are read back and written to the planes
 #pragma unroll
-                    for (int q = 0; q < 8; ++q) {
+                for (int q = 0; q < 8; ++q) {
+                    if ((dirty >> q) & 1u) {
                         raw[q] = make_uint4(col[(4 * q) * kPixThreads], col[(4 * q + 1) * kPixThreads],
                                             col[(4 * q + 2) * kPixThreads], col[(4 * q + 3) * kPixThreads]);
                         if (q == 0 && kDcMode != 0) *reinterpret_cast<uint4*>(P.head + blk * 8) = raw[0];

@@ -269,6 +269,7 @@ def test_record_cache_reopens_the_same_record_and_only_that(rec0, rec1_small):
     try:
         dec = Decoder(rec0.bytes)
         host = dec.host                                   # keep the pinned bytes: the identity includes their address
+        dec.out = torch.zeros(dec.out_bytes, dtype=torch.uint8, device="cuda")    # bytes between images are never written
         want = dec.decode(7).clone()
         torch.cuda.synchronize()
         dec.close()
