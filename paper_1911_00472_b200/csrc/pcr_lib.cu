@@ -601,7 +601,7 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     r->item_begin.assign((size_t)r->n_slices * G, 0); r->item_count.assign((size_t)r->n_slices * G, 0);
     // A scan that is one restart interval of at least this many bytes goes to the kernels for long
     // intervals; DC refinement scans have a kernel of their own and no items at all.
-    uint32_t long_min = 1024;
+    uint32_t long_min = 64;
     if (const char* e = getenv("PCR_LONG_MIN_BYTES")) long_min = (uint32_t)std::max(0, atoi(e));
     auto is_long = [&](int s, uint32_t i) {
         const ScanScript& sc = r->script[s];

@@ -414,10 +414,17 @@ __device__ __forceinline__ bool wait_at_least(const volatile uint32_t* flag, uin
     return false;
 }
 
+// Entry of the chain's own lookup table on the next kChainLutBits bits, made from the Huffman table:
+// bits 0..4 = bits to skip (code, plus the sign bit of a new coefficient), 5..8 = run r, 9 = a new
+// coefficient follows the run; 0 = everything else (end-of-band runs, codes longer than the index,
+// undefined codes), which takes the general path.
 struct ChainShared {
     HuffTabT<kChainLutBits> tab;
+    uint32_t quick[1 << kChainLutBits];
     uint32_t ring[kChainRing];
     uint64_t h[32];
+    uint8_t zpos[64][32];              // [i][block]: position of the block's i-th still-zero coefficient of the band
+    uint8_t nz[32];                    // how many there are
     uint2 rec[kChainRecs];             // {bit position behind the sign bit, corrections | position << 7 | new << 13}
     uint32_t first[33];                // first record of each block of the batch
 };
@@ -444,6 +451,12 @@ __global__ void __launch_bounds__(32 * kGroupWarps) ac_refine_group_kernel(Param
     ChainShared& sh = s_sh[wid];
     volatile uint32_t* my_progress = &s_progress[wid];
     build_hufftab(sh.tab, P.rec + sd.tab_off[0], lane);
+    for (int i = lane; i < (1 << kChainLutBits); i += 32) {
+        const uint32_t e = sh.tab.lut[i], len = e >> 8, rs = e & 255u, newc = rs & 1u, r = rs >> 4;
+        const bool plain = e != 0 && (rs & 14u) == 0 && (newc || r == 15u);   // a run followed by a new coefficient, or sixteen zeros
+        sh.quick[i] = plain ? ((len + newc) | (r << 5) | (newc << 9)) : 0u;
+    }
+    __syncwarp();
     const uint32_t* segtab = P.seg_start + sd.seg_base;
     const uint32_t bstart = segtab[0], bend = segtab[1] - 2u;
     if (bstart < sd.data_off || bend > sd.data_end || bend < bstart) {
@@ -475,7 +488,6 @@ __global__ void __launch_bounds__(32 * kGroupWarps) ac_refine_group_kernel(Param
     }
     uint64_t* outp = P.aux + ax.base + g.loff[c] * 4ull;
     uint32_t* ring = sh.ring;
-    const uint16_t* lut = sh.tab.lut;
     uint32_t wr = rd0;                                         // next word to fetch
     ChainBits B;
     B.ring = ring; B.w0 = B.w1 = B.w2 = 0; B.o = 0; B.rd = rd0; B.base = rd0;
@@ -496,7 +508,22 @@ __global__ void __launch_bounds__(32 * kGroupWarps) ac_refine_group_kernel(Param
             if (src1) v |= __ldcg(src1 + (uint64_t)bi * st1);
             if (src2) v |= __ldcg(src2 + (uint64_t)bi * st2);
             if (src3) v |= __ldcg(src3 + (uint64_t)bi * st3);
-            sh.h[lane] = v & band;
+            v &= band;
+            sh.h[lane] = v;
+            // the positions of the band that are still zero, in order: the target of a run r is then one
+            // table look-up for lane 0 (the (r+1)-th of those not yet passed).  (Listing the few non-zero
+            // positions instead and stepping over them measured 18 % slower: the steps sit on lane 0's chain.)
+            const uint64_t z = ~v & band;
+            uint32_t n = 0;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t w = half ? (uint32_t)(z >> 32) : (uint32_t)z;
+                while (w) {
+                    sh.zpos[n++][lane] = (uint8_t)(32 * half + __ffs((int)w) - 1);
+                    w &= w - 1u;
+                }
+            }
+            sh.nz[lane] = (uint8_t)n;
         }
         const uint32_t rd_now = __shfl_sync(full, B.rd - (primed ? 3u : 0u), 0);   // lane 0's reader: w0 is the oldest word still in use
         while (wr - rd_now + 32u <= (uint32_t)kChainRing) {
@@ -512,53 +539,47 @@ __global__ void __launch_bounds__(32 * kGroupWarps) ac_refine_group_kernel(Param
             for (; nd < nblk; ++nd) {
                 if (wr - B.rd < kChainBlockWords || nrec > (uint32_t)kChainRecs - 64u) break;   // fetch more / flush first
                 sh.first[nd] = nrec;
-                uint64_t Hs = sh.h[nd] >> Ss;                  // non-zero positions; bit 0 = the position that comes next
-                uint32_t k = Ss, rem = Se - Ss + 1u;
+                // k: the position that comes next; zi: how many of the block's zero positions lie below it
+                const uint32_t nz = sh.nz[nd];
+                uint32_t k = Ss, zi = 0;
                 if (eobrun == 0) {
-                    while (rem) {
+                    while (k <= Se) {
                         const uint32_t win = B.win();
-                        uint32_t e = lut[win >> (32 - kChainLutBits)];
-                        if (e == 0) { e = huff_lookup(sh.tab, win); if (e == 0) { err = kErrCorrupt; break; } }
-                        const uint32_t len = e >> 8, rs = e & 255u;
-                        if (rs & 14u) { err = kErrCorrupt; break; }   // a refinement symbol has size 0 or 1
-                        const uint32_t newc = rs & 1u, r = rs >> 4;
-                        if (rs < 0xF0u && !newc) {             // end of band for this block and eobrun - 1 more
-                            eobrun = 1u << r;
-                            if (r) eobrun += (win << len) >> (32u - r);
-                            B.skip(len + r);
-                            break;
-                        }
-                        B.skip(len + newc);                    // the sign comes before the correction bits
-                        // distance d of the (r+1)-th position that is still zero: d = r + (non-zero positions up to d),
-                        // iterated from d = r; the count reached is the number of correction bits that follow
-                        uint32_t d = r, cnt = 0;
-                        {
-                            const uint32_t lo = (uint32_t)Hs;
-                            bool settled = false;
-                            while (d < 32u) {
-                                cnt = (uint32_t)__popc(lo & ((2u << d) - 1u));
-                                if (r + cnt == d) { settled = true; break; }
-                                d = r + cnt;
+                        uint32_t q = sh.quick[win >> (32 - kChainLutBits)];
+                        if (q == 0) {                          // not a plain (run, new coefficient) symbol
+                            const uint32_t e = huff_lookup(sh.tab, win);
+                            const uint32_t len = e >> 8, rs = e & 255u, newc = rs & 1u, r = rs >> 4;
+                            if (e == 0 || (rs & 14u)) { err = kErrCorrupt; break; }   // a refinement symbol has size 0 or 1
+                            if (!newc && r < 15u) {            // end of band for this block and eobrun - 1 more
+                                eobrun = 1u << r;
+                                if (r) eobrun += (win << len) >> (32u - r);
+                                B.skip(len + r);
+                                break;
                             }
-                            while (!settled) {                 // beyond the low word (d <= 78)
-                                cnt = (uint32_t)__popcll(Hs & low_mask((int)d + 1));
-                                if (r + cnt == d) break;
-                                d = r + cnt;
-                            }
+                            q = (len + newc) | (r << 5) | (newc << 9);   // a code longer than the table's index
                         }
-                        uint32_t flag = newc;
-                        if (d >= rem) { d = rem; cnt = (uint32_t)__popcll(Hs); flag = 0; }   // past the band: nothing new
-                        sh.rec[nrec++] = make_uint2(B.pos(), cnt | ((k + d) << 7) | (flag << 13));
+                        B.skip(q & 31u);                       // the code and, for a new coefficient, its sign
+                        const uint32_t r = (q >> 5) & 15u, t = zi + r;
+                        uint32_t cnt, pos, flag;
+                        if (t < nz) {                          // the target: the (r+1)-th zero position from here
+                            pos = sh.zpos[t][nd];
+                            cnt = pos - k - r;                 // the non-zero positions passed: one correction bit each
+                            flag = q >> 9;
+                            zi = t + 1u;
+                        } else {                               // past the band: the rest is passed over, nothing new
+                            pos = Se + 1u;
+                            cnt = pos - k - (nz - zi);
+                            flag = 0;
+                            zi = nz;
+                        }
+                        sh.rec[nrec++] = make_uint2(B.pos(), cnt | ((pos & 63u) << 7) | (flag << 13));
                         if (cnt > 32u) { B.skip(32u); B.skip(cnt - 32u); } else B.skip(cnt);
-                        const uint32_t adv = min(d + 1u, rem);
-                        k += adv;
-                        rem -= adv;
-                        Hs >>= adv;                            // adv <= 63
+                        k = pos + 1u;
                     }
                 }
                 if (err) break;
-                if (rem) {                                     // inside an end-of-band run: corrections for the rest of the band
-                    const uint32_t cnt = (uint32_t)__popcll(Hs);
+                if (k <= Se) {                                 // inside an end-of-band run: corrections for the rest of the band
+                    const uint32_t cnt = Se + 1u - k - (nz - zi);
                     sh.rec[nrec++] = make_uint2(B.pos(), cnt);
                     if (cnt > 32u) { B.skip(32u); B.skip(cnt - 32u); } else B.skip(cnt);
                     --eobrun;

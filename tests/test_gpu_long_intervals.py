@@ -48,7 +48,7 @@ def _compare_every_k(rec, min_bytes, monkeypatch):
         dec.close()
 
 
-@pytest.mark.parametrize("min_bytes", [0, 1024])
+@pytest.mark.parametrize("min_bytes", [0, 1 << 20])
 def test_ham_shaped_small(rec3_small, min_bytes, monkeypatch):
     _compare_every_k(rec3_small, min_bytes, monkeypatch)
 

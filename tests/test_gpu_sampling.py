@@ -56,7 +56,7 @@ def test_with_restart_markers(name, config):
 
 
 @pytest.mark.parametrize("name", sorted(SAMPLINGS))
-@pytest.mark.parametrize("min_bytes", [0, 1024])
+@pytest.mark.parametrize("min_bytes", [0, 1 << 20])
 def test_without_restart_markers(name, min_bytes, monkeypatch):
     with pcr_synth.sampling(*SAMPLINGS[name]):
         rec = pcr_synth.make_record(3, n_images=2, restart_rows=False)
