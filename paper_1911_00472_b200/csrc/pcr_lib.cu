@@ -606,7 +606,7 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     auto is_long = [&](int s, uint32_t i) {
         const ScanScript& sc = r->script[s];
         const ScanDesc& sd = scans[(size_t)s * N + i];
-        if (sc.Ss == 0 && sc.Se == 63) return false;           // a baseline record's sequential scan
+        (void)sc;
         return sd.nseg == 1 && sd.data_end - sd.data_off >= long_min;
     };
     // the AC refinements of one component of one image go together: all of them one interval each,
@@ -1071,10 +1071,18 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
                 if (!count) begin = rec->item_begin[(size_t)g * G + s];
                 count += rec->item_count[(size_t)g * G + s];
             }
-            if (count && sequential) {
-                if (roi) sequential_kernel<true><<<(count + kSeqWarps - 1) / kSeqWarps, 32 * kSeqWarps, 0, q>>>(P, begin, count);
-                else sequential_kernel<false><<<(count + kSeqWarps - 1) / kSeqWarps, 32 * kSeqWarps, 0, q>>>(P, begin, count);
-                ++g_launches;
+            if (sequential) {
+                if (count) {
+                    if (roi) sequential_kernel<true><<<(count + kSeqWarps - 1) / kSeqWarps, 32 * kSeqWarps, 0, q>>>(P, begin, count);
+                    else sequential_kernel<false><<<(count + kSeqWarps - 1) / kSeqWarps, 32 * kSeqWarps, 0, q>>>(P, begin, count);
+                    ++g_launches;
+                }
+                const int s0 = rec->wave_scans[w][0];      // the record's one scan
+                const uint32_t lc = (s0 >= k0 && s0 < k) ? rec->long_count[(size_t)g * G + s0] : 0u;
+                if (lc) {                                  // images whose scan is one long restart interval
+                    sequential_long_kernel<<<(lc + kSeqLongWarps - 1) / kSeqLongWarps, 32 * kSeqLongWarps, 0, q>>>(P, rec->d_long + rec->long_begin[(size_t)g * G + s0], lc);
+                    ++g_launches;
+                }
                 return true;
             }
             if (count) {

@@ -2,7 +2,7 @@
 // markers: one entropy-coded segment per image and scan), and the DC refinement scans of any record.
 //
 // A Huffman stream is a serial chain, so a whole scan on one lane takes tens of thousands of
-// dependent steps.  Three kernels shorten or remove that chain:
+// dependent steps.  These kernels shorten or remove that chain:
 //
 //  * dc_refine_kernel: a DC refinement scan carries exactly one raw bit per block, so after
 //    unstuffing bit j of a restart interval is block j of the interval in scan order: one thread
@@ -17,6 +17,7 @@
 //    the true beginning, so after round r lanes 0..r are exact).  A prefix sum of the blocks each
 //    lane finished (and of the DC differences per component) gives every lane its first block and
 //    its predictors, and a last pass decodes once more and writes.
+//  * sequential_long_kernel: the same scheme for the one scan of a baseline JPEG.
 //  * ac_refine_group_kernel: an AC refinement cannot be entered in the middle (how many correction
 //    bits follow a symbol depends on which coefficients of the block are already non-zero, i.e. on
 //    the block number).  One warp per scan: lane 0 walks the chain with ordinary branches (no other
@@ -345,6 +346,158 @@ __global__ void __launch_bounds__(32 * kLongWarps) first_pass_long_kernel(Params
         ac_first_span<true>(tab, base, pos, k, my_end, Ss, Se, pos_x, k_x, nb, W, bad);
         if (all < total) bad = true;                                         // the stream ends before the last block
     }
+    if (__any_sync(full, bad) && lane == 0) atomicMin(&P.status[img], kErrCorrupt);
+}
+
+// ---------------------------------------------------------------------------------------
+// A sequential (baseline) scan that is one restart interval: the same scheme as the first passes.
+// The state a lane hands on is (bit position, block of the MCU, zigzag position inside the block;
+// 0 = the block's DC symbol comes next); every lane counts the blocks it finishes and sums the DC
+// differences it reads per component.
+// ---------------------------------------------------------------------------------------
+struct SeqWrite {
+    int16_t* head;
+    int16_t* planes;
+    uint64_t coff[3];
+    uint32_t bw[3];
+    uint32_t mcu_w;
+    uint32_t hs, vs;
+    uint32_t n, n1;        // next block of the scan in scan order (the one being decoded), one past the last
+    int pred[3];
+};
+
+template <bool kWrite>
+__device__ __forceinline__ void seq_span(const HuffTab* tabs4, uint32_t slots, uint32_t slots_ac, int nc, const uint32_t* base,
+                                         uint32_t pos, int j, int k, uint32_t pos_end, uint32_t& pos_out, int& j_out, int& k_out,
+                                         uint32_t& nblk, int& sum0, int& sum1, int& sum2, SeqWrite& W, bool& bad) {
+    WordReader br;
+    br.init(base, pos);
+    const int ny = (int)(W.hs * W.vs), bpm = nc == 3 ? ny + 2 : 1;
+    uint32_t nb = 0;
+    int s0 = 0, s1 = 0, s2 = 0;
+    uint32_t mrow = 0, mcol = 0;
+    if (kWrite) { const uint32_t m = W.n / (uint32_t)bpm; mrow = m / W.mcu_w; mcol = m - mrow * W.mcu_w; }
+    bool stop = kWrite && W.n >= W.n1;
+    while (!stop && br.pos() < pos_end) {
+        br.refill();
+        const uint32_t win = br.top32();
+        const int c = nc == 3 ? (j < ny ? 0 : j - ny + 1) : 0;
+        const bool is_dc = k == 0;
+        const int ti = is_dc ? (int)((slots >> (2 * c)) & 1u) : 2 + (int)((slots_ac >> (2 * c)) & 1u);
+        const uint32_t e = huff_lookup(tabs4[ti], win);
+        const int len = (int)(e >> 8), r = is_dc ? 0 : (int)(e >> 4) & 15, sz = is_dc ? (int)(e & 255u) : (int)(e & 15u);
+        const bool is_coef = sz != 0, is_zrl = !is_dc && sz == 0 && r == 15, is_eob = !is_dc && sz == 0 && r == 0;
+        const int kk = k + r;
+        if (e == 0 || sz > 15 || (!is_dc && !is_coef && !is_zrl && !is_eob) || (is_coef && kk > 63)) {
+            if (kWrite) { bad = true; break; }
+            br.skip(1);
+            continue;
+        }
+        const int extra = is_coef ? sz : 0;
+        const int v = extend_bits(top_bits(win << len, extra), extra);
+        br.skip(len + extra);
+        uint64_t blk = 0;
+        if (kWrite) {
+            if (nc == 3 && c == 0) blk = W.coff[0] + (uint64_t)(W.vs * mrow + ((uint32_t)j >> (W.hs - 1u))) * W.bw[0] + W.hs * mcol + ((uint32_t)j & (W.hs - 1u));
+            else blk = W.coff[c] + (uint64_t)mrow * W.bw[c] + mcol;
+        }
+        if (is_dc) {
+            if (c == 0) s0 += v; else if (c == 1) s1 += v; else s2 += v;
+            if (kWrite) {
+                const int pv = (c == 0 ? W.pred[0] : (c == 1 ? W.pred[1] : W.pred[2])) + v;
+                if (c == 0) W.pred[0] = pv; else if (c == 1) W.pred[1] = pv; else W.pred[2] = pv;
+                W.head[blk * 8] = (int16_t)pv;
+            }
+            k = 1;
+        } else if (is_coef) {
+            if (kWrite) {
+                if (kk < 8) W.head[blk * 8 + kk] = (int16_t)v;
+                else W.planes[blk * 64 + kk] = (int16_t)v;
+            }
+            k = kk + 1;
+        } else if (is_zrl) {
+            k += 16;
+        }
+        if (is_eob || k > 63) {                               // block finished
+            k = 0;
+            ++nb;
+            if (kWrite && ++W.n >= W.n1) stop = true;
+            if (++j == bpm) {
+                j = 0;
+                if (kWrite) { if (++mcol == W.mcu_w) { mcol = 0; ++mrow; } }
+            }
+        }
+    }
+    pos_out = br.pos();
+    j_out = j;
+    k_out = k;
+    nblk = nb;
+    sum0 = s0; sum1 = s1; sum2 = s2;
+}
+
+constexpr int kSeqLongWarps = 2;
+
+__global__ void __launch_bounds__(32 * kSeqLongWarps) sequential_long_kernel(Params P, const uint32_t* __restrict__ list, uint32_t count) {
+    __shared__ HuffTab tabs[kSeqLongWarps][4];                // DC 0, DC 1, AC 0, AC 1
+    const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t it = blockIdx.x * kSeqLongWarps + wid;
+    if (it >= count) return;                                   // whole warp
+    const uint32_t si = list[it];
+    const int img = (int)(si % (uint32_t)P.N);
+    const ScanDesc sd = P.scans[si];
+    const ImgDesc im = P.imgs[img];
+    const Geometry g = make_geometry(im, P);
+    const uint32_t mcu_w = g.mx, total = g.mx * g.my;
+    const uint32_t bpm = P.nc == 3 ? (uint32_t)(P.hs * P.vs + 2) : 1u;
+    const unsigned full = 0xffffffffu;
+    build_hufftab(tabs[wid][0], P.rec + sd.tab_off[0], lane);
+    if (sd.tab_off[1]) build_hufftab(tabs[wid][1], P.rec + sd.tab_off[1], lane);
+    build_hufftab(tabs[wid][2], P.rec + sd.tab_ac[0], lane);
+    if (sd.tab_ac[1]) build_hufftab(tabs[wid][3], P.rec + sd.tab_ac[1], lane);
+    const uint32_t* segtab = P.seg_start + sd.seg_base;
+    const uint32_t bstart = segtab[0], bend = segtab[1] - 2u;
+    if (bstart < sd.data_off || bend > sd.data_end || bend < bstart) {
+        if (lane == 0) atomicMin(&P.status[img], kErrCorrupt);
+        return;
+    }
+    const uint32_t* base = reinterpret_cast<const uint32_t*>(P.ubuf) + (bstart >> 2);
+    const uint32_t lead = 8u * (bstart & 3u), endbit = lead + 8u * (bend - bstart);
+    const uint32_t nwords = (endbit + 31u) >> 5;
+    const uint32_t S = 32u * max(8u, (nwords + 31u) / 32u);
+    const uint32_t my_begin = min(max((uint32_t)lane * S, lead), endbit), my_end = min(((uint32_t)lane + 1u) * S, endbit);
+    bool bad = false;
+    SeqWrite W;
+    W.head = P.head; W.planes = P.planes; W.mcu_w = mcu_w; W.hs = (uint32_t)P.hs; W.vs = (uint32_t)P.vs;
+#pragma unroll
+    for (int c = 0; c < 3; ++c) { W.coff[c] = g.coff[c]; W.bw[c] = g.bw[c]; W.pred[c] = 0; }
+    W.n = 0; W.n1 = total * bpm;
+    uint32_t pos = my_begin, pos_x = my_begin, nb = 0;
+    int j = 0, k = 0, j_x = 0, k_x = 0, a0 = 0, a1 = 0, a2 = 0;
+    bool again = true;
+    for (int round = 0; round < 33; ++round) {
+        if (again) seq_span<false>(tabs[wid], sd.slots, sd.slots_ac, P.nc, base, pos, j, k, my_end, pos_x, j_x, k_x, nb, a0, a1, a2, W, bad);
+        const uint32_t ppos = min(__shfl_up_sync(full, pos_x, 1), endbit);
+        const int pj = __shfl_up_sync(full, j_x, 1), pk = __shfl_up_sync(full, k_x, 1);
+        again = lane > 0 && (ppos != pos || pj != j || pk != k);
+        if (again) { pos = ppos; j = pj; k = pk; }
+        if (!__any_sync(full, again)) break;
+    }
+    uint32_t nin = nb;
+    int b0 = a0, b1 = a1, b2 = a2;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t on = __shfl_up_sync(full, nin, d);
+        const int o0 = __shfl_up_sync(full, b0, d), o1 = __shfl_up_sync(full, b1, d), o2 = __shfl_up_sync(full, b2, d);
+        if (lane >= d) { nin += on; b0 += o0; b1 += o1; b2 += o2; }
+    }
+    const uint32_t all = __shfl_sync(full, nin, 31);
+    W.n = min(nin - nb, W.n1); W.pred[0] = b0 - a0; W.pred[1] = b1 - a1; W.pred[2] = b2 - a2;
+    // the place inside the MCU follows from the block number (equal to the handed-on state unless the
+    // stream is damaged; taking it from the block number keeps every store inside the image)
+    if ((nb || k) && (uint32_t)j != W.n % bpm) bad = true;
+    j = (int)(W.n % bpm);
+    seq_span<true>(tabs[wid], sd.slots, sd.slots_ac, P.nc, base, pos, j, k, my_end, pos_x, j_x, k_x, nb, a0, a1, a2, W, bad);
+    if (all < total * bpm) bad = true;                         // the stream ends before the last block
     if (__any_sync(full, bad) && lane == 0) atomicMin(&P.status[img], kErrCorrupt);
 }
 
