@@ -70,7 +70,7 @@ def whole_job_rate(images_this_rank: int, steps: int, ms_this_rank: float, world
     return total * steps / (ms / 1000.0)
 
 
-def algorithmic_bytes(scans, infos, k: int):
+def algorithmic_bytes(scans, infos, k: int, chains: bool = False):
     """Bytes the method has to move for one decode at fidelity k, per stage.
 
     scans: [(ncomp, comp0, Ss, Se, Ah, wave, group_bytes)], infos: [(W, H)].
@@ -80,10 +80,13 @@ def algorithmic_bytes(scans, infos, k: int):
                  refinement).  The refinement's share is what the method has to move for that
                  step; this implementation moves it in the pixel kernel, which folds the
                  refinement side data into the planes before it transforms a block.
+      chains   : (records without restart markers) the AC refinements' share of the above, when the
+                 library runs them as one stage of their own
       clear    : 128 bytes per block
       pixels   : 128 bytes per block read + 3 bytes per pixel written
     """
     out = {"index": 0.0, "clear": 0.0, "pixels": 0.0}
+    ac_refine = {}
     blocks_pad = 0
     blocks_unp = [0, 0, 0]
     px = 0
@@ -105,7 +108,14 @@ def algorithmic_bytes(scans, infos, k: int):
         nb = blocks_pad if ncomp > 1 else blocks_unp[comp0]
         key = f"entropy{wave}"
         out[key] = out.get(key, 0.0) + gbytes + 2.0 * band * nb * (2 if Ah else 1)
+        if Ah and Ss > 0:
+            ac_refine[key] = ac_refine.get(key, 0.0) + gbytes + 4.0 * band * nb
     out["total"] = sum(out.values())
+    if chains:          # the AC refinements ran as one stage of their own: their share moves there
+        out["chains"] = 0.0
+        for key, v in ac_refine.items():
+            out[key] -= v
+            out["chains"] += v
     return out
 
 
@@ -770,7 +780,7 @@ def main():
             stage_ms[name] = stage_ms.get(name, 0.0) + t / reps
             stage_n[name] = nl
     binding.pcr_set_profiling(dec.handle, False)
-    model = algorithmic_bytes(scans, infos, k)
+    model = algorithmic_bytes(scans, infos, k, chains=stage_n.get("chains", 0) > 0)
     kernels = {n: t for n, t in stage_ms.items() if stage_n.get(n, 0) > 0}
     dom = max(kernels, key=kernels.get)
     peak, peak_src = hbm_peak()

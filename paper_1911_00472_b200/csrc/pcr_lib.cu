@@ -155,8 +155,11 @@ struct pcr_record {
     // groups sorted by slice (all refinement scans of the component that a call decodes, in one CTA)
     std::vector<uint32_t> long_begin, long_count;               // [n_slices][G]
     uint32_t* d_long = nullptr;
-    std::vector<uint32_t> group_begin, group_count;             // [n_slices]
-    uint32_t* d_group = nullptr;
+    uint32_t n_groups = 0;                                      // (image, component) pairs whose AC refinements are chains
+    uint32_t* d_group = nullptr;                                // luminance first, most bytes first
+    uint32_t* d_chain_sync = nullptr;                           // queue counters and progress words of the chain launch
+    int n_sms = 1;
+    cudaEvent_t ev_chain = nullptr;
     std::vector<cudaStream_t> streams;                          // one per slice
     std::vector<cudaEvent_t> ev_index;                          // [n_waves] index of wave w done (side stream)
     cudaEvent_t ev_start = nullptr;                             // index of the first wave done
@@ -390,6 +393,8 @@ void free_device(pcr_record* r) {
     r->streams.clear();
     if (r->ev_start) pool_event_put(r->ev_start, r->device);
     r->ev_start = nullptr;
+    if (r->ev_chain) pool_event_put(r->ev_chain, r->device);
+    r->ev_chain = nullptr;
     for (cudaEvent_t e : r->ev_index) pool_event_put(e, r->device);
     r->ev_index.clear();
     if (r->ev_fork) pool_event_put(r->ev_fork, r->device);
@@ -631,7 +636,6 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     };
     std::vector<uint32_t> longs, groups;
     r->long_begin.assign((size_t)r->n_slices * G, 0); r->long_count.assign((size_t)r->n_slices * G, 0);
-    r->group_begin.assign(r->n_slices, 0); r->group_count.assign(r->n_slices, 0);
     for (int g = 0; g < r->n_slices; ++g) {
         for (int w = 0; w < r->n_waves; ++w)
             for (int s : r->wave_scans[w]) {
@@ -642,12 +646,24 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
                     if (is_long(s, order[pos])) longs.push_back((uint32_t)(s * N + order[pos]));
                 r->long_count[(size_t)g * G + s] = (uint32_t)longs.size() - r->long_begin[(size_t)g * G + s];
             }
-        r->group_begin[g] = (uint32_t)groups.size();
-        for (int c = 0; c < 3; ++c)                            // luminance first: its chains are the longest
-            for (uint32_t pos = r->slice_img[g]; pos < r->slice_img[g + 1]; ++pos)
-                if (grouped[(size_t)order[pos] * 3 + c]) groups.push_back(((uint32_t)c << 28) | order[pos]);
-        r->group_count[g] = (uint32_t)groups.size() - r->group_begin[g];
     }
+    // one list for the whole record: luminance first (its chains are the longest), within a
+    // component the images with the most refinement bytes first
+    for (int c = 0; c < 3; ++c) {
+        std::vector<std::pair<uint64_t, uint32_t>> byw;
+        for (uint32_t i = 0; i < N; ++i) {
+            if (!grouped[(size_t)i * 3 + c]) continue;
+            uint64_t bytes = 0;
+            for (uint32_t s = 0; s < G; ++s) {
+                const ScanScript& sc = r->script[s];
+                if (sc.Ss > 0 && sc.Ah != 0 && sc.comp[0] == c) bytes += scans[(size_t)s * N + i].data_end - scans[(size_t)s * N + i].data_off;
+            }
+            byw.push_back({bytes, i});
+        }
+        std::stable_sort(byw.begin(), byw.end(), [](const std::pair<uint64_t, uint32_t>& a, const std::pair<uint64_t, uint32_t>& b) { return a.first > b.first; });
+        for (auto& e : byw) groups.push_back(((uint32_t)c << 28) | e.second);
+    }
+    r->n_groups = (uint32_t)groups.size();
     for (int g = 0; g < r->n_slices; ++g)
         for (int w = 0; w < r->n_waves; ++w)
             for (int s : r->wave_scans[w]) {
@@ -753,6 +769,11 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     if ((rc = upload(r, &r->d_items, items))) return rc;
     if ((rc = upload(r, &r->d_long, longs))) return rc;
     if ((rc = upload(r, &r->d_group, groups))) return rc;
+    if (r->n_groups) {
+        if ((rc = take(r, &r->d_chain_sync, (size_t)(4 + 4 * (size_t)r->n_groups) * 4))) return rc;
+        if (cudaDeviceGetAttribute(&r->n_sms, cudaDevAttrMultiProcessorCount, r->device) != cudaSuccess) return PCR_E_CUDA;
+        if (cudaFuncSetAttribute(ac_refine_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kChainMaxWarps * sizeof(ChainShared))) != cudaSuccess) return PCR_E_CUDA;
+    }
     if ((rc = upload(r, &r->d_qtab, qtab))) return rc;
     if ((rc = upload(r, &r->d_unit_prefix, unit_prefix))) return rc;
     if ((rc = take(r, &r->d_units, (size_t)std::max<uint32_t>(r->n_units, 1) * sizeof(Unit)))) return rc;
@@ -773,6 +794,7 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
         if (!(r->clear_stream = pool_stream_get(r->device))) return PCR_E_CUDA;
         if (!(r->ev_clear = pool_event_get(r->device))) return PCR_E_CUDA;
         if (!(r->ev_start = pool_event_get(r->device))) return PCR_E_CUDA;
+        if (!(r->ev_chain = pool_event_get(r->device))) return PCR_E_CUDA;
         for (int w = 0; w < r->n_waves; ++w) {
             cudaEvent_t e;
             if (!(e = pool_event_get(r->device))) return PCR_E_CUDA;
@@ -989,6 +1011,9 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
     for (int s = k0; s < k; ++s)
         if (rec->script[s].Ss > 0 && rec->script[s].Ah > 0 && (first_refine_wave < 0 || rec->wave_of_scan[s] < first_refine_wave))
             first_refine_wave = rec->wave_of_scan[s];
+    const bool chains = first_refine_wave >= 0 && rec->n_groups > 0;
+    int chain_depth = 6;                        // warps per scheduler of the chain launch (at most kChainMaxWarps / 4)
+    if (const char* e = getenv("PCR_CHAIN_DEPTH")) chain_depth = std::max(1, std::min(kChainMaxWarps / 4, atoi(e)));
     bool dc_only = true, head_only = true;      // no AC scan at all / no scan beyond zigzag position 7
     for (int s = 0; s < k; ++s) {
         if (rec->script[s].Ss > 0 || rec->script[s].Se > 0) dc_only = false;
@@ -1023,13 +1048,6 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
         unstuff_index_kernel<<<(warps + 7) / 8, 256, 0, q>>>(P, sl, (int)i0, (int)(i1 - i0));
         ++g_launches;
         return 1;
-    };
-    // the restart-interval index (and unstuffed copy) of waves w0.. is complete before what follows on q
-    auto wait_index_from = [&](int w0, cudaStream_t q) -> bool {
-        if (!pipelined) return true;                 // indexed up front on the same stream
-        for (int w = std::max(w0, 1); w < rec->n_waves; ++w)
-            if (indexed[w] && cudaStreamWaitEvent(q, rec->ev_index[w], 0) != cudaSuccess) return false;
-        return true;
     };
     auto run_stage = [&](int stage, int g, cudaStream_t q) -> bool {
         const uint32_t i0 = rec->slice_img[g], i1 = rec->slice_img[g + 1];
@@ -1107,16 +1125,8 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
                     ++g_launches;
                 }
             }
-            // ... all their AC refinements of this call in the wave of the first one (a refinement
-            // depends on first passes, which every wave-0 launch above has finished, and on earlier
-            // refinements of its component, which run in the same CTA) ...
-            if (w == first_refine_wave && rec->group_count[g]) {
-                if (!wait_index_from(w + 1, q)) return false;    // the launch reads scans of later waves too
-                int warps = std::max(fl.n[0], std::max(fl.n[1], fl.n[2]));
-                ac_refine_group_kernel<<<rec->group_count[g], 32 * warps, (size_t)warps * sizeof(ChainShared), q>>>(P, fl, rec->d_group + rec->group_begin[g]);
-                ++g_launches;
-            }
-            // ... and the DC refinement scans of every record
+            // ... (their AC refinements follow in one launch for the whole record, once every slice
+            // has finished its waves) and the DC refinement scans of every record
             for (int s : rec->wave_scans[w]) {
                 if (s >= k) break;
                 const ScanScript& sc = rec->script[s];
@@ -1130,7 +1140,19 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
         }
         Params Q = P;
         Q.units = P.units + u0;
-        if (stage == 2 + W) return true;      // the refinement side data is folded in by the pixel kernel
+        if (stage == 2 + W) {
+            // the AC refinements of scans that are one long restart interval: one persistent launch
+            // for all slices (the first slice's stream carries it; the caller has joined the others)
+            if (g != 0 || !chains) return true;
+            const int levels = std::max(fl.n[0], std::max(fl.n[1], fl.n[2]));
+            const int rounds = std::max(1, chain_depth / levels);
+            const int warps = 4 * rounds * levels;
+            if (cudaMemsetAsync(rec->d_chain_sync, 0, (size_t)(4 + 4 * (size_t)rec->n_groups) * 4, q) != cudaSuccess) return false;
+            const unsigned grid = std::min<unsigned>((unsigned)rec->n_sms, (rec->n_groups + 3u) / 4u);
+            ac_refine_group_kernel<<<grid, 32 * warps, (size_t)warps * sizeof(ChainShared), q>>>(P, fl, rec->d_group, rec->n_groups, rec->d_chain_sync, levels, rounds);
+            ++g_launches;
+            return true;
+        }
         if (nu) {
             const unsigned grid = nu;
             uint8_t* o8 = static_cast<uint8_t*>(out);
@@ -1187,7 +1209,7 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
     };
     auto launched_in = [&](int stage) -> int {      // kernel launches of a stage over all slices (for the profile)
         if (stage == 0) return 0;
-        if (stage == 2 + W) return 0;
+        if (stage == 2 + W) return chains ? 1 : 0;
         if (stage >= 2 && stage < 2 + W) {
             bool any = false;
             for (int s : rec->wave_scans[stage - 2]) if (s >= k0 && s < k) any = true;
@@ -1216,7 +1238,7 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
             if (stage == 0) snprintf(name, sizeof name, "clear");
             else if (stage == 1) snprintf(name, sizeof name, "index");
             else if (stage < 2 + W) snprintf(name, sizeof name, "entropy%d", stage - 2);
-            else if (stage == 2 + W) snprintf(name, sizeof name, "finalize");
+            else if (stage == 2 + W) snprintf(name, sizeof name, "chains");
             else snprintf(name, sizeof name, "pixels");
             const int nl = launched_in(stage);
             if (stage <= 1 || stage == n_stages - 1 || nl) mark(name, nl);
@@ -1257,13 +1279,30 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
             indexed[w] = li > 0;
             if (li > 0 && cudaEventRecord(rec->ev_index[w], rec->clear_stream) != cudaSuccess) return PCR_E_CUDA;
         }
+        // with a chain launch the slices meet once: it follows the entropy waves of all of them
+        const int meet = chains ? 2 + W : n_stages;
         for (int g = 0; g < rec->n_slices; ++g) {
             cudaStream_t q = rec->streams[g];
             if (cudaStreamWaitEvent(q, rec->ev_start, 0) != cudaSuccess) return PCR_E_CUDA;
-            for (int stage = 0; stage < n_stages; ++stage)
+            for (int stage = 0; stage < meet; ++stage)
                 if (!run_stage(stage, g, q)) return PCR_E_CUDA;
             if (cudaEventRecord(rec->ev_join[g], q) != cudaSuccess) return PCR_E_CUDA;
-            if (cudaStreamWaitEvent(st, rec->ev_join[g], 0) != cudaSuccess) return PCR_E_CUDA;
+            if (!chains && cudaStreamWaitEvent(st, rec->ev_join[g], 0) != cudaSuccess) return PCR_E_CUDA;
+        }
+        if (chains) {
+            cudaStream_t q0 = rec->streams[0];
+            for (int g = 1; g < rec->n_slices; ++g)
+                if (cudaStreamWaitEvent(q0, rec->ev_join[g], 0) != cudaSuccess) return PCR_E_CUDA;
+            if (!run_stage(2 + W, 0, q0)) return PCR_E_CUDA;
+            if (cudaEventRecord(rec->ev_chain, q0) != cudaSuccess) return PCR_E_CUDA;
+            for (int g = 0; g < rec->n_slices; ++g) {
+                cudaStream_t q = rec->streams[g];
+                if (g && cudaStreamWaitEvent(q, rec->ev_chain, 0) != cudaSuccess) return PCR_E_CUDA;
+                for (int stage = 3 + W; stage < n_stages; ++stage)
+                    if (!run_stage(stage, g, q)) return PCR_E_CUDA;
+                if (cudaEventRecord(rec->ev_join[g], q) != cudaSuccess) return PCR_E_CUDA;
+                if (cudaStreamWaitEvent(st, rec->ev_join[g], 0) != cudaSuccess) return PCR_E_CUDA;
+            }
         }
         // the side and copy streams rejoin the caller's stream too (implied by the slices' waits
         // whenever they carried work; stated so that every fork is joined)

@@ -524,6 +524,7 @@ __global__ void __launch_bounds__(32 * kSeqLongWarps) sequential_long_kernel(Par
 // a CTA, so both are resident while either waits.
 // ---------------------------------------------------------------------------------------
 constexpr int kGroupWarps = 4;           // refinement scans of one component in one call (pcr_open admits four)
+constexpr int kChainMaxWarps = 24;       // warps of the persistent refinement launch: at most six per scheduler
 constexpr int kChainRing = 128;          // words of bitstream per warp in shared memory
 constexpr int kChainRecs = 192;          // symbol records per batch of blocks
 constexpr int kChainLutBits = 9;         // refinement alphabets are small (runs 0..15 with size 0 or 1): short codes
@@ -534,22 +535,22 @@ constexpr int kErrTimeout = -4;
 struct ChainBits {
     const uint32_t* ring;
     uint32_t w0, w1, w2;   // the word the next bit lies in and the two after it
-    uint32_t o;            // bits of w0 already consumed (0..31)
+    uint32_t bits;         // position of the next bit, counted from the first bit of the interval's first word
     uint32_t rd;           // ring word that follows w2 (absolute word index)
-    uint32_t base;         // first word of the interval
     __device__ __forceinline__ void init(const uint32_t* r, uint32_t first, uint32_t lead) {
         ring = r;
-        base = first;
         w0 = r[first & (kChainRing - 1)]; w1 = r[(first + 1) & (kChainRing - 1)]; w2 = r[(first + 2) & (kChainRing - 1)];
         rd = first + 3;
-        o = lead;
+        bits = lead;
     }
-    __device__ __forceinline__ uint32_t win() const { return __funnelshift_l(w1, w0, o); }   // the next 32 bits
-    __device__ __forceinline__ void skip(uint32_t n) {        // n <= 32
-        o += n;
-        if (o >= 32u) { o -= 32u; w0 = w1; w1 = w2; w2 = ring[rd & (kChainRing - 1)]; ++rd; }
+    __device__ __forceinline__ uint32_t win() const { return __funnelshift_l(w1, w0, bits); }   // the next 32 bits (shift taken mod 32)
+    __device__ __forceinline__ void skip(uint32_t n) {        // n <= 96 (the third word is only prefetched)
+        const uint32_t nb = bits + n;
+        uint32_t adv = (nb >> 5) - (bits >> 5);
+        bits = nb;
+        while (adv) { w0 = w1; w1 = w2; w2 = ring[rd & (kChainRing - 1)]; ++rd; --adv; }
     }
-    __device__ __forceinline__ uint32_t pos() const { return (rd - 3u - base) * 32u + o; }   // bits from the first bit of the interval's first word
+    __device__ __forceinline__ uint32_t pos() const { return bits; }
 };
 
 // the n bits (1..32) at bit position p (counted from the first bit of word `base`) of the ring
@@ -568,9 +569,10 @@ __device__ __forceinline__ bool wait_at_least(const volatile uint32_t* flag, uin
 }
 
 // Entry of the chain's own lookup table on the next kChainLutBits bits, made from the Huffman table:
-// bits 0..4 = bits to skip (code, plus the sign bit of a new coefficient), 5..8 = run r, 9 = a new
-// coefficient follows the run; 0 = everything else (end-of-band runs, codes longer than the index,
-// undefined codes), which takes the general path.
+// bits 0..4 = bits to skip (code, plus the sign bit of a new coefficient), 5..11 = run r, 15 = a new
+// coefficient follows the run; the end of band of a single block is entered as a run of 64 without a
+// new coefficient (it passes over the rest of the band like a run that overshoots); 0 = everything
+// else (longer end-of-band runs, codes longer than the index, undefined codes): the general path.
 struct ChainShared {
     HuffTabT<kChainLutBits> tab;
     uint32_t quick[1 << kChainLutBits];
@@ -578,21 +580,28 @@ struct ChainShared {
     uint64_t h[32];
     uint8_t zpos[64][32];              // [i][block]: position of the block's i-th still-zero coefficient of the band
     uint8_t nz[32];                    // how many there are
-    uint2 rec[kChainRecs];             // {bit position behind the sign bit, corrections | position << 7 | new << 13}
+    uint2 rec[kChainRecs];             // {bit position behind the sign bit, corrections | position << 8 | new << 15}
     uint32_t first[33];                // first record of each block of the batch
 };
 
-__global__ void __launch_bounds__(32 * kGroupWarps) ac_refine_group_kernel(Params P, FinalizeList fl, const uint32_t* __restrict__ list) {
-    extern __shared__ __align__(16) unsigned char s_dyn[];     // one ChainShared per warp of the launch
-    ChainShared* s_sh = reinterpret_cast<ChainShared*>(s_dyn);
-    __shared__ uint32_t s_progress[kGroupWarps];              // blocks whose side data each warp has written
-    const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t entry = list[blockIdx.x];
-    const int c = (int)(entry >> 28), img = (int)(entry & 0x0FFFFFFFu);
-    if (threadIdx.x < kGroupWarps) s_progress[threadIdx.x] = 0;
-    __syncthreads();
-    if (wid >= fl.n[c]) return;                                // whole warp: fewer scans than warps
-    const int s = fl.scan[c][wid];
+// Polls *flag (another warp's progress word in global memory) until it reaches `need`; `seen` keeps
+// the last value read, so that a consumer that is behind anyway polls once per many batches.
+__device__ __forceinline__ bool wait_progress(const volatile uint32_t* flag, uint32_t need, uint32_t& seen, uint32_t limit) {
+    if (seen >= need) return true;
+    for (uint32_t i = 0; i < limit; ++i) {
+        seen = *flag;
+        if (seen >= need) return true;
+        __nanosleep(64);
+    }
+    return false;
+}
+
+// One refinement scan (level `level` of the component's refinements in this call) of one (image,
+// component): the chain on lane 0, the rest of the warp around it.  progress = the group's four
+// progress words in global memory (zero before the launch).
+__device__ __forceinline__ void refine_chain(const Params& P, const FinalizeList& fl, ChainShared& sh, int c, int img, int level,
+                                             uint32_t* progress, int lane) {
+    const int s = fl.scan[c][level];
     const uint32_t si = (uint32_t)s * (uint32_t)P.N + (uint32_t)img;
     const ScanDesc sd = P.scans[si];
     const ScanScript sc = P.script[s];
@@ -601,13 +610,13 @@ __global__ void __launch_bounds__(32 * kGroupWarps) ac_refine_group_kernel(Param
     const uint32_t Ss = (uint32_t)sc.Ss, Se = (uint32_t)sc.Se;
     const uint32_t mcu_w = g.ubw[c], total = g.ubw[c] * g.ubh[c], bw = g.bw[c];
     const unsigned full = 0xffffffffu;
-    ChainShared& sh = s_sh[wid];
-    volatile uint32_t* my_progress = &s_progress[wid];
+    volatile uint32_t* my_progress = progress + level;
+    __syncwarp(full);                                          // the previous job's readers of the tables are done
     build_hufftab(sh.tab, P.rec + sd.tab_off[0], lane);
     for (int i = lane; i < (1 << kChainLutBits); i += 32) {
         const uint32_t e = sh.tab.lut[i], len = e >> 8, rs = e & 255u, newc = rs & 1u, r = rs >> 4;
-        const bool plain = e != 0 && (rs & 14u) == 0 && (newc || r == 15u);   // a run followed by a new coefficient, or sixteen zeros
-        sh.quick[i] = plain ? ((len + newc) | (r << 5) | (newc << 9)) : 0u;
+        const bool plain = e != 0 && (rs & 14u) == 0 && (newc || r == 15u || r == 0u);   // run + new coefficient, sixteen zeros, end of band
+        sh.quick[i] = plain ? ((len + newc) | ((rs == 0u ? 64u : r) << 5) | (newc << 15)) : 0u;
     }
     __syncwarp();
     const uint32_t* segtab = P.seg_start + sd.seg_base;
@@ -621,18 +630,19 @@ __global__ void __launch_bounds__(32 * kGroupWarps) ac_refine_group_kernel(Param
     const uint32_t limit = lead + 8u * (bend - bstart);        // first bit behind the interval, counted from word rd0
     const uint32_t wlim = ((bend + 3u) >> 2) + 2u;             // words beyond are not read (zeros instead)
     // masks of the positions that are already non-zero: the union of up to four earlier scans; a
-    // source that this CTA decodes itself is waited for (prod* = its progress word)
+    // source that this launch decodes itself (an earlier level of the group) is waited for
+    // (prod* = its progress word)
     const ScanAux ax = P.saux[s];
     const uint64_t band = low_mask((int)Se + 1) & ~low_mask((int)Ss);
     const uint64_t* src0 = nullptr; const uint64_t* src1 = nullptr; const uint64_t* src2 = nullptr; const uint64_t* src3 = nullptr;
     uint32_t st0 = 0, st1 = 0, st2 = 0, st3 = 0;
-    const volatile uint32_t* prod0 = nullptr; const volatile uint32_t* prod1 = nullptr;
+    const volatile uint32_t* prod0 = nullptr; const volatile uint32_t* prod1 = nullptr; const volatile uint32_t* prod2 = nullptr;
     {
         auto producer = [&](int scan) -> const volatile uint32_t* {
-            for (int w = 0; w < wid; ++w) if (fl.scan[c][w] == scan) return &s_progress[w];
+            for (int w = 0; w < level; ++w) if (fl.scan[c][w] == scan) return progress + w;
             return nullptr;
         };
-        auto note = [&](const volatile uint32_t* p) { if (p) { if (!prod0) prod0 = p; else prod1 = p; } };
+        auto note = [&](const volatile uint32_t* p) { if (p) { if (!prod0) prod0 = p; else if (!prod1) prod1 = p; else prod2 = p; } };
         const ScanAux x0 = P.saux[ax.src[0]];
         src0 = P.aux + x0.base + g.loff[c] * x0.stride; st0 = x0.stride; note(producer(ax.src[0]));
         if (ax.nsrc > 1) { const ScanAux x = P.saux[ax.src[1]]; src1 = P.aux + x.base + g.loff[c] * x.stride; st1 = x.stride; note(producer(ax.src[1])); }
@@ -643,15 +653,16 @@ __global__ void __launch_bounds__(32 * kGroupWarps) ac_refine_group_kernel(Param
     uint32_t* ring = sh.ring;
     uint32_t wr = rd0;                                         // next word to fetch
     ChainBits B;
-    B.ring = ring; B.w0 = B.w1 = B.w2 = 0; B.o = 0; B.rd = rd0; B.base = rd0;
-    uint32_t eobrun = 0, m = 0;
+    B.ring = ring; B.w0 = B.w1 = B.w2 = 0; B.bits = 0; B.rd = rd0;
+    uint32_t eobrun = 0, m = 0, seen0 = 0, seen1 = 0, seen2 = 0;
     int err = 0;
     bool primed = false;
     while (m < total && !err) {
         // ---- all lanes: the masks of the next 32 blocks (once their producers have written them), the ring topped up
         const uint32_t nblk = min(32u, total - m);
-        if (prod0 && !wait_at_least(prod0, m + nblk, kSpinLimit)) { err = kErrTimeout; break; }
-        if (prod1 && !wait_at_least(prod1, m + nblk, kSpinLimit)) { err = kErrTimeout; break; }
+        if (prod0 && !wait_progress(prod0, m + nblk, seen0, kSpinLimit)) { err = kErrTimeout; break; }
+        if (prod1 && !wait_progress(prod1, m + nblk, seen1, kSpinLimit)) { err = kErrTimeout; break; }
+        if (prod2 && !wait_progress(prod2, m + nblk, seen2, kSpinLimit)) { err = kErrTimeout; break; }
         __threadfence();
         uint32_t bi = 0;
         if ((uint32_t)lane < nblk) {
@@ -709,32 +720,32 @@ __global__ void __launch_bounds__(32 * kGroupWarps) ac_refine_group_kernel(Param
                                 B.skip(len + r);
                                 break;
                             }
-                            q = (len + newc) | (r << 5) | (newc << 9);   // a code longer than the table's index
+                            q = (len + newc) | (r << 5) | (newc << 15);   // a code longer than the table's index
                         }
-                        B.skip(q & 31u);                       // the code and, for a new coefficient, its sign
-                        const uint32_t r = (q >> 5) & 15u, t = zi + r;
-                        uint32_t cnt, pos, flag;
+                        const uint32_t r = (q >> 5) & 127u, t = zi + r;
+                        const uint32_t p1 = B.pos() + (q & 31u);   // behind the code and, for a new coefficient, its sign
+                        uint32_t cnt, y;
                         if (t < nz) {                          // the target: the (r+1)-th zero position from here
-                            pos = sh.zpos[t][nd];
+                            const uint32_t pos = sh.zpos[t][nd];
                             cnt = pos - k - r;                 // the non-zero positions passed: one correction bit each
-                            flag = q >> 9;
+                            y = cnt | (pos << 8) | (q & 0x8000u);
                             zi = t + 1u;
+                            k = pos + 1u;
                         } else {                               // past the band: the rest is passed over, nothing new
-                            pos = Se + 1u;
-                            cnt = pos - k - (nz - zi);
-                            flag = 0;
+                            cnt = Se + 1u - k - (nz - zi);
+                            y = cnt;
                             zi = nz;
+                            k = Se + 1u;
                         }
-                        sh.rec[nrec++] = make_uint2(B.pos(), cnt | ((pos & 63u) << 7) | (flag << 13));
-                        if (cnt > 32u) { B.skip(32u); B.skip(cnt - 32u); } else B.skip(cnt);
-                        k = pos + 1u;
+                        sh.rec[nrec++] = make_uint2(p1, y);
+                        B.skip((q & 31u) + cnt);               // code, sign and correction bits in one step
                     }
                 }
                 if (err) break;
                 if (k <= Se) {                                 // inside an end-of-band run: corrections for the rest of the band
                     const uint32_t cnt = Se + 1u - k - (nz - zi);
                     sh.rec[nrec++] = make_uint2(B.pos(), cnt);
-                    if (cnt > 32u) { B.skip(32u); B.skip(cnt - 32u); } else B.skip(cnt);
+                    B.skip(cnt);
                     --eobrun;
                 }
                 if (B.pos() > limit) { err = kErrCorrupt; break; }   // read past the end of the interval
@@ -752,8 +763,8 @@ __global__ void __launch_bounds__(32 * kGroupWarps) ac_refine_group_kernel(Param
             for (uint32_t i = sh.first[lane]; i < sh.first[lane + 1]; ++i) {
                 const uint2 rc = sh.rec[i];
                 uint32_t n = rc.y & 127u;
-                if (rc.y >> 13) {
-                    const uint64_t bit = 1ull << ((rc.y >> 7) & 63u);
+                if (rc.y >> 15) {
+                    const uint64_t bit = 1ull << ((rc.y >> 8) & 63u);
                     Nw |= bit;
                     if (ring_bits(ring, rd0, rc.x - 1u, 1u)) NS |= bit;
                 }
@@ -778,8 +789,50 @@ __global__ void __launch_bounds__(32 * kGroupWarps) ac_refine_group_kernel(Param
         if (lane == 0) *my_progress = m;
     }
     if (lane == 0) {
+        __threadfence();
         *my_progress = 0xFFFFFFFFu;                            // a scan that failed must not keep a later one waiting
         if (err) atomicMin(&P.status[img], err);
+    }
+}
+
+// Persistent launch: one CTA per SM, 4 * rounds * levels warps, warp w on scheduler w % 4.  The
+// groups ((image, component) pairs, luminance first, large images first) are dealt to four queues,
+// one per scheduler (group gi is in queue gi % 4); within a queue every group is followed through
+// its levels (the refinement scans of the component that this call decodes, in script order), so a
+// producer is always taken before its consumer.  The first `rounds` groups of each CTA's schedulers
+// are assigned statically (group r * 4 * CTAs + 4 * CTA + q in round r: every scheduler of the
+// device gets one long luminance chain before any gets a second, and a group's levels start
+// together in one CTA); after that a warp that has finished takes the next entry of its queue from
+// a counter in global memory.  sync: four queue counters, then four progress words per group, all
+// zero before the launch.
+__global__ void __launch_bounds__(32 * kChainMaxWarps, 1) ac_refine_group_kernel(Params P, FinalizeList fl, const uint32_t* __restrict__ list,
+                                                                                 uint32_t n_groups, uint32_t* __restrict__ sync, int levels, int rounds) {
+    extern __shared__ __align__(16) unsigned char s_dyn[];     // one ChainShared per warp of the launch
+    ChainShared* s_sh = reinterpret_cast<ChainShared*>(s_dyn);
+    const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t q = (uint32_t)wid & 3u, slot = (uint32_t)wid >> 2;
+    const uint32_t per_round = 4u * gridDim.x, statics = per_round * (uint32_t)rounds;
+    uint32_t* progress = sync + 4;
+    bool first = true;
+    for (;;) {
+        uint32_t gi;
+        int level;
+        if (first) {
+            first = false;
+            gi = (slot / (uint32_t)levels) * per_round + 4u * blockIdx.x + q;
+            level = (int)(slot % (uint32_t)levels);
+        } else {
+            uint32_t t = 0;
+            if (lane == 0) t = atomicAdd(&sync[q], 1u);
+            t = __shfl_sync(0xffffffffu, t, 0);
+            gi = statics + 4u * (t / (uint32_t)levels) + q;
+            level = (int)(t % (uint32_t)levels);
+        }
+        if (gi >= n_groups) break;                             // the queue is empty (entries only grow)
+        const uint32_t entry = list[gi];
+        const int c = (int)(entry >> 28), img = (int)(entry & 0x0FFFFFFFu);
+        if (level >= fl.n[c]) continue;                        // this component has fewer refinements
+        refine_chain(P, fl, s_sh[wid], c, img, level, progress + 4ull * gi, lane);
     }
 }
 
