@@ -772,7 +772,7 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
     if (r->n_groups) {
         if ((rc = take(r, &r->d_chain_sync, (size_t)(4 + 4 * (size_t)r->n_groups) * 4))) return rc;
         if (cudaDeviceGetAttribute(&r->n_sms, cudaDevAttrMultiProcessorCount, r->device) != cudaSuccess) return PCR_E_CUDA;
-        if (cudaFuncSetAttribute(ac_refine_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kChainMaxWarps * sizeof(ChainShared))) != cudaSuccess) return PCR_E_CUDA;
+        if (cudaFuncSetAttribute(ac_refine_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kChainPairs * sizeof(ChainShared))) != cudaSuccess) return PCR_E_CUDA;
     }
     if ((rc = upload(r, &r->d_qtab, qtab))) return rc;
     if ((rc = upload(r, &r->d_unit_prefix, unit_prefix))) return rc;
@@ -1012,8 +1012,8 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
         if (rec->script[s].Ss > 0 && rec->script[s].Ah > 0 && (first_refine_wave < 0 || rec->wave_of_scan[s] < first_refine_wave))
             first_refine_wave = rec->wave_of_scan[s];
     const bool chains = first_refine_wave >= 0 && rec->n_groups > 0;
-    int chain_depth = 6;                        // warps per scheduler of the chain launch (at most kChainMaxWarps / 4)
-    if (const char* e = getenv("PCR_CHAIN_DEPTH")) chain_depth = std::max(1, std::min(kChainMaxWarps / 4, atoi(e)));
+    int chain_depth = kChainPairs / 4;          // chains per scheduler of the chain launch
+    if (const char* e = getenv("PCR_CHAIN_DEPTH")) chain_depth = std::max(1, std::min(kChainPairs / 4, atoi(e)));
     bool dc_only = true, head_only = true;      // no AC scan at all / no scan beyond zigzag position 7
     for (int s = 0; s < k; ++s) {
         if (rec->script[s].Ss > 0 || rec->script[s].Se > 0) dc_only = false;
@@ -1146,10 +1146,10 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
             if (g != 0 || !chains) return true;
             const int levels = std::max(fl.n[0], std::max(fl.n[1], fl.n[2]));
             const int rounds = std::max(1, chain_depth / levels);
-            const int warps = 4 * rounds * levels;
+            const int pairs = 4 * rounds * levels;          // chains per CTA: a decoding and a helper warp each
             if (cudaMemsetAsync(rec->d_chain_sync, 0, (size_t)(4 + 4 * (size_t)rec->n_groups) * 4, q) != cudaSuccess) return false;
             const unsigned grid = std::min<unsigned>((unsigned)rec->n_sms, (rec->n_groups + 3u) / 4u);
-            ac_refine_group_kernel<<<grid, 32 * warps, (size_t)warps * sizeof(ChainShared), q>>>(P, fl, rec->d_group, rec->n_groups, rec->d_chain_sync, levels, rounds);
+            ac_refine_group_kernel<<<grid, 64 * pairs, (size_t)pairs * sizeof(ChainShared), q>>>(P, fl, rec->d_group, rec->n_groups, rec->d_chain_sync, levels, rounds);
             ++g_launches;
             return true;
         }

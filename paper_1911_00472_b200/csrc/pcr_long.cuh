@@ -524,9 +524,9 @@ __global__ void __launch_bounds__(32 * kSeqLongWarps) sequential_long_kernel(Par
 // a CTA, so both are resident while either waits.
 // ---------------------------------------------------------------------------------------
 constexpr int kGroupWarps = 4;           // refinement scans of one component in one call (pcr_open admits four)
-constexpr int kChainMaxWarps = 24;       // warps of the persistent refinement launch: at most six per scheduler
-constexpr int kChainRing = 128;          // words of bitstream per warp in shared memory
-constexpr int kChainRecs = 192;          // symbol records per batch of blocks
+constexpr int kChainPairs = 16;          // chains per CTA of the persistent refinement launch (four per scheduler), two warps each
+constexpr int kChainRing = 256;          // words of bitstream per chain in shared memory
+constexpr int kChainRecs = 512;          // symbol records per batch of blocks (four bytes each)
 constexpr int kChainLutBits = 9;         // refinement alphabets are small (runs 0..15 with size 0 or 1): short codes
 constexpr uint32_t kChainBlockWords = 44;   // a block never needs more: 63 symbols of at most 17 bits, 3 sixteen-zero runs, one run length, 63 correction bits
 constexpr uint32_t kSpinLimit = 1u << 22;   // polls (of at least 64 ns) before a wait gives up
@@ -573,15 +573,30 @@ __device__ __forceinline__ bool wait_at_least(const volatile uint32_t* flag, uin
 // coefficient follows the run; the end of band of a single block is entered as a run of 64 without a
 // new coefficient (it passes over the rest of the band like a run that overshoots); 0 = everything
 // else (longer end-of-band runs, codes longer than the index, undefined codes): the general path.
+struct ChainLists {
+    uint64_t h[32];                    // positions of the band that are already non-zero, per block of the batch
+    uint8_t zpos[64][32];              // [i][block]: position of the block's i-th still-zero coefficient of the band
+    uint8_t nz[32];                    // how many there are
+};
+struct ChainRecs {
+    uint32_t rec[kChainRecs];          // corrections | position << 8 | new << 15 | (bit position behind the sign bit - base) << 16
+    uint32_t first[33];                // first record of each block of the batch
+    uint32_t base;                     // bit position at which the batch starts
+};
+struct ChainMail {                     // what the two warps of a chain tell each other at a meeting point
+    uint32_t nd, rd, err_c;            // decoder: blocks it decoded, oldest ring word it still needs, error
+    uint32_t wr, err_h;                // helper: the ring is filled up to this word, error
+};
 struct ChainShared {
     HuffTabT<kChainLutBits> tab;
     uint32_t quick[1 << kChainLutBits];
     uint32_t ring[kChainRing];
-    uint64_t h[32];
-    uint8_t zpos[64][32];              // [i][block]: position of the block's i-th still-zero coefficient of the band
-    uint8_t nz[32];                    // how many there are
-    uint2 rec[kChainRecs];             // {bit position behind the sign bit, corrections | position << 8 | new << 15}
-    uint32_t first[33];                // first record of each block of the batch
+    ChainLists lists[2];               // the batch being decoded and the one being prepared
+    ChainRecs recs[2];                 // the batch being decoded and the one being turned into side data
+    ChainMail mail[2];                 // by parity of the meeting point
+    uint32_t job_gi, job_level;        // the pair's job (job_gi = 0xFFFFFFFF: none left)
+    uint32_t Ss, Se, total, rd0, lead, limit;   // of the job, for the decoder
+    volatile uint32_t phase_c, phase_h;         // meeting points each side has reached
 };
 
 // Polls *flag (another warp's progress word in global memory) until it reaches `need`; `seen` keeps
@@ -596,121 +611,76 @@ __device__ __forceinline__ bool wait_progress(const volatile uint32_t* flag, uin
     return false;
 }
 
-// One refinement scan (level `level` of the component's refinements in this call) of one (image,
-// component): the chain on lane 0, the rest of the warp around it.  progress = the group's four
-// progress words in global memory (zero before the launch).
-__device__ __forceinline__ void refine_chain(const Params& P, const FinalizeList& fl, ChainShared& sh, int c, int img, int level,
-                                             uint32_t* progress, int lane) {
-    const int s = fl.scan[c][level];
-    const uint32_t si = (uint32_t)s * (uint32_t)P.N + (uint32_t)img;
-    const ScanDesc sd = P.scans[si];
-    const ScanScript sc = P.script[s];
-    const ImgDesc im = P.imgs[img];
-    const Geometry g = make_geometry(im, P);
-    const uint32_t Ss = (uint32_t)sc.Ss, Se = (uint32_t)sc.Se;
-    const uint32_t mcu_w = g.ubw[c], total = g.ubw[c] * g.ubh[c], bw = g.bw[c];
-    const unsigned full = 0xffffffffu;
-    volatile uint32_t* my_progress = progress + level;
-    __syncwarp(full);                                          // the previous job's readers of the tables are done
-    build_hufftab(sh.tab, P.rec + sd.tab_off[0], lane);
-    for (int i = lane; i < (1 << kChainLutBits); i += 32) {
-        const uint32_t e = sh.tab.lut[i], len = e >> 8, rs = e & 255u, newc = rs & 1u, r = rs >> 4;
-        const bool plain = e != 0 && (rs & 14u) == 0 && (newc || r == 15u || r == 0u);   // run + new coefficient, sixteen zeros, end of band
-        sh.quick[i] = plain ? ((len + newc) | ((rs == 0u ? 64u : r) << 5) | (newc << 15)) : 0u;
-    }
+// Meeting point k of a chain's two warps: each side announces that it has arrived (everything it
+// wrote to shared memory before is visible to the other behind the meeting) and waits, with a
+// bounded number of polls, for the other.  false: the partner never came.
+__device__ __forceinline__ bool meet_decoder(ChainShared& sh, uint32_t k) {          // one thread
+    __threadfence_block();
+    sh.phase_c = k;
+    const bool ok = wait_at_least(&sh.phase_h, k, kSpinLimit);
+    __threadfence_block();
+    return ok;
+}
+__device__ __forceinline__ bool meet_helper(ChainShared& sh, uint32_t k, int lane) {  // a whole warp
     __syncwarp();
-    const uint32_t* segtab = P.seg_start + sd.seg_base;
-    const uint32_t bstart = segtab[0], bend = segtab[1] - 2u;
-    if (bstart < sd.data_off || bend > sd.data_end || bend < bstart) {
-        if (lane == 0) { atomicMin(&P.status[img], kErrCorrupt); *my_progress = 0xFFFFFFFFu; }   // nobody waits for this scan
-        return;
-    }
-    const uint32_t* words = reinterpret_cast<const uint32_t*>(P.ubuf);
-    const uint32_t rd0 = bstart >> 2, lead = 8u * (bstart & 3u);
-    const uint32_t limit = lead + 8u * (bend - bstart);        // first bit behind the interval, counted from word rd0
-    const uint32_t wlim = ((bend + 3u) >> 2) + 2u;             // words beyond are not read (zeros instead)
-    // masks of the positions that are already non-zero: the union of up to four earlier scans; a
-    // source that this launch decodes itself (an earlier level of the group) is waited for
-    // (prod* = its progress word)
-    const ScanAux ax = P.saux[s];
-    const uint64_t band = low_mask((int)Se + 1) & ~low_mask((int)Ss);
-    const uint64_t* src0 = nullptr; const uint64_t* src1 = nullptr; const uint64_t* src2 = nullptr; const uint64_t* src3 = nullptr;
-    uint32_t st0 = 0, st1 = 0, st2 = 0, st3 = 0;
-    const volatile uint32_t* prod0 = nullptr; const volatile uint32_t* prod1 = nullptr; const volatile uint32_t* prod2 = nullptr;
-    {
-        auto producer = [&](int scan) -> const volatile uint32_t* {
-            for (int w = 0; w < level; ++w) if (fl.scan[c][w] == scan) return progress + w;
-            return nullptr;
-        };
-        auto note = [&](const volatile uint32_t* p) { if (p) { if (!prod0) prod0 = p; else if (!prod1) prod1 = p; else prod2 = p; } };
-        const ScanAux x0 = P.saux[ax.src[0]];
-        src0 = P.aux + x0.base + g.loff[c] * x0.stride; st0 = x0.stride; note(producer(ax.src[0]));
-        if (ax.nsrc > 1) { const ScanAux x = P.saux[ax.src[1]]; src1 = P.aux + x.base + g.loff[c] * x.stride; st1 = x.stride; note(producer(ax.src[1])); }
-        if (ax.nsrc > 2) { const ScanAux x = P.saux[ax.src[2]]; src2 = P.aux + x.base + g.loff[c] * x.stride; st2 = x.stride; note(producer(ax.src[2])); }
-        if (ax.nsrc > 3) { const ScanAux x = P.saux[ax.src[3]]; src3 = P.aux + x.base + g.loff[c] * x.stride; st3 = x.stride; note(producer(ax.src[3])); }
-    }
-    uint64_t* outp = P.aux + ax.base + g.loff[c] * 4ull;
-    uint32_t* ring = sh.ring;
-    uint32_t wr = rd0;                                         // next word to fetch
-    ChainBits B;
-    B.ring = ring; B.w0 = B.w1 = B.w2 = 0; B.bits = 0; B.rd = rd0;
-    uint32_t eobrun = 0, m = 0, seen0 = 0, seen1 = 0, seen2 = 0;
-    int err = 0;
-    bool primed = false;
-    while (m < total && !err) {
-        // ---- all lanes: the masks of the next 32 blocks (once their producers have written them), the ring topped up
-        const uint32_t nblk = min(32u, total - m);
-        if (prod0 && !wait_progress(prod0, m + nblk, seen0, kSpinLimit)) { err = kErrTimeout; break; }
-        if (prod1 && !wait_progress(prod1, m + nblk, seen1, kSpinLimit)) { err = kErrTimeout; break; }
-        if (prod2 && !wait_progress(prod2, m + nblk, seen2, kSpinLimit)) { err = kErrTimeout; break; }
-        __threadfence();
-        uint32_t bi = 0;
-        if ((uint32_t)lane < nblk) {
-            const uint32_t x = m + lane, row = x / mcu_w;
-            bi = row * bw + (x - row * mcu_w);
-            uint64_t v = __ldcg(src0 + (uint64_t)bi * st0);    // not through L1: a line may hold blocks written later
-            if (src1) v |= __ldcg(src1 + (uint64_t)bi * st1);
-            if (src2) v |= __ldcg(src2 + (uint64_t)bi * st2);
-            if (src3) v |= __ldcg(src3 + (uint64_t)bi * st3);
-            v &= band;
-            sh.h[lane] = v;
-            // the positions of the band that are still zero, in order: the target of a run r is then one
-            // table look-up for lane 0 (the (r+1)-th of those not yet passed).  (Listing the few non-zero
-            // positions instead and stepping over them measured 18 % slower: the steps sit on lane 0's chain.)
-            const uint64_t z = ~v & band;
-            uint32_t n = 0;
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                uint32_t w = half ? (uint32_t)(z >> 32) : (uint32_t)z;
-                while (w) {
-                    sh.zpos[n++][lane] = (uint8_t)(32 * half + __ffs((int)w) - 1);
-                    w &= w - 1u;
-                }
+    if (lane == 0) { __threadfence_block(); sh.phase_h = k; }
+    const bool ok = __all_sync(0xffffffffu, wait_at_least(&sh.phase_c, k, kSpinLimit));
+    __threadfence_block();
+    return ok;
+}
+
+// The decoding side of a chain: one thread.  It takes the pair's jobs (first the statically assigned
+// one, then tickets of its scheduler's queue), and per job follows the bit stream batch by batch:
+// the lists of still-zero positions of a batch come from the helper, the symbol records go back to it.
+__device__ __forceinline__ void chain_decoder(const FinalizeList& fl, ChainShared& sh, const uint32_t* __restrict__ list, uint32_t n_groups,
+                                              uint32_t* sync, uint32_t levels, uint32_t rounds, uint32_t q, uint32_t slot) {
+    const uint32_t per_round = 4u * gridDim.x, statics = per_round * rounds;
+    uint32_t mk = 0;                                           // meeting points so far
+    bool first_job = true;
+    for (;;) {
+        uint32_t gi, level;
+        for (;;) {
+            if (first_job) {
+                first_job = false;
+                gi = (slot / levels) * per_round + 4u * blockIdx.x + q;
+                level = slot % levels;
+            } else {
+                const uint32_t t = atomicAdd(&sync[q], 1u);
+                gi = statics + 4u * (t / levels) + q;
+                level = t % levels;
             }
-            sh.nz[lane] = (uint8_t)n;
+            if (gi >= n_groups) { gi = 0xFFFFFFFFu; break; }  // the queue is empty (entries only grow)
+            if ((int)level < fl.n[list[gi] >> 28]) break;      // (a component with fewer refinements has no such level)
         }
-        const uint32_t rd_now = __shfl_sync(full, B.rd - (primed ? 3u : 0u), 0);   // lane 0's reader: w0 is the oldest word still in use
-        while (wr - rd_now + 32u <= (uint32_t)kChainRing) {
-            ring[(wr + lane) & (kChainRing - 1)] = wr + lane < wlim ? __ldg(words + wr + lane) : 0u;
-            wr += 32u;
-        }
-        __syncwarp(full);
-        // ---- lane 0: the chain
-        uint32_t nd = 0;
-        if (lane == 0) {
-            if (!primed) { B.init(ring, rd0, lead); primed = true; }
-            uint32_t nrec = 0;
+        sh.job_gi = gi; sh.job_level = level;
+        if (!meet_decoder(sh, ++mk)) return;                   // the helper has the job
+        if (gi == 0xFFFFFFFFu) return;
+        if (!meet_decoder(sh, ++mk)) return;                   // tables, first lists and ring are ready
+        if (sh.mail[mk & 1u].err_h) continue;                  // a scan whose bounds are off: the helper reports it
+        uint32_t wr = sh.mail[mk & 1u].wr;
+        const uint32_t Ss = sh.Ss, Se = sh.Se, total = sh.total, limit = sh.limit;
+        ChainBits B;
+        B.init(sh.ring, sh.rd0, sh.lead);
+        uint32_t eobrun = 0, m = 0, p = 0;
+        for (;;) {
+            const uint32_t nblk = min(32u, total - m);
+            const ChainLists& L = sh.lists[p];
+            ChainRecs& R = sh.recs[p];
+            uint32_t nrec = 0, nd = 0;
+            int err = 0;
+            const uint32_t base = B.pos();                     // a batch spans fewer than 2^16 bits (32 blocks of kChainBlockWords words)
+            R.base = base;
             for (; nd < nblk; ++nd) {
                 if (wr - B.rd < kChainBlockWords || nrec > (uint32_t)kChainRecs - 64u) break;   // fetch more / flush first
-                sh.first[nd] = nrec;
+                R.first[nd] = nrec;
                 // k: the position that comes next; zi: how many of the block's zero positions lie below it
-                const uint32_t nz = sh.nz[nd];
+                const uint32_t nz = L.nz[nd];
                 uint32_t k = Ss, zi = 0;
                 if (eobrun == 0) {
                     while (k <= Se) {
                         const uint32_t win = B.win();
-                        uint32_t q = sh.quick[win >> (32 - kChainLutBits)];
-                        if (q == 0) {                          // not a plain (run, new coefficient) symbol
+                        uint32_t qe = sh.quick[win >> (32 - kChainLutBits)];
+                        if (qe == 0) {                         // not a plain (run, new coefficient) symbol
                             const uint32_t e = huff_lookup(sh.tab, win);
                             const uint32_t len = e >> 8, rs = e & 255u, newc = rs & 1u, r = rs >> 4;
                             if (e == 0 || (rs & 14u)) { err = kErrCorrupt; break; }   // a refinement symbol has size 0 or 1
@@ -720,15 +690,15 @@ __device__ __forceinline__ void refine_chain(const Params& P, const FinalizeList
                                 B.skip(len + r);
                                 break;
                             }
-                            q = (len + newc) | (r << 5) | (newc << 15);   // a code longer than the table's index
+                            qe = (len + newc) | (r << 5) | (newc << 15);   // a code longer than the table's index
                         }
-                        const uint32_t r = (q >> 5) & 127u, t = zi + r;
-                        const uint32_t p1 = B.pos() + (q & 31u);   // behind the code and, for a new coefficient, its sign
+                        const uint32_t r = (qe >> 5) & 127u, t = zi + r;
+                        const uint32_t p1 = B.pos() - base + (qe & 31u);   // behind the code and, for a new coefficient, its sign
                         uint32_t cnt, y;
                         if (t < nz) {                          // the target: the (r+1)-th zero position from here
-                            const uint32_t pos = sh.zpos[t][nd];
+                            const uint32_t pos = L.zpos[t][nd];
                             cnt = pos - k - r;                 // the non-zero positions passed: one correction bit each
-                            y = cnt | (pos << 8) | (q & 0x8000u);
+                            y = cnt | (pos << 8) | (qe & 0x8000u);
                             zi = t + 1u;
                             k = pos + 1u;
                         } else {                               // past the band: the rest is passed over, nothing new
@@ -737,102 +707,242 @@ __device__ __forceinline__ void refine_chain(const Params& P, const FinalizeList
                             zi = nz;
                             k = Se + 1u;
                         }
-                        sh.rec[nrec++] = make_uint2(p1, y);
-                        B.skip((q & 31u) + cnt);               // code, sign and correction bits in one step
+                        R.rec[nrec++] = (p1 << 16) | y;
+                        B.skip((qe & 31u) + cnt);              // code, sign and correction bits in one step
                     }
                 }
                 if (err) break;
                 if (k <= Se) {                                 // inside an end-of-band run: corrections for the rest of the band
                     const uint32_t cnt = Se + 1u - k - (nz - zi);
-                    sh.rec[nrec++] = make_uint2(B.pos(), cnt);
+                    R.rec[nrec++] = ((B.pos() - base) << 16) | cnt;
                     B.skip(cnt);
                     --eobrun;
                 }
                 if (B.pos() > limit) { err = kErrCorrupt; break; }   // read past the end of the interval
             }
-            sh.first[nd] = nrec;
-        }
-        __syncwarp(full);
-        nd = __shfl_sync(full, nd, 0);
-        err = __shfl_sync(full, err, 0);
-        // ---- all lanes: one block each, records -> side data
-        bool over = false;
-        if ((uint32_t)lane < nd) {
-            uint64_t cstr = 0, Nw = 0, NS = 0;
-            uint32_t cn = 0;
-            for (uint32_t i = sh.first[lane]; i < sh.first[lane + 1]; ++i) {
-                const uint2 rc = sh.rec[i];
-                uint32_t n = rc.y & 127u;
-                if (rc.y >> 15) {
-                    const uint64_t bit = 1ull << ((rc.y >> 8) & 63u);
-                    Nw |= bit;
-                    if (ring_bits(ring, rd0, rc.x - 1u, 1u)) NS |= bit;
-                }
-                if (cn + n > 64u) { over = true; break; }
-                cn += n;
-                uint32_t p = rc.x;
-                while (n) {
-                    const uint32_t q = min(n, 32u);
-                    cstr = (cstr << q) | (uint64_t)ring_bits(ring, rd0, p, q);
-                    p += q; n -= q;
-                }
+            R.first[nd] = nrec;
+            ++mk;
+            sh.mail[mk & 1u].nd = nd; sh.mail[mk & 1u].rd = B.rd - 3u; sh.mail[mk & 1u].err_c = (uint32_t)err;
+            if (!meet_decoder(sh, mk)) return;
+            wr = sh.mail[mk & 1u].wr;
+            if (err || sh.mail[mk & 1u].err_h) break;
+            m += nd;
+            if (nd == nblk) {
+                p ^= 1u;
+                if (m >= total) break;
+            } else {                                           // stopped early: the helper lists the blocks from m again
+                if (!meet_decoder(sh, ++mk)) return;
+                wr = sh.mail[mk & 1u].wr;
+                if (sh.mail[mk & 1u].err_h) break;
+                p ^= 1u;
             }
-            if (cn) cstr <<= 64u - cn;                         // first correction bit at bit 63
-            ulonglong2* o = reinterpret_cast<ulonglong2*>(outp + (uint64_t)bi * 4);
-            o[0] = make_ulonglong2((sh.h[lane] | Nw), cstr);
-            o[1] = make_ulonglong2(Nw, NS);
         }
-        if (__any_sync(full, over)) err = kErrCorrupt;
-        m += nd;
-        __threadfence();                                       // the side data before the count
-        __syncwarp(full);
-        if (lane == 0) *my_progress = m;
-    }
-    if (lane == 0) {
-        __threadfence();
-        *my_progress = 0xFFFFFFFFu;                            // a scan that failed must not keep a later one waiting
-        if (err) atomicMin(&P.status[img], err);
     }
 }
 
-// Persistent launch: one CTA per SM, 4 * rounds * levels warps, warp w on scheduler w % 4.  The
-// groups ((image, component) pairs, luminance first, large images first) are dealt to four queues,
-// one per scheduler (group gi is in queue gi % 4); within a queue every group is followed through
-// its levels (the refinement scans of the component that this call decodes, in script order), so a
-// producer is always taken before its consumer.  The first `rounds` groups of each CTA's schedulers
-// are assigned statically (group r * 4 * CTAs + 4 * CTA + q in round r: every scheduler of the
-// device gets one long luminance chain before any gets a second, and a group's levels start
-// together in one CTA); after that a warp that has finished takes the next entry of its queue from
-// a counter in global memory.  sync: four queue counters, then four progress words per group, all
-// zero before the launch.
-__global__ void __launch_bounds__(32 * kChainMaxWarps, 1) ac_refine_group_kernel(Params P, FinalizeList fl, const uint32_t* __restrict__ list,
-                                                                                 uint32_t n_groups, uint32_t* __restrict__ sync, int levels, int rounds) {
-    extern __shared__ __align__(16) unsigned char s_dyn[];     // one ChainShared per warp of the launch
-    ChainShared* s_sh = reinterpret_cast<ChainShared*>(s_dyn);
-    const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t q = (uint32_t)wid & 3u, slot = (uint32_t)wid >> 2;
-    const uint32_t per_round = 4u * gridDim.x, statics = per_round * (uint32_t)rounds;
-    uint32_t* progress = sync + 4;
-    bool first = true;
+// The helper side of a chain: a whole warp.  Per job it builds the tables, then stays one batch ahead
+// of the decoder with the masks and lists of still-zero positions (waiting, with bounded polls, for
+// an earlier refinement of the same blocks when this launch decodes that too), keeps the ring of
+// bitstream words filled, and one batch behind it turns the symbol records into side data.
+__device__ __forceinline__ void chain_helper(const Params& P, const FinalizeList& fl, ChainShared& sh, const uint32_t* __restrict__ list,
+                                             uint32_t* progress_all, int lane) {
+    const unsigned full = 0xffffffffu;
+    uint32_t mk = 0;
     for (;;) {
-        uint32_t gi;
-        int level;
-        if (first) {
-            first = false;
-            gi = (slot / (uint32_t)levels) * per_round + 4u * blockIdx.x + q;
-            level = (int)(slot % (uint32_t)levels);
-        } else {
-            uint32_t t = 0;
-            if (lane == 0) t = atomicAdd(&sync[q], 1u);
-            t = __shfl_sync(0xffffffffu, t, 0);
-            gi = statics + 4u * (t / (uint32_t)levels) + q;
-            level = (int)(t % (uint32_t)levels);
-        }
-        if (gi >= n_groups) break;                             // the queue is empty (entries only grow)
+        if (!meet_helper(sh, ++mk, lane)) return;
+        const uint32_t gi = sh.job_gi;
+        const int level = (int)sh.job_level;
+        if (gi == 0xFFFFFFFFu) return;
         const uint32_t entry = list[gi];
         const int c = (int)(entry >> 28), img = (int)(entry & 0x0FFFFFFFu);
-        if (level >= fl.n[c]) continue;                        // this component has fewer refinements
-        refine_chain(P, fl, s_sh[wid], c, img, level, progress + 4ull * gi, lane);
+        uint32_t* progress = progress_all + 4ull * gi;
+        volatile uint32_t* my_progress = progress + level;
+        const int s = fl.scan[c][level];
+        const ScanDesc sd = P.scans[(uint32_t)s * (uint32_t)P.N + (uint32_t)img];
+        const ScanScript sc = P.script[s];
+        const Geometry g = make_geometry(P.imgs[img], P);
+        const uint32_t Ss = (uint32_t)sc.Ss, Se = (uint32_t)sc.Se;
+        const uint32_t mcu_w = g.ubw[c], total = g.ubw[c] * g.ubh[c], bw = g.bw[c];
+        build_hufftab(sh.tab, P.rec + sd.tab_off[0], lane);
+        for (int i = lane; i < (1 << kChainLutBits); i += 32) {
+            const uint32_t e = sh.tab.lut[i], len = e >> 8, rs = e & 255u, newc = rs & 1u, r = rs >> 4;
+            const bool plain = e != 0 && (rs & 14u) == 0 && (newc || r == 15u || r == 0u);   // run + new coefficient, sixteen zeros, end of band
+            sh.quick[i] = plain ? ((len + newc) | ((rs == 0u ? 64u : r) << 5) | (newc << 15)) : 0u;
+        }
+        const uint32_t* segtab = P.seg_start + sd.seg_base;
+        const uint32_t bstart = segtab[0], bend = segtab[1] - 2u;
+        const bool bad = bstart < sd.data_off || bend > sd.data_end || bend < bstart;
+        const uint32_t* words = reinterpret_cast<const uint32_t*>(P.ubuf);
+        const uint32_t rd0 = bstart >> 2, lead = 8u * (bstart & 3u);
+        const uint32_t wlim = ((bend + 3u) >> 2) + 2u;         // words beyond are not read (zeros instead)
+        if (lane == 0) {
+            sh.Ss = Ss; sh.Se = Se; sh.total = total; sh.rd0 = rd0; sh.lead = lead;
+            sh.limit = lead + 8u * (bend - bstart);            // first bit behind the interval, counted from word rd0
+        }
+        // masks of the positions that are already non-zero: the union of up to four earlier scans; a
+        // source that this launch decodes itself (an earlier level of the group) is waited for
+        // (prod* = its progress word)
+        const ScanAux ax = P.saux[s];
+        const uint64_t band = low_mask((int)Se + 1) & ~low_mask((int)Ss);
+        const uint64_t* src0 = nullptr; const uint64_t* src1 = nullptr; const uint64_t* src2 = nullptr; const uint64_t* src3 = nullptr;
+        uint32_t st0 = 0, st1 = 0, st2 = 0, st3 = 0;
+        const volatile uint32_t* prod0 = nullptr; const volatile uint32_t* prod1 = nullptr; const volatile uint32_t* prod2 = nullptr;
+        {
+            auto producer = [&](int scan) -> const volatile uint32_t* {
+                for (int w = 0; w < level; ++w) if (fl.scan[c][w] == scan) return progress + w;
+                return nullptr;
+            };
+            auto note = [&](const volatile uint32_t* q) { if (q) { if (!prod0) prod0 = q; else if (!prod1) prod1 = q; else prod2 = q; } };
+            const ScanAux x0 = P.saux[ax.src[0]];
+            src0 = P.aux + x0.base + g.loff[c] * x0.stride; st0 = x0.stride; note(producer(ax.src[0]));
+            if (ax.nsrc > 1) { const ScanAux x = P.saux[ax.src[1]]; src1 = P.aux + x.base + g.loff[c] * x.stride; st1 = x.stride; note(producer(ax.src[1])); }
+            if (ax.nsrc > 2) { const ScanAux x = P.saux[ax.src[2]]; src2 = P.aux + x.base + g.loff[c] * x.stride; st2 = x.stride; note(producer(ax.src[2])); }
+            if (ax.nsrc > 3) { const ScanAux x = P.saux[ax.src[3]]; src3 = P.aux + x.base + g.loff[c] * x.stride; st3 = x.stride; note(producer(ax.src[3])); }
+        }
+        uint64_t* outp = P.aux + ax.base + g.loff[c] * 4ull;
+        uint32_t* ring = sh.ring;
+        uint32_t wr = rd0, seen0 = 0, seen1 = 0, seen2 = 0;
+        int err = bad ? kErrCorrupt : 0;
+        auto block_index = [&](uint32_t x) { const uint32_t row = x / mcu_w; return row * bw + (x - row * mcu_w); };
+        // the masks of blocks m0 .. m0 + 31 and their lists of still-zero positions
+        auto gather = [&](uint32_t m0, ChainLists& L) -> int {
+            const uint32_t nblk = min(32u, total - m0);
+            if (prod0 && !wait_progress(prod0, m0 + nblk, seen0, kSpinLimit)) return kErrTimeout;
+            if (prod1 && !wait_progress(prod1, m0 + nblk, seen1, kSpinLimit)) return kErrTimeout;
+            if (prod2 && !wait_progress(prod2, m0 + nblk, seen2, kSpinLimit)) return kErrTimeout;
+            __threadfence();
+            if ((uint32_t)lane < nblk) {
+                const uint32_t bi = block_index(m0 + lane);
+                uint64_t v = __ldcg(src0 + (uint64_t)bi * st0);    // not through L1: a line may hold blocks written later
+                if (src1) v |= __ldcg(src1 + (uint64_t)bi * st1);
+                if (src2) v |= __ldcg(src2 + (uint64_t)bi * st2);
+                if (src3) v |= __ldcg(src3 + (uint64_t)bi * st3);
+                v &= band;
+                L.h[lane] = v;
+                // the positions of the band that are still zero, in order: the target of a run r is then one
+                // table look-up for the decoder (the (r+1)-th of those not yet passed).  (Listing the few non-zero
+                // positions instead and stepping over them measured 18 % slower: the steps sit on the chain.)
+                const uint64_t z = ~v & band;
+                uint32_t n = 0;
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    uint32_t w = half ? (uint32_t)(z >> 32) : (uint32_t)z;
+                    while (w) {
+                        L.zpos[n++][lane] = (uint8_t)(32 * half + __ffs((int)w) - 1);
+                        w &= w - 1u;
+                    }
+                }
+                L.nz[lane] = (uint8_t)n;
+            }
+            return 0;
+        };
+        // the ring filled as far as it goes while word `oldest` is still needed
+        auto top_up = [&](uint32_t oldest) {
+            while (wr - oldest + 32u <= (uint32_t)kChainRing) {
+                ring[(wr + lane) & (kChainRing - 1)] = wr + lane < wlim ? __ldg(words + wr + lane) : 0u;
+                wr += 32u;
+            }
+        };
+        // the records of blocks m0 .. m0 + nd - 1 -> side data, one block per lane; then the count
+        auto side_data = [&](uint32_t m0, uint32_t nd, const ChainRecs& R, const ChainLists& L) {
+            bool over = false;
+            if ((uint32_t)lane < nd) {
+                uint64_t cstr = 0, Nw = 0, NS = 0;
+                uint32_t cn = 0;
+                for (uint32_t i = R.first[lane]; i < R.first[lane + 1]; ++i) {
+                    const uint32_t rc = R.rec[i], at = R.base + (rc >> 16);
+                    uint32_t n = rc & 127u;
+                    if (rc & 0x8000u) {
+                        const uint64_t bit = 1ull << ((rc >> 8) & 63u);
+                        Nw |= bit;
+                        if (ring_bits(ring, rd0, at - 1u, 1u)) NS |= bit;
+                    }
+                    if (cn + n > 64u) { over = true; break; }
+                    cn += n;
+                    uint32_t bp = at;
+                    while (n) {
+                        const uint32_t nn = min(n, 32u);
+                        cstr = (cstr << nn) | (uint64_t)ring_bits(ring, rd0, bp, nn);
+                        bp += nn; n -= nn;
+                    }
+                }
+                if (cn) cstr <<= 64u - cn;                     // first correction bit at bit 63
+                ulonglong2* o = reinterpret_cast<ulonglong2*>(outp + (uint64_t)block_index(m0 + lane) * 4);
+                o[0] = make_ulonglong2((L.h[lane] | Nw), cstr);
+                o[1] = make_ulonglong2(Nw, NS);
+            }
+            if (__any_sync(full, over)) err = kErrCorrupt;
+            __threadfence();                                   // the side data before the count
+            __syncwarp(full);
+            if (lane == 0) *my_progress = m0 + nd;
+        };
+        if (!bad) {
+            err = gather(0, sh.lists[0]);
+            top_up(rd0);
+        }
+        ++mk;
+        if (lane == 0) { sh.mail[mk & 1u].wr = wr; sh.mail[mk & 1u].err_h = (uint32_t)err; }
+        if (!meet_helper(sh, mk, lane)) return;
+        uint32_t m = 0, p = 0, rd_c = rd0, pend_m = 0, pend_n = 0, pend_p = 0;
+        while (!err) {
+            const uint32_t nblk = min(32u, total - m);
+            if (pend_n) { side_data(pend_m, pend_n, sh.recs[pend_p], sh.lists[pend_p]); pend_n = 0; }
+            top_up(rd_c);
+            if (m + nblk < total) { const int e = gather(m + nblk, sh.lists[p ^ 1u]); if (!err) err = e; }
+            ++mk;
+            if (lane == 0) { sh.mail[mk & 1u].wr = wr; sh.mail[mk & 1u].err_h = (uint32_t)err; }
+            if (!meet_helper(sh, mk, lane)) return;
+            const uint32_t nd = sh.mail[mk & 1u].nd;
+            const int err_c = (int)sh.mail[mk & 1u].err_c;
+            rd_c = sh.mail[mk & 1u].rd;
+            if (err || err_c) { if (!err) err = err_c; break; }
+            if (nd == nblk) {
+                pend_m = m; pend_n = nd; pend_p = p;
+                p ^= 1u;
+                m += nd;
+                if (m >= total) { side_data(pend_m, pend_n, sh.recs[pend_p], sh.lists[pend_p]); break; }
+            } else {                                           // the decoder stopped early: its records now, the lists from m again
+                if (nd) side_data(m, nd, sh.recs[p], sh.lists[p]);
+                m += nd;
+                top_up(rd_c);
+                { const int e = gather(m, sh.lists[p ^ 1u]); if (!err) err = e; }
+                ++mk;
+                if (lane == 0) { sh.mail[mk & 1u].wr = wr; sh.mail[mk & 1u].err_h = (uint32_t)err; }
+                if (!meet_helper(sh, mk, lane)) return;
+                p ^= 1u;
+            }
+        }
+        __syncwarp(full);
+        if (lane == 0) {
+            __threadfence();
+            *my_progress = 0xFFFFFFFFu;                        // a scan that failed must not keep a later one waiting
+            if (err) atomicMin(&P.status[img], err);
+        }
+    }
+}
+
+// Persistent launch: one CTA per SM with `pairs` chains, each a decoding warp (one thread of it
+// works) and a helper warp; warp w and its helper w + pairs sit on scheduler w % 4.  The groups
+// ((image, component) pairs, luminance first, most bytes first) are dealt to four queues, one per
+// scheduler (group gi is in queue gi % 4); within a queue every group is followed through its levels
+// (the refinement scans of the component that this call decodes, in script order), so a producer is
+// always taken before its consumer.  The first `rounds` groups of each CTA's schedulers are assigned
+// statically (group r * 4 * CTAs + 4 * CTA + q in round r: every scheduler of the device gets one
+// long luminance chain before any gets a second, and a group's levels start together in one CTA);
+// after that a decoder that has finished takes the next entry of its queue from a counter in global
+// memory.  sync: four queue counters, then four progress words per group, all zero before the launch.
+__global__ void __launch_bounds__(64 * kChainPairs, 1) ac_refine_group_kernel(Params P, FinalizeList fl, const uint32_t* __restrict__ list,
+                                                                              uint32_t n_groups, uint32_t* __restrict__ sync, int levels, int rounds) {
+    extern __shared__ __align__(16) unsigned char s_dyn[];     // one ChainShared per chain
+    ChainShared* s_sh = reinterpret_cast<ChainShared*>(s_dyn);
+    const int pairs = (int)(blockDim.x >> 6);
+    const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if ((int)threadIdx.x < pairs) { s_sh[threadIdx.x].phase_c = 0; s_sh[threadIdx.x].phase_h = 0; }
+    __syncthreads();
+    if (wid < pairs) {
+        if (lane == 0) chain_decoder(fl, s_sh[wid], list, n_groups, sync, (uint32_t)levels, (uint32_t)rounds, (uint32_t)wid & 3u, (uint32_t)wid >> 2);
+    } else {
+        chain_helper(P, fl, s_sh[wid - pairs], list, sync + 4, lane);
     }
 }
 
