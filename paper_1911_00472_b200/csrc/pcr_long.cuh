@@ -535,22 +535,27 @@ constexpr int kErrTimeout = -4;
 struct ChainBits {
     const uint32_t* ring;
     uint32_t w0, w1, w2;   // the word the next bit lies in and the two after it
-    uint32_t bits;         // position of the next bit, counted from the first bit of the interval's first word
-    uint32_t rd;           // ring word that follows w2 (absolute word index)
+    uint32_t bits;         // position of the next bit, counted from the first bit of ring word `org`
+    uint32_t org;          // absolute index of that word (moved up at the start of every batch)
     __device__ __forceinline__ void init(const uint32_t* r, uint32_t first, uint32_t lead) {
         ring = r;
         w0 = r[first & (kChainRing - 1)]; w1 = r[(first + 1) & (kChainRing - 1)]; w2 = r[(first + 2) & (kChainRing - 1)];
-        rd = first + 3;
+        org = first;
         bits = lead;
     }
     __device__ __forceinline__ uint32_t win() const { return __funnelshift_l(w1, w0, bits); }   // the next 32 bits (shift taken mod 32)
-    __device__ __forceinline__ void skip(uint32_t n) {        // n <= 96 (the third word is only prefetched)
-        const uint32_t nb = bits + n;
-        uint32_t adv = (nb >> 5) - (bits >> 5);
+    __device__ __forceinline__ uint32_t word() const { return org + (bits >> 5); }               // absolute index of the word of the next bit
+    __device__ __forceinline__ void skip(uint32_t n) {
+        const uint32_t nb = bits + n, adv = (nb >> 5) - (bits >> 5);
         bits = nb;
-        while (adv) { w0 = w1; w1 = w2; w2 = ring[rd & (kChainRing - 1)]; ++rd; --adv; }
+        if (adv) {
+            const uint32_t wi = org + (nb >> 5);
+            if (adv == 1u) { w0 = w1; w1 = w2; }
+            else { w0 = ring[wi & (kChainRing - 1)]; w1 = ring[(wi + 1u) & (kChainRing - 1)]; }
+            w2 = ring[(wi + 2u) & (kChainRing - 1)];
+        }
     }
-    __device__ __forceinline__ uint32_t pos() const { return bits; }
+    __device__ __forceinline__ void rebase() { org += bits >> 5; bits &= 31u; }
 };
 
 // the n bits (1..32) at bit position p (counted from the first bit of word `base`) of the ring
@@ -559,11 +564,12 @@ __device__ __forceinline__ uint32_t ring_bits(const uint32_t* ring, uint32_t bas
     return __funnelshift_l(b, a, p & 31u) >> (32u - n);
 }
 
-// Polls *flag until it reaches `need`; false after `limit` polls.
-__device__ __forceinline__ bool wait_at_least(const volatile uint32_t* flag, uint32_t need, uint32_t limit) {
+// Polls *flag until it reaches `need`, sleeping `ns` nanoseconds between polls; false after `limit` polls.
+__device__ __forceinline__ bool wait_at_least(const volatile uint32_t* flag, uint32_t need, uint32_t limit, uint32_t ns = 64) {
+#pragma unroll 1
     for (uint32_t i = 0; i < limit; ++i) {
         if (*flag >= need) return true;
-        __nanosleep(64);
+        __nanosleep(ns);
     }
     return false;
 }
@@ -573,10 +579,13 @@ __device__ __forceinline__ bool wait_at_least(const volatile uint32_t* flag, uin
 // coefficient follows the run; the end of band of a single block is entered as a run of 64 without a
 // new coefficient (it passes over the rest of the band like a run that overshoots); 0 = everything
 // else (longer end-of-band runs, codes longer than the index, undefined codes): the general path.
+__device__ __noinline__ uint32_t chain_lookup(const HuffTabT<kChainLutBits>& tab, uint32_t win) { return huff_lookup(tab, win); }
+
 struct ChainLists {
     uint64_t h[32];                    // positions of the band that are already non-zero, per block of the batch
-    uint8_t zpos[64][32];              // [i][block]: position of the block's i-th still-zero coefficient of the band
-    uint8_t nz[32];                    // how many there are
+    uint8_t zpos[64][32];              // [i][block]: position of the block's i-th still-zero coefficient of the band, minus i;
+                                       // entry nz: Se + 1 - nz (as if position Se + 1 followed)
+    uint8_t nz[32];                    // how many such positions there are (at most 63)
 };
 struct ChainRecs {
     uint32_t rec[kChainRecs];          // corrections | position << 8 | new << 15 | (bit position behind the sign bit - base) << 16
@@ -603,6 +612,7 @@ struct ChainShared {
 // the last value read, so that a consumer that is behind anyway polls once per many batches.
 __device__ __forceinline__ bool wait_progress(const volatile uint32_t* flag, uint32_t need, uint32_t& seen, uint32_t limit) {
     if (seen >= need) return true;
+#pragma unroll 1
     for (uint32_t i = 0; i < limit; ++i) {
         seen = *flag;
         if (seen >= need) return true;
@@ -624,7 +634,10 @@ __device__ __forceinline__ bool meet_decoder(ChainShared& sh, uint32_t k) {     
 __device__ __forceinline__ bool meet_helper(ChainShared& sh, uint32_t k, int lane) {  // a whole warp
     __syncwarp();
     if (lane == 0) { __threadfence_block(); sh.phase_h = k; }
-    const bool ok = __all_sync(0xffffffffu, wait_at_least(&sh.phase_c, k, kSpinLimit));
+    // (long sleeps: the helper is far ahead of the decoder, and its polls would take issue slots from the chains)
+    bool ok = true;
+    if (lane == 0) ok = wait_at_least(&sh.phase_c, k, kSpinLimit, 512);
+    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
     __threadfence_block();
     return ok;
 }
@@ -666,22 +679,36 @@ __device__ __forceinline__ void chain_decoder(const FinalizeList& fl, ChainShare
             const uint32_t nblk = min(32u, total - m);
             const ChainLists& L = sh.lists[p];
             ChainRecs& R = sh.recs[p];
-            uint32_t nrec = 0, nd = 0;
-            int err = 0;
-            const uint32_t base = B.pos();                     // a batch spans fewer than 2^16 bits (32 blocks of kChainBlockWords words)
+            // positions inside a batch count from the word the batch starts in (fewer than 2^16 bits: 32
+            // blocks of kChainBlockWords words)
+            B.rebase();
+            const uint32_t base = (B.org - sh.rd0) * 32u;
             R.base = base;
+            // a block is only begun while kChainBlockWords words lie ahead in the ring and the interval has
+            // not ended: one comparison for both, told apart behind the loop
+            const uint32_t avail = wr - B.org;
+            const uint32_t pause_bits = avail > kChainBlockWords + 2u ? (avail - (kChainBlockWords + 2u)) << 5 : 0u;
+            const uint32_t end_bits = limit >= base ? limit - base + 1u : 0u;      // first position that is past the end
+            const uint32_t stop_bits = min(pause_bits, end_bits);
+            uint32_t* recp = R.rec;
+            uint32_t* const rec_stop = R.rec + (kChainRecs - 64);
+            uint32_t nd = 0;
+            int err = 0;
             for (; nd < nblk; ++nd) {
-                if (wr - B.rd < kChainBlockWords || nrec > (uint32_t)kChainRecs - 64u) break;   // fetch more / flush first
-                R.first[nd] = nrec;
-                // k: the position that comes next; zi: how many of the block's zero positions lie below it
+                if (B.bits >= stop_bits || recp > rec_stop) break;
+                R.first[nd] = (uint32_t)(recp - R.rec);
+                // zi: how many of the block's still-zero positions are passed; ep: the list entry of the last
+                // one reached (entry t = position - t, so that the difference of two entries is the number of
+                // non-zero positions between them: one correction bit each)
                 const uint32_t nz = L.nz[nd];
-                uint32_t k = Ss, zi = 0;
+                uint32_t zi = 0, ep = Ss;
+                bool band_done = false;
                 if (eobrun == 0) {
-                    while (k <= Se) {
+                    for (;;) {
                         const uint32_t win = B.win();
                         uint32_t qe = sh.quick[win >> (32 - kChainLutBits)];
                         if (qe == 0) {                         // not a plain (run, new coefficient) symbol
-                            const uint32_t e = huff_lookup(sh.tab, win);
+                            const uint32_t e = chain_lookup(sh.tab, win);
                             const uint32_t len = e >> 8, rs = e & 255u, newc = rs & 1u, r = rs >> 4;
                             if (e == 0 || (rs & 14u)) { err = kErrCorrupt; break; }   // a refinement symbol has size 0 or 1
                             if (!newc && r < 15u) {            // end of band for this block and eobrun - 1 more
@@ -692,37 +719,30 @@ __device__ __forceinline__ void chain_decoder(const FinalizeList& fl, ChainShare
                             }
                             qe = (len + newc) | (r << 5) | (newc << 15);   // a code longer than the table's index
                         }
-                        const uint32_t r = (qe >> 5) & 127u, t = zi + r;
-                        const uint32_t p1 = B.pos() - base + (qe & 31u);   // behind the code and, for a new coefficient, its sign
-                        uint32_t cnt, y;
-                        if (t < nz) {                          // the target: the (r+1)-th zero position from here
-                            const uint32_t pos = L.zpos[t][nd];
-                            cnt = pos - k - r;                 // the non-zero positions passed: one correction bit each
-                            y = cnt | (pos << 8) | (qe & 0x8000u);
-                            zi = t + 1u;
-                            k = pos + 1u;
-                        } else {                               // past the band: the rest is passed over, nothing new
-                            cnt = Se + 1u - k - (nz - zi);
-                            y = cnt;
-                            zi = nz;
-                            k = Se + 1u;
-                        }
-                        R.rec[nrec++] = (p1 << 16) | y;
-                        B.skip((qe & 31u) + cnt);              // code, sign and correction bits in one step
+                        // the target: the (r+1)-th still-zero position from here; a run past the last one ends
+                        // at the list's closing entry (position Se + 1)
+                        const uint32_t t = min(zi + ((qe >> 5) & 127u), nz);
+                        const uint32_t e = L.zpos[t][nd];
+                        const uint32_t cnt = e - ep, pos = e + t, n1 = qe & 31u;
+                        *recp++ = ((B.bits + n1) << 16) | (pos << 8) | (qe & 0x8000u) | cnt;
+                        B.skip(n1 + cnt);                      // code, sign and correction bits in one step
+                        zi = t + 1u;
+                        ep = e;
+                        if (pos >= Se) { band_done = true; break; }
                     }
                 }
                 if (err) break;
-                if (k <= Se) {                                 // inside an end-of-band run: corrections for the rest of the band
-                    const uint32_t cnt = Se + 1u - k - (nz - zi);
-                    R.rec[nrec++] = ((B.pos() - base) << 16) | cnt;
+                if (!band_done) {                              // inside an end-of-band run: corrections for the rest of the band
+                    const uint32_t cnt = L.zpos[nz][nd] - ep;
+                    *recp++ = (B.bits << 16) | cnt;
                     B.skip(cnt);
                     --eobrun;
                 }
-                if (B.pos() > limit) { err = kErrCorrupt; break; }   // read past the end of the interval
             }
-            R.first[nd] = nrec;
+            R.first[nd] = (uint32_t)(recp - R.rec);
+            if (!err && B.bits >= end_bits) err = kErrCorrupt;     // read past the end of the interval
             ++mk;
-            sh.mail[mk & 1u].nd = nd; sh.mail[mk & 1u].rd = B.rd - 3u; sh.mail[mk & 1u].err_c = (uint32_t)err;
+            sh.mail[mk & 1u].nd = nd; sh.mail[mk & 1u].rd = B.word(); sh.mail[mk & 1u].err_c = (uint32_t)err;
             if (!meet_decoder(sh, mk)) return;
             wr = sh.mail[mk & 1u].wr;
             if (err || sh.mail[mk & 1u].err_h) break;
@@ -828,10 +848,12 @@ __device__ __forceinline__ void chain_helper(const Params& P, const FinalizeList
                 for (int half = 0; half < 2; ++half) {
                     uint32_t w = half ? (uint32_t)(z >> 32) : (uint32_t)z;
                     while (w) {
-                        L.zpos[n++][lane] = (uint8_t)(32 * half + __ffs((int)w) - 1);
+                        L.zpos[n][lane] = (uint8_t)(32 * half + __ffs((int)w) - 1 - (int)n);
+                        ++n;
                         w &= w - 1u;
                     }
                 }
+                L.zpos[n][lane] = (uint8_t)(Se + 1u - n);      // closing entry: behind the band
                 L.nz[lane] = (uint8_t)n;
             }
             return 0;
@@ -853,6 +875,7 @@ __device__ __forceinline__ void chain_helper(const Params& P, const FinalizeList
                     const uint32_t rc = R.rec[i], at = R.base + (rc >> 16);
                     uint32_t n = rc & 127u;
                     if (rc & 0x8000u) {
+                        if (((rc >> 8) & 127u) > Se) { over = true; break; }   // a new coefficient behind the band
                         const uint64_t bit = 1ull << ((rc >> 8) & 63u);
                         Nw |= bit;
                         if (ring_bits(ring, rd0, at - 1u, 1u)) NS |= bit;
