@@ -1121,7 +1121,7 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
                     lc += rec->long_count[(size_t)g * G + s];
                 }
                 if (lc) {
-                    first_pass_long_kernel<<<(lc + kLongWarps - 1) / kLongWarps, 32 * kLongWarps, 0, q>>>(P, rec->d_long + lb, lc);
+                    first_pass_long_kernel<<<lc, 32 * kLongWarps, 0, q>>>(P, rec->d_long + lb, lc);
                     ++g_launches;
                 }
             }
@@ -1182,14 +1182,14 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
                 ++g_launches;
             } else if (!targs) {
                 if (dc_only && rec->widths_mult16) dc_pixel_kernel<false><<<grid, 128, 0, q>>>(Q, o8);
-                else if (dc_only) pixel_kernel<false, 2><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+                else if (dc_only) dc_pixel_kernel<false, false><<<grid, 128, 0, q>>>(Q, o8);
                 else if (head_only && any_refine) pixel_kernel<true, 3><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
                 else if (head_only) pixel_kernel<false, 3><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
                 else if (any_refine) pixel_kernel<true, 1><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
                 else pixel_kernel<false, 1><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
             } else {
                 if (dc_only && rec->widths_mult16) dc_pixel_kernel<true><<<grid, 128, 0, q>>>(Q, o8);
-                else if (dc_only) pixel_kernel<false, 2, true><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
+                else if (dc_only) dc_pixel_kernel<true, false><<<grid, 128, 0, q>>>(Q, o8);
                 else if (head_only && any_refine) pixel_kernel<true, 3, true><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
                 else if (head_only) pixel_kernel<false, 3, true><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);
                 else if (any_refine) pixel_kernel<true, 1, true><<<grid, kPixThreads, 0, q>>>(Q, fl, o8);

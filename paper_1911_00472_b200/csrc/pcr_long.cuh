@@ -114,7 +114,10 @@ struct WordReader {
     __device__ __forceinline__ uint32_t pos() const { return rd * 32u - (uint32_t)nbits; }
 };
 
-constexpr int kLongWarps = 3;
+#ifndef PCR_LONG_WARPS
+#define PCR_LONG_WARPS 2
+#endif
+constexpr int kLongWarps = PCR_LONG_WARPS;   // warps per scan in first_pass_long_kernel: 32 subsequences each
 
 // What one lane needs to write the coefficients of an AC first pass.
 struct AcWrite {
@@ -248,12 +251,37 @@ __device__ __forceinline__ void dc_first_span(const HuffTab* tabs2, uint32_t slo
     sum0 = s0; sum1 = s1; sum2 = s2;
 }
 
-// One warp per listed (scan, image) whose scan is one restart interval; first passes only.
+// Exclusive prefix sum over the CTA's threads in thread order (warp scans, then the warps' totals
+// through shared memory); total = the sum over all threads.  Every thread of the CTA calls it.
+template <class T>
+__device__ __forceinline__ T cta_exclusive_sum(T v, T* s_tmp, int wid, int lane, int warps, T& total) {
+    const unsigned full = 0xffffffffu;
+    T inc = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const T o = __shfl_up_sync(full, inc, d);
+        if (lane >= d) inc += o;
+    }
+    __syncthreads();                                           // s_tmp may still be read from the previous call
+    if (lane == 31) s_tmp[wid] = inc;
+    __syncthreads();
+    T before = 0, all = 0;
+    for (int w = 0; w < warps; ++w) { const T t = s_tmp[w]; if (w < wid) before += t; all += t; }
+    total = all;
+    return before + inc - v;
+}
+
+// One CTA of kLongWarps warps per listed (scan, image) whose scan is one restart interval; first
+// passes only.  The interval is cut into 32 * kLongWarps subsequences, one per thread.
 __global__ void __launch_bounds__(32 * kLongWarps) first_pass_long_kernel(Params P, const uint32_t* __restrict__ list, uint32_t count) {
-    __shared__ HuffTab tabs[kLongWarps][2];
-    const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t it = blockIdx.x * kLongWarps + wid;
-    if (it >= count) return;                                   // whole warp
+    __shared__ HuffTab tabs[2];
+    __shared__ uint32_t s_pos[kLongWarps];                     // end state of every warp's last lane, for the next warp's first
+    __shared__ int s_state[kLongWarps];
+    __shared__ uint32_t s_u[kLongWarps];
+    __shared__ int s_i[kLongWarps];
+    const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
+    const uint32_t it = blockIdx.x;
+    if (it >= count) return;                                   // whole CTA
     const uint32_t si = list[it];
     const int s = (int)(si / (uint32_t)P.N), img = (int)(si % (uint32_t)P.N);
     const ScanDesc sd = P.scans[si];
@@ -266,21 +294,32 @@ __global__ void __launch_bounds__(32 * kLongWarps) first_pass_long_kernel(Params
     const uint32_t mcu_h = inter ? g.my : g.ubh[c0];
     const uint32_t total = mcu_w * mcu_h;                      // MCUs of the scan (one interval)
     const unsigned full = 0xffffffffu;
-    build_hufftab(tabs[wid][0], P.rec + sd.tab_off[0], lane);
-    if (sd.tab_off[1]) build_hufftab(tabs[wid][1], P.rec + sd.tab_off[1], lane);
+    if (wid == 0) build_hufftab(tabs[0], P.rec + sd.tab_off[0], lane);
+    if (wid == (kLongWarps > 1 ? 1 : 0) && sd.tab_off[1]) build_hufftab(tabs[1], P.rec + sd.tab_off[1], lane);
+    __syncthreads();
     const uint32_t* segtab = P.seg_start + sd.seg_base;
     const uint32_t bstart = segtab[0], bend = segtab[1] - 2u;
-    if (bstart < sd.data_off || bend > sd.data_end || bend < bstart) {
-        if (lane == 0) atomicMin(&P.status[img], kErrCorrupt);
+    if (bstart < sd.data_off || bend > sd.data_end || bend < bstart) {   // (the same for every thread)
+        if (tid == 0) atomicMin(&P.status[img], kErrCorrupt);
         return;
     }
     const uint32_t* base = reinterpret_cast<const uint32_t*>(P.ubuf) + (bstart >> 2);
     const uint32_t lead = 8u * (bstart & 3u), endbit = lead + 8u * (bend - bstart);
-    // 32 subsequences of S bits (whole words, at least 8 of them)
+    // subsequences of S bits (whole words, at least 8 of them)
+    constexpr uint32_t kSubs = 32u * kLongWarps;
     const uint32_t nwords = (endbit + 31u) >> 5;
-    const uint32_t S = 32u * max(8u, (nwords + 31u) / 32u);
-    const uint32_t my_begin = min(max((uint32_t)lane * S, lead), endbit), my_end = min(((uint32_t)lane + 1u) * S, endbit);
+    const uint32_t S = 32u * max(8u, (nwords + kSubs - 1u) / kSubs);
+    const uint32_t my_begin = min(max((uint32_t)tid * S, lead), endbit), my_end = min(((uint32_t)tid + 1u) * S, endbit);
     bool bad = false;
+    // the state the previous thread ended in (its last lane's through shared memory for a warp's first lane)
+    auto handed_on = [&](uint32_t pos_x, int st_x, uint32_t& ppos, int& pst) {
+        if (lane == 31) { s_pos[wid] = pos_x; s_state[wid] = st_x; }
+        __syncthreads();
+        ppos = __shfl_up_sync(full, pos_x, 1);
+        pst = __shfl_up_sync(full, st_x, 1);
+        if (lane == 0 && wid > 0) { ppos = s_pos[wid - 1]; pst = s_state[wid - 1]; }
+        ppos = min(ppos, endbit);
+    };
     if (dc) {
         DcWrite W;
         W.head = P.head; W.mcu_w = mcu_w; W.Al = sc.Al; W.hs = (uint32_t)P.hs; W.vs = (uint32_t)P.vs;
@@ -288,33 +327,29 @@ __global__ void __launch_bounds__(32 * kLongWarps) first_pass_long_kernel(Params
 #pragma unroll
         for (int c = 0; c < 3; ++c) { W.coff[c] = g.coff[c]; W.bw[c] = g.bw[c]; W.pred[c] = 0; }
         W.n = 0; W.n1 = total * bpm;
-        uint32_t pos = my_begin, pos_x, nb;
-        int j = 0, j_x, a0, a1, a2;
+        uint32_t pos = my_begin, pos_x = my_begin, nb = 0;
+        int j = 0, j_x = 0, a0 = 0, a1 = 0, a2 = 0;
         bool again = true;
-        for (int round = 0; round < 33; ++round) {
-            if (again) dc_first_span<false>(tabs[wid], sd.slots, inter, c0, base, pos, j, my_end, pos_x, j_x, nb, a0, a1, a2, W, bad);
-            const uint32_t ppos = min(__shfl_up_sync(full, pos_x, 1), endbit);
-            const int pj = __shfl_up_sync(full, j_x, 1);
-            again = lane > 0 && (ppos != pos || pj != j);
+        for (int round = 0; round <= (int)kSubs; ++round) {
+            if (again) dc_first_span<false>(tabs, sd.slots, inter, c0, base, pos, j, my_end, pos_x, j_x, nb, a0, a1, a2, W, bad);
+            uint32_t ppos; int pj;
+            handed_on(pos_x, j_x, ppos, pj);
+            again = tid > 0 && (ppos != pos || pj != j);
             if (again) { pos = ppos; j = pj; }
-            if (!__any_sync(full, again)) break;
+            if (!__syncthreads_or(again)) break;
         }
-        // first block and predictors of every lane: exclusive prefix sums
-        uint32_t nin = nb;
-        int b0 = a0, b1 = a1, b2 = a2;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const uint32_t on = __shfl_up_sync(full, nin, d);
-            const int o0 = __shfl_up_sync(full, b0, d), o1 = __shfl_up_sync(full, b1, d), o2 = __shfl_up_sync(full, b2, d);
-            if (lane >= d) { nin += on; b0 += o0; b1 += o1; b2 += o2; }
-        }
-        const uint32_t all = __shfl_sync(full, nin, 31);
-        W.n = min(nin - nb, W.n1); W.pred[0] = b0 - a0; W.pred[1] = b1 - a1; W.pred[2] = b2 - a2;
+        // first block and predictors of every thread: exclusive prefix sums
+        uint32_t all;
+        int t0, t1, t2;
+        W.n = min(cta_exclusive_sum(nb, s_u, wid, lane, kLongWarps, all), W.n1);
+        W.pred[0] = cta_exclusive_sum(a0, s_i, wid, lane, kLongWarps, t0);
+        W.pred[1] = cta_exclusive_sum(a1, s_i, wid, lane, kLongWarps, t1);
+        W.pred[2] = cta_exclusive_sum(a2, s_i, wid, lane, kLongWarps, t2);
         // the place inside the MCU follows from the block number (equal to the handed-on state unless
         // the stream is damaged; taking it from the block number keeps every store inside the image)
         if (nb && (uint32_t)j != W.n % bpm) bad = true;
         j = (int)(W.n % bpm);
-        dc_first_span<true>(tabs[wid], sd.slots, inter, c0, base, pos, j, my_end, pos_x, j_x, nb, a0, a1, a2, W, bad);
+        dc_first_span<true>(tabs, sd.slots, inter, c0, base, pos, j, my_end, pos_x, j_x, nb, a0, a1, a2, W, bad);
         if (all < total * bpm) bad = true;                     // the stream ends before the last block
     } else {
         const int c = c0, Ss = sc.Ss, Se = sc.Se;
@@ -323,30 +358,24 @@ __global__ void __launch_bounds__(32 * kLongWarps) first_pass_long_kernel(Params
         W.plane = P.planes + g.coff[c] * 64; W.headp = P.head + g.coff[c] * 8;
         W.maskp = reinterpret_cast<unsigned long long*>(P.aux + ax.base + g.loff[c]);
         W.mcu_w = mcu_w; W.bw = g.bw[c]; W.m = 0; W.m1 = total; W.p1 = 1 << sc.Al;
-        const HuffTab& tab = tabs[wid][0];
-        uint32_t pos = my_begin, pos_x, nb;
-        int k = Ss, k_x;
+        const HuffTab& tab = tabs[0];
+        uint32_t pos = my_begin, pos_x = my_begin, nb = 0;
+        int k = Ss, k_x = Ss;
         bool again = true;
-        for (int round = 0; round < 33; ++round) {
+        for (int round = 0; round <= (int)kSubs; ++round) {
             if (again) ac_first_span<false>(tab, base, pos, k, my_end, Ss, Se, pos_x, k_x, nb, W, bad);
-            const uint32_t ppos = min(__shfl_up_sync(full, pos_x, 1), endbit);
-            const int pk = __shfl_up_sync(full, k_x, 1);
-            again = lane > 0 && (ppos != pos || pk != k);
+            uint32_t ppos; int pk;
+            handed_on(pos_x, k_x, ppos, pk);
+            again = tid > 0 && (ppos != pos || pk != k);
             if (again) { pos = ppos; k = pk; }
-            if (!__any_sync(full, again)) break;
+            if (!__syncthreads_or(again)) break;
         }
-        uint32_t nin = nb;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const uint32_t on = __shfl_up_sync(full, nin, d);
-            if (lane >= d) nin += on;
-        }
-        const uint32_t all = __shfl_sync(full, nin, 31);
-        W.m = min(nin - nb, total);
+        uint32_t all;
+        W.m = min(cta_exclusive_sum(nb, s_u, wid, lane, kLongWarps, all), total);
         ac_first_span<true>(tab, base, pos, k, my_end, Ss, Se, pos_x, k_x, nb, W, bad);
         if (all < total) bad = true;                                         // the stream ends before the last block
     }
-    if (__any_sync(full, bad) && lane == 0) atomicMin(&P.status[img], kErrCorrupt);
+    if (__syncthreads_or(bad) && tid == 0) atomicMin(&P.status[img], kErrCorrupt);
 }
 
 // ---------------------------------------------------------------------------------------

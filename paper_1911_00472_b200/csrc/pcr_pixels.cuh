@@ -416,7 +416,11 @@ __global__ void __launch_bounds__(kPixThreads, PCR_PIX_MIN_CTAS) pixel_kernel(Pa
 // arithmetic as the general kernel: the transform collapses to its k = 0 term, samples clamp to
 // 0..255), then every thread writes 16-byte vectors whose bytes are picked from the two triples
 // of the vector's MCU half-row.  48 bytes per MCU row = 3 vectors, so a vector never leaves its MCU.
-template <bool kRoi>
+// kAligned = false: images of any width.  A row of the unit then starts at any byte address: every
+// thread takes one 16-byte-aligned chunk of global memory that the row touches, builds its four
+// words from the triples of the (at most two) pixels each word covers, and stores the chunk whole
+// when it lies inside the row, byte by byte at the row's two ends.
+template <bool kRoi, bool kAligned = true>
 __global__ void __launch_bounds__(128) dc_pixel_kernel(Params P, uint8_t* __restrict__ out) {
     __shared__ uint32_t s_tri[2][2 * kPixMcus];        // [block row of the MCU row][block column]: R | G << 8 | B << 16
     const int tid = threadIdx.x;
@@ -451,6 +455,62 @@ __global__ void __launch_bounds__(128) dc_pixel_kernel(Params P, uint8_t* __rest
     const int nrows = min(16, (int)im.H - 16 * (int)un.mrow);
     const size_t gpitch = (size_t)im.W * 3;
     uint8_t* gbase = out + im.out_off + ((uint64_t)(16 * un.mrow) * im.W + 16 * (uint64_t)un.mcol0) * 3;
+    if (!kAligned) {
+        const int len = 3 * min(16 * nm, (int)im.W - 16 * (int)un.mcol0);      // bytes of the unit in one output row
+        // the four bytes at offset o of a row (o may lie up to 15 bytes before the row or behind its end:
+        // those bytes are not stored, their pixels are clamped into the unit): pixel px from channel ph
+        // on, then pixel px + 1
+        auto word_at = [&](const uint32_t* tri, int o) {
+            const int oo = o + 24;
+            const int px = (int)(((uint32_t)oo * 0xAAABu) >> 17) - 8, ph = oo - 3 * (px + 8);
+            const uint32_t A = tri[min(max(px, 0), 16 * nm - 1) >> 3], Bt = tri[min(max(px + 1, 0), 16 * nm - 1) >> 3];
+            return __byte_perm(A, Bt, ph == 0 ? 0x4210u : (ph == 1 ? 0x5421u : 0x6542u));
+        };
+        // chunks that lie inside the row: whole 16-byte stores
+        constexpr int kInner = (3 * 16 * kPixMcus) / 16 - 1;
+        for (int i = tid; i < nrows * kInner; i += 128) {
+            const int row = i / kInner, slot = 1 + (i - row * kInner);
+            uint8_t* g = gbase + row * gpitch;                                  // first byte of the row
+            const int lead = (int)(reinterpret_cast<uintptr_t>(g) & 15u);
+            if (16 * slot + 16 > lead + len) continue;                          // the row's last chunk, or behind it
+            const int o0 = 16 * slot - lead;                                    // the chunk's first byte, counted from g
+            const uint32_t* tri = s_tri[row >> 3];
+            uint32_t w[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int o = o0 + 4 * j;
+                const int px = (int)(((uint32_t)o * 0xAAABu) >> 17), ph = o - 3 * px;
+                const uint32_t A = tri[px >> 3], Bt = tri[(px + 1) >> 3];
+                w[j] = __byte_perm(A, Bt, ph == 0 ? 0x4210u : (ph == 1 ? 0x5421u : 0x6542u));
+            }
+            *reinterpret_cast<uint4*>(g + o0) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+        // the first and the last chunk of every row: whole words where they lie inside, else bytes
+        if (tid < 2 * nrows) {
+            const int row = tid >> 1;
+            uint8_t* g = gbase + row * gpitch;
+            const int lead = (int)(reinterpret_cast<uintptr_t>(g) & 15u);
+            const int nch = (lead + len + 15) >> 4;
+            const int slot = (tid & 1) ? nch - 1 : 0;
+            if (!(tid & 1) || nch > 1) {
+                const int o0 = 16 * slot - lead;
+                const uint32_t* tri = s_tri[row >> 3];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int o = o0 + 4 * j;
+                    const uint32_t w = word_at(tri, o);
+                    if (o >= 0 && o + 4 <= len) {
+                        *reinterpret_cast<uint32_t*>(g + o) = w;
+                    } else {
+#pragma unroll
+                        for (int b = 0; b < 4; ++b)
+                            if (o + b >= 0 && o + b < len) g[o + b] = (uint8_t)(w >> (8 * b));
+                    }
+                }
+            }
+        }
+        return;
+    }
     const int vec = 3 * nm;                                 // 16-byte vectors per output row of this unit
     for (int i = tid; i < nrows * vec; i += 128) {
         const int row = i / vec, v = i - row * vec, mcu = v / 3, kk = v - 3 * mcu;

@@ -66,7 +66,7 @@ def test_full_record_every_pixel(config, oracle_pool):
     offsets = [int(inf.out_offset) for inf in dec.info]
     try:
         with tempfile.TemporaryDirectory() as td:
-            for k in (10, 5):
+            for k in (10, 5, 1):
                 want = oracle_record_pixels(pool, workers, rec.bytes, td, offsets, dec.out_bytes, k)
                 dec.out = torch.zeros(dec.out_bytes, dtype=torch.uint8, device="cuda")     # gaps between images stay zero
                 got = dec.decode(k)

@@ -54,6 +54,14 @@ def test_tiny_record_random_crops_every_k(rec0):
         _check(rec0, k, crops, 24, range(rec0.n_images))
 
 
+def test_widths_that_are_no_multiple_of_sixteen_dc_only():
+    # k = 1 takes the DC-only pixel kernel; with such widths an output row starts at any byte address
+    rec = pcr_synth.make_record(2, n_images=6)
+    assert any(w % 16 for w, _ in _dims(rec))
+    crops = pcr_synth.random_resized_crops(_dims(rec), 5)
+    _check(rec, 1, crops, 32, range(rec.n_images))
+
+
 def test_full_image_identity_size(rec0):
     # crop = whole image, size = image size: the tensor is the normalised decode itself
     crops = np.array([[0, 0, w, h, i & 1] for i, (w, h) in enumerate(_dims(rec0))], dtype=np.uint32)
