@@ -785,7 +785,7 @@ def main():
     dom = max(kernels, key=kernels.get)
     peak, peak_src = hbm_peak()
     achieved = model[dom] / (kernels[dom] * 1e-3) / 1e9
-    traffic = measured_traffic(dom, k, n_img)
+    traffic = measured_traffic(dom, k, n_img) if wl == WORKLOAD else None      # the capture is of the ImageNet-shaped record
     whole = model["total"] / (ms_max / args.steps * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": traffic, "peak_source": peak_src, "kernel_ms": kernels[dom],
