@@ -7,23 +7,24 @@
 //  * dc_refine_kernel: a DC refinement scan carries exactly one raw bit per block, so after
 //    unstuffing bit j of a restart interval is block j of the interval in scan order: one thread
 //    per MCU, no chain at all.  Used for every record.
-//  * first_pass_long_kernel: DC and AC first passes.  One warp per (scan, image); the segment is cut
-//    into 32 subsequences of equal bit length and every lane decodes its own.  A lane that starts
-//    in the middle of the stream does not know where a code begins nor which coefficient (or which
-//    block of the MCU) it is at; it starts anyway, and because Huffman streams re-synchronise, its
-//    state at the end of its subsequence is usually right.  The lanes then hand their end states on:
-//    a lane whose predecessor ended in a state other than the one it started from decodes again
-//    from there; the rounds stop when nothing changes (at the latest after 32: lane 0 starts at
-//    the true beginning, so after round r lanes 0..r are exact).  A prefix sum of the blocks each
-//    lane finished (and of the DC differences per component) gives every lane its first block and
-//    its predictors, and a last pass decodes once more and writes.
+//  * first_pass_long_kernel: DC and AC first passes.  One small CTA per (scan, image); the segment is
+//    cut into one subsequence of equal bit length per thread and every thread decodes its own.  A
+//    thread that starts in the middle of the stream does not know where a code begins nor which
+//    coefficient (or which block of the MCU) it is at; it starts anyway, and because Huffman streams
+//    re-synchronise, its state at the end of its subsequence is often right.  The threads then hand
+//    their end states on: a thread whose predecessor ended in a state other than the one it started
+//    from decodes again from there; the rounds stop when nothing changes (thread 0 starts at the
+//    true beginning, so after round r threads 0..r are exact).  A prefix sum of the blocks each
+//    thread finished (and of the DC differences per component) gives every thread its first block
+//    and its predictors, and a last pass decodes once more and writes.
 //  * sequential_long_kernel: the same scheme for the one scan of a baseline JPEG.
 //  * ac_refine_group_kernel: an AC refinement cannot be entered in the middle (how many correction
 //    bits follow a symbol depends on which coefficients of the block are already non-zero, i.e. on
-//    the block number).  One warp per scan: lane 0 walks the chain with ordinary branches (no other
-//    lane shares its instruction stream), the other lanes fetch the bitstream into a shared-memory
-//    ring, gather the masks of the next 32 blocks and turn lane 0's symbol records into side data.
-//    The refinements of one component share a CTA and run behind one another, block by block.
+//    the block number).  A scan is one chain: one thread follows it with ordinary branches, a
+//    helper warp fetches the bitstream into a shared-memory ring, prepares the masks of the next 32
+//    blocks and turns the thread's symbol records into side data.  All chains of a record run in
+//    one persistent launch that deals them to the SMs' schedulers evenly; the refinements of one
+//    component run behind one another, block by block.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -531,26 +532,26 @@ __global__ void __launch_bounds__(32 * kSeqLongWarps) sequential_long_kernel(Par
 }
 
 // ---------------------------------------------------------------------------------------
-// AC refinements of scans that are one restart interval.  One CTA per listed (image,
-// component), one warp per refinement scan of that component that the call decodes (at most
-// four, in scan order).  Side data written per block is that of entropy_kernel's refinement
-// branch: {non-zero mask of the band after the scan, correction bits in reading order from bit
-// 63 down, newly non-zero positions, the positive ones among them}.
+// AC refinements of scans that are one restart interval.  The unit of work is a chain: one
+// refinement scan of one (image, component) group; a group has at most four (its "levels", in
+// scan order).  Side data written per block is that of entropy_kernel's refinement branch:
+// {non-zero mask of the band after the scan, correction bits in reading order from bit 63 down,
+// newly non-zero positions, the positive ones among them}.
 //
-// The time of a scan is the number of instructions lane 0 executes per symbol (a warp or two
-// per scheduler: every instruction waits for the one before), so lane 0 only follows the chain:
-// Huffman symbol -> run r -> position of the (r+1)-th still-zero coefficient -> number of
-// correction bits passed -> next symbol.  For every symbol it leaves a record {bit position
-// behind the sign, new position, number of correction bits}; afterwards all lanes turn the
-// records of 32 blocks into the side data in parallel (one lane per block, reading sign and
-// correction bits back from the ring).
+// The time of a chain is the number of instructions one thread executes per symbol (every
+// instruction waits for the one before), so the decoding thread only follows the chain: Huffman
+// symbol -> run r -> position of the (r+1)-th still-zero coefficient -> number of correction bits
+// passed -> next symbol.  For every symbol it leaves a record {bit position behind the sign, new
+// position, number of correction bits}; the chain's helper warp lists the still-zero positions
+// of the next 32 blocks meanwhile and afterwards turns the records of 32 blocks into the side
+// data (one lane per block, reading sign and correction bits back from the ring).
 //
 // A later refinement of the same component needs the masks the earlier one leaves, block by
-// block.  Both walk the same block grid in the same order, so the later warp runs behind the
-// earlier one instead of after it: every warp publishes the number of blocks whose side data it
-// has written (shared memory, after a fence), and a warp that depends on it waits, with a bounded
-// number of polls, until the blocks it is about to read are there.  Producer and consumer share
-// a CTA, so both are resident while either waits.
+// block.  Both walk the same block grid in the same order, so the later chain runs behind the
+// earlier one instead of after it: every chain publishes the number of blocks whose side data it
+// has written (global memory, after a fence), and a helper that depends on it waits, with a
+// bounded number of polls, until the blocks it is about to read are there.  A chain is only
+// started after the chains it depends on (queue order), so its producer is running or done.
 // ---------------------------------------------------------------------------------------
 constexpr int kGroupWarps = 4;           // refinement scans of one component in one call (pcr_open admits four)
 constexpr int kChainPairs = 16;          // chains per CTA of the persistent refinement launch (four per scheduler), two warps each
