@@ -52,8 +52,9 @@ extern "C" {
                                segment overrun, wrong number of restart markers                   */
 #define PCR_E_TIMEOUT (-4)  /* a bounded device-side wait gave up: in records without restart
                                markers a refinement scan follows, block by block, the earlier
-                               refinement of the same component that another warp of its CTA
-                               decodes; its polls for that warp's progress are counted          */
+                               refinement of the same component that other warps of the same
+                               launch decode, and a scan's decoding thread and helper warp meet
+                               once per batch of blocks; the polls of these waits are counted   */
 #define PCR_E_CUDA (-5)     /* a CUDA runtime call failed                                        */
 #define PCR_E_NOMEM (-6)    /* host or device allocation failed                                  */
 

@@ -553,7 +553,6 @@ __global__ void __launch_bounds__(32 * kSeqLongWarps) sequential_long_kernel(Par
 // bounded number of polls, until the blocks it is about to read are there.  A chain is only
 // started after the chains it depends on (queue order), so its producer is running or done.
 // ---------------------------------------------------------------------------------------
-constexpr int kGroupWarps = 4;           // refinement scans of one component in one call (pcr_open admits four)
 constexpr int kChainPairs = 16;          // chains per CTA of the persistent refinement launch (four per scheduler), two warps each
 constexpr int kChainRing = 256;          // words of bitstream per chain in shared memory
 constexpr int kChainRecs = 512;          // symbol records per batch of blocks (four bytes each)
