@@ -95,9 +95,16 @@ def test_all_zero_and_saturated_streams(monkeypatch):
     _compare_every_k(rec, 0, monkeypatch)
 
 
-@pytest.mark.parametrize("name", ["spectral4", "mixed6", "deep14"])
+# four AC refinements of the luminance (the most one call decodes per component), two of each chroma component
+SCRIPT_FOUR_LEVELS = [((0, 1, 2), 0, 0, 0, 0), ((0,), 1, 63, 0, 4), ((1,), 1, 63, 0, 2), ((2,), 1, 63, 0, 2),
+                      ((0,), 1, 63, 4, 3), ((0,), 1, 63, 3, 2), ((1,), 1, 63, 2, 1), ((2,), 1, 63, 2, 1),
+                      ((0,), 1, 63, 2, 1), ((0,), 1, 63, 1, 0), ((1,), 1, 63, 1, 0), ((2,), 1, 63, 1, 0)]
+
+
+@pytest.mark.parametrize("name", ["spectral4", "mixed6", "deep14", "four_levels"])
 def test_other_scripts_without_restart_markers(name, monkeypatch):
-    scripts = {"spectral4": pcr_synth.SCRIPT_SPECTRAL_4, "mixed6": pcr_synth.SCRIPT_MIXED_6, "deep14": pcr_synth.SCRIPT_DEEP_14}
+    scripts = {"spectral4": pcr_synth.SCRIPT_SPECTRAL_4, "mixed6": pcr_synth.SCRIPT_MIXED_6, "deep14": pcr_synth.SCRIPT_DEEP_14,
+               "four_levels": SCRIPT_FOUR_LEVELS}
     with pcr_synth.scan_script(scripts[name]):
         rec = pcr_synth.make_record(3, n_images=2, restart_rows=False)
     _compare_every_k(rec, 0, monkeypatch)
