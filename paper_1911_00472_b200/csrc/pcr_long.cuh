@@ -120,6 +120,105 @@ struct WordReader {
 #endif
 constexpr int kLongWarps = PCR_LONG_WARPS;   // warps per scan in first_pass_long_kernel: 32 subsequences each
 
+// ---------------------------------------------------------------------------------------
+// The search passes of first_pass_long_kernel (a thread decodes its subsequence only to learn in which
+// state it ends and how many blocks it finishes) are the serial part of that kernel: when a stream
+// does not re-synchronise (a stretch of equally long symbols, in which a shifted reading stays shifted)
+// the true state moves on by one subsequence per round.  So they are kept short: a lookup table that
+// already holds what the search needs of a symbol, and a reader of three words in registers.
+// ---------------------------------------------------------------------------------------
+struct GlobalBits {
+    const uint32_t* w;     // base word (global memory; the neighbouring threads share its cache lines)
+    uint32_t w0, w1, w2;   // the word the next bit lies in and the two after it
+    uint32_t bits;         // position of the next bit, counted from the first bit of the base word
+    __device__ __forceinline__ void init(const uint32_t* base, uint32_t pos) {
+        w = base;
+        bits = pos;
+        const uint32_t i = pos >> 5;
+        w0 = __ldg(w + i); w1 = __ldg(w + i + 1); w2 = __ldg(w + i + 2);
+    }
+    __device__ __forceinline__ uint32_t win() const { return __funnelshift_l(w1, w0, bits); }   // the next 32 bits (shift taken mod 32)
+    __device__ __forceinline__ void skip(uint32_t n) {        // n < 32: at most one word further
+        const uint32_t nb = bits + n;
+        if ((nb ^ bits) >> 5) { w0 = w1; w1 = w2; w2 = __ldg(w + (nb >> 5) + 2); }
+        bits = nb;
+    }
+};
+
+// What the search of an AC first pass needs of a symbol (a HuffTab entry (length << 8) | (run << 4 | size)):
+// bits 0..4 bits to skip (code and extra bits), 5..8 positions the symbol moves on minus one (run + 1 for
+// a coefficient, 16 for sixteen zeros), 9 end of band, 10..13 its run-length exponent.
+constexpr uint32_t kSearchEob = 0x200u;
+__device__ __forceinline__ uint32_t ac_search_entry(uint32_t t) {
+    if (t == 0) return 0;
+    const uint32_t len = t >> 8, r = (t >> 4) & 15u, sz = t & 15u;
+    if (sz) return (len + sz) | (r << 5);
+    if (r == 15u) return len | (15u << 5);
+    return (len + r) | kSearchEob | (r << 10);
+}
+
+// Search pass of an AC first pass: the symbols that START in [pos, pos_end), from zigzag position k.
+// An undefined code is skipped by one bit and a coefficient beyond the band ends the block (the thread
+// is then reading from a wrong entry point and only has to arrive somewhere).
+__device__ __forceinline__ void ac_search_span(const HuffTab& tab, const uint16_t* slut, const uint32_t* base, uint32_t pos, int k,
+                                               uint32_t pos_end, int Ss, int Se, uint32_t& pos_out, int& k_out, uint32_t& nblk) {
+    GlobalBits B;
+    B.init(base, pos);
+    uint32_t nb = 0;
+    while (B.bits < pos_end) {
+        const uint32_t win = B.win();
+        uint32_t e = slut[win >> (32 - kLutBits)];
+        if (e == 0) {                                          // a code longer than the table's index, or none
+            e = ac_search_entry(huff_lookup(tab, win));
+            if (e == 0) { B.skip(1); continue; }
+        }
+        if (e & kSearchEob) {
+            const uint32_t r = e >> 10;
+            nb += r ? (1u << r) + ((win << ((e & 31u) - r)) >> (32u - r)) : 1u;
+            k = Ss;
+        } else {
+            const int nk = k + (int)((e >> 5) & 15u) + 1;
+            if (nk > Se) { ++nb; k = Ss; } else k = nk;
+        }
+        B.skip(e & 31u);
+    }
+    pos_out = B.bits;
+    k_out = k;
+    nblk = nb;
+}
+
+// Search pass of a DC first pass.  dlut: per table, (length << 4) | size of the codes of at most kLutBits
+// bits; tbits: bit j = the table of the j-th block of an MCU; cpack: two bits per j = its component.
+__device__ __forceinline__ void dc_search_span(const HuffTab* tabs2, const uint8_t* dlut, uint32_t tbits, uint32_t cpack, int bpm,
+                                               const uint32_t* base, uint32_t pos, int j, uint32_t pos_end, uint32_t& pos_out,
+                                               int& j_out, uint32_t& nblk, int& sum0, int& sum1, int& sum2) {
+    GlobalBits B;
+    B.init(base, pos);
+    uint32_t nb = 0;
+    int s0 = 0, s1 = 0, s2 = 0;
+    while (B.bits < pos_end) {
+        const uint32_t win = B.win();
+        const uint32_t tsel = (tbits >> j) & 1u;
+        const uint32_t e = dlut[(tsel << kLutBits) + (win >> (32 - kLutBits))];
+        int len = (int)(e >> 4), sz = (int)(e & 15u);
+        if (e == 0) {
+            const uint32_t t = huff_lookup(tabs2[tsel], win);
+            len = (int)(t >> 8); sz = (int)(t & 255u);
+            if (t == 0 || sz > 15) { B.skip(1); continue; }
+        }
+        const int d = extend_bits(top_bits(win << len, sz), sz);
+        const uint32_t c = (cpack >> (2 * j)) & 3u;
+        s0 += c == 0u ? d : 0; s1 += c == 1u ? d : 0; s2 += c == 2u ? d : 0;
+        B.skip((uint32_t)(len + sz));
+        ++nb;
+        if (++j == bpm) j = 0;
+    }
+    pos_out = B.bits;
+    j_out = j;
+    nblk = nb;
+    sum0 = s0; sum1 = s1; sum2 = s2;
+}
+
 // What one lane needs to write the coefficients of an AC first pass.
 struct AcWrite {
     int16_t* plane;        // the component's lines
@@ -280,6 +379,7 @@ __global__ void __launch_bounds__(32 * kLongWarps) first_pass_long_kernel(Params
     __shared__ int s_state[kLongWarps];
     __shared__ uint32_t s_u[kLongWarps];
     __shared__ int s_i[kLongWarps];
+    __shared__ __align__(4) uint16_t s_lut[1 << kLutBits];    // the search pass's table (AC), or two byte tables (DC)
     const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
     const uint32_t it = blockIdx.x;
     if (it >= count) return;                                   // whole CTA
@@ -297,6 +397,16 @@ __global__ void __launch_bounds__(32 * kLongWarps) first_pass_long_kernel(Params
     const unsigned full = 0xffffffffu;
     if (wid == 0) build_hufftab(tabs[0], P.rec + sd.tab_off[0], lane);
     if (wid == (kLongWarps > 1 ? 1 : 0) && sd.tab_off[1]) build_hufftab(tabs[1], P.rec + sd.tab_off[1], lane);
+    __syncthreads();
+    if (dc) {
+        uint8_t* dl = reinterpret_cast<uint8_t*>(s_lut);
+        for (int i = tid; i < (2 << kLutBits); i += 32 * kLongWarps) {
+            const uint32_t t = ((i >> kLutBits) == 0 || sd.tab_off[1]) ? tabs[i >> kLutBits].lut[i & ((1 << kLutBits) - 1)] : 0u;
+            dl[i] = (uint8_t)((t != 0 && (t & 255u) <= 15u) ? ((t >> 8) << 4) | (t & 15u) : 0u);
+        }
+    } else {
+        for (int i = tid; i < (1 << kLutBits); i += 32 * kLongWarps) s_lut[i] = (uint16_t)ac_search_entry(tabs[0].lut[i]);
+    }
     __syncthreads();
     const uint32_t* segtab = P.seg_start + sd.seg_base;
     const uint32_t bstart = segtab[0], bend = segtab[1] - 2u;
@@ -328,11 +438,18 @@ __global__ void __launch_bounds__(32 * kLongWarps) first_pass_long_kernel(Params
 #pragma unroll
         for (int c = 0; c < 3; ++c) { W.coff[c] = g.coff[c]; W.bw[c] = g.bw[c]; W.pred[c] = 0; }
         W.n = 0; W.n1 = total * bpm;
+        // per block of the MCU: its table (one bit) and its component (two bits)
+        uint32_t tbits = 0, cpack = 0;
+        for (uint32_t jj = 0; jj < bpm; ++jj) {
+            const uint32_t ny = (uint32_t)(P.hs * P.vs), ci = inter ? (jj < ny ? 0u : jj - ny + 1u) : 0u;
+            tbits |= ((sd.slots >> (2u * ci)) & 1u) << jj;
+            cpack |= (inter ? ci : (uint32_t)c0) << (2u * jj);
+        }
         uint32_t pos = my_begin, pos_x = my_begin, nb = 0;
         int j = 0, j_x = 0, a0 = 0, a1 = 0, a2 = 0;
         bool again = true;
         for (int round = 0; round <= (int)kSubs; ++round) {
-            if (again) dc_first_span<false>(tabs, sd.slots, inter, c0, base, pos, j, my_end, pos_x, j_x, nb, a0, a1, a2, W, bad);
+            if (again) dc_search_span(tabs, reinterpret_cast<const uint8_t*>(s_lut), tbits, cpack, (int)bpm, base, pos, j, my_end, pos_x, j_x, nb, a0, a1, a2);
             uint32_t ppos; int pj;
             handed_on(pos_x, j_x, ppos, pj);
             again = tid > 0 && (ppos != pos || pj != j);
@@ -364,7 +481,7 @@ __global__ void __launch_bounds__(32 * kLongWarps) first_pass_long_kernel(Params
         int k = Ss, k_x = Ss;
         bool again = true;
         for (int round = 0; round <= (int)kSubs; ++round) {
-            if (again) ac_first_span<false>(tab, base, pos, k, my_end, Ss, Se, pos_x, k_x, nb, W, bad);
+            if (again) ac_search_span(tab, s_lut, base, pos, k, my_end, Ss, Se, pos_x, k_x, nb);
             uint32_t ppos; int pk;
             handed_on(pos_x, k_x, ppos, pk);
             again = tid > 0 && (ppos != pos || pk != k);
