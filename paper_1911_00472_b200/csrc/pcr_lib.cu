@@ -1012,8 +1012,7 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
         if (rec->script[s].Ss > 0 && rec->script[s].Ah > 0 && (first_refine_wave < 0 || rec->wave_of_scan[s] < first_refine_wave))
             first_refine_wave = rec->wave_of_scan[s];
     const bool chains = first_refine_wave >= 0 && rec->n_groups > 0;
-    int chain_depth = kChainPairs / 4;          // chains per scheduler of the chain launch
-    if (const char* e = getenv("PCR_CHAIN_DEPTH")) chain_depth = std::max(1, std::min(kChainPairs / 4, atoi(e)));
+    const int chain_depth = kChainPairs / 4;    // chains per scheduler of the chain launch
     bool dc_only = true, head_only = true;      // no AC scan at all / no scan beyond zigzag position 7
     for (int s = 0; s < k; ++s) {
         if (rec->script[s].Ss > 0 || rec->script[s].Se > 0) dc_only = false;
