@@ -466,6 +466,22 @@ __global__ void __launch_bounds__(128) dc_pixel_kernel(Params P, uint8_t* __rest
             const uint32_t A = tri[min(max(px, 0), 16 * nm - 1) >> 3], Bt = tri[min(max(px + 1, 0), 16 * nm - 1) >> 3];
             return __byte_perm(A, Bt, ph == 0 ? 0x4210u : (ph == 1 ? 0x5421u : 0x6542u));
         };
+        // the bytes of one output row of the unit, once per block row (the eight pixel rows of a block row are
+        // equal), with 16 bytes of margin on either side so that a chunk may begin before the row or end behind it
+        constexpr int kPatWords = (16 + 3 * 16 * kPixMcus + 16) / 4;
+        __shared__ __align__(16) uint32_t s_pat[2][kPatWords];
+        for (int i = tid; i < 2 * kPatWords; i += 128) {
+            const int br = i / kPatWords, wi = i - br * kPatWords;
+            s_pat[br][wi] = word_at(s_tri[br], 4 * wi - 16);
+        }
+        __syncthreads();
+        // the 16 bytes of a row from offset o on (o >= -16): five pattern words, shifted into place
+        auto chunk_at = [&](const uint32_t* pat, int o) {
+            const int sb = o + 16, a = 8 * (sb & 3);
+            const uint32_t* q = pat + (sb >> 2);
+            const uint32_t p0 = q[0], p1 = q[1], p2 = q[2], p3 = q[3], p4 = q[4];
+            return make_uint4(__funnelshift_r(p0, p1, a), __funnelshift_r(p1, p2, a), __funnelshift_r(p2, p3, a), __funnelshift_r(p3, p4, a));
+        };
         // chunks that lie inside the row: whole 16-byte stores
         constexpr int kInner = (3 * 16 * kPixMcus) / 16 - 1;
         for (int i = tid; i < nrows * kInner; i += 128) {
@@ -474,16 +490,7 @@ __global__ void __launch_bounds__(128) dc_pixel_kernel(Params P, uint8_t* __rest
             const int lead = (int)(reinterpret_cast<uintptr_t>(g) & 15u);
             if (16 * slot + 16 > lead + len) continue;                          // the row's last chunk, or behind it
             const int o0 = 16 * slot - lead;                                    // the chunk's first byte, counted from g
-            const uint32_t* tri = s_tri[row >> 3];
-            uint32_t w[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int o = o0 + 4 * j;
-                const int px = (int)(((uint32_t)o * 0xAAABu) >> 17), ph = o - 3 * px;
-                const uint32_t A = tri[px >> 3], Bt = tri[(px + 1) >> 3];
-                w[j] = __byte_perm(A, Bt, ph == 0 ? 0x4210u : (ph == 1 ? 0x5421u : 0x6542u));
-            }
-            *reinterpret_cast<uint4*>(g + o0) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4*>(g + o0) = chunk_at(s_pat[row >> 3], o0);
         }
         // the first and the last chunk of every row: whole words where they lie inside, else bytes
         if (tid < 2 * nrows) {
@@ -494,17 +501,17 @@ __global__ void __launch_bounds__(128) dc_pixel_kernel(Params P, uint8_t* __rest
             const int slot = (tid & 1) ? nch - 1 : 0;
             if (!(tid & 1) || nch > 1) {
                 const int o0 = 16 * slot - lead;
-                const uint32_t* tri = s_tri[row >> 3];
+                const uint4 v = chunk_at(s_pat[row >> 3], o0);
+                const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const int o = o0 + 4 * j;
-                    const uint32_t w = word_at(tri, o);
                     if (o >= 0 && o + 4 <= len) {
-                        *reinterpret_cast<uint32_t*>(g + o) = w;
+                        *reinterpret_cast<uint32_t*>(g + o) = w4[j];
                     } else {
 #pragma unroll
                         for (int b = 0; b < 4; ++b)
-                            if (o + b >= 0 && o + b < len) g[o + b] = (uint8_t)(w >> (8 * b));
+                            if (o + b >= 0 && o + b < len) g[o + b] = (uint8_t)(w4[j] >> (8 * b));
                     }
                 }
             }
