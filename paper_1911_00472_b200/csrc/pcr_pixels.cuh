@@ -388,21 +388,40 @@ __global__ void __launch_bounds__(kPixThreads, PCR_PIX_MIN_CTAS) pixel_kernel(Pa
             *reinterpret_cast<uint4*>(gbase + row * gpitch + 16 * c) = *reinterpret_cast<const uint4*>(s_stage + row * kStagePitch + 16 * c);
         }
     } else {
-        const int wid = tid >> 5, lane = tid & 31;
-        for (int row = wid; row < nrows; row += kPixThreads / 32) {
+        // rows at any byte address.  The 16-byte-aligned chunks of global memory that lie inside a row:
+        // five staged words shifted into place, one 16-byte store
+        constexpr int kInner = (3 * 128) / 16 - 1;
+        for (int i = tid; i < nrows * kInner; i += kPixThreads) {
+            const int row = i / kInner, slot = 1 + (i - row * kInner);
             uint8_t* gp = gbase + row * gpitch;
-            const int a = (int)(reinterpret_cast<uintptr_t>(gp) & 3u);
-            const uint8_t* srow = s_stage + row * kStagePitch;
-            const uint32_t* sw = reinterpret_cast<const uint32_t*>(srow);
-            const int nw = (a + nbytes + 3) >> 2;
-            for (int i = lane; i < nw; i += 32) {
-                const int sb = 4 * i - a;                     // first staged byte of this output word
-                if (sb >= 0 && sb + 4 <= nbytes) {
-                    const uint32_t lo = sw[sb >> 2], hi = sw[(sb >> 2) + 1];   // the spare bytes keep hi in bounds
-                    const uint32_t v = a ? __funnelshift_r(lo, hi, 8 * (sb & 3)) : lo;
-                    *reinterpret_cast<uint32_t*>(gp + sb) = v;
-                } else {
-                    for (int b = max(sb, 0); b < min(sb + 4, nbytes); ++b) gp[b] = srow[b];
+            const int lead = (int)(reinterpret_cast<uintptr_t>(gp) & 15u);
+            if (16 * slot + 16 > lead + nbytes) continue;     // the row's last chunk, or behind it
+            const int o0 = 16 * slot - lead;                  // the chunk's first byte, counted from the row's first
+            const uint32_t* q = reinterpret_cast<const uint32_t*>(s_stage + row * kStagePitch) + (o0 >> 2);
+            const int sh = 8 * (o0 & 3);
+            const uint32_t p0 = q[0], p1 = q[1], p2 = q[2], p3 = q[3], p4 = q[4];   // (the spare bytes keep p4 in bounds)
+            *reinterpret_cast<uint4*>(gp + o0) = make_uint4(__funnelshift_r(p0, p1, sh), __funnelshift_r(p1, p2, sh),
+                                                            __funnelshift_r(p2, p3, sh), __funnelshift_r(p3, p4, sh));
+        }
+        // the first and the last chunk of every row: whole words where they lie inside the row, else bytes
+        if (tid < 2 * nrows) {
+            const int row = tid >> 1;
+            uint8_t* gp = gbase + row * gpitch;
+            const int lead = (int)(reinterpret_cast<uintptr_t>(gp) & 15u);
+            const int nch = (lead + nbytes + 15) >> 4;
+            if (!(tid & 1) || nch > 1) {
+                const int o0 = 16 * ((tid & 1) ? nch - 1 : 0) - lead;
+                const uint8_t* srow = s_stage + row * kStagePitch;
+                const uint32_t* sw = reinterpret_cast<const uint32_t*>(srow);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int sb = o0 + 4 * j;                // first staged byte of this output word
+                    if (sb >= 0 && sb + 4 <= nbytes) {
+                        const uint32_t lo = sw[sb >> 2], hi = sw[(sb >> 2) + 1];   // the spare bytes keep hi in bounds
+                        *reinterpret_cast<uint32_t*>(gp + sb) = __funnelshift_r(lo, hi, 8 * (sb & 3));
+                    } else {
+                        for (int b = max(sb, 0); b < min(sb + 4, nbytes); ++b) gp[b] = srow[b];
+                    }
                 }
             }
         }
