@@ -591,16 +591,21 @@ int open_impl(const uint8_t* rec, size_t len, pcr_record* r) {
         for (int g = 0; g <= r->n_slices; ++g) r->slice_img[g] = (uint32_t)((uint64_t)N * g / r->n_slices);
     }
     // Processing order of the images: a slice is a run of this order.  The time a slice needs for
-    // its entropy waves is set by its longest restart interval, i.e. by its widest image, so the
-    // images are sorted by decreasing width: slices of narrow images finish their waves early and
-    // their pixel stage overlaps the waves of the wide ones.
+    // its entropy waves is set by its longest restart intervals, so the images are sorted by their
+    // entropy-coded bytes per MCU row, most first: the slice of the heaviest rows starts first, slices
+    // of light images finish their waves early and their pixel stage overlaps the waves of the heavy
+    // ones.  (By width alone, the first version of this order: 2 % slower on the ImageNet-shaped record.)
     std::vector<uint32_t> order(N);
     for (uint32_t i = 0; i < N; ++i) order[i] = i;
-    if (r->n_slices > 1)
-        std::stable_sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) {
-            if (imgs[a].mx != imgs[b].mx) return imgs[a].mx > imgs[b].mx;
-            return imgs[a].my > imgs[b].my;
-        });
+    if (r->n_slices > 1) {
+        std::vector<double> key(N);
+        for (uint32_t i = 0; i < N; ++i) {
+            uint64_t b = 0;
+            for (uint32_t s2 = 0; s2 < G; ++s2) b += scans[(size_t)s2 * N + i].data_end - scans[(size_t)s2 * N + i].data_off;
+            key[i] = (double)b / (double)std::max<uint32_t>(1, imgs[i].my);
+        }
+        std::stable_sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) { return key[a] > key[b]; });
+    }
     std::vector<Item> items;
     items.reserve((size_t)(segs / 24 + (uint64_t)N * G));
     r->item_begin.assign((size_t)r->n_slices * G, 0); r->item_count.assign((size_t)r->n_slices * G, 0);
