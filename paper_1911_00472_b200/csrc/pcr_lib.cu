@@ -1102,7 +1102,7 @@ static int decode_range(pcr_record* rec, int k0, int k, void* out, void* stream,
                 const int s0 = rec->wave_scans[w][0];      // the record's one scan
                 const uint32_t lc = (s0 >= k0 && s0 < k) ? rec->long_count[(size_t)g * G + s0] : 0u;
                 if (lc) {                                  // images whose scan is one long restart interval
-                    sequential_long_kernel<<<(lc + kSeqLongWarps - 1) / kSeqLongWarps, 32 * kSeqLongWarps, 0, q>>>(P, rec->d_long + rec->long_begin[(size_t)g * G + s0], lc);
+                    sequential_long_kernel<<<lc, 32 * kSeqLongWarps, 0, q>>>(P, rec->d_long + rec->long_begin[(size_t)g * G + s0], lc);
                     ++g_launches;
                 }
                 return true;

@@ -582,13 +582,21 @@ __device__ __forceinline__ void seq_span(const HuffTab* tabs4, uint32_t slots, u
     sum0 = s0; sum1 = s1; sum2 = s2;
 }
 
-constexpr int kSeqLongWarps = 2;
+#ifndef PCR_SEQ_LONG_WARPS
+#define PCR_SEQ_LONG_WARPS 4
+#endif
+constexpr int kSeqLongWarps = PCR_SEQ_LONG_WARPS;   // warps per image in sequential_long_kernel: 32 subsequences each
 
+// One CTA of kSeqLongWarps warps per listed image whose (one) sequential scan is one restart interval.
 __global__ void __launch_bounds__(32 * kSeqLongWarps) sequential_long_kernel(Params P, const uint32_t* __restrict__ list, uint32_t count) {
-    __shared__ HuffTab tabs[kSeqLongWarps][4];                // DC 0, DC 1, AC 0, AC 1
-    const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t it = blockIdx.x * kSeqLongWarps + wid;
-    if (it >= count) return;                                   // whole warp
+    __shared__ HuffTab tabs[4];                                // DC 0, DC 1, AC 0, AC 1
+    __shared__ uint32_t s_pos[kSeqLongWarps];                  // end state of every warp's last lane, for the next warp's first
+    __shared__ int s_state[kSeqLongWarps];
+    __shared__ uint32_t s_u[kSeqLongWarps];
+    __shared__ int s_i[kSeqLongWarps];
+    const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
+    const uint32_t it = blockIdx.x;
+    if (it >= count) return;                                   // whole CTA
     const uint32_t si = list[it];
     const int img = (int)(si % (uint32_t)P.N);
     const ScanDesc sd = P.scans[si];
@@ -597,21 +605,24 @@ __global__ void __launch_bounds__(32 * kSeqLongWarps) sequential_long_kernel(Par
     const uint32_t mcu_w = g.mx, total = g.mx * g.my;
     const uint32_t bpm = P.nc == 3 ? (uint32_t)(P.hs * P.vs + 2) : 1u;
     const unsigned full = 0xffffffffu;
-    build_hufftab(tabs[wid][0], P.rec + sd.tab_off[0], lane);
-    if (sd.tab_off[1]) build_hufftab(tabs[wid][1], P.rec + sd.tab_off[1], lane);
-    build_hufftab(tabs[wid][2], P.rec + sd.tab_ac[0], lane);
-    if (sd.tab_ac[1]) build_hufftab(tabs[wid][3], P.rec + sd.tab_ac[1], lane);
+    // four tables, built by the warps in turn
+    for (int t = wid; t < 4; t += kSeqLongWarps) {
+        const uint32_t off = t == 0 ? sd.tab_off[0] : (t == 1 ? sd.tab_off[1] : (t == 2 ? sd.tab_ac[0] : sd.tab_ac[1]));
+        if (off) build_hufftab(tabs[t], P.rec + off, lane);
+    }
+    __syncthreads();
     const uint32_t* segtab = P.seg_start + sd.seg_base;
     const uint32_t bstart = segtab[0], bend = segtab[1] - 2u;
-    if (bstart < sd.data_off || bend > sd.data_end || bend < bstart) {
-        if (lane == 0) atomicMin(&P.status[img], kErrCorrupt);
+    if (bstart < sd.data_off || bend > sd.data_end || bend < bstart) {   // (the same for every thread)
+        if (tid == 0) atomicMin(&P.status[img], kErrCorrupt);
         return;
     }
     const uint32_t* base = reinterpret_cast<const uint32_t*>(P.ubuf) + (bstart >> 2);
     const uint32_t lead = 8u * (bstart & 3u), endbit = lead + 8u * (bend - bstart);
+    constexpr uint32_t kSubs = 32u * kSeqLongWarps;
     const uint32_t nwords = (endbit + 31u) >> 5;
-    const uint32_t S = 32u * max(8u, (nwords + 31u) / 32u);
-    const uint32_t my_begin = min(max((uint32_t)lane * S, lead), endbit), my_end = min(((uint32_t)lane + 1u) * S, endbit);
+    const uint32_t S = 32u * max(8u, (nwords + kSubs - 1u) / kSubs);
+    const uint32_t my_begin = min(max((uint32_t)tid * S, lead), endbit), my_end = min(((uint32_t)tid + 1u) * S, endbit);
     bool bad = false;
     SeqWrite W;
     W.head = P.head; W.planes = P.planes; W.mcu_w = mcu_w; W.hs = (uint32_t)P.hs; W.vs = (uint32_t)P.vs;
@@ -621,31 +632,33 @@ __global__ void __launch_bounds__(32 * kSeqLongWarps) sequential_long_kernel(Par
     uint32_t pos = my_begin, pos_x = my_begin, nb = 0;
     int j = 0, k = 0, j_x = 0, k_x = 0, a0 = 0, a1 = 0, a2 = 0;
     bool again = true;
-    for (int round = 0; round < 33; ++round) {
-        if (again) seq_span<false>(tabs[wid], sd.slots, sd.slots_ac, P.nc, base, pos, j, k, my_end, pos_x, j_x, k_x, nb, a0, a1, a2, W, bad);
-        const uint32_t ppos = min(__shfl_up_sync(full, pos_x, 1), endbit);
-        const int pj = __shfl_up_sync(full, j_x, 1), pk = __shfl_up_sync(full, k_x, 1);
-        again = lane > 0 && (ppos != pos || pj != j || pk != k);
-        if (again) { pos = ppos; j = pj; k = pk; }
-        if (!__any_sync(full, again)) break;
+    for (int round = 0; round <= (int)kSubs; ++round) {
+        if (again) seq_span<false>(tabs, sd.slots, sd.slots_ac, P.nc, base, pos, j, k, my_end, pos_x, j_x, k_x, nb, a0, a1, a2, W, bad);
+        // the state the previous thread ended in (block of the MCU and zigzag position in one word)
+        const int st_x = j_x * 64 + k_x;
+        if (lane == 31) { s_pos[wid] = pos_x; s_state[wid] = st_x; }
+        __syncthreads();
+        uint32_t ppos = __shfl_up_sync(full, pos_x, 1);
+        int pst = __shfl_up_sync(full, st_x, 1);
+        if (lane == 0 && wid > 0) { ppos = s_pos[wid - 1]; pst = s_state[wid - 1]; }
+        ppos = min(ppos, endbit);
+        again = tid > 0 && (ppos != pos || pst != j * 64 + k);
+        if (again) { pos = ppos; j = pst >> 6; k = pst & 63; }
+        if (!__syncthreads_or(again)) break;
     }
-    uint32_t nin = nb;
-    int b0 = a0, b1 = a1, b2 = a2;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const uint32_t on = __shfl_up_sync(full, nin, d);
-        const int o0 = __shfl_up_sync(full, b0, d), o1 = __shfl_up_sync(full, b1, d), o2 = __shfl_up_sync(full, b2, d);
-        if (lane >= d) { nin += on; b0 += o0; b1 += o1; b2 += o2; }
-    }
-    const uint32_t all = __shfl_sync(full, nin, 31);
-    W.n = min(nin - nb, W.n1); W.pred[0] = b0 - a0; W.pred[1] = b1 - a1; W.pred[2] = b2 - a2;
+    uint32_t all;
+    int t0, t1, t2;
+    W.n = min(cta_exclusive_sum(nb, s_u, wid, lane, kSeqLongWarps, all), W.n1);
+    W.pred[0] = cta_exclusive_sum(a0, s_i, wid, lane, kSeqLongWarps, t0);
+    W.pred[1] = cta_exclusive_sum(a1, s_i, wid, lane, kSeqLongWarps, t1);
+    W.pred[2] = cta_exclusive_sum(a2, s_i, wid, lane, kSeqLongWarps, t2);
     // the place inside the MCU follows from the block number (equal to the handed-on state unless the
     // stream is damaged; taking it from the block number keeps every store inside the image)
     if ((nb || k) && (uint32_t)j != W.n % bpm) bad = true;
     j = (int)(W.n % bpm);
-    seq_span<true>(tabs[wid], sd.slots, sd.slots_ac, P.nc, base, pos, j, k, my_end, pos_x, j_x, k_x, nb, a0, a1, a2, W, bad);
+    seq_span<true>(tabs, sd.slots, sd.slots_ac, P.nc, base, pos, j, k, my_end, pos_x, j_x, k_x, nb, a0, a1, a2, W, bad);
     if (all < total * bpm) bad = true;                         // the stream ends before the last block
-    if (__any_sync(full, bad) && lane == 0) atomicMin(&P.status[img], kErrCorrupt);
+    if (__syncthreads_or(bad) && tid == 0) atomicMin(&P.status[img], kErrCorrupt);
 }
 
 // ---------------------------------------------------------------------------------------
