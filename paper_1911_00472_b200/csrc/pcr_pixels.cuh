@@ -82,6 +82,16 @@ __device__ __forceinline__ uint32_t pack4_sat(int v0, int v1, int v2, int v3) {
     return w;
 }
 
+// bytes {clamp(v0 + 128), ..., clamp(v3 + 128)}, clamp to 0..255, for any 32-bit v: clamping v to
+// -128..127 and flipping the byte's top bit is the same as adding 128 and clamping to 0..255, and it
+// needs no addition that could overflow for v near the ends of the 32-bit range
+__device__ __forceinline__ uint32_t pack4_sat_plus128(int v0, int v1, int v2, int v3) {
+    uint32_t hi, w;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(v3), "r"(v2), "r"(0));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(v1), "r"(v0), "r"(hi));
+    return w ^ 0x80808080u;
+}
+
 // kRefine: first fold the side data of the AC refinement scans (see ScanAux) into the block, in
 // scan order, and write the updated 128-byte line back, so the planes in device memory hold the
 // final coefficients.  The thread parks its line in shared memory for that (word w of thread t
@@ -166,8 +176,8 @@ __global__ void __launch_bounds__(kPixThreads, PCR_PIX_MIN_CTAS) pixel_kernel(Pa
             constexpr uint32_t K4 = 5793;
             const int F = (int)P.head[blk * 8] * (int)s_q[comp][0];
             const int T = (int)(K4 * (uint32_t)F + (1u << 11)) >> 12;
-            const int smp = (int)(K4 * (uint32_t)T + (1u << 15) + (128u << 16)) >> 16;
-            const uint32_t w = pack4_sat(smp, smp, smp, smp);
+            const int smp = (int)(K4 * (uint32_t)T + (1u << 15)) >> 16;
+            const uint32_t w = pack4_sat_plus128(smp, smp, smp, smp);
             uint8_t* dst;
             int pitch;
             if (comp == 0) { dst = &s_y[yr * 8][yc * 8]; pitch = 128; }
@@ -286,7 +296,7 @@ __global__ void __launch_bounds__(kPixThreads, PCR_PIX_MIN_CTAS) pixel_kernel(Pa
 #pragma unroll
             for (int u = 0; u < 8; ++u)
                 idct8(v[u], v[8 + u], v[16 + u], v[24 + u], v[32 + u], v[40 + u], v[48 + u], v[56 + u], 1u << 11, 12);
-            // pass 2: rows; the +128 level shift rides in the rounding constant
+            // pass 2: rows; the +128 level shift is part of the packing
             uint8_t* dst;
             int pitch;
             if (kStage == 1) { dst = cplane; pitch = 8 * (int)im.mx; }
@@ -295,9 +305,9 @@ __global__ void __launch_bounds__(kPixThreads, PCR_PIX_MIN_CTAS) pixel_kernel(Pa
 #pragma unroll
             for (int y = 0; y < 8; ++y) {
                 idct8(v[8 * y], v[8 * y + 1], v[8 * y + 2], v[8 * y + 3], v[8 * y + 4], v[8 * y + 5], v[8 * y + 6], v[8 * y + 7],
-                      (1u << 15) + (128u << 16), 16);
-                const uint32_t lo = pack4_sat((int)v[8 * y], (int)v[8 * y + 1], (int)v[8 * y + 2], (int)v[8 * y + 3]);
-                const uint32_t hi = pack4_sat((int)v[8 * y + 4], (int)v[8 * y + 5], (int)v[8 * y + 6], (int)v[8 * y + 7]);
+                      1u << 15, 16);
+                const uint32_t lo = pack4_sat_plus128((int)v[8 * y], (int)v[8 * y + 1], (int)v[8 * y + 2], (int)v[8 * y + 3]);
+                const uint32_t hi = pack4_sat_plus128((int)v[8 * y + 4], (int)v[8 * y + 5], (int)v[8 * y + 6], (int)v[8 * y + 7]);
                 *reinterpret_cast<uint2*>(dst + y * pitch) = make_uint2(lo, hi);
             }
         }
@@ -458,7 +468,7 @@ __global__ void __launch_bounds__(128) dc_pixel_kernel(Params P, uint8_t* __rest
         auto sample = [&](uint64_t blk, int comp) {
             const int F = (int)P.head[blk * 8] * (int)q[64 * comp];
             const int T = (int)(K4 * (uint32_t)F + (1u << 11)) >> 12;
-            const int smp = (int)(K4 * (uint32_t)T + (1u << 15) + (128u << 16)) >> 16;
+            const int smp = ((int)(K4 * (uint32_t)T + (1u << 15)) >> 16) + 128;
             return min(max(smp, 0), 255);
         };
         const uint64_t mcus = (uint64_t)im.mx * im.my;

@@ -298,3 +298,44 @@ def test_record_cache_reopens_the_same_record_and_only_that(rec0, rec1_small):
         other.close()
     finally:
         binding.pcr_set_record_cache(0)
+
+
+def test_samples_near_the_end_of_the_32_bit_range():
+    """Coefficients no image produces: a luminance DC of 2040 under a quantiser of 128 gives a sample of
+    32644 before the level shift, so the second transform pass ends within 128 << 16 of 2^31.  The oracle
+    rounds, shifts, adds 128 and clamps (255); a kernel that folds the 128 into the rounding constant
+    wraps there (0).  Dense +-1023 fields at odd sizes beside it (4:2:0 and 4:4:0)."""
+    import torch
+    from paper_1911_00472_b200 import Decoder
+    rng = np.random.default_rng(21)
+    qy = np.ones(64, dtype=np.uint8); qy[0] = 128
+    qc = np.ones(64, dtype=np.uint8)
+    for samp in ((2, 2, 3), (1, 2, 3)):
+        with pcr_synth.sampling(*samp):
+            dims = [(24, 16), (183, 70), (61, 35)]
+            coeffs = []
+            for n, (w, h) in enumerate(dims):
+                nb = pcr_synth.num_blocks(w, h)
+                if n == 0:
+                    c = np.zeros((nb, 64), dtype=np.int16)
+                    c[:, 0] = 2040
+                else:
+                    c = rng.integers(-1023, 1024, size=(nb, 64)).astype(np.int16)
+                coeffs.append(c)
+            rec = pcr_synth.record_from_coeffs(dims, coeffs, qtables=(qy, qc))
+            rec2 = pcr_synth.record_from_coeffs(dims[1:], coeffs[1:])
+        for r in (rec, rec2):
+            dec = Decoder(r.bytes)
+            try:
+                for k in (1, dec.n_groups):
+                    out = dec.decode(k).cpu().numpy()
+                    assert dec.status() == (-1, 0)
+                    for i in range(r.n_images):
+                        _, want = O.decode_image(r.bytes, i, k)
+                        inf = dec.info[i]
+                        got = out[inf.out_offset:inf.out_offset + inf.out_bytes].reshape(inf.height, inf.width, 3)
+                        assert np.array_equal(got, want), (samp, i, k, np.argwhere(got != want)[:3])
+            finally:
+                dec.close()
+    _, rgb = O.decode_image(rec.bytes, 0, 10)
+    assert rgb[0, 0, 0] == 255          # (the case is the one described: the oracle saturates high)
